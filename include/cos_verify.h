@@ -1,0 +1,155 @@
+/*
+ * cos_verify.h -- C ABI of the CoS verification step for NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper: "Fast Large Language Model Collaborative Decoding via
+ * Speculation", Sec. 3.1-3.2):
+ *   for every row b of a batch and every one of the gamma+1 positions j, read the
+ *   logits of n models over the vocabulary, form the combined distribution r
+ *   (Eq. 3: weighted probability ensemble, Eq. 4, or a logit-level combination,
+ *   Eq. 5, optionally restricted to a plausibility mask), test the draft token x
+ *   with  u <= min(1, r(x) / q(x))  against the proposer's distribution q (Eq. 6),
+ *   find the first rejected position of the row, and emit there a token drawn from
+ *   norm(max(0, r - q)) (text after Eq. 6, App. A.1), or, when all gamma drafts pass,
+ *   a bonus token for position gamma (Sec. 3.1).  Temperature T tempers every
+ *   softmax; T = 0 is greedy decoding with one-hot distributions (Sec. 4.1).
+ *
+ * All pointers in cos_verify_args are DEVICE pointers owned by the caller unless a
+ * function says otherwise.  No function here synchronises the device except
+ * cos_verify_create, cos_verify_destroy and cos_verify_run_host.
+ */
+#ifndef COS_VERIFY_H
+#define COS_VERIFY_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define COS_MAX_MODELS 8
+
+typedef struct cos_verify_ctx cos_verify_ctx; /* opaque; owns only device scratch */
+
+typedef enum {
+  COS_OK = 0,
+  COS_ERR_INVALID_ARG = 1, /* null pointer, value out of range, inconsistent config   */
+  COS_ERR_UNSUPPORTED = 2, /* valid request this build does not implement             */
+  COS_ERR_ALIGNMENT = 3,   /* a pointer is not aligned to its element type            */
+  COS_ERR_CUDA = 4,        /* a CUDA runtime call failed; see cos_verify_last_error   */
+  COS_ERR_NOMEM = 5        /* host or device allocation failed                        */
+} cos_status;
+
+/* combination function C / C' of Eq. 3 */
+enum {
+  COS_COMBINE_PROB_ENSEMBLE = 0, /* r = sum_i w_i softmax(l_i / T)              (Eq. 4)            */
+  COS_COMBINE_LOGIT_LINEAR = 1   /* r = softmax_M((sum_i w_i l_i) / T)          (Eq. 5; also logit */
+                                 /*     interpolation of an aligned / base model pair)             */
+};
+
+enum { COS_DTYPE_F32 = 0, COS_DTYPE_BF16 = 1 };
+
+/* bits of row_status[b]; only positions up to and including the row's first rejection report */
+enum {
+  COS_ROW_NONFINITE = 1,      /* a distribution was NaN/Inf: that position counts as rejected, token -1 */
+  COS_ROW_BAD_DRAFT = 2,      /* draft token outside [0, vocab): rejected, residual still sampled       */
+  COS_ROW_Q_ZERO = 4,         /* q(draft) == 0: ratio taken as +inf if r(draft) > 0, else 0             */
+  COS_ROW_RESIDUAL_EMPTY = 8  /* rejected but max(0, r - q) == 0 everywhere: token drawn from r         */
+};
+
+/* bits of cos_verify_args.flags */
+enum {
+  COS_RUN_ALL_RESIDUALS = 1 /* compute the residual mass S = sum max(0, r - q) = 1 - alpha (Eq. 7) at  */
+                            /* every draft position and report it in diag, not only where it is needed */
+};
+
+typedef struct {
+  int32_t n;                       /* number of models, 1..COS_MAX_MODELS                               */
+  int32_t combine;                 /* COS_COMBINE_*                                                     */
+  float weights[COS_MAX_MODELS];   /* w_i.  Ensemble: w_i >= 0, |sum - 1| <= 1e-6.  Logit-linear: any   */
+                                   /* finite values (contrastive decoding is (1, -mu), Eq. 5).          */
+  int32_t mask_model;              /* logit-linear only: index e of the model whose probabilities gate  */
+                                   /* the vocabulary, or -1 for no mask                                 */
+  float mask_alpha;                /* in (0, 1]: keep x with l_e(x) >= max_x l_e(x) + ln(mask_alpha)    */
+  float temperature;               /* T >= 0; 0 = greedy (lowest index wins ties)                       */
+  int32_t gamma;                   /* proposal length, >= 0; every row has gamma + 1 positions          */
+  int32_t vocab;                   /* V >= 1                                                            */
+  int32_t max_batch;               /* largest batch a run may pass, >= 1                                */
+  int32_t dtype;                   /* COS_DTYPE_* of the logits                                         */
+  int32_t device;                  /* CUDA device ordinal                                               */
+  int32_t cluster_size;            /* thread blocks that share one (row, position): 1, 2, 4, 8 or 16;   */
+                                   /* 0 lets the library choose from the vocabulary size                */
+  int32_t host_staging;            /* non-zero: also allocate device staging for cos_verify_run_host    */
+} cos_verify_config;
+
+typedef struct {
+  const void* logits;          /* [n][B][gamma+1][V], element (i,b,j,x) at                              */
+                               /*   i*stride_model + b*stride_row + j*stride_pos + x   (in elements)    */
+  int64_t stride_model, stride_row, stride_pos;
+  const int32_t* draft_tokens; /* [B][gamma]; may be NULL when gamma == 0                               */
+  const int32_t* proposer;     /* [B], index in [0, n) of the model that proposed the row's drafts      */
+  int32_t batch;               /* B, 1..max_batch                                                       */
+  int32_t flags;               /* COS_RUN_* bits                                                        */
+  int64_t row_base;            /* global index of row 0 (for row-sharded batches); enters the RNG only  */
+  uint64_t seed, offset;       /* Philox4x32-10 key and counter words 2-3; counter words 0-1 are        */
+                               /* (row_base + b, j).  Word 0 of the output feeds the accept test, word  */
+                               /* 1 the residual / bonus sample, each as u = (2*(w>>9)+1) * 2^-24.      */
+  int32_t* accept_count;       /* out [B]: number of accepted drafts a, 0..gamma                        */
+  int32_t* out_tokens;         /* out [B][gamma+1]: a accepted drafts, then the resampled (a < gamma)   */
+                               /* or bonus (a == gamma) token, then -1 padding                          */
+  uint32_t* row_status;        /* out [B]: COS_ROW_* bits                                               */
+  float* diag;                 /* optional out [B][gamma+1][4]: ratio r(x)/q(x), r(x), q(x) at the      */
+                               /* draft, and S where it was computed (NaN elsewhere); may be NULL       */
+  float* dump_r;               /* optional test hook, out [B][gamma+1][V]: the combined distribution;   */
+                               /* forces the full second sweep everywhere; may be NULL                  */
+} cos_verify_args;
+
+typedef struct {
+  int32_t cluster_size;      /* thread blocks per (row, position)                                     */
+  int32_t threads_per_block;
+  int32_t max_clusters;      /* clusters that can be resident at once on the device                   */
+  int32_t sm_count;
+  int32_t launches_per_run;  /* kernels cos_verify_run enqueues per call                              */
+  int32_t reserved[3];
+} cos_verify_info;
+
+/*
+ * Validate the configuration, select the device, allocate scratch sized for
+ * max_batch * (gamma + 1) positions and return a context in *out.
+ * Errors: COS_ERR_INVALID_ARG (with the reason available from cos_verify_last_error(NULL)),
+ * COS_ERR_CUDA, COS_ERR_NOMEM.  One context serves one stream at a time.
+ */
+cos_status cos_verify_create(const cos_verify_config* config, cos_verify_ctx** out);
+
+/*
+ * Enqueue one verification pass (Eq. 3-6 and the rejection / bonus rule of Sec. 3.1) for
+ * args->batch rows on `cuda_stream` (a cudaStream_t; NULL is the default stream) and
+ * return without waiting.  Outputs are valid once the stream has reached this point.
+ * Host-detected problems return an error code and enqueue nothing; data-dependent
+ * problems are reported per row in row_status and never trap the device.
+ * Runs that share a context must be ordered on one stream.
+ */
+cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* args, void* cuda_stream);
+
+/*
+ * Same operation with every pointer in `args` a HOST pointer (pinned memory makes the
+ * copies asynchronous): copies logits, drafts and proposers to staging owned by the
+ * context, runs, copies accept_count / out_tokens / row_status (and diag if given)
+ * back and waits for the stream.  Requires config.host_staging != 0 and contiguous
+ * logits (stride_pos = V, stride_row = (gamma+1) V, stride_model = B (gamma+1) V).
+ * dump_r is not supported here.
+ */
+cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args, void* cuda_stream);
+
+/* Launch geometry chosen at creation. */
+cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info);
+
+/* Free the context and its scratch (waits for the device). NULL is allowed. */
+cos_status cos_verify_destroy(cos_verify_ctx* ctx);
+
+/* Text of the last error on this context, or of the last failed create when ctx is NULL. */
+const char* cos_verify_last_error(const cos_verify_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COS_VERIFY_H */

@@ -1,0 +1,228 @@
+"""ctypes binding of include/cos_verify.h: argument marshalling only.
+
+torch supplies device memory and the stream; all arithmetic happens in the CUDA library.
+Loading fails loudly if the library cannot be built or opened.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional, Sequence
+
+from . import build as _build
+
+COS_MAX_MODELS = 8
+COS_OK = 0
+COS_COMBINE_PROB_ENSEMBLE = 0
+COS_COMBINE_LOGIT_LINEAR = 1
+COS_DTYPE_F32 = 0
+COS_DTYPE_BF16 = 1
+COS_ROW_NONFINITE = 1
+COS_ROW_BAD_DRAFT = 2
+COS_ROW_Q_ZERO = 4
+COS_ROW_RESIDUAL_EMPTY = 8
+COS_RUN_ALL_RESIDUALS = 1
+
+_STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR_ALIGNMENT",
+                 4: "COS_ERR_CUDA", 5: "COS_ERR_NOMEM"}
+
+EXPORTS = ("cos_verify_create", "cos_verify_run", "cos_verify_run_host", "cos_verify_get_info",
+           "cos_verify_destroy", "cos_verify_last_error")
+
+
+class CosVerifyError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{_STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+class cos_verify_config(ctypes.Structure):
+    _fields_ = [
+        ("n", ctypes.c_int32), ("combine", ctypes.c_int32), ("weights", ctypes.c_float * COS_MAX_MODELS),
+        ("mask_model", ctypes.c_int32), ("mask_alpha", ctypes.c_float), ("temperature", ctypes.c_float),
+        ("gamma", ctypes.c_int32), ("vocab", ctypes.c_int32), ("max_batch", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("device", ctypes.c_int32), ("cluster_size", ctypes.c_int32),
+        ("host_staging", ctypes.c_int32),
+    ]
+
+
+class cos_verify_args(ctypes.Structure):
+    _fields_ = [
+        ("logits", ctypes.c_void_p), ("stride_model", ctypes.c_int64), ("stride_row", ctypes.c_int64),
+        ("stride_pos", ctypes.c_int64), ("draft_tokens", ctypes.c_void_p), ("proposer", ctypes.c_void_p),
+        ("batch", ctypes.c_int32), ("flags", ctypes.c_int32), ("row_base", ctypes.c_int64),
+        ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64), ("accept_count", ctypes.c_void_p),
+        ("out_tokens", ctypes.c_void_p), ("row_status", ctypes.c_void_p), ("diag", ctypes.c_void_p),
+        ("dump_r", ctypes.c_void_p),
+    ]
+
+
+class cos_verify_info(ctypes.Structure):
+    _fields_ = [
+        ("cluster_size", ctypes.c_int32), ("threads_per_block", ctypes.c_int32), ("max_clusters", ctypes.c_int32),
+        ("sm_count", ctypes.c_int32), ("launches_per_run", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+    ]
+
+
+_lib = None
+
+
+def load_library(rebuild: bool = False) -> ctypes.CDLL:
+    """Build (if stale) and open libcos_verify.so; raises if either step fails."""
+    global _lib
+    if _lib is not None and not rebuild:
+        return _lib
+    path = _build.build(force=rebuild)
+    lib = ctypes.CDLL(path)
+    lib.cos_verify_create.argtypes = [ctypes.POINTER(cos_verify_config), ctypes.POINTER(ctypes.c_void_p)]
+    lib.cos_verify_create.restype = ctypes.c_int
+    lib.cos_verify_run.argtypes = [ctypes.c_void_p, ctypes.POINTER(cos_verify_args), ctypes.c_void_p]
+    lib.cos_verify_run.restype = ctypes.c_int
+    lib.cos_verify_run_host.argtypes = [ctypes.c_void_p, ctypes.POINTER(cos_verify_args), ctypes.c_void_p]
+    lib.cos_verify_run_host.restype = ctypes.c_int
+    lib.cos_verify_get_info.argtypes = [ctypes.c_void_p, ctypes.POINTER(cos_verify_info)]
+    lib.cos_verify_get_info.restype = ctypes.c_int
+    lib.cos_verify_destroy.argtypes = [ctypes.c_void_p]
+    lib.cos_verify_destroy.restype = ctypes.c_int
+    lib.cos_verify_last_error.argtypes = [ctypes.c_void_p]
+    lib.cos_verify_last_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _dtype_code(torch_dtype) -> int:
+    import torch
+    if torch_dtype == torch.float32:
+        return COS_DTYPE_F32
+    if torch_dtype == torch.bfloat16:
+        return COS_DTYPE_BF16
+    raise ValueError(f"logits must be float32 or bfloat16, not {torch_dtype}")
+
+
+class CosVerifier:
+    """One verification context (cos_verify_create ... cos_verify_destroy).
+
+    run() takes device tensors and returns device tensors; run_host() takes host tensors
+    (pinned for asynchronous copies) and returns host tensors, the copies being part of the call.
+    """
+
+    def __init__(self, n: int, combine: int, weights: Sequence[float], temperature: float, gamma: int,
+                 vocab: int, max_batch: int, dtype, mask_model: int = -1, mask_alpha: float = 1.0,
+                 device: int = 0, cluster_size: int = 0, host_staging: bool = False):
+        self._lib = load_library()
+        self._ctx = ctypes.c_void_p()
+        cfg = cos_verify_config()
+        cfg.n, cfg.combine = n, combine
+        for i, w in enumerate(list(weights)[:COS_MAX_MODELS]):
+            cfg.weights[i] = w
+        cfg.mask_model, cfg.mask_alpha, cfg.temperature = mask_model, mask_alpha, temperature
+        cfg.gamma, cfg.vocab, cfg.max_batch = gamma, vocab, max_batch
+        cfg.dtype = dtype if isinstance(dtype, int) else _dtype_code(dtype)
+        cfg.device, cfg.cluster_size, cfg.host_staging = device, cluster_size, int(host_staging)
+        self.cfg = cfg
+        st = self._lib.cos_verify_create(ctypes.byref(cfg), ctypes.byref(self._ctx))
+        if st != COS_OK:
+            msg = self._lib.cos_verify_last_error(None).decode()
+            self._ctx = ctypes.c_void_p()
+            raise CosVerifyError(st, msg)
+
+    # -- helpers ---------------------------------------------------------------------
+    def _check(self, st: int):
+        if st != COS_OK:
+            raise CosVerifyError(st, self._lib.cos_verify_last_error(self._ctx).decode())
+
+    def info(self) -> dict:
+        inf = cos_verify_info()
+        self._check(self._lib.cos_verify_get_info(self._ctx, ctypes.byref(inf)))
+        return {k: getattr(inf, k) for k in ("cluster_size", "threads_per_block", "max_clusters", "sm_count",
+                                             "launches_per_run")}
+
+    def _fill_args(self, logits, drafts, proposer, seed, offset, row_base, flags, outs) -> cos_verify_args:
+        n, B, P, V = logits.shape
+        if n != self.cfg.n or P != self.cfg.gamma + 1 or V != self.cfg.vocab:
+            raise ValueError(f"logits shape {tuple(logits.shape)} does not match the context")
+        if logits.stride(3) != 1:
+            raise ValueError("the vocabulary axis of logits must be contiguous")
+        if _dtype_code(logits.dtype) != self.cfg.dtype:
+            raise ValueError("logits dtype does not match the context")
+        a = cos_verify_args()
+        a.logits = logits.data_ptr()
+        a.stride_model, a.stride_row, a.stride_pos = logits.stride(0), logits.stride(1), logits.stride(2)
+        a.draft_tokens = drafts.data_ptr() if (drafts is not None and drafts.numel() > 0) else None
+        a.proposer = proposer.data_ptr()
+        a.batch, a.flags, a.row_base = B, flags, row_base
+        a.seed, a.offset = seed & 0xFFFFFFFFFFFFFFFF, offset & 0xFFFFFFFFFFFFFFFF
+        a.accept_count = outs["accept_count"].data_ptr()
+        a.out_tokens = outs["out_tokens"].data_ptr()
+        a.row_status = outs["row_status"].data_ptr()
+        a.diag = outs["diag"].data_ptr() if "diag" in outs else None
+        a.dump_r = outs["r"].data_ptr() if "r" in outs else None
+        return a
+
+    @staticmethod
+    def _alloc_outs(B, P, V, device, diag, dump_r, pin=False):
+        import torch
+        kw = dict(device=device)
+        if pin:
+            kw["pin_memory"] = True
+        outs = {
+            "accept_count": torch.empty(B, dtype=torch.int32, **kw),
+            "out_tokens": torch.empty((B, P), dtype=torch.int32, **kw),
+            "row_status": torch.empty(B, dtype=torch.int32, **kw),
+        }
+        if diag:
+            outs["diag"] = torch.empty((B, P, 4), dtype=torch.float32, **kw)
+        if dump_r:
+            outs["r"] = torch.empty((B, P, V), dtype=torch.float32, **kw)
+        return outs
+
+    # -- the calls -------------------------------------------------------------------
+    def run(self, logits, drafts, proposer, seed: int, offset: int, row_base: int = 0, flags: int = 0,
+            diag: bool = False, dump_r: bool = False, outs: Optional[dict] = None, stream=None) -> dict:
+        """cos_verify_run on device tensors; asynchronous on `stream` (default: torch's current stream)."""
+        import torch
+        if not logits.is_cuda:
+            raise ValueError("run() needs device tensors; use run_host() for host tensors")
+        for t, name in ((drafts, "drafts"), (proposer, "proposer")):
+            if t is not None and t.numel() > 0 and (t.dtype != torch.int32 or not t.is_contiguous() or not t.is_cuda):
+                raise ValueError(f"{name} must be a contiguous int32 device tensor")
+        n, B, P, V = logits.shape
+        if outs is None:
+            outs = self._alloc_outs(B, P, V, logits.device, diag, dump_r)
+        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs)
+        s = torch.cuda.current_stream(logits.device) if stream is None else stream
+        self._check(self._lib.cos_verify_run(self._ctx, ctypes.byref(a), ctypes.c_void_p(s.cuda_stream)))
+        return outs
+
+    def run_host(self, logits, drafts, proposer, seed: int, offset: int, row_base: int = 0, flags: int = 0,
+                 diag: bool = False, outs: Optional[dict] = None, stream=None) -> dict:
+        """cos_verify_run_host on host tensors: copies in, runs, copies out, waits."""
+        import torch
+        if logits.is_cuda or not logits.is_contiguous():
+            raise ValueError("run_host() needs contiguous host tensors")
+        for t, name in ((drafts, "drafts"), (proposer, "proposer")):
+            if t is not None and t.numel() > 0 and (t.dtype != torch.int32 or not t.is_contiguous() or t.is_cuda):
+                raise ValueError(f"{name} must be a contiguous int32 host tensor")
+        n, B, P, V = logits.shape
+        if outs is None:
+            outs = self._alloc_outs(B, P, V, "cpu", diag, False, pin=True)
+        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs)
+        s = torch.cuda.current_stream(self.cfg.device) if stream is None else stream
+        self._check(self._lib.cos_verify_run_host(self._ctx, ctypes.byref(a), ctypes.c_void_p(s.cuda_stream)))
+        return outs
+
+    def close(self):
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            self._lib.cos_verify_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
