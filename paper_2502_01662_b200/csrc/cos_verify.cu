@@ -16,6 +16,8 @@
 //            fp64 prefix sums, locate u * S, rescan one warp's run for the token;
 //   publish  per-unit result, and the last unit of a row to arrive runs the
 //            first-rejection scan and writes the row's outputs.
+// Units are handed out from a global counter (a cluster draws its next unit while it sweeps
+// the current one), because units that must draw a token take several times longer.
 // Nothing in the kernel spins on memory: blocks meet only at hardware cluster barriers.
 
 #include <cooperative_groups.h>
@@ -40,6 +42,10 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kMaxSlots = COS_MAX_MODELS + 2;
 constexpr int kMaxCluster = 16;
 constexpr int kNoReject = 0x7fffffff;
+constexpr double kBigShare = 1.0 / 1024.0;  // probabilities above 2^-10 get fp64 treatment in sweep 2
+constexpr int kRingVecs = 8;                 // 16-byte vectors per lane staged ahead in sweep 2 (4 KB per warp)
+constexpr int kRingBytes = kWarps * kRingVecs * 32 * 16;
+constexpr int kRec = 64;                     // running totals recorded per warp in sweep 2
 
 enum Mode { kEnsembleSample = 0, kLogitSample = 1, kEnsembleGreedy = 2, kLogitGreedy = 3 };
 
@@ -67,7 +73,7 @@ struct KParams {
   float* diag;
   float* dump_r;
   // scratch owned by the context
-  unsigned* work_counter;  // monotonically increasing across runs
+  unsigned* work_counter;  // units are handed out from here; grows by num_units every run
   unsigned work_base;      // its value when this run starts
   int* row_arrivals;       // [B], zero between runs
   int* first_rej;          // [B], kNoReject between runs
@@ -85,10 +91,26 @@ __device__ __forceinline__ float ex2_approx(float x) {
 
 __device__ __forceinline__ uint4 ldg_stream16(const void* p) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+  asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
   return v;
+}
+
+__device__ __forceinline__ int ld_relaxed_gpu(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* g) {
+  unsigned sa = static_cast<unsigned>(__cvta_generic_to_shared(smem));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
 template <int DT>
@@ -205,44 +227,52 @@ struct Xchg {  // one per block and barrier parity; peers read it through DSMEM
   SoftPart soft[kMaxSlots];
   ArgPart arg[kMaxSlots];
   double cta_total;
-  int bcast[4];
+  int known;  // rank 0 only: earliest rejected position of the row seen so far
+  int next;   // rank 0 only: the unit this cluster takes after the current one
 };
 
 struct Decision {  // written by thread 0 of every block, identically
   int accept, status, want_sample, cand;
-  int natoms;
+  int natoms, need2;
   int atom_tok[COS_MAX_MODELS];
   double atom_mass[COS_MAX_MODELS];
-  double ratio, r_d, q_d, S, u_smp;
+  double ratio, r_d, q_d, S;
 };
 
 struct Shared {
   Xchg x[2];
   SoftPart wsoft[kWarps][kMaxSlots];
   ArgPart warg[kWarps][kMaxSlots];
-  double wtot[kWarps];       // this block's per-warp totals of sweep 2
-  double wincl[kWarps];      // their running sum
-  SoftPart fsoft[kMaxSlots]; // merged over the cluster
+  double wtot[kWarps];        // this block's per-warp totals of sweep 2
+  double wincl[kWarps];       // their running sum
+  double srun[kWarps][kRec];  // a warp's running total after each group of steps
+  SoftPart fsoft[kMaxSlots];  // merged over the cluster
   ArgPart farg[kMaxSlots];
+  double pdraft[kMaxSlots];   // probability of the draft token under each merged softmax
   float a_scale[COS_MAX_MODELS];  // w_i / Z_i (ensemble) for sweep 2
   float a_ref[COS_MAX_MODELS];
+  float a_resid[COS_MAX_MODELS];  // coefficient of e_i in r - q
   Decision dec;
-  double target, base;  // sweep-2 search: u*S and the mass before the winning warp
+  double u_acc, u_smp;
+  double target, base;  // sweep-2 search: u*S and the mass before the winning block
   int win_rank, win_warp;
-  int need2, next_unit;
+  int known_local, known;
+  int next_local, next;
   float thr32;  // plausibility threshold rounded up to fp32
+  float big_thr[kMaxSlots];  // sweep 2: terms above this share of a normaliser are redone in fp64
   float ldraft[COS_MAX_MODELS];  // the n logits at the draft token, fetched before sweep 1
 };
 
-// lane accumulator of the online softmax in the base-2 domain
+// lane accumulator of a softmax normaliser in the base-2 domain: s = sum 2^(v*c - ref)
 struct LaneSoft {
   float ref, s;
   __device__ __forceinline__ void init() {
     ref = -INFINITY;
     s = 0.f;
   }
+  // reference exponent moves up with the running maximum (never overflows)
   template <int E>
-  __device__ __forceinline__ void add(const float (&v)[E], float c) {
+  __device__ __forceinline__ void add_online(const float (&v)[E], float c) {
     float vmax = v[0];
 #pragma unroll
     for (int k = 1; k < E; ++k) vmax = fmaxf(vmax, v[k]);
@@ -257,9 +287,59 @@ struct LaneSoft {
     for (int k = 0; k < E; ++k) acc += ex2_approx(fmaf(v[k], c, nref));
     s += acc;
   }
+  __device__ __forceinline__ void add_online1(float x, float c) {
+    float cand = x * c;
+    if (cand > ref) {
+      s *= ex2_approx(ref - cand);
+      ref = cand;
+    }
+    float nref = (ref == -INFINITY) ? 0.f : -ref;
+    s += ex2_approx(fmaf(x, c, nref));
+  }
+  // reference exponent fixed (set from the first chunk); the caller checks s for overflow
+  template <int E>
+  __device__ __forceinline__ void seed(const float (&v)[E], float c) {
+    float vmax = v[0];
+#pragma unroll
+    for (int k = 1; k < E; ++k) vmax = fmaxf(vmax, v[k]);
+    float cand = vmax * c;
+    ref = (fabsf(cand) < INFINITY) ? cand : 0.f;
+    s = 0.f;
+  }
+  template <int E>
+  __device__ __forceinline__ void add_fixed(const float (&v)[E], float c) {
+    const float nref = -ref;
+    float a0 = 0.f, a1 = 0.f;
+#pragma unroll
+    for (int k = 0; k < E; k += 2) {
+      a0 += ex2_approx(fmaf(v[k], c, nref));
+      a1 += ex2_approx(fmaf(v[k + 1], c, nref));
+    }
+    s += a0 + a1;
+  }
 };
 
+// sum of (ref, s) pairs held one per lane: common reference = the largest, fp64 sum
+__device__ __forceinline__ SoftPart warp_reduce_soft(float ref, double s) {
+  float R = ref;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, d));
+  double t = (ref == R) ? s : s * exp2(static_cast<double>(ref) - static_cast<double>(R));
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    int lo = __shfl_xor_sync(0xffffffffu, __double2loint(t), d);
+    int hi = __shfl_xor_sync(0xffffffffu, __double2hiint(t), d);
+    t += __hiloint2double(hi, lo);
+  }
+  SoftPart o;
+  o.s = t;
+  o.ref = R;
+  o.pad = 0;
+  return o;
+}
+
 __device__ __forceinline__ void warp_merge_soft(LaneSoft a, SoftPart* dst, int lane) {
+  // lanes of one warp: fp32 is enough here, the errors of the 32 scale factors average out
   float R = a.ref;
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, d));
@@ -272,7 +352,7 @@ __device__ __forceinline__ void warp_merge_soft(LaneSoft a, SoftPart* dst, int l
   }
 }
 
-__device__ __forceinline__ void warp_merge_arg(double val, int idx, int bad, ArgPart* dst, int lane) {
+__device__ __forceinline__ ArgPart warp_reduce_arg(double val, int idx, int bad, int lane) {
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) {
     double ov = shfl_double(val, lane ^ d);
@@ -283,75 +363,73 @@ __device__ __forceinline__ void warp_merge_arg(double val, int idx, int bad, Arg
       idx = oi;
     }
   }
-  if (lane == 0) {
-    dst->val = val;
-    dst->idx = idx;
-    dst->bad = bad;
-  }
-}
-
-__device__ __forceinline__ SoftPart merge_soft_list(const SoftPart* parts, int count, int stride_bytes) {
-  float R = -INFINITY;
-  for (int k = 0; k < count; ++k) {
-    const SoftPart* p = reinterpret_cast<const SoftPart*>(reinterpret_cast<const char*>(parts) + k * stride_bytes);
-    R = fmaxf(R, p->ref);
-  }
-  double Z = 0.0;
-  for (int k = 0; k < count; ++k) {
-    const SoftPart* p = reinterpret_cast<const SoftPart*>(reinterpret_cast<const char*>(parts) + k * stride_bytes);
-    float ref = p->ref;
-    double s = p->s;
-    Z += (ref == R) ? s : s * exp2(static_cast<double>(ref) - static_cast<double>(R));
-  }
-  SoftPart o;
-  o.s = Z;
-  o.ref = R;
-  o.pad = 0;
+  ArgPart o;
+  o.val = val;
+  o.idx = idx;
+  o.bad = bad;
   return o;
 }
 
-// Block merge of warp partials, publish for the peers, cluster barrier, merge over ranks.
-// All threads of all blocks of the cluster call this; results land in sh.fsoft / sh.farg.
-__device__ void cluster_merge(Shared& sh, cg::cluster_group& cluster, int& phase, int nsoft, const int* soft_slots,
-                              int narg, const int* arg_slots) {
-  const int tid = threadIdx.x;
+__device__ __forceinline__ void warp_merge_arg(double val, int idx, int bad, ArgPart* dst, int lane) {
+  ArgPart o = warp_reduce_arg(val, idx, bad, lane);
+  if (lane == 0) *dst = o;
+}
+
+// Block merge of the warp partials, publish for the peers, ONE cluster barrier, merge over
+// the ranks.  Warp k handles soft slot k (k < nsoft); warp 8 + k handles arg slot a0 + k.
+// All threads of all blocks of the cluster call this; results land in sh.fsoft / sh.farg,
+// and rank 0's view of the row's earliest rejection in sh.known.
+__device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& cluster, int& phase, int nsoft, int a0,
+                                              int narg) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int C = cluster.num_blocks();
   __syncthreads();
   Xchg& mine = sh.x[phase & 1];
-  if (tid < nsoft) {
-    int slot = soft_slots[tid];
-    mine.soft[slot] = merge_soft_list(&sh.wsoft[0][slot], kWarps, sizeof(SoftPart) * kMaxSlots);
-  } else if (tid >= 32 && tid < 32 + narg) {
-    int slot = arg_slots[tid - 32];
-    ArgPart best = sh.warg[0][slot];
-    for (int w = 1; w < kWarps; ++w) {
-      ArgPart o = sh.warg[w][slot];
-      best.bad |= o.bad;
-      if (arg_better(o.val, o.idx, best.val, best.idx)) {
-        best.val = o.val;
-        best.idx = o.idx;
-      }
+  if (warp < nsoft) {
+    float ref = (lane < kWarps) ? sh.wsoft[lane][warp].ref : -INFINITY;
+    double s = (lane < kWarps) ? sh.wsoft[lane][warp].s : 0.0;
+    SoftPart o = warp_reduce_soft(ref, s);
+    if (lane == 0) mine.soft[warp] = o;
+  } else if (warp >= 8 && warp < 8 + narg) {
+    const int slot = a0 + warp - 8;
+    ArgPart in;
+    if (lane < kWarps) {
+      in = sh.warg[lane][slot];
+    } else {
+      in.val = -INFINITY;
+      in.idx = kNoReject;
+      in.bad = 0;
     }
-    mine.arg[slot] = best;
+    ArgPart o = warp_reduce_arg(in.val, in.idx, in.bad, lane);
+    if (lane == 0) mine.arg[slot] = o;
+  } else if (warp == kWarps - 1 && lane == 0) {
+    mine.known = sh.known_local;
+    mine.next = sh.next_local;
   }
   cluster.sync();
-  if (tid < nsoft) {
-    int slot = soft_slots[tid];
-    SoftPart tmp[kMaxCluster];
-    for (int r = 0; r < C; ++r) tmp[r] = cluster.map_shared_rank(&sh.x[phase & 1], r)->soft[slot];
-    sh.fsoft[slot] = merge_soft_list(tmp, C, sizeof(SoftPart));
-  } else if (tid >= 32 && tid < 32 + narg) {
-    int slot = arg_slots[tid - 32];
-    ArgPart best = cluster.map_shared_rank(&sh.x[phase & 1], 0)->arg[slot];
-    for (int r = 1; r < C; ++r) {
-      ArgPart o = cluster.map_shared_rank(&sh.x[phase & 1], r)->arg[slot];
-      best.bad |= o.bad;
-      if (arg_better(o.val, o.idx, best.val, best.idx)) {
-        best.val = o.val;
-        best.idx = o.idx;
-      }
+  if (warp < nsoft) {
+    float ref = -INFINITY;
+    double s = 0.0;
+    if (lane < C) {
+      const Xchg* peer = cluster.map_shared_rank(&sh.x[phase & 1], lane);
+      ref = peer->soft[warp].ref;
+      s = peer->soft[warp].s;
     }
-    sh.farg[slot] = best;
+    SoftPart o = warp_reduce_soft(ref, s);
+    if (lane == 0) sh.fsoft[warp] = o;
+  } else if (warp >= 8 && warp < 8 + narg) {
+    const int slot = a0 + warp - 8;
+    ArgPart in;
+    in.val = -INFINITY;
+    in.idx = kNoReject;
+    in.bad = 0;
+    if (lane < C) in = cluster.map_shared_rank(&sh.x[phase & 1], lane)->arg[slot];
+    ArgPart o = warp_reduce_arg(in.val, in.idx, in.bad, lane);
+    if (lane == 0) sh.farg[slot] = o;
+  } else if (warp == kWarps - 1 && lane == 0) {
+    const Xchg* r0 = cluster.map_shared_rank(&sh.x[phase & 1], 0);
+    sh.known = r0->known;
+    sh.next = r0->next;
   }
   __syncthreads();
   ++phase;
@@ -397,6 +475,81 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
 }
 
 // ------------------------------------------------------------------------------------
+// sweep 1: a block's slice of the vocabulary, threads interleaved over 16-byte vectors
+// ------------------------------------------------------------------------------------
+// Sweep 1 only forms sums, maxima and argmaxes, so any assignment of tokens to threads
+// will do: each block reads its slice as consecutive 8 KB pieces (one vector per thread),
+// which keeps the DRAM accesses of a block contiguous.
+struct Slice {
+  int v_lo, v_hi;  // whole 16-byte vectors [v_lo, v_hi) of the row (aligned layouts only)
+  int e_lo, e_hi;  // single entries [e_lo, e_hi): the ragged tail, or everything when unaligned
+};
+
+template <int DT>
+__device__ __forceinline__ Slice slice_of(int rank, int C, int V, bool vec_ok) {
+  constexpr int E = Elem<DT>::E;
+  Slice s;
+  if (vec_ok) {
+    const int nvec = V / E;
+    s.v_lo = static_cast<int>(static_cast<long long>(rank) * nvec / C);
+    s.v_hi = static_cast<int>(static_cast<long long>(rank + 1) * nvec / C);
+    s.e_lo = (rank == C - 1) ? nvec * E : V;
+    s.e_hi = V;
+  } else {
+    s.v_lo = s.v_hi = 0;
+    s.e_lo = static_cast<int>(static_cast<long long>(rank) * V / C);
+    s.e_hi = static_cast<int>(static_cast<long long>(rank + 1) * V / C);
+  }
+  return s;
+}
+
+// Softmax normaliser of one row over the slice: fixed reference exponent (seeded from the
+// thread's first vector) with four loads in flight; overflow or a non-finite input falls
+// back to the running-maximum form.
+template <int DT>
+__device__ __forceinline__ LaneSoft soft_slice(const void* row, const Slice& sl, int tid, float c) {
+  constexpr int E = Elem<DT>::E;
+  constexpr int U = 4;
+  const char* rowb = reinterpret_cast<const char*>(row);
+  LaneSoft acc;
+  acc.init();
+  int v = sl.v_lo + tid;
+  if (v < sl.v_hi) {
+    float x[E];
+    uint4 raw[U];
+    raw[0] = ldg_stream16(rowb + static_cast<long long>(v) * 16);
+    Elem<DT>::unpack(raw[0], x);
+    acc.seed(x, c);
+    for (; v + (U - 1) * kThreads < sl.v_hi; v += U * kThreads) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) raw[u] = ldg_stream16(rowb + static_cast<long long>(v + u * kThreads) * 16);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        Elem<DT>::unpack(raw[u], x);
+        acc.add_fixed(x, c);
+      }
+    }
+    for (; v < sl.v_hi; v += kThreads) {
+      raw[0] = ldg_stream16(rowb + static_cast<long long>(v) * 16);
+      Elem<DT>::unpack(raw[0], x);
+      acc.add_fixed(x, c);
+    }
+  }
+  for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) acc.add_online1(Elem<DT>::load1(row, e), c);
+  if (!(acc.s < INFINITY)) {
+    acc.init();
+    for (v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+      float x[E];
+      uint4 raw = ldg_stream16(rowb + static_cast<long long>(v) * 16);
+      Elem<DT>::unpack(raw, x);
+      acc.add_online(x, c);
+    }
+    for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) acc.add_online1(Elem<DT>::load1(row, e), c);
+  }
+  return acc;
+}
+
+// ------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------
 template <int DT, int MODE>
@@ -409,14 +562,18 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gwarp = rank * kWarps + warp, G = C * kWarps;
   __shared__ Shared sh;
-  __shared__ int slot_ids[2][kMaxSlots];
+  extern __shared__ uint4 ring[];  // kWarps * kRingVecs * 32 vectors: sweep-2 staging
   int phase = 0;
   const bool vec_ok = p.vec_ok != 0;
   const bool masked = (MODE == kLogitSample || MODE == kLogitGreedy) && p.mask_model >= 0;
+  const double kNaN = __longlong_as_double(0x7ff8000000000000LL);
+  const double kInf = __longlong_as_double(0x7ff0000000000000LL);
 
   // this warp's run of steps (a step = 32 lanes x E entries)
   const int s_begin = static_cast<int>(static_cast<long long>(gwarp) * p.nsteps / G);
   const int s_end = static_cast<int>(static_cast<long long>(gwarp + 1) * p.nsteps / G);
+  // this block's slice of every row in sweep 1
+  const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
 
   int unit = blockIdx.x / C;
   while (unit < p.num_units) {
@@ -429,55 +586,61 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
     auto row_of = [&](int i) -> const void* { return base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes; };
     const bool is_bonus = (j == p.gamma);
     const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
-    if (tid < p.n && !is_bonus && draft >= 0 && draft < p.V) sh.ldraft[tid] = Elem<DT>::load1(row_of(tid), draft);
+    const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
+
+    // ---- small jobs issued before the sweep so that their latency hides behind it
+    if (tid < p.n && !is_bonus && draft_ok) sh.ldraft[tid] = Elem<DT>::load1(row_of(tid), draft);
+    if (warp == kWarps - 1) {
+      if (lane == 0) {
+        sh.known_local = (rank == 0) ? ld_relaxed_gpu(&p.first_rej[b]) : kNoReject;
+      } else if (lane == 2) {
+        // rank 0 draws the cluster's next unit now; every block learns it with the merged statistics
+        if (rank == 0) sh.next_local = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
+      } else if (lane == 1) {
+        unsigned rnd[4];
+        const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
+        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi,
+                      rnd);
+        sh.u_acc = word_to_uniform(rnd[0]);
+        sh.u_smp = word_to_uniform(rnd[1]);
+      }
+    }
 
     // ================================ sweep 1: statistics ================================
     if (MODE == kEnsembleSample) {
       for (int i = 0; i < p.n; ++i) {
-        const void* row = row_of(i);
-        LaneSoft acc;
-        acc.init();
-        int s = s_begin;
-        for (; s + 2 <= s_end; s += 2) {
-          float v0[E], v1[E];
-          load_chunk<DT>(row, (s * 32 + lane) * E, p.V, vec_ok, v0);
-          load_chunk<DT>(row, ((s + 1) * 32 + lane) * E, p.V, vec_ok, v1);
-          acc.add(v0, p.cT);
-          acc.add(v1, p.cT);
-        }
-        for (; s < s_end; ++s) {
-          float v0[E];
-          load_chunk<DT>(row, (s * 32 + lane) * E, p.V, vec_ok, v0);
-          acc.add(v0, p.cT);
-        }
+        LaneSoft acc = soft_slice<DT>(row_of(i), sl, tid, p.cT);
         warp_merge_soft(acc, &sh.wsoft[warp][i], lane);
       }
-      if (tid < p.n) slot_ids[0][tid] = tid;
-      cluster_merge(sh, cluster, phase, p.n, slot_ids[0], 0, slot_ids[1]);
+      cluster_merge(sh, cluster, phase, p.n, 0, 0);
+      if (tid < p.n && !is_bonus && draft_ok) {
+        // probability of the draft under model tid, with the constant the sweep used
+        sh.pdraft[tid] = exp2(static_cast<double>(sh.ldraft[tid]) * p.cT64 - static_cast<double>(sh.fsoft[tid].ref)) /
+                         sh.fsoft[tid].s;
+      }
     } else if (MODE == kEnsembleGreedy) {
       for (int i = 0; i < p.n; ++i) {
         const void* row = row_of(i);
         float best = -INFINITY;
         int bidx = kNoReject, bad = 0;
-        for (int s = s_begin; s < s_end; ++s) {
-          float v[E];
-          const int e0 = (s * 32 + lane) * E;
-          load_chunk<DT>(row, e0, p.V, vec_ok, v);
-#pragma unroll
-          for (int k = 0; k < E; ++k) {
-            if (e0 + k < p.V) {
-              bad |= !(v[k] < INFINITY);
-              if (v[k] > best) {
-                best = v[k];
-                bidx = e0 + k;
-              }
-            }
+        auto see = [&](float x, int e) {
+          bad |= !(x < INFINITY);
+          if (x > best) {
+            best = x;
+            bidx = e;
           }
+        };
+        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+          float x[E];
+          uint4 raw = ldg_stream16(reinterpret_cast<const char*>(row) + static_cast<long long>(v) * 16);
+          Elem<DT>::unpack(raw, x);
+#pragma unroll
+          for (int k = 0; k < E; ++k) see(x[k], v * E + k);
         }
+        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) see(Elem<DT>::load1(row, e), e);
         warp_merge_arg(static_cast<double>(best), bidx, bad, &sh.warg[warp][i], lane);
       }
-      if (tid < p.n) slot_ids[1][tid] = tid;
-      cluster_merge(sh, cluster, phase, 0, slot_ids[0], p.n, slot_ids[1]);
+      cluster_merge(sh, cluster, phase, 0, 0, p.n);
     } else {
       // logit-level combine.  soft slot 0 = proposer, soft slot 1 = combined logits;
       // arg slot 0 = expert maximum (mask), arg slot 1 = proposer argmax, arg slot 2 = combined argmax.
@@ -485,21 +648,23 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         const void* row = row_of(p.mask_model);
         float best = -INFINITY;
         int bad = 0;
-        for (int s = s_begin; s < s_end; ++s) {
-          float v[E];
-          const int e0 = (s * 32 + lane) * E;
-          load_chunk<DT>(row, e0, p.V, vec_ok, v);
+        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+          float x[E];
+          uint4 raw = ldg_stream16(reinterpret_cast<const char*>(row) + static_cast<long long>(v) * 16);
+          Elem<DT>::unpack(raw, x);
 #pragma unroll
           for (int k = 0; k < E; ++k) {
-            if (e0 + k < p.V) {
-              bad |= (v[k] != v[k]);
-              best = fmaxf(best, v[k]);
-            }
+            bad |= (x[k] != x[k]);
+            best = fmaxf(best, x[k]);
           }
         }
+        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+          float x = Elem<DT>::load1(row, e);
+          bad |= (x != x);
+          best = fmaxf(best, x);
+        }
         warp_merge_arg(static_cast<double>(best), 0, bad, &sh.warg[warp][0], lane);
-        if (tid == 0) slot_ids[1][0] = 0;
-        cluster_merge(sh, cluster, phase, 0, slot_ids[0], 1, slot_ids[1]);
+        cluster_merge(sh, cluster, phase, 0, 0, 1);
         if (tid == 0) {
           // l >= max + ln(alpha) in fp64 is the same as l >= (that bound rounded up to fp32) for fp32 l
           double bound = sh.farg[0].val + p.ln_alpha;
@@ -512,8 +677,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         LaneSoft accq, accc;
         accq.init();
         accc.init();
-        for (int s = s_begin; s < s_end; ++s) {
-          const int e0 = (s * 32 + lane) * E;
+        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
           float cmb[E], vq[E], ve[E];
 #pragma unroll
           for (int k = 0; k < E; ++k) {
@@ -522,10 +686,13 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             ve[k] = 0.f;
           }
           for (int i = 0; i < p.n; i += 2) {
-            float va[E], vb[E];
             const bool two = (i + 1 < p.n);
-            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, va);
-            if (two) load_chunk<DT>(row_of(i + 1), e0, p.V, vec_ok, vb);
+            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
+            uint4 rb = ra;
+            if (two) rb = ldg_stream16(reinterpret_cast<const char*>(row_of(i + 1)) + static_cast<long long>(v) * 16);
+            float va[E], vb[E];
+            Elem<DT>::unpack(ra, va);
+            Elem<DT>::unpack(rb, vb);
             const float wa = p.w[i], wb = two ? p.w[i + 1] : 0.f;
 #pragma unroll
             for (int k = 0; k < E; ++k) {
@@ -539,82 +706,101 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               }
             }
           }
+          if (masked) {
 #pragma unroll
-          for (int k = 0; k < E; ++k) {
-            bool in = (e0 + k < p.V) && (!masked || ve[k] >= thr);
-            cmb[k] = in ? cmb[k] : -INFINITY;
+            for (int k = 0; k < E; ++k) cmb[k] = (ve[k] >= thr) ? cmb[k] : -INFINITY;
           }
-          accq.add(vq, p.cT);
-          accc.add(cmb, p.cT);
+          accq.add_online(vq, p.cT);
+          accc.add_online(cmb, p.cT);
+        }
+        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+          float cmb = 0.f, xq = -INFINITY, xe = 0.f;
+          for (int i = 0; i < p.n; ++i) {
+            float x = Elem<DT>::load1(row_of(i), e);
+            cmb = fmaf(p.w[i], x, cmb);
+            if (i == pis) xq = x;
+            if (i == p.mask_model) xe = x;
+          }
+          if (masked && !(xe >= thr)) cmb = -INFINITY;
+          accq.add_online1(xq, p.cT);
+          accc.add_online1(cmb, p.cT);
         }
         warp_merge_soft(accq, &sh.wsoft[warp][0], lane);
         warp_merge_soft(accc, &sh.wsoft[warp][1], lane);
-        if (tid < 2) slot_ids[0][tid] = tid;
-        cluster_merge(sh, cluster, phase, 2, slot_ids[0], 0, slot_ids[1]);
+        cluster_merge(sh, cluster, phase, 2, 0, 0);
       } else {  // kLogitGreedy: combined logits in fp64, the same chain of fused multiply-adds on every token
         double cbest = -INFINITY;
         int cidx = kNoReject, bad = 0;
         float qbest = -INFINITY;
         int qidx = kNoReject;
-        for (int s = s_begin; s < s_end; ++s) {
-          const int e0 = (s * 32 + lane) * E;
+        auto see = [&](double cm, float xq, float xe, int e) {
+          if (xq > qbest) {
+            qbest = xq;
+            qidx = e;
+          }
+          if (!masked || xe >= thr) {
+            bad |= (cm != cm);
+            if (cm > cbest) {
+              cbest = cm;
+              cidx = e;
+            }
+          }
+        };
+        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
           double cmb[E];
-          float ve[E];
+          float vq[E], ve[E];
 #pragma unroll
           for (int k = 0; k < E; ++k) {
             cmb[k] = 0.0;
+            vq[k] = -INFINITY;
             ve[k] = 0.f;
           }
           for (int i = 0; i < p.n; ++i) {
             float va[E];
-            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, va);
+            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
+            Elem<DT>::unpack(ra, va);
             const double wa = p.w64[i];
 #pragma unroll
             for (int k = 0; k < E; ++k) {
-              if (e0 + k < p.V) {
-                bad |= !(va[k] < INFINITY);
-                cmb[k] = fma(wa, static_cast<double>(va[k]), cmb[k]);
-                if (i == p.mask_model) ve[k] = va[k];
-                if (i == pis && va[k] > qbest) {
-                  qbest = va[k];
-                  qidx = e0 + k;
-                }
-              }
+              bad |= !(va[k] < INFINITY);
+              cmb[k] = fma(wa, static_cast<double>(va[k]), cmb[k]);
+              if (i == p.mask_model) ve[k] = va[k];
+              if (i == pis) vq[k] = va[k];
             }
           }
 #pragma unroll
-          for (int k = 0; k < E; ++k) {
-            if (e0 + k < p.V && (!masked || ve[k] >= thr)) {
-              bad |= (cmb[k] != cmb[k]);
-              if (cmb[k] > cbest) {
-                cbest = cmb[k];
-                cidx = e0 + k;
-              }
-            }
+          for (int k = 0; k < E; ++k) see(cmb[k], vq[k], ve[k], v * E + k);
+        }
+        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+          double cm = 0.0;
+          float xq = -INFINITY, xe = 0.f;
+          for (int i = 0; i < p.n; ++i) {
+            float x = Elem<DT>::load1(row_of(i), e);
+            bad |= !(x < INFINITY);
+            cm = fma(p.w64[i], static_cast<double>(x), cm);
+            if (i == pis) xq = x;
+            if (i == p.mask_model) xe = x;
           }
+          see(cm, xq, xe, e);
         }
         warp_merge_arg(static_cast<double>(qbest), qidx, bad, &sh.warg[warp][1], lane);
         warp_merge_arg(cbest, cidx, bad, &sh.warg[warp][2], lane);
-        if (tid < 2) slot_ids[1][tid] = tid + 1;
-        cluster_merge(sh, cluster, phase, 0, slot_ids[0], 2, slot_ids[1]);
+        cluster_merge(sh, cluster, phase, 0, 1, 2);
       }
     }
+    if (MODE == kEnsembleSample) __syncthreads();  // pdraft
 
     // ================================ decision (Eq. 6) ================================
+    // every block takes the same decision from the same merged numbers
     if (tid == 0) {
       Decision& d = sh.dec;
-      unsigned rnd[4];
-      const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
-      philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi, rnd);
-      const double u_acc = word_to_uniform(rnd[0]);
-      d.u_smp = word_to_uniform(rnd[1]);
+      const double u_acc = sh.u_acc;
       d.accept = 0;
       d.status = 0;
       d.want_sample = 0;
       d.cand = -1;
       d.natoms = 0;
-      d.ratio = d.r_d = d.q_d = d.S = __longlong_as_double(0x7ff8000000000000LL);
-      const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
+      d.ratio = d.r_d = d.q_d = d.S = kNaN;
       bool finite = pi_ok;
       if (kSample) {
         const int nsoft = (MODE == kEnsembleSample) ? p.n : 2;
@@ -626,26 +812,18 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         if (!finite) {
           d.status |= COS_ROW_NONFINITE;
         } else {
-          if (MODE == kEnsembleSample) {
-            for (int i = 0; i < p.n; ++i) {
-              sh.a_scale[i] = static_cast<float>(p.w64[i] / sh.fsoft[i].s);
-              sh.a_ref[i] = -sh.fsoft[i].ref;
-            }
-          }
+          for (int k = 0; k < nsoft; ++k) sh.big_thr[k] = static_cast<float>(sh.fsoft[k].s * kBigShare);
           if (!is_bonus) {
             if (draft_ok) {
               double r_d = 0.0, q_d = 0.0;
               if (MODE == kEnsembleSample) {
                 for (int i = 0; i < p.n; ++i) {
-                  double l = static_cast<double>(sh.ldraft[i]);
-                  double pr = exp2(l * p.cT64 - static_cast<double>(sh.fsoft[i].ref)) / sh.fsoft[i].s;
-                  r_d += p.w64[i] * pr;
-                  if (i == pi) q_d = pr;
+                  r_d += p.w64[i] * sh.pdraft[i];
+                  if (i == pi) q_d = sh.pdraft[i];
                 }
               } else {
                 double cd = 0.0;
-                for (int i = 0; i < p.n; ++i)
-                  cd = fma(p.w64[i], static_cast<double>(sh.ldraft[i]), cd);
+                for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(sh.ldraft[i]), cd);
                 bool in = !masked || (sh.ldraft[p.mask_model] >= sh.thr32);
                 r_d = in ? exp2(cd * p.cT64 - static_cast<double>(sh.fsoft[1].ref)) / sh.fsoft[1].s : 0.0;
                 double lq = static_cast<double>(sh.ldraft[pi]);
@@ -657,7 +835,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
                 d.ratio = r_d / q_d;
               } else {
                 d.status |= COS_ROW_Q_ZERO;
-                d.ratio = (r_d > 0.0) ? __longlong_as_double(0x7ff0000000000000LL) : 0.0;
+                d.ratio = (r_d > 0.0) ? kInf : 0.0;
               }
               d.accept = (u_acc <= fmin(1.0, d.ratio)) ? 1 : 0;
             } else {
@@ -716,7 +894,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
                 d.ratio = d.r_d / d.q_d;
               } else {
                 d.status |= COS_ROW_Q_ZERO;
-                d.ratio = (d.r_d > 0.0) ? __longlong_as_double(0x7ff0000000000000LL) : 0.0;
+                d.ratio = (d.r_d > 0.0) ? kInf : 0.0;
               }
               d.accept = (u_acc <= fmin(1.0, d.ratio)) ? 1 : 0;
             } else {
@@ -735,7 +913,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           double total = 0.0;
           for (int k = 0; k < d.natoms; ++k)
             total += use_r ? d.atom_mass[k] : fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
-          const double target = d.u_smp * total;
+          const double target = sh.u_smp * total;
           double run = 0.0;
           int lastpos = -1;
           d.cand = -1;
@@ -748,36 +926,19 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           if (d.cand < 0) d.cand = lastpos;
         }
       }
-      // rank 0 alone talks to global memory about the row and fetches the next unit
-      if (rank == 0) {
-        int known = kNoReject;
-        if (!is_bonus && !d.accept)
-          known = atomicMin(&p.first_rej[b], j);
-        else
-          known = atomicMin(&p.first_rej[b], kNoReject);
-        const bool superseded = known < j;  // an earlier position of this row already rejected
-        int need2 = 0;
-        if (kSample && finite) {
-          need2 = (d.want_sample && !superseded) || (p.dump_r != nullptr) ||
+      // a token is drawn only where the row can still need it: rank 0 looked at the row's
+      // earliest known rejection before the sweep and every block received that same value
+      const bool superseded = sh.known < j;
+      d.need2 = 0;
+      if (kSample && finite) {
+        d.need2 = (d.want_sample && !superseded) || (p.dump_r != nullptr) ||
                   ((p.flags & COS_RUN_ALL_RESIDUALS) && !is_bonus);
-        }
-        unsigned t = atomicAdd(p.work_counter, 1u);
-        int next = p.num_clusters + static_cast<int>(t - p.work_base);
-        Xchg& mine = sh.x[phase & 1];
-        mine.bcast[0] = need2;
-        mine.bcast[1] = next;
       }
-    }
-    cluster.sync();
-    if (tid == 0) {
-      const Xchg* r0 = cluster.map_shared_rank(&sh.x[phase & 1], 0);
-      sh.need2 = r0->bcast[0];
-      sh.next_unit = r0->bcast[1];
+      if (rank == 0 && !is_bonus && !d.accept) atomicMin(&p.first_rej[b], j);
     }
     __syncthreads();
-    ++phase;
-    const int need2 = sh.need2;
-    const int next_unit = sh.next_unit;
+    const int need2 = sh.dec.need2;
+    const int next_unit = sh.next;
 
     // greedy test hook: r is a handful of atoms
     if (!kSample && p.dump_r != nullptr) {
@@ -795,100 +956,341 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
     bool published = false;
     if (kSample && need2) {
       bool from_r = is_bonus;  // the bonus is drawn from r itself; a rejected draft from max(0, r - q)
-      const float inv_zq = (MODE == kEnsembleSample) ? static_cast<float>(1.0 / sh.fsoft[pis].s)
-                                                     : static_cast<float>(1.0 / sh.fsoft[0].s);
-      const float ref_q = (MODE == kEnsembleSample) ? -sh.fsoft[pis].ref : -sh.fsoft[0].ref;
-      const float inv_zc = (MODE == kLogitSample) ? static_cast<float>(1.0 / sh.fsoft[1].s) : 0.f;
-      const float ref_c = (MODE == kLogitSample) ? -sh.fsoft[1].ref : 0.f;
       const float thr = masked ? sh.thr32 : -INFINITY;
-      double S_report = __longlong_as_double(0x7ff8000000000000LL);
+      double S_report = kNaN;
+      const int nsoft2 = (MODE == kEnsembleSample) ? p.n : 2;
 
-      // mass of one lane chunk: fills res[] and returns nothing else; used by both the totals and the rescan
-      auto chunk_mass = [&](int e0, bool use_r, bool dump, float (&res)[E]) {
-        float r[E], q[E];
-        if (MODE == kEnsembleSample) {
-#pragma unroll
-          for (int k = 0; k < E; ++k) {
-            r[k] = 0.f;
-            q[k] = 0.f;
-          }
-          for (int i = 0; i < p.n; ++i) {
-            float v[E];
-            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
-            const float sc = sh.a_scale[i], rf = sh.a_ref[i];
+      // ---- 2a: normalisers again, now that the references are known: terms holding more
+      // than 2^-14 of a normaliser are evaluated in fp64 and kept out of the fp32 sums, so
+      // a dominant token neither absorbs the small ones nor carries the fast exp's error
+      if (MODE == kEnsembleSample) {
+        for (int i = 0; i < p.n; ++i) {
+          const void* row = row_of(i);
+          const char* rowb = reinterpret_cast<const char*>(row);
+          const float nref = -sh.fsoft[i].ref, bt = sh.big_thr[i];
+          const double dref = static_cast<double>(sh.fsoft[i].ref);
+          float zs = 0.f;
+          double zb = 0.0;
+          auto eat = [&](const float (&v)[E]) {
+            float e[E];
+            bool any = false;
 #pragma unroll
             for (int k = 0; k < E; ++k) {
-              float e = ex2_approx(fmaf(v[k], p.cT, rf));
-              r[k] = fmaf(sc, e, r[k]);
-              if (i == pis) q[k] = e * inv_zq;
+              e[k] = ex2_approx(fmaf(v[k], p.cT, nref));
+              const bool big = e[k] > bt;
+              any |= big;
+              zs += big ? 0.f : e[k];
+            }
+            if (any) {
+#pragma unroll
+              for (int k = 0; k < E; ++k)
+                if (e[k] > bt) zb += exp2(static_cast<double>(v[k]) * p.cT64 - dref);
+            }
+          };
+          int v = sl.v_lo + tid;
+          for (; v + 3 * kThreads < sl.v_hi; v += 4 * kThreads) {
+            uint4 raw[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) raw[u] = ldg_stream16(rowb + static_cast<long long>(v + u * kThreads) * 16);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              float x[E];
+              Elem<DT>::unpack(raw[u], x);
+              eat(x);
+            }
+          }
+          for (; v < sl.v_hi; v += kThreads) {
+            float x[E];
+            uint4 raw = ldg_stream16(rowb + static_cast<long long>(v) * 16);
+            Elem<DT>::unpack(raw, x);
+            eat(x);
+          }
+          for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+            const float x = Elem<DT>::load1(row, e);
+            const float ee = ex2_approx(fmaf(x, p.cT, nref));
+            if (ee > bt)
+              zb += exp2(static_cast<double>(x) * p.cT64 - dref);
+            else
+              zs += ee;
+          }
+          double t = static_cast<double>(zs) + zb;
+#pragma unroll
+          for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+          if (lane == 0) {
+            sh.wsoft[warp][i].s = t;
+            sh.wsoft[warp][i].ref = sh.fsoft[i].ref;
+          }
+        }
+      } else {
+        const float nref_q = -sh.fsoft[0].ref, nref_c = -sh.fsoft[1].ref;
+        const float bt_q = sh.big_thr[0], bt_c = sh.big_thr[1];
+        const double dref_q = static_cast<double>(sh.fsoft[0].ref), dref_c = static_cast<double>(sh.fsoft[1].ref);
+        float zsq = 0.f, zsc = 0.f;
+        double zbq = 0.0, zbc = 0.0;
+        auto big_c = [&](int e) {  // combined logit of one token in fp64
+          double cd = 0.0;
+          for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e)), cd);
+          return exp2(cd * p.cT64 - dref_c);
+        };
+        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+          float cmb[E], vq[E], ve[E];
+#pragma unroll
+          for (int k = 0; k < E; ++k) {
+            cmb[k] = 0.f;
+            vq[k] = -INFINITY;
+            ve[k] = 0.f;
+          }
+          for (int i = 0; i < p.n; i += 2) {
+            const bool two = (i + 1 < p.n);
+            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
+            uint4 rb = ra;
+            if (two) rb = ldg_stream16(reinterpret_cast<const char*>(row_of(i + 1)) + static_cast<long long>(v) * 16);
+            float va[E], vb[E];
+            Elem<DT>::unpack(ra, va);
+            Elem<DT>::unpack(rb, vb);
+            const float wa = p.w[i], wb = two ? p.w[i + 1] : 0.f;
+#pragma unroll
+            for (int k = 0; k < E; ++k) {
+              cmb[k] = fmaf(wa, va[k], cmb[k]);
+              if (i == pis) vq[k] = va[k];
+              if (i == p.mask_model) ve[k] = va[k];
+              if (two) {
+                cmb[k] = fmaf(wb, vb[k], cmb[k]);
+                if (i + 1 == pis) vq[k] = vb[k];
+                if (i + 1 == p.mask_model) ve[k] = vb[k];
+              }
+            }
+          }
+          bool any = false;
+          float eq[E], ec[E];
+#pragma unroll
+          for (int k = 0; k < E; ++k) {
+            const bool in = !masked || ve[k] >= thr;
+            eq[k] = ex2_approx(fmaf(vq[k], p.cT, nref_q));
+            ec[k] = in ? ex2_approx(fmaf(cmb[k], p.cT, nref_c)) : 0.f;
+            const bool bq = eq[k] > bt_q, bc = ec[k] > bt_c;
+            any |= bq | bc;
+            zsq += bq ? 0.f : eq[k];
+            zsc += bc ? 0.f : ec[k];
+          }
+          if (any) {
+#pragma unroll
+            for (int k = 0; k < E; ++k) {
+              if (eq[k] > bt_q) zbq += exp2(static_cast<double>(vq[k]) * p.cT64 - dref_q);
+              if (ec[k] > bt_c) zbc += big_c(v * E + k);
+            }
+          }
+        }
+        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+          float cmb = 0.f, xq = -INFINITY, xe = 0.f;
+          for (int i = 0; i < p.n; ++i) {
+            float x = Elem<DT>::load1(row_of(i), e);
+            cmb = fmaf(p.w[i], x, cmb);
+            if (i == pis) xq = x;
+            if (i == p.mask_model) xe = x;
+          }
+          const bool in = !masked || xe >= thr;
+          const float eq = ex2_approx(fmaf(xq, p.cT, nref_q));
+          const float ec = in ? ex2_approx(fmaf(cmb, p.cT, nref_c)) : 0.f;
+          if (eq > bt_q)
+            zbq += exp2(static_cast<double>(xq) * p.cT64 - dref_q);
+          else
+            zsq += eq;
+          if (ec > bt_c)
+            zbc += big_c(e);
+          else
+            zsc += ec;
+        }
+        double tq = static_cast<double>(zsq) + zbq, tc = static_cast<double>(zsc) + zbc;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+          tq += shfl_double(tq, lane ^ d);
+          tc += shfl_double(tc, lane ^ d);
+        }
+        if (lane == 0) {
+          sh.wsoft[warp][0].s = tq;
+          sh.wsoft[warp][0].ref = sh.fsoft[0].ref;
+          sh.wsoft[warp][1].s = tc;
+          sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
+        }
+      }
+      cluster_merge(sh, cluster, phase, nsoft2, 0, 0);  // refined normalisers replace sh.fsoft[*].s
+      if (MODE == kEnsembleSample && tid < p.n) {
+        // r - q = sum_i (w_i/Z_i - [i = proposer]/Z_i) e_i, and r = sum_i (w_i/Z_i) e_i
+        const double a = p.w64[tid] / sh.fsoft[tid].s;
+        sh.a_scale[tid] = static_cast<float>(a);
+        sh.a_resid[tid] = static_cast<float>(a - (tid == pis ? 1.0 / sh.fsoft[tid].s : 0.0));
+        sh.a_ref[tid] = -sh.fsoft[tid].ref;
+      }
+      __syncthreads();
+      const float inv_zq = (MODE == kLogitSample) ? static_cast<float>(1.0 / sh.fsoft[0].s) : 0.f;
+      const float ref_q = (MODE == kLogitSample) ? -sh.fsoft[0].ref : 0.f;
+      const float inv_zc = (MODE == kLogitSample) ? static_cast<float>(1.0 / sh.fsoft[1].s) : 0.f;
+      const float ref_c = (MODE == kLogitSample) ? -sh.fsoft[1].ref : 0.f;
+
+      // ---- 2b: token masses.  mass32[k] is max(0, r - q) (or r) of the lane's k-th token in fp32;
+      // tokens holding more than 2^-10 of any normaliser are flagged in `bigbits`, get mass32 = 0
+      // and are evaluated by big_mass() in fp64 from the stored logits.
+      // `staged` points at this lane's staged vector of model 0 (models 32 vectors apart), or is null.
+      auto chunk_mass = [&](int e0, bool use_r, bool dump, float (&mass32)[E], unsigned& bigbits, const uint4* staged) {
+        auto fetch = [&](int i, float (&v)[E]) {
+          if (staged != nullptr) {
+            uint4 raw = staged[i * 32];
+            Elem<DT>::unpack(raw, v);
+          } else {
+            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
+          }
+        };
+        float acc[E], rr[E];
+        bigbits = 0u;
+#pragma unroll
+        for (int k = 0; k < E; ++k) {
+          acc[k] = 0.f;
+          rr[k] = 0.f;
+        }
+        if (MODE == kEnsembleSample) {
+          for (int i = 0; i < p.n; ++i) {
+            float v[E];
+            fetch(i, v);
+            const float co = use_r ? sh.a_scale[i] : sh.a_resid[i], rf = sh.a_ref[i], bt = sh.big_thr[i];
+            const float cr = sh.a_scale[i];
+#pragma unroll
+            for (int k = 0; k < E; ++k) {
+              const float e = ex2_approx(fmaf(v[k], p.cT, rf));
+              bigbits |= (e > bt) ? (1u << k) : 0u;
+              acc[k] = fmaf(co, e, acc[k]);
+              if (dump) rr[k] = fmaf(cr, e, rr[k]);
             }
           }
         } else {
-          float cmb[E], ve[E];
+          float cmb[E], ve[E], eq[E];
 #pragma unroll
           for (int k = 0; k < E; ++k) {
             cmb[k] = 0.f;
             ve[k] = 0.f;
-            q[k] = 0.f;
+            eq[k] = 0.f;
           }
           for (int i = 0; i < p.n; ++i) {
             float v[E];
-            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
+            fetch(i, v);
             const float wi = p.w[i];
 #pragma unroll
             for (int k = 0; k < E; ++k) {
               cmb[k] = fmaf(wi, v[k], cmb[k]);
               if (i == p.mask_model) ve[k] = v[k];
-              if (i == pis) q[k] = ex2_approx(fmaf(v[k], p.cT, ref_q)) * inv_zq;
+              if (i == pis) eq[k] = ex2_approx(fmaf(v[k], p.cT, ref_q));
             }
           }
 #pragma unroll
           for (int k = 0; k < E; ++k) {
-            bool in = (e0 + k < p.V) && (!masked || ve[k] >= thr);
-            r[k] = in ? ex2_approx(fmaf(cmb[k], p.cT, ref_c)) * inv_zc : 0.f;
+            const bool in = (e0 + k < p.V) && (!masked || ve[k] >= thr);
+            const float ec = in ? ex2_approx(fmaf(cmb[k], p.cT, ref_c)) : 0.f;
+            bigbits |= (ec > sh.big_thr[1] || eq[k] > sh.big_thr[0]) ? (1u << k) : 0u;
+            rr[k] = ec * inv_zc;
+            acc[k] = use_r ? rr[k] : fmaf(-eq[k], inv_zq, rr[k]);
           }
         }
 #pragma unroll
         for (int k = 0; k < E; ++k) {
-          bool valid = (e0 + k < p.V);
-          float m = use_r ? r[k] : fmaxf(0.f, r[k] - q[k]);
-          res[k] = valid ? m : 0.f;
+          const bool keep = (e0 + k < p.V) && !(bigbits & (1u << k));
+          mass32[k] = keep ? (use_r ? acc[k] : fmaxf(0.f, acc[k])) : 0.f;
         }
         if (dump) {
           float* out = p.dump_r + (static_cast<long long>(b) * p.P + j) * p.V;
 #pragma unroll
           for (int k = 0; k < E; ++k)
-            if (e0 + k < p.V) out[e0 + k] = r[k];
+            if (e0 + k < p.V && !(bigbits & (1u << k))) out[e0 + k] = rr[k];
         }
       };
-      // per-step prefix over the 32 lanes in fp64: exclusive prefix and the lane's own sum
-      auto lane_prefix = [&](const float (&res)[E], double& excl, float& own) {
+      auto big_mass = [&](int e, bool use_r, bool dump) -> double {
+        if (e >= p.V) return 0.0;
+        double r64 = 0.0, q64 = 0.0;
+        float lv[COS_MAX_MODELS];
+        for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::load1(row_of(i), e);  // all loads first
+        if (MODE == kEnsembleSample) {
+          for (int i = 0; i < p.n; ++i) {
+            double pr = exp2(static_cast<double>(lv[i]) * p.cT64 - static_cast<double>(sh.fsoft[i].ref)) / sh.fsoft[i].s;
+            r64 += p.w64[i] * pr;
+            if (i == pis) q64 = pr;
+          }
+        } else {
+          double cd = 0.0;
+          for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(lv[i]), cd);
+          bool in = !masked || (lv[p.mask_model] >= thr);
+          r64 = in ? exp2(cd * p.cT64 - static_cast<double>(sh.fsoft[1].ref)) / sh.fsoft[1].s : 0.0;
+          q64 = exp2(static_cast<double>(lv[pis]) * p.cT64 - static_cast<double>(sh.fsoft[0].ref)) / sh.fsoft[0].s;
+        }
+        if (dump) p.dump_r[(static_cast<long long>(b) * p.P + j) * p.V + e] = static_cast<float>(r64);
+        return use_r ? r64 : fmax(0.0, r64 - q64);
+      };
+      // a lane's mass of one step: fp32 sum of the small tokens in token order plus the big ones in fp64
+      auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, bool dump) -> double {
         float ls = 0.f;
 #pragma unroll
-        for (int k = 0; k < E; ++k) ls += res[k];
-        own = ls;
-        double inc = static_cast<double>(ls);
+        for (int k = 0; k < E; ++k) ls += mass32[k];
+        double own = static_cast<double>(ls);
+        if (bigbits) {
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-          double o = shfl_up_double(inc, d);
-          if (lane >= d) inc += o;
+          for (int k = 0; k < E; ++k)
+            if (bigbits & (1u << k)) own += big_mass(e0 + k, use_r, dump);
         }
-        excl = shfl_up_double(inc, 1);
-        if (lane == 0) excl = 0.0;
+        return own;
       };
 
+      // running totals are recorded every gsz steps; the search below re-reads one such group
+      const int nst = s_end - s_begin;
+      const int gsz = (nst + kRec - 1) / kRec > 4 ? (nst + kRec - 1) / kRec : 4;
+      const int ngrp = (nst + gsz - 1) / gsz;
       for (int attempt = 0; attempt < 2; ++attempt) {
         const bool dump = (p.dump_r != nullptr) && attempt == 0;
-        double wrun = 0.0;  // this warp's total, accumulated step by step
-        for (int s = s_begin; s < s_end; ++s) {
-          float res[E];
-          chunk_mass((s * 32 + lane) * E, from_r, dump, res);
-          double excl;
-          float own;
-          lane_prefix(res, excl, own);
-          double step_total = shfl_double(excl + static_cast<double>(own), 31);
-          wrun += step_total;
+        double wrun = 0.0;   // this warp's total, accumulated group by group
+        double lacc = 0.0;   // this lane's mass within the current group
+        // vectors of the coming steps are staged in shared memory with cp.async so that a warp
+        // keeps several loads in flight although it consumes its run in token order
+        const int depth = (p.n <= 2) ? 4 : (p.n <= 4 ? 2 : 1);
+        const int nfull = vec_ok ? p.V / (32 * E) : 0;
+        const int fe = (s_end < nfull) ? s_end : nfull;  // steps [s_begin, fe) go through the ring
+        uint4* myring = ring + static_cast<size_t>(warp) * kRingVecs * 32 + lane;
+        auto stage = [&](int s) {  // issue the loads of step s into its ring slot
+          const int slot = ((s - s_begin) % depth) * p.n;
+          for (int i = 0; i < p.n; ++i)
+            cp_async16(&myring[(slot + i) * 32],
+                       reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(s * 32 + lane) * 16);
+        };
+        for (int t = 0; t < depth; ++t) {
+          if (s_begin + t < fe) stage(s_begin + t);
+          cp_async_commit();
         }
+        for (int s = s_begin; s < s_end; ++s) {
+          float mass32[E];
+          unsigned bigbits;
+          const int e0 = (s * 32 + lane) * E;
+          if (s < fe) {
+            if (depth == 4)
+              cp_async_wait<3>();
+            else if (depth == 2)
+              cp_async_wait<1>();
+            else
+              cp_async_wait<0>();
+            const int slot = ((s - s_begin) % depth) * p.n;
+            chunk_mass(e0, from_r, dump, mass32, bigbits, &myring[slot * 32]);
+            if (s + depth < fe) stage(s + depth);
+            cp_async_commit();
+          } else {
+            chunk_mass(e0, from_r, dump, mass32, bigbits, nullptr);
+          }
+          lacc += lane_mass(e0, mass32, bigbits, from_r, dump);
+          const int done = s - s_begin + 1;
+          if (done % gsz == 0 || s + 1 == s_end) {
+            double t = lacc;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+            wrun += t;
+            if (lane == 0) sh.srun[warp][(done - 1) / gsz] = wrun;
+            lacc = 0.0;
+          }
+        }
+        cp_async_wait<0>();
         if (lane == 0) sh.wtot[warp] = wrun;
         __syncthreads();
         if (tid == 0) {
@@ -905,7 +1307,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           for (int r = 0; r < C; ++r) tot[r] = cluster.map_shared_rank(&sh.x[phase & 1], r)->cta_total;
           double S = 0.0;
           for (int r = 0; r < C; ++r) S += tot[r];
-          const double target = sh.dec.u_smp * S;
+          const double target = sh.u_smp * S;
           double cp = 0.0;
           int wr = -1, ww = -1;
           double wbase = 0.0;
@@ -915,6 +1317,16 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               wbase = cp;
             }
             cp += tot[r];
+          }
+          if (wr < 0 && S > 0.0) {  // rounding corner: last block with mass
+            cp = 0.0;
+            for (int r = 0; r < C; ++r) {
+              if (tot[r] > 0.0) {
+                wr = r;
+                wbase = cp;
+              }
+              cp += tot[r];
+            }
           }
           if (wr == rank) {
             for (int w = 0; w < kWarps; ++w) {
@@ -943,6 +1355,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         if (sh.win_rank == -2 && !from_r) {
           // no residual mass although a token is needed: draw from r instead
           from_r = true;
+          __syncthreads();
           if (tid == 0 && !sh.dec.accept) sh.dec.status |= COS_ROW_RESIDUAL_EMPTY;
           __syncthreads();
           continue;
@@ -950,38 +1363,71 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         break;
       }
 
-      // the winning warp walks its run again and finds the token
+      // the winning warp finds the group of steps from the recorded totals, then walks that group
+      // again step by step with an fp64 prefix over the lanes and a walk over the lane's tokens
       if (sh.win_rank == rank && sh.win_warp == warp) {
         const double target = sh.target;
         const double lex = (warp > 0) ? sh.wincl[warp - 1] : 0.0;
         const double cbase = sh.base;
-        double R = 0.0;
+        int grp = -1;
+        for (int g0 = 0; g0 < ngrp && grp < 0; g0 += 32) {
+          const int g = g0 + lane;
+          const double prev = (g > 0 && g < ngrp) ? sh.srun[warp][g - 1] : 0.0;
+          const bool ok = (g < ngrp) && (sh.srun[warp][g < ngrp ? g : 0] > prev) &&
+                          (cbase + (lex + sh.srun[warp][g < ngrp ? g : 0]) >= target);
+          const unsigned m = __ballot_sync(0xffffffffu, ok);
+          if (m) grp = g0 + __ffs(m) - 1;
+        }
+        if (grp < 0) {  // rounding corner: last group with mass
+          for (int g = ngrp - 1; g >= 0 && grp < 0; --g)
+            if (sh.srun[warp][g] > (g > 0 ? sh.srun[warp][g - 1] : 0.0)) grp = g;
+          if (grp < 0) grp = 0;
+        }
+        double R = (grp > 0) ? sh.srun[warp][grp - 1] : 0.0;
         int token = -1, last_pos = -1;
-        for (int s = s_begin; s < s_end && token < 0; ++s) {
-          float res[E];
+        const int rs_begin = s_begin + grp * gsz;
+        const int rs_end = (rs_begin + gsz < s_end) ? rs_begin + gsz : s_end;
+        for (int s = rs_begin; s < rs_end && token < 0; ++s) {
+          float mass32[E];
+          unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
-          chunk_mass(e0, from_r, false, res);
-          double excl;
-          float own;
-          lane_prefix(res, excl, own);
-          const double incl = excl + static_cast<double>(own);
+          chunk_mass(e0, from_r, false, mass32, bigbits, nullptr);
+          // per-token masses of this lane in fp64 (big tokens from their fp64 evaluation)
+          double m64[E];
+#pragma unroll
+          for (int k = 0; k < E; ++k) m64[k] = static_cast<double>(mass32[k]);
+          if (bigbits) {
+#pragma unroll
+            for (int k = 0; k < E; ++k)
+              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, from_r, false);
+          }
+          const double own = lane_mass(e0, mass32, bigbits, from_r, false);
+          double inc = own;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            double o = shfl_up_double(inc, d);
+            if (lane >= d) inc += o;
+          }
+          double excl = shfl_up_double(inc, 1);
+          if (lane == 0) excl = 0.0;
+          const double incl = excl + own;
           const double step_total = shfl_double(incl, 31);
-          const bool hit = (own > 0.f) && (cbase + (lex + (R + incl)) >= target);
+          const bool hit = (own > 0.0) && (cbase + (lex + (R + incl)) >= target);
           unsigned hits = __ballot_sync(0xffffffffu, hit);
-          unsigned pos_lanes = __ballot_sync(0xffffffffu, own > 0.f);
-          const bool step_hit = (cbase + (lex + (R + step_total)) >= target) && pos_lanes != 0u;
-          if (step_hit) {
+          unsigned pos_lanes = __ballot_sync(0xffffffffu, own > 0.0);
+          const bool last_chance = (s + 1 == rs_end);
+          if (hits != 0u || (last_chance && pos_lanes != 0u)) {
             int src = hits ? (__ffs(hits) - 1) : (31 - __clz(pos_lanes));
             int found = -1;
             if (lane == src) {
-              float part = 0.f;
+              double part = 0.0;
               int lastk = -1;
 #pragma unroll
               for (int k = 0; k < E; ++k) {
-                part += res[k];
-                if (res[k] > 0.f) {
+                part += m64[k];
+                if (m64[k] > 0.0) {
                   lastk = k;
-                  if (found < 0 && cbase + (lex + (R + (excl + static_cast<double>(part)))) >= target) found = e0 + k;
+                  if (found < 0 && cbase + (lex + (R + (excl + part))) >= target) found = e0 + k;
                 }
               }
               if (found < 0) found = e0 + lastk;
@@ -992,7 +1438,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             int lp = -1;
 #pragma unroll
             for (int k = 0; k < E; ++k)
-              if (res[k] > 0.f) lp = e0 + k;
+              if (m64[k] > 0.0) lp = e0 + k;
             last_pos = __shfl_sync(0xffffffffu, lp, src);
           }
           R += step_total;
@@ -1009,7 +1455,8 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       const Decision& d = sh.dec;
       publish_unit(p, b, j, d.accept, d.status, d.cand, d.ratio, d.r_d, d.q_d, d.S);
     }
-    __syncthreads();
+    // No barrier here: everything the next unit writes before its first block barrier
+    // (ldraft, known_local, next_local, u_acc/u_smp, warp partials) is read only before this point.
     unit = next_unit;
   }
   cluster.sync();  // no block leaves while a peer may still read its shared memory
@@ -1028,9 +1475,9 @@ struct cos_verify_ctx {
   int max_clusters;
   int sm_count;
   unsigned work_base;
+  unsigned* d_work_counter;
   bool scratch_dirty;
   // device scratch
-  unsigned* d_work_counter;
   int* d_row_arrivals;
   int* d_first_rej;
   int4* d_unit_res;
@@ -1170,6 +1617,11 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   }
   ctx->sm_count = prop.multiProcessorCount;
   KernelFn fn = pick_kernel(config->dtype, mode_of(*config));
+  e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+  if (e != cudaSuccess) {
+    delete ctx;
+    return cuda_fail(nullptr, "cudaFuncSetAttribute(shared memory)", e);
+  }
   if (ctx->cluster > 8) {
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) {
@@ -1181,6 +1633,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(ctx->cluster * ctx->sm_count, 1, 1);
     lc.blockDim = dim3(kThreads, 1, 1);
+    lc.dynamicSmemBytes = kRingBytes;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = ctx->cluster;
@@ -1322,6 +1775,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * ctx->cluster, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = kRingBytes;
   lc.stream = stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
@@ -1333,8 +1787,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   ctx->scratch_dirty = true;  // cleared below once the launch is known to be queued
   e = cudaLaunchKernelEx(&lc, fn, p);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch", e);
-  // every unit is fetched exactly once from the counter or assigned statically, and every
-  // cluster that ran fetches once past the end
+  // every cluster starts on the unit of its own index and draws once after each unit it finishes,
+  // so a run draws exactly num_units numbers from the counter
   ctx->work_base += static_cast<unsigned>(p.num_units);
   ctx->scratch_dirty = false;
   return COS_OK;
