@@ -140,6 +140,38 @@ cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* args, void
  */
 cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args, void* cuda_stream);
 
+/*
+ * The same verification pass for callers that must not allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for deployment only.)
+ *
+ * cos_verify_create reserves its scratch with cudaMalloc.  Some hosts of this library cannot
+ * do that at the point where they need a verification: an inference engine that has handed
+ * the whole device to its own memory pool, or a serving loop in which the device-wide
+ * synchronisation that cudaMalloc / cudaFree imply would stall every other stream.  This call
+ * needs no context: the kernel's scratch (work counter, per-row arrival counters and
+ * earliest-rejection words, per-position results) lives in an array that is part of the
+ * library image, COS_STATIC_SCRATCH_BYTES long, resident on every device that loads the
+ * library until the process exits.  The call performs no cudaMalloc, cudaFree or other
+ * device allocation; `config` is read on every call (max_batch and host_staging are ignored).
+ *
+ * Limits: args->batch <= COS_STATIC_MAX_BATCH and args->batch * (gamma + 1) <=
+ * COS_STATIC_MAX_POSITIONS; anything larger returns COS_ERR_INVALID_ARG with the reason in
+ * cos_verify_last_error(NULL) and enqueues nothing.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
+ * sets kernel attributes; make that first call outside any stream capture.  Every call
+ * re-initialises the part of the array that must start clean (memset on `cuda_stream`)
+ * before the kernel, so a call does not depend on what the previous one left behind.
+ * All calls on a device share the one array: two calls that overlap on the GPU (different
+ * streams without an ordering between them) race and give undefined results.  Calls ordered
+ * on one stream, or otherwise serialised, are safe.  Inputs, outputs and semantics are those
+ * of cos_verify_run.
+ */
+#define COS_STATIC_MAX_BATCH 1024
+#define COS_STATIC_MAX_POSITIONS 8192
+#define COS_STATIC_SCRATCH_BYTES (256 + 8 * COS_STATIC_MAX_BATCH + 16 * COS_STATIC_MAX_POSITIONS)
+cos_status cos_verify_run_static(const cos_verify_config* config, const cos_verify_args* args, void* cuda_stream);
+
 /* Launch geometry chosen at creation. */
 cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info);
 

@@ -226,3 +226,50 @@ class CosVerifier:
 
     def __exit__(self, *exc):
         self.close()
+
+
+def run_static(n: int, combine: int, weights: Sequence[float], temperature: float, gamma: int, vocab: int,
+               logits, drafts, proposer, seed: int, offset: int, mask_model: int = -1, mask_alpha: float = 1.0,
+               device: int = 0, cluster_size: int = 0, row_base: int = 0, flags: int = 0, outs: dict = None,
+               stream=None) -> dict:
+    """cos_verify_run_static: one verification pass with no context and no device allocation.
+
+    For hosts that cannot call cudaMalloc where they verify (a device fully owned by an engine's
+    memory pool, or a serving loop that must avoid the device-wide stall of cudaMalloc/cudaFree):
+    the kernel's scratch is an array built into the library.  `outs` must hold the preallocated
+    output tensors ("accept_count" [B], "out_tokens" [B, gamma+1], "row_status" [B], all int32,
+    optionally "diag" [B, gamma+1, 4] float32) so that this wrapper allocates nothing either.
+    Limits: B <= 1024 and B * (gamma + 1) <= 8192.  Calls share the built-in array, so calls
+    that overlap on the GPU race; order them on one stream.
+    """
+    import torch
+    lib = load_library()
+    lib.cos_verify_run_static.argtypes = [ctypes.POINTER(cos_verify_config), ctypes.POINTER(cos_verify_args),
+                                          ctypes.c_void_p]
+    lib.cos_verify_run_static.restype = ctypes.c_int
+    cfg = cos_verify_config()
+    cfg.n, cfg.combine = n, combine
+    for i, w in enumerate(list(weights)[:COS_MAX_MODELS]):
+        cfg.weights[i] = w
+    cfg.mask_model, cfg.mask_alpha, cfg.temperature = mask_model, mask_alpha, temperature
+    cfg.gamma, cfg.vocab, cfg.max_batch = gamma, vocab, logits.shape[1]
+    cfg.dtype, cfg.device, cfg.cluster_size, cfg.host_staging = _dtype_code(logits.dtype), device, cluster_size, 0
+    if outs is None:
+        raise ValueError("run_static needs preallocated outputs (it must not allocate)")
+    a = cos_verify_args()
+    a.logits = logits.data_ptr()
+    a.stride_model, a.stride_row, a.stride_pos = logits.stride(0), logits.stride(1), logits.stride(2)
+    a.draft_tokens = drafts.data_ptr() if (drafts is not None and drafts.numel() > 0) else None
+    a.proposer = proposer.data_ptr()
+    a.batch, a.flags, a.row_base = logits.shape[1], flags, row_base
+    a.seed, a.offset = seed & 0xFFFFFFFFFFFFFFFF, offset & 0xFFFFFFFFFFFFFFFF
+    a.accept_count = outs["accept_count"].data_ptr()
+    a.out_tokens = outs["out_tokens"].data_ptr()
+    a.row_status = outs["row_status"].data_ptr()
+    a.diag = outs["diag"].data_ptr() if "diag" in outs else None
+    a.dump_r = None
+    s = torch.cuda.current_stream(logits.device) if stream is None else stream
+    st = lib.cos_verify_run_static(ctypes.byref(cfg), ctypes.byref(a), ctypes.c_void_p(s.cuda_stream))
+    if st != COS_OK:
+        raise CosVerifyError(st, lib.cos_verify_last_error(None).decode())
+    return outs

@@ -1888,3 +1888,153 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
 extern "C" const char* cos_verify_last_error(const cos_verify_ctx* ctx) {
   return ctx ? ctx->err.c_str() : g_create_error.c_str();
 }
+
+// ------------------------------------------------------------------------------------
+// verification without a context and without any device allocation
+// ------------------------------------------------------------------------------------
+namespace {
+
+// Scratch of the context-free entry point.  It is part of the library image: every device
+// that loads the library holds these COS_STATIC_SCRATCH_BYTES until the process exits.
+// Layout: [0, 256) work counter | row arrival counters | earliest-rejection words | unit results.
+static __device__ __align__(256) unsigned char g_static_scratch[COS_STATIC_SCRATCH_BYTES];
+
+constexpr int kStaticMaxDevices = 64;
+// Device address of g_static_scratch per device.  In host code the symbol itself is only a
+// stand-in, never an address a kernel may use, so the address is asked for once per device.
+unsigned char* g_static_addr[kStaticMaxDevices];
+bool g_static_ready[kStaticMaxDevices];
+
+cos_status static_fail(cos_status st, const char* msg) {
+  g_create_error = msg;
+  return st;
+}
+
+}  // namespace
+
+extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, const cos_verify_args* a,
+                                            void* cuda_stream) {
+  if (!config || !a) return static_fail(COS_ERR_INVALID_ARG, "null argument");
+  cos_verify_config c = *config;
+  c.max_batch = COS_STATIC_MAX_BATCH;  // the array, not the caller, bounds the batch here
+  if (!validate_config(c, &g_create_error)) return COS_ERR_INVALID_ARG;
+  if (a->batch < 1 || a->batch > COS_STATIC_MAX_BATCH)
+    return static_fail(COS_ERR_INVALID_ARG, "batch exceeds COS_STATIC_MAX_BATCH (1024) of the built-in scratch");
+  const long long units = static_cast<long long>(a->batch) * (c.gamma + 1);
+  if (units > COS_STATIC_MAX_POSITIONS)
+    return static_fail(COS_ERR_INVALID_ARG,
+                       "batch * (gamma + 1) exceeds COS_STATIC_MAX_POSITIONS (8192) of the built-in scratch");
+  if (c.device < 0 || c.device >= kStaticMaxDevices) return static_fail(COS_ERR_INVALID_ARG, "device ordinal out of range");
+  if (!a->logits || !a->proposer || !a->accept_count || !a->out_tokens || !a->row_status)
+    return static_fail(COS_ERR_INVALID_ARG, "null device pointer");
+  if (c.gamma > 0 && !a->draft_tokens) return static_fail(COS_ERR_INVALID_ARG, "draft_tokens is null although gamma > 0");
+  if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return static_fail(COS_ERR_INVALID_ARG, "negative stride");
+  if (a->flags & ~COS_RUN_ALL_RESIDUALS) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
+  const int eb = elem_bytes(c.dtype);
+  if (reinterpret_cast<uintptr_t>(a->logits) % eb) return static_fail(COS_ERR_ALIGNMENT, "logits pointer not aligned to its element type");
+  if (reinterpret_cast<uintptr_t>(a->proposer) % 4 || reinterpret_cast<uintptr_t>(a->accept_count) % 4 ||
+      reinterpret_cast<uintptr_t>(a->out_tokens) % 4 || reinterpret_cast<uintptr_t>(a->row_status) % 4 ||
+      (a->draft_tokens && reinterpret_cast<uintptr_t>(a->draft_tokens) % 4) ||
+      (a->diag && reinterpret_cast<uintptr_t>(a->diag) % 4) || (a->dump_r && reinterpret_cast<uintptr_t>(a->dump_r) % 4))
+    return static_fail(COS_ERR_ALIGNMENT, "an int32/float pointer is not 4-byte aligned");
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaSetDevice(c.device);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaSetDevice", e);
+  KernelFn fn = pick_kernel(c.dtype, mode_of(c));
+  const int cluster = choose_cluster(c);
+  if (!g_static_ready[c.device]) {
+    // once per device, with that device current: the device address of the built-in array
+    void* addr = nullptr;
+    e = cudaGetSymbolAddress(&addr, g_static_scratch);
+    if (e != cudaSuccess || addr == nullptr) return cuda_fail(nullptr, "cudaGetSymbolAddress(built-in scratch)", e);
+    g_static_addr[c.device] = static_cast<unsigned char*>(addr);
+    g_static_ready[c.device] = true;
+  }
+  e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+  if (e == cudaSuccess && cluster > 8)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaFuncSetAttribute", e);
+
+  cudaLaunchConfig_t lc = {};
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cluster;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = kRingBytes;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  int sm_count = 0;
+  e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c.device);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaDeviceGetAttribute", e);
+  lc.gridDim = dim3(static_cast<unsigned>(cluster * sm_count), 1, 1);
+  int max_clusters = 0;
+  e = cudaOccupancyMaxActiveClusters(&max_clusters, reinterpret_cast<const void*>(fn), &lc);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "cudaOccupancyMaxActiveClusters", e);
+  if (max_clusters < 1) return static_fail(COS_ERR_UNSUPPORTED, "no cluster of the requested size fits on the device");
+
+  // carve the array; what must start clean is cleared on the caller's stream before the kernel
+  unsigned char* basep = g_static_addr[c.device];
+  unsigned* d_counter = reinterpret_cast<unsigned*>(basep);
+  int* d_arrivals = reinterpret_cast<int*>(basep + 256);
+  int* d_first_rej = d_arrivals + COS_STATIC_MAX_BATCH;
+  int4* d_unit_res = reinterpret_cast<int4*>(basep + 256 + 8 * COS_STATIC_MAX_BATCH);
+  e = cudaMemsetAsync(d_counter, 0, sizeof(unsigned), stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_arrivals, 0, static_cast<size_t>(a->batch) * sizeof(int), stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_first_rej, 0x7f, static_cast<size_t>(a->batch) * sizeof(int), stream);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "clearing the built-in scratch", e);
+
+  KParams p;
+  memset(&p, 0, sizeof(p));
+  p.logits = a->logits;
+  p.s_model = a->stride_model;
+  p.s_row = a->stride_row;
+  p.s_pos = a->stride_pos;
+  p.drafts = a->draft_tokens;
+  p.proposer = a->proposer;
+  p.n = c.n;
+  p.V = c.vocab;
+  p.gamma = c.gamma;
+  p.P = c.gamma + 1;
+  p.B = a->batch;
+  p.mask_model = (c.combine == COS_COMBINE_LOGIT_LINEAR) ? c.mask_model : -1;
+  const int E = entries_per_vec(c.dtype);
+  p.vec_ok = (reinterpret_cast<uintptr_t>(a->logits) % 16 == 0) && ((a->stride_model * eb) % 16 == 0) &&
+             ((a->stride_row * eb) % 16 == 0) && ((a->stride_pos * eb) % 16 == 0);
+  p.nsteps = (c.vocab + 32 * E - 1) / (32 * E);
+  p.flags = a->flags;
+  p.num_units = static_cast<int>(units);
+  p.num_clusters = p.num_units < max_clusters ? p.num_units : max_clusters;
+  for (int i = 0; i < COS_MAX_MODELS; ++i) {
+    p.w[i] = (i < c.n) ? c.weights[i] : 0.f;
+    p.w64[i] = static_cast<double>(p.w[i]);
+  }
+  if (c.temperature > 0.0f) {
+    p.cT = static_cast<float>(1.4426950408889634 / static_cast<double>(c.temperature));
+    p.cT64 = static_cast<double>(p.cT);
+  }
+  p.ln_alpha = (p.mask_model >= 0) ? log(static_cast<double>(c.mask_alpha)) : 0.0;
+  p.seed_lo = static_cast<unsigned>(a->seed);
+  p.seed_hi = static_cast<unsigned>(a->seed >> 32);
+  p.off_lo = static_cast<unsigned>(a->offset);
+  p.off_hi = static_cast<unsigned>(a->offset >> 32);
+  p.row_base = a->row_base;
+  p.accept_count = a->accept_count;
+  p.out_tokens = a->out_tokens;
+  p.row_status = a->row_status;
+  p.diag = a->diag;
+  p.dump_r = a->dump_r;
+  p.work_counter = d_counter;
+  p.work_base = 0;  // the counter was just cleared
+  p.row_arrivals = d_arrivals;
+  p.first_rej = d_first_rej;
+  p.unit_res = d_unit_res;
+
+  lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * cluster, 1, 1);
+  lc.stream = stream;
+  e = cudaLaunchKernelEx(&lc, fn, p);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch", e);
+  return COS_OK;
+}
