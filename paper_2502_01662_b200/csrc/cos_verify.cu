@@ -9,7 +9,7 @@
 //            merge lane -> warp -> block -> cluster (the last two in fp64, across blocks
 //            through distributed shared memory);
 //   decide   the accept test of Eq. 6 in fp64 from the merged statistics and the logits at
-//            the draft token; rank 0 records the row's earliest known rejection;
+//            the draft token;
 //   sweep 2  only where a token must be drawn (first rejected position of a row, or the
 //            bonus position when nothing earlier was rejected): re-read the unit (it is
 //            still in L2), form r and q per token, residual max(0, r - q), warp-ordered
@@ -49,6 +49,13 @@ constexpr int kRec = 64;                     // running totals recorded per warp
 
 enum Mode { kEnsembleSample = 0, kLogitSample = 1, kEnsembleGreedy = 2, kLogitGreedy = 3 };
 
+struct UnitStats {  // what stage 1 needs from stage 0 about one (row, position)
+  double s[COS_MAX_MODELS];   // normalisers sum 2^(arg - ref)
+  float ref[COS_MAX_MODELS];  // reference exponents
+  float thr32;                // plausibility threshold
+  int pad[3];
+};
+
 struct KParams {
   const void* logits;
   long long s_model, s_row, s_pos;  // element strides
@@ -60,6 +67,8 @@ struct KParams {
   int nsteps;   // ceil(V / (32 * E))
   int flags;
   int num_units, num_clusters;
+  int stage;     // 0: statistics, decisions, row scan (every unit); 1: draw tokens for the listed units
+  int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
   double w64[COS_MAX_MODELS];
   float cT;       // log2(e) / T in fp32 (T > 0)
@@ -76,8 +85,11 @@ struct KParams {
   unsigned* work_counter;  // units are handed out from here; grows by num_units every run
   unsigned work_base;      // its value when this run starts
   int* row_arrivals;       // [B], zero between runs
-  int* first_rej;          // [B], kNoReject between runs
-  int4* unit_res;          // [B*P]: x = accept flag, y = status bits, z = candidate token
+  int4* unit_res;          // [B*P]: x = accept flag, y = status bits, z = candidate token, w = a token can be drawn
+  int* job_count;          // units that stage 1 must process (this run's counter)
+  int* job_reset;          // the other run parity's counter, cleared by stage 0
+  int2* jobs;              // x = b * P + j, y = 1 if the drawn token is the row's output at position j
+  UnitStats* ustats;       // [B*P]: merged statistics of sweep 1, read back by stage 1
 };
 
 // ------------------------------------------------------------------------------------
@@ -94,12 +106,6 @@ __device__ __forceinline__ uint4 ldg_stream16(const void* p) {
   asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(p));
-  return v;
-}
-
-__device__ __forceinline__ int ld_relaxed_gpu(const int* p) {
-  int v;
-  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p));
   return v;
 }
 
@@ -227,13 +233,13 @@ struct Xchg {  // one per block and barrier parity; peers read it through DSMEM
   SoftPart soft[kMaxSlots];
   ArgPart arg[kMaxSlots];
   double cta_total;
-  int known;  // rank 0 only: earliest rejected position of the row seen so far
+  int pad;
   int next;   // rank 0 only: the unit this cluster takes after the current one
 };
 
 struct Decision {  // written by thread 0 of every block, identically
   int accept, status, want_sample, cand;
-  int natoms, need2;
+  int natoms, need2, drawable;
   int atom_tok[COS_MAX_MODELS];
   double atom_mass[COS_MAX_MODELS];
   double ratio, r_d, q_d, S;
@@ -256,7 +262,6 @@ struct Shared {
   double u_acc, u_smp;
   double target, base;  // sweep-2 search: u*S and the mass before the winning block
   int win_rank, win_warp;
-  int known_local, known;
   int next_local, next;
   float thr32;  // plausibility threshold rounded up to fp32
   float big_thr[kMaxSlots];  // sweep 2: terms above this share of a normaliser are redone in fp64
@@ -378,7 +383,7 @@ __device__ __forceinline__ void warp_merge_arg(double val, int idx, int bad, Arg
 // Block merge of the warp partials, publish for the peers, ONE cluster barrier, merge over
 // the ranks.  Warp k handles soft slot k (k < nsoft); warp 8 + k handles arg slot a0 + k.
 // All threads of all blocks of the cluster call this; results land in sh.fsoft / sh.farg,
-// and rank 0's view of the row's earliest rejection in sh.known.
+// and the cluster's next unit (drawn by rank 0) in sh.next.
 __device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& cluster, int& phase, int nsoft, int a0,
                                               int narg) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -403,7 +408,6 @@ __device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& clu
     ArgPart o = warp_reduce_arg(in.val, in.idx, in.bad, lane);
     if (lane == 0) mine.arg[slot] = o;
   } else if (warp == kWarps - 1 && lane == 0) {
-    mine.known = sh.known_local;
     mine.next = sh.next_local;
   }
   cluster.sync();
@@ -428,7 +432,6 @@ __device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& clu
     if (lane == 0) sh.farg[slot] = o;
   } else if (warp == kWarps - 1 && lane == 0) {
     const Xchg* r0 = cluster.map_shared_rank(&sh.x[phase & 1], 0);
-    sh.known = r0->known;
     sh.next = r0->next;
   }
   __syncthreads();
@@ -438,17 +441,28 @@ __device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& clu
 // ------------------------------------------------------------------------------------
 // publishing a unit and the per-row first-rejection scan (Sec. 3.1)
 // ------------------------------------------------------------------------------------
-__device__ void publish_unit(const KParams& p, int b, int j, int accept, int status, int cand, double ratio,
-                             double r_d, double q_d, double S) {
+__device__ __forceinline__ void push_job(const KParams& p, int idx, int emit) {
+  const int k = atomicAdd(p.job_count, 1);
+  if (k < p.max_jobs) p.jobs[k] = make_int2(idx, emit);
+}
+
+// Stage 0: record a unit's decision; the last unit of a row to arrive scans for the first
+// rejection, writes the row's outputs and, where a token has to be drawn, lists that unit
+// for stage 1 (which fills in out_tokens[b][a]).
+__device__ void publish_unit(const KParams& p, int b, int j, int accept, int status, int cand, int drawable,
+                             double ratio, double r_d, double q_d, double S) {
+  const int idx = b * p.P + j;
   if (p.diag) {
-    float* d = p.diag + (static_cast<long long>(b) * p.P + j) * 4;
+    float* d = p.diag + static_cast<long long>(idx) * 4;
     d[0] = static_cast<float>(ratio);
     d[1] = static_cast<float>(r_d);
     d[2] = static_cast<float>(q_d);
     d[3] = static_cast<float>(S);
   }
-  int4 res = make_int4(accept, status, cand, 0);
-  __stcg(&p.unit_res[b * p.P + j], res);
+  int4 res = make_int4(accept, status, cand, drawable);
+  __stcg(&p.unit_res[idx], res);
+  // test hooks: the combined distribution everywhere, or the residual mass at every draft position
+  if (drawable && (p.dump_r != nullptr || ((p.flags & COS_RUN_ALL_RESIDUALS) && j < p.gamma))) push_job(p, idx, 0);
   __threadfence();
   int prev = atomicAdd(&p.row_arrivals[b], 1);
   if (prev != p.P - 1) return;
@@ -456,13 +470,14 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
   __threadfence();
   int a = p.gamma;
   unsigned st = 0;
-  int tok = -1;
+  int tok = -1, draw = 0;
   for (int k = 0; k < p.P; ++k) {
     int4 u = __ldcg(&p.unit_res[b * p.P + k]);
     st |= static_cast<unsigned>(u.y);
     if (k == p.gamma || !u.x) {
       a = k;
       tok = u.z;
+      draw = u.w;
       break;
     }
   }
@@ -471,7 +486,7 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
   for (int k = 0; k < p.P; ++k) o[k] = (k < a) ? p.drafts[b * p.gamma + k] : (k == a ? tok : -1);
   p.row_status[b] = st;
   p.row_arrivals[b] = 0;  // leave the scratch ready for the next run
-  p.first_rej[b] = kNoReject;
+  if (draw) push_job(p, b * p.P + a, 1);
 }
 
 // ------------------------------------------------------------------------------------
@@ -575,9 +590,30 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   // this block's slice of every row in sweep 1
   const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
 
-  int unit = blockIdx.x / C;
-  while (unit < p.num_units) {
-    const int j = unit / p.B, b = unit % p.B;  // earlier positions of every row come first
+  const int cluster_id = blockIdx.x / C;
+  int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
+  if (p.stage == 0) {
+    if (blockIdx.x == 0 && tid == 0) *p.job_reset = 0;  // the list of the next run starts empty
+  } else {
+    njobs = *p.job_count;
+    njobs = njobs < p.max_jobs ? njobs : p.max_jobs;
+  }
+  while (true) {
+    int j, b;
+    if (p.stage == 0) {
+      if (unit >= p.num_units) break;
+      j = unit / p.B;  // earlier positions of every row come first
+      b = unit % p.B;
+    } else {
+      const int job = cluster_id + job_it * p.num_clusters;
+      if (job >= njobs) break;
+      const int2 jb = p.jobs[job];
+      ++job_it;
+      emit = jb.y;
+      b = jb.x / p.P;
+      j = jb.x % p.P;
+    }
+    const int uidx = b * p.P + j;
     const int pi = p.proposer[b];
     const bool pi_ok = (pi >= 0 && pi < p.n);
     const int pis = pi_ok ? pi : 0;
@@ -588,12 +624,11 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
     const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
     const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
 
+    if (p.stage == 0) {
     // ---- small jobs issued before the sweep so that their latency hides behind it
     if (tid < p.n && !is_bonus && draft_ok) sh.ldraft[tid] = Elem<DT>::load1(row_of(tid), draft);
     if (warp == kWarps - 1) {
-      if (lane == 0) {
-        sh.known_local = (rank == 0) ? ld_relaxed_gpu(&p.first_rej[b]) : kNoReject;
-      } else if (lane == 2) {
+      if (lane == 2) {
         // rank 0 draws the cluster's next unit now; every block learns it with the merged statistics
         if (rank == 0) sh.next_local = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
       } else if (lane == 1) {
@@ -926,17 +961,48 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           if (d.cand < 0) d.cand = lastpos;
         }
       }
-      // a token is drawn only where the row can still need it: rank 0 looked at the row's
-      // earliest known rejection before the sweep and every block received that same value
-      const bool superseded = sh.known < j;
-      d.need2 = 0;
-      if (kSample && finite) {
-        d.need2 = (d.want_sample && !superseded) || (p.dump_r != nullptr) ||
-                  ((p.flags & COS_RUN_ALL_RESIDUALS) && !is_bonus);
-      }
-      if (rank == 0 && !is_bonus && !d.accept) atomicMin(&p.first_rej[b], j);
+      d.need2 = 0;  // tokens are drawn by stage 1, for the one position per row that needs it
+      d.drawable = (kSample && finite) ? 1 : 0;
     }
     __syncthreads();
+    // rank 0 keeps the merged statistics for stage 1 and reports the unit
+    if (rank == 0) {
+      const int nkeep = (MODE == kEnsembleSample) ? p.n : (MODE == kLogitSample ? 2 : 0);
+      if (tid < nkeep) {
+        p.ustats[uidx].s[tid] = sh.fsoft[tid].s;
+        p.ustats[uidx].ref[tid] = sh.fsoft[tid].ref;
+      }
+      if (tid == 32 && nkeep > 0) p.ustats[uidx].thr32 = masked ? sh.thr32 : 0.f;
+    }
+    } else {
+      // stage 1: the statistics of this unit were merged by stage 0
+      const int nkeep = (MODE == kEnsembleSample) ? p.n : 2;
+      if (tid < nkeep) {
+        sh.fsoft[tid].s = p.ustats[uidx].s[tid];
+        sh.fsoft[tid].ref = p.ustats[uidx].ref[tid];
+        sh.big_thr[tid] = static_cast<float>(sh.fsoft[tid].s * kBigShare);
+      }
+      if (tid == 32) {
+        const int4 ur = __ldcg(&p.unit_res[uidx]);
+        Decision& d = sh.dec;
+        d.accept = ur.x;
+        d.status = ur.y;
+        d.want_sample = 1;
+        d.cand = -1;
+        d.natoms = 0;
+        d.need2 = 1;
+        d.drawable = 1;
+        d.ratio = d.r_d = d.q_d = d.S = kNaN;
+        sh.thr32 = p.ustats[uidx].thr32;
+        unsigned rnd[4];
+        const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
+        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi,
+                      rnd);
+        sh.u_smp = word_to_uniform(rnd[1]);
+        sh.next = 0;
+      }
+      __syncthreads();
+    }
     const int need2 = sh.dec.need2;
     const int next_unit = sh.next;
 
@@ -1445,18 +1511,25 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         }
         if (token < 0) token = last_pos;
         if (lane == 0) {
-          const Decision& d = sh.dec;
-          publish_unit(p, b, j, d.accept, d.status, token, d.ratio, d.r_d, d.q_d, S_report);
+          // stage 1 result: the row's token at its first rejection (or bonus), and the residual mass
+          if (emit) {
+            p.out_tokens[uidx] = token;
+            if (sh.dec.status & COS_ROW_RESIDUAL_EMPTY) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_RESIDUAL_EMPTY));
+          }
+          if (p.diag) p.diag[static_cast<long long>(uidx) * 4 + 3] = static_cast<float>(S_report);
         }
       }
       published = (sh.win_rank >= 0);  // otherwise nothing had mass: rank 0 reports token -1 below
     }
-    if (!published && rank == 0 && tid == 0) {
+    if (p.stage == 0 && rank == 0 && tid == 0) {
       const Decision& d = sh.dec;
-      publish_unit(p, b, j, d.accept, d.status, d.cand, d.ratio, d.r_d, d.q_d, d.S);
+      publish_unit(p, b, j, d.accept, d.status, d.cand, d.drawable, d.ratio, d.r_d, d.q_d, d.S);
     }
+    (void)published;
     // No barrier here: everything the next unit writes before its first block barrier
-    // (ldraft, known_local, next_local, u_acc/u_smp, warp partials) is read only before this point.
+    // (ldraft, next_local, u_acc/u_smp, warp partials) is read only before this point; stage 1
+    // starts every unit with a block barrier of its own.
+    if (p.stage == 1) __syncthreads();
     unit = next_unit;
   }
   cluster.sync();  // no block leaves while a peer may still read its shared memory
@@ -1471,16 +1544,19 @@ thread_local std::string g_create_error;
 
 struct cos_verify_ctx {
   cos_verify_config cfg;
-  int cluster;
-  int max_clusters;
+  int cluster_draw;     // blocks per unit in stage 1
+  int max_clusters[5];  // resident clusters for cluster sizes 1, 2, 4, 8, 16 (0 = not available)
   int sm_count;
   unsigned work_base;
+  unsigned run_parity;
   unsigned* d_work_counter;
   bool scratch_dirty;
   // device scratch
   int* d_row_arrivals;
-  int* d_first_rej;
   int4* d_unit_res;
+  int* d_job_count;  // two counters, used alternately by successive runs
+  int2* d_jobs;
+  UnitStats* d_ustats;
   // optional staging for host-pointer runs
   void* d_logits;
   int* d_drafts;
@@ -1569,6 +1645,49 @@ int choose_cluster(const cos_verify_config& c) {
   return cs;
 }
 
+int log2i(int c) { return c >= 16 ? 4 : (c >= 8 ? 3 : (c >= 4 ? 2 : (c >= 2 ? 1 : 0))); }
+
+// Stage 0 streams best with one block per unit (long contiguous reads, no cluster barrier);
+// more blocks per unit only when there are too few units to occupy the device.
+int choose_stream_cluster(const cos_verify_config& c, int units, int sm_count) {
+  if (c.cluster_size > 0) return c.cluster_size;
+  const int cap = choose_cluster(c);
+  int cs = 1;
+  while (cs < cap && units * cs < sm_count) cs <<= 1;
+  return cs;
+}
+
+cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int* out) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(cluster * sm_count, 1, 1);
+  lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = kRingBytes;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cluster;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaOccupancyMaxActiveClusters(out, reinterpret_cast<const void*>(fn), &lc);
+}
+
+cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, cudaStream_t stream) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * cluster, 1, 1);
+  lc.blockDim = dim3(kThreads, 1, 1);
+  lc.dynamicSmemBytes = kRingBytes;
+  lc.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = cluster;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, fn, p);
+}
+
 cos_status cuda_fail(cos_verify_ctx* ctx, const char* what, cudaError_t e) {
   char buf[256];
   snprintf(buf, sizeof(buf), "%s: %s", what, cudaGetErrorString(e));
@@ -1583,10 +1702,10 @@ cos_status init_scratch(cos_verify_ctx* ctx, cudaStream_t stream) {
   const size_t rows = static_cast<size_t>(ctx->cfg.max_batch);
   cudaError_t e = cudaMemsetAsync(ctx->d_work_counter, 0, sizeof(unsigned), stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_row_arrivals, 0, rows * sizeof(int), stream);
-  // kNoReject = 0x7fffffff is not a byte pattern; 0x7f7f7f7f is large enough to mean "no rejection yet"
-  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_first_rej, 0x7f, rows * sizeof(int), stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_job_count, 0, 2 * sizeof(int), stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "scratch reset", e);
   ctx->work_base = 0;
+  ctx->run_parity = 0;
   ctx->scratch_dirty = false;
   return COS_OK;
 }
@@ -1608,7 +1727,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     return COS_ERR_NOMEM;
   }
   ctx->cfg = *config;
-  ctx->cluster = choose_cluster(*config);
+  ctx->cluster_draw = choose_cluster(*config);
   cudaDeviceProp prop;
   e = cudaGetDeviceProperties(&prop, config->device);
   if (e != cudaSuccess) {
@@ -1622,43 +1741,41 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     delete ctx;
     return cuda_fail(nullptr, "cudaFuncSetAttribute(shared memory)", e);
   }
-  if (ctx->cluster > 8) {
+  if (config->cluster_size > 8) {
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) {
       delete ctx;
       return cuda_fail(nullptr, "cluster size above 8 not available", e);
     }
   }
-  {
-    cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(ctx->cluster * ctx->sm_count, 1, 1);
-    lc.blockDim = dim3(kThreads, 1, 1);
-    lc.dynamicSmemBytes = kRingBytes;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = ctx->cluster;
-    at[0].val.clusterDim.y = 1;
-    at[0].val.clusterDim.z = 1;
-    lc.attrs = at;
-    lc.numAttrs = 1;
+  for (int k = 0; k < 5; ++k) {
+    const int cs = 1 << k;
+    ctx->max_clusters[k] = 0;
+    if (cs == 16 && config->cluster_size != 16) continue;
     int nc = 0;
-    e = cudaOccupancyMaxActiveClusters(&nc, reinterpret_cast<const void*>(fn), &lc);
-    if (e != cudaSuccess || nc < 1) {
-      delete ctx;
-      if (e == cudaSuccess) {
-        g_create_error = "no cluster of the requested size fits on the device";
-        return COS_ERR_UNSUPPORTED;
-      }
-      return cuda_fail(nullptr, "cudaOccupancyMaxActiveClusters", e);
+    e = query_clusters(fn, cs, ctx->sm_count, &nc);
+    if (e != cudaSuccess) {
+      (void)cudaGetLastError();
+      nc = 0;
     }
-    ctx->max_clusters = nc;
+    ctx->max_clusters[k] = nc;
+  }
+  {
+    const int need = config->cluster_size > 0 ? config->cluster_size : 1;
+    if (ctx->max_clusters[log2i(need)] < 1 || ctx->max_clusters[log2i(ctx->cluster_draw)] < 1) {
+      delete ctx;
+      g_create_error = "no cluster of the requested size fits on the device";
+      return COS_ERR_UNSUPPORTED;
+    }
   }
   const size_t rows = static_cast<size_t>(config->max_batch), P = static_cast<size_t>(config->gamma) + 1;
   bool ok = true;
   ok = ok && cudaMalloc(&ctx->d_work_counter, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_row_arrivals, rows * sizeof(int)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->d_first_rej, rows * sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_unit_res, rows * P * sizeof(int4)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_job_count, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_jobs, (rows * P + rows) * sizeof(int2)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_ustats, rows * P * sizeof(UnitStats)) == cudaSuccess;
   if (ok && config->host_staging) {
     const size_t V = static_cast<size_t>(config->vocab);
     ok = ok && cudaMalloc(&ctx->d_logits, static_cast<size_t>(config->n) * rows * P * V * elem_bytes(config->dtype)) == cudaSuccess;
@@ -1745,7 +1862,6 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.nsteps = (c.vocab + 32 * E - 1) / (32 * E);
   p.flags = a->flags;
   p.num_units = a->batch * (c.gamma + 1);
-  p.num_clusters = p.num_units < ctx->max_clusters ? p.num_units : ctx->max_clusters;
   for (int i = 0; i < COS_MAX_MODELS; ++i) {
     p.w[i] = (i < c.n) ? c.weights[i] : 0.f;
     p.w64[i] = static_cast<double>(p.w[i]);
@@ -1768,28 +1884,43 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.work_counter = ctx->d_work_counter;
   p.work_base = ctx->work_base;
   p.row_arrivals = ctx->d_row_arrivals;
-  p.first_rej = ctx->d_first_rej;
   p.unit_res = ctx->d_unit_res;
+  p.job_count = ctx->d_job_count + (ctx->run_parity & 1u);
+  p.job_reset = ctx->d_job_count + ((ctx->run_parity & 1u) ^ 1u);
+  p.jobs = ctx->d_jobs;
+  p.ustats = ctx->d_ustats;
+  p.max_jobs = p.num_units + a->batch;
 
   KernelFn fn = pick_kernel(c.dtype, mode_of(c));
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * ctx->cluster, 1, 1);
-  lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = kRingBytes;
-  lc.stream = stream;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = ctx->cluster;
-  at[0].val.clusterDim.y = 1;
-  at[0].val.clusterDim.z = 1;
-  lc.attrs = at;
-  lc.numAttrs = 1;
-  ctx->scratch_dirty = true;  // cleared below once the launch is known to be queued
-  e = cudaLaunchKernelEx(&lc, fn, p);
-  if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch", e);
+  const int mode = mode_of(c);
+  const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
+  // stage 0: every unit once (statistics, accept tests, row scans)
+  const int c0 = choose_stream_cluster(c, p.num_units, ctx->sm_count);
+  const int mc0 = ctx->max_clusters[log2i(c0)];
+  if (mc0 < 1) {
+    ctx->err = "no cluster of the chosen size fits on the device";
+    return COS_ERR_UNSUPPORTED;
+  }
+  p.stage = 0;
+  p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
+  ctx->scratch_dirty = true;  // cleared below once the launches are known to be queued
+  e = launch_stage(fn, p, c0, stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
+  if (draws) {
+    // stage 1: the units listed by stage 0 (one per row, or all of them under the test hooks)
+    const int c1 = ctx->cluster_draw;
+    const int mc1 = ctx->max_clusters[log2i(c1)];
+    const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
+    const int most = all ? p.max_jobs : a->batch;
+    p.stage = 1;
+    p.num_clusters = most < mc1 ? most : mc1;
+    e = launch_stage(fn, p, c1, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 1)", e);
+  }
   // every cluster starts on the unit of its own index and draws once after each unit it finishes,
   // so a run draws exactly num_units numbers from the counter
   ctx->work_base += static_cast<unsigned>(p.num_units);
+  ctx->run_parity ^= 1u;
   ctx->scratch_dirty = false;
   return COS_OK;
 }
@@ -1857,11 +1988,12 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
 extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info) {
   if (!ctx || !info) return COS_ERR_INVALID_ARG;
   memset(info, 0, sizeof(*info));
-  info->cluster_size = ctx->cluster;
+  info->cluster_size = choose_stream_cluster(ctx->cfg, ctx->cfg.max_batch * (ctx->cfg.gamma + 1), ctx->sm_count);
   info->threads_per_block = kThreads;
-  info->max_clusters = ctx->max_clusters;
+  info->max_clusters = ctx->max_clusters[log2i(info->cluster_size)];
   info->sm_count = ctx->sm_count;
-  info->launches_per_run = 1;
+  info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? 2 : 1;
+  info->reserved[0] = ctx->cluster_draw;
   return COS_OK;
 }
 
@@ -1871,7 +2003,9 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   (void)cudaDeviceSynchronize();
   cudaFree(ctx->d_work_counter);
   cudaFree(ctx->d_row_arrivals);
-  cudaFree(ctx->d_first_rej);
+  cudaFree(ctx->d_job_count);
+  cudaFree(ctx->d_jobs);
+  cudaFree(ctx->d_ustats);
   cudaFree(ctx->d_unit_res);
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_drafts);
@@ -1896,7 +2030,7 @@ namespace {
 
 // Scratch of the context-free entry point.  It is part of the library image: every device
 // that loads the library holds these COS_STATIC_SCRATCH_BYTES until the process exits.
-// Layout: [0, 256) work counter | row arrival counters | earliest-rejection words | unit results.
+// Layout: [0, 256) work and job counters | row arrival counters | unit results | job list | unit statistics.
 static __device__ __align__(256) unsigned char g_static_scratch[COS_STATIC_SCRATCH_BYTES];
 
 constexpr int kStaticMaxDevices = 64;
@@ -1942,7 +2076,6 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   cudaError_t e = cudaSetDevice(c.device);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaSetDevice", e);
   KernelFn fn = pick_kernel(c.dtype, mode_of(c));
-  const int cluster = choose_cluster(c);
   if (!g_static_ready[c.device]) {
     // once per device, with that device current: the device address of the built-in array
     void* addr = nullptr;
@@ -1952,38 +2085,32 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     g_static_ready[c.device] = true;
   }
   e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
-  if (e == cudaSuccess && cluster > 8)
+  if (e == cudaSuccess && c.cluster_size > 8)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaFuncSetAttribute", e);
-
-  cudaLaunchConfig_t lc = {};
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = cluster;
-  at[0].val.clusterDim.y = 1;
-  at[0].val.clusterDim.z = 1;
-  lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = kRingBytes;
-  lc.attrs = at;
-  lc.numAttrs = 1;
   int sm_count = 0;
   e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c.device);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaDeviceGetAttribute", e);
-  lc.gridDim = dim3(static_cast<unsigned>(cluster * sm_count), 1, 1);
-  int max_clusters = 0;
-  e = cudaOccupancyMaxActiveClusters(&max_clusters, reinterpret_cast<const void*>(fn), &lc);
+  const int c0 = choose_stream_cluster(c, static_cast<int>(units), sm_count);
+  const int c1 = choose_cluster(c);
+  int mc0 = 0, mc1 = 0;
+  e = query_clusters(fn, c0, sm_count, &mc0);
+  if (e == cudaSuccess) e = query_clusters(fn, c1, sm_count, &mc1);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaOccupancyMaxActiveClusters", e);
-  if (max_clusters < 1) return static_fail(COS_ERR_UNSUPPORTED, "no cluster of the requested size fits on the device");
+  if (mc0 < 1 || mc1 < 1) return static_fail(COS_ERR_UNSUPPORTED, "no cluster of the requested size fits on the device");
 
-  // carve the array; what must start clean is cleared on the caller's stream before the kernel
+  // carve the array; what must start clean is cleared on the caller's stream before the kernels
   unsigned char* basep = g_static_addr[c.device];
   unsigned* d_counter = reinterpret_cast<unsigned*>(basep);
+  int* d_job_count = reinterpret_cast<int*>(basep + 16);
   int* d_arrivals = reinterpret_cast<int*>(basep + 256);
-  int* d_first_rej = d_arrivals + COS_STATIC_MAX_BATCH;
-  int4* d_unit_res = reinterpret_cast<int4*>(basep + 256 + 8 * COS_STATIC_MAX_BATCH);
-  e = cudaMemsetAsync(d_counter, 0, sizeof(unsigned), stream);
+  int4* d_unit_res = reinterpret_cast<int4*>(basep + 256 + 4 * COS_STATIC_MAX_BATCH);
+  int2* d_jobs = reinterpret_cast<int2*>(reinterpret_cast<unsigned char*>(d_unit_res) + 16 * COS_STATIC_MAX_POSITIONS);
+  UnitStats* d_ustats = reinterpret_cast<UnitStats*>(reinterpret_cast<unsigned char*>(d_jobs) +
+                                                      8 * (COS_STATIC_MAX_POSITIONS + COS_STATIC_MAX_BATCH));
+  static_assert(sizeof(UnitStats) == 112, "COS_STATIC_SCRATCH_BYTES assumes 112 bytes of statistics per position");
+  e = cudaMemsetAsync(basep, 0, 256, stream);  // work counter and both job counters
   if (e == cudaSuccess) e = cudaMemsetAsync(d_arrivals, 0, static_cast<size_t>(a->batch) * sizeof(int), stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(d_first_rej, 0x7f, static_cast<size_t>(a->batch) * sizeof(int), stream);
   if (e != cudaSuccess) return cuda_fail(nullptr, "clearing the built-in scratch", e);
 
   KParams p;
@@ -2006,7 +2133,6 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.nsteps = (c.vocab + 32 * E - 1) / (32 * E);
   p.flags = a->flags;
   p.num_units = static_cast<int>(units);
-  p.num_clusters = p.num_units < max_clusters ? p.num_units : max_clusters;
   for (int i = 0; i < COS_MAX_MODELS; ++i) {
     p.w[i] = (i < c.n) ? c.weights[i] : 0.f;
     p.w64[i] = static_cast<double>(p.w[i]);
@@ -2029,12 +2155,24 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.work_counter = d_counter;
   p.work_base = 0;  // the counter was just cleared
   p.row_arrivals = d_arrivals;
-  p.first_rej = d_first_rej;
   p.unit_res = d_unit_res;
+  p.job_count = d_job_count;
+  p.job_reset = d_job_count + 1;
+  p.jobs = d_jobs;
+  p.ustats = d_ustats;
+  p.max_jobs = p.num_units + a->batch;
 
-  lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * cluster, 1, 1);
-  lc.stream = stream;
-  e = cudaLaunchKernelEx(&lc, fn, p);
-  if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch", e);
+  p.stage = 0;
+  p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
+  e = launch_stage(fn, p, c0, stream);
+  if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (stage 0)", e);
+  if (mode_of(c) == kEnsembleSample || mode_of(c) == kLogitSample) {
+    const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
+    const int most = all ? p.max_jobs : a->batch;
+    p.stage = 1;
+    p.num_clusters = most < mc1 ? most : mc1;
+    e = launch_stage(fn, p, c1, stream);
+    if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (stage 1)", e);
+  }
   return COS_OK;
 }
