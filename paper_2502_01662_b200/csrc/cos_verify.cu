@@ -69,8 +69,6 @@ struct KParams {
   int num_units, num_clusters;
   int stage;     // 0: statistics, decisions, row scan (every unit); 1: draw tokens for the listed units
   int max_jobs;  // capacity of the job list
-  int resident;  // stage 1 keeps the block's slice of the unit in shared memory
-  int nv_cap;    // vectors per model reserved for that slice
   float w[COS_MAX_MODELS];
   double w64[COS_MAX_MODELS];
   float cT;       // log2(e) / T in fp32 (T > 0)
@@ -591,12 +589,6 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   const int s_end = static_cast<int>(static_cast<long long>(gwarp + 1) * p.nsteps / G);
   // this block's slice of every row in sweep 1
   const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
-  // stage 1 with a resident slice: the block owns the vectors of its warps' runs
-  const bool res_on = (p.stage == 1) && (p.resident != 0);
-  const int nvec_all = p.V / E;
-  const int rv_lo = static_cast<int>(static_cast<long long>(rank) * kWarps * p.nsteps / G) * 32;
-  const int rv_hi_raw = static_cast<int>(static_cast<long long>(rank + 1) * kWarps * p.nsteps / G) * 32;
-  const int rv_hi = rv_hi_raw < nvec_all ? rv_hi_raw : nvec_all;
 
   const int cluster_id = blockIdx.x / C;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
@@ -1009,16 +1001,6 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         sh.u_smp = word_to_uniform(rnd[1]);
         sh.next = 0;
       }
-      if (res_on) {
-        // the block's slice of all n rows goes to shared memory once; every later pass reads it there
-        for (int i = 0; i < p.n; ++i) {
-          const char* rowb = reinterpret_cast<const char*>(row_of(i));
-          for (int v = rv_lo + tid; v < rv_hi; v += kThreads)
-            cp_async16(&ring[static_cast<size_t>(i) * p.nv_cap + (v - rv_lo)], rowb + static_cast<long long>(v) * 16);
-        }
-        cp_async_commit();
-        cp_async_wait<0>();
-      }
       __syncthreads();
     }
     const int need2 = sh.dec.need2;
@@ -1071,32 +1053,23 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
                 if (e[k] > bt) zb += exp2(static_cast<double>(v[k]) * p.cT64 - dref);
             }
           };
-          if (res_on) {
-            for (int v = rv_lo + tid; v < rv_hi; v += kThreads) {
+          int v = sl.v_lo + tid;
+          for (; v + 3 * kThreads < sl.v_hi; v += 4 * kThreads) {
+            uint4 raw[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) raw[u] = ldg_stream16(rowb + static_cast<long long>(v + u * kThreads) * 16);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
               float x[E];
-              uint4 raw = ring[static_cast<size_t>(i) * p.nv_cap + (v - rv_lo)];
-              Elem<DT>::unpack(raw, x);
+              Elem<DT>::unpack(raw[u], x);
               eat(x);
             }
-          } else {
-            int v = sl.v_lo + tid;
-            for (; v + 3 * kThreads < sl.v_hi; v += 4 * kThreads) {
-              uint4 raw[4];
-#pragma unroll
-              for (int u = 0; u < 4; ++u) raw[u] = ldg_stream16(rowb + static_cast<long long>(v + u * kThreads) * 16);
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                float x[E];
-                Elem<DT>::unpack(raw[u], x);
-                eat(x);
-              }
-            }
-            for (; v < sl.v_hi; v += kThreads) {
-              float x[E];
-              uint4 raw = ldg_stream16(rowb + static_cast<long long>(v) * 16);
-              Elem<DT>::unpack(raw, x);
-              eat(x);
-            }
+          }
+          for (; v < sl.v_hi; v += kThreads) {
+            float x[E];
+            uint4 raw = ldg_stream16(rowb + static_cast<long long>(v) * 16);
+            Elem<DT>::unpack(raw, x);
+            eat(x);
           }
           for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
             const float x = Elem<DT>::load1(row, e);
@@ -1125,8 +1098,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e)), cd);
           return exp2(cd * p.cT64 - dref_c);
         };
-        const int a_lo = res_on ? rv_lo : sl.v_lo, a_hi = res_on ? rv_hi : sl.v_hi;
-        for (int v = a_lo + tid; v < a_hi; v += kThreads) {
+        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
           float cmb[E], vq[E], ve[E];
 #pragma unroll
           for (int k = 0; k < E; ++k) {
@@ -1136,15 +1108,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           }
           for (int i = 0; i < p.n; i += 2) {
             const bool two = (i + 1 < p.n);
-            uint4 ra, rb;
-            if (res_on) {
-              ra = ring[static_cast<size_t>(i) * p.nv_cap + (v - rv_lo)];
-              rb = two ? ring[static_cast<size_t>(i + 1) * p.nv_cap + (v - rv_lo)] : ra;
-            } else {
-              ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
-              rb = ra;
-              if (two) rb = ldg_stream16(reinterpret_cast<const char*>(row_of(i + 1)) + static_cast<long long>(v) * 16);
-            }
+            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
+            uint4 rb = ra;
+            if (two) rb = ldg_stream16(reinterpret_cast<const char*>(row_of(i + 1)) + static_cast<long long>(v) * 16);
             float va[E], vb[E];
             Elem<DT>::unpack(ra, va);
             Elem<DT>::unpack(rb, vb);
@@ -1231,12 +1197,11 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       // ---- 2b: token masses.  mass32[k] is max(0, r - q) (or r) of the lane's k-th token in fp32;
       // tokens holding more than 2^-10 of any normaliser are flagged in `bigbits`, get mass32 = 0
       // and are evaluated by big_mass() in fp64 from the stored logits.
-      // `staged` points at this lane's vector of model 0 in shared memory (models `stride` vectors apart), or is null.
-      auto chunk_mass = [&](int e0, bool use_r, bool dump, float (&mass32)[E], unsigned& bigbits, const uint4* staged,
-                            int stride) {
+      // `staged` points at this lane's staged vector of model 0 (models 32 vectors apart), or is null.
+      auto chunk_mass = [&](int e0, bool use_r, bool dump, float (&mass32)[E], unsigned& bigbits, const uint4* staged) {
         auto fetch = [&](int i, float (&v)[E]) {
           if (staged != nullptr) {
-            uint4 raw = staged[static_cast<size_t>(i) * stride];
+            uint4 raw = staged[i * 32];
             Elem<DT>::unpack(raw, v);
           } else {
             load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
@@ -1340,7 +1305,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
 
       // running totals are recorded every gsz steps; the search below re-reads one such group
       const int nst = s_end - s_begin;
-      const int gsz = (nst + kRec - 1) / kRec > 1 ? (nst + kRec - 1) / kRec : 1;
+      const int gsz = (nst + kRec - 1) / kRec > 4 ? (nst + kRec - 1) / kRec : 4;
       const int ngrp = (nst + gsz - 1) / gsz;
       for (int attempt = 0; attempt < 2; ++attempt) {
         const bool dump = (p.dump_r != nullptr) && attempt == 0;
@@ -1350,7 +1315,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         // keeps several loads in flight although it consumes its run in token order
         const int depth = (p.n <= 2) ? 4 : (p.n <= 4 ? 2 : 1);
         const int nfull = vec_ok ? p.V / (32 * E) : 0;
-        const int fe = res_on ? s_begin : ((s_end < nfull) ? s_end : nfull);  // steps [s_begin, fe) go through the ring
+        const int fe = (s_end < nfull) ? s_end : nfull;  // steps [s_begin, fe) go through the ring
         uint4* myring = ring + static_cast<size_t>(warp) * kRingVecs * 32 + lane;
         auto stage = [&](int s) {  // issue the loads of step s into its ring slot
           const int slot = ((s - s_begin) % depth) * p.n;
@@ -1366,10 +1331,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           float mass32[E];
           unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
-          if (res_on) {
-            const int vi = s * 32 + lane;
-            chunk_mass(e0, from_r, dump, mass32, bigbits, (vi < rv_hi) ? &ring[vi - rv_lo] : nullptr, p.nv_cap);
-          } else if (s < fe) {
+          if (s < fe) {
             if (depth == 4)
               cp_async_wait<3>();
             else if (depth == 2)
@@ -1377,11 +1339,11 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             else
               cp_async_wait<0>();
             const int slot = ((s - s_begin) % depth) * p.n;
-            chunk_mass(e0, from_r, dump, mass32, bigbits, &myring[slot * 32], 32);
+            chunk_mass(e0, from_r, dump, mass32, bigbits, &myring[slot * 32]);
             if (s + depth < fe) stage(s + depth);
             cp_async_commit();
           } else {
-            chunk_mass(e0, from_r, dump, mass32, bigbits, nullptr, 0);
+            chunk_mass(e0, from_r, dump, mass32, bigbits, nullptr);
           }
           lacc += lane_mass(e0, mass32, bigbits, from_r, dump);
           const int done = s - s_begin + 1;
@@ -1495,8 +1457,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           float mass32[E];
           unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
-          chunk_mass(e0, from_r, false, mass32, bigbits,
-                     (res_on && (s * 32 + lane) < rv_hi) ? &ring[s * 32 + lane - rv_lo] : nullptr, p.nv_cap);
+          chunk_mass(e0, from_r, false, mass32, bigbits, nullptr);
           // per-token masses of this lane in fp64 (big tokens from their fp64 evaluation)
           double m64[E];
 #pragma unroll
@@ -1584,9 +1545,6 @@ thread_local std::string g_create_error;
 struct cos_verify_ctx {
   cos_verify_config cfg;
   int cluster_draw;     // blocks per unit in stage 1
-  int draw_nv_cap;      // > 0: stage 1 keeps the slice in shared memory, this many vectors per model
-  int draw_smem;        // dynamic shared memory of a resident stage 1
-  int draw_max_clusters;
   int max_clusters[5];  // resident clusters for cluster sizes 1, 2, 4, 8, 16 (0 = not available)
   int sm_count;
   unsigned work_base;
@@ -1689,19 +1647,6 @@ int choose_cluster(const cos_verify_config& c) {
 
 int log2i(int c) { return c >= 16 ? 4 : (c >= 8 ? 3 : (c >= 4 ? 2 : (c >= 2 ? 1 : 0))); }
 
-// Stage 1 keeps a block's slice of the unit in shared memory when it fits: vectors reserved per model
-// (0 = does not fit, stage 1 then streams from global memory).
-constexpr int kResidentMaxBytes = 200 * 1024;
-int resident_nv_cap(const cos_verify_config& c, int cluster) {
-  const int E = entries_per_vec(c.dtype);
-  if (c.vocab % E != 0) return 0;
-  const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
-  const int G = cluster * kWarps;
-  const int cap = ((nsteps * kWarps + G - 1) / G + 1) * 32;
-  if (static_cast<long long>(cap) * 16 * c.n > kResidentMaxBytes) return 0;
-  return cap;
-}
-
 // Stage 0 streams best with one block per unit (long contiguous reads, no cluster barrier);
 // more blocks per unit only when there are too few units to occupy the device.
 int choose_stream_cluster(const cos_verify_config& c, int units, int sm_count) {
@@ -1712,23 +1657,11 @@ int choose_stream_cluster(const cos_verify_config& c, int units, int sm_count) {
   return cs;
 }
 
-// The dynamic shared memory limit of a kernel is only ever raised: contexts and the
-// context-free entry point share the kernels, and a later, smaller request must not undo
-// what an earlier context relies on.
-int g_smem_limit[64][2][4];
-cudaError_t raise_dynamic_smem(KernelFn fn, int device, int dtype, int mode, int bytes) {
-  if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
-  if (g_smem_limit[device][dtype][mode] >= bytes) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  if (e == cudaSuccess) g_smem_limit[device][dtype][mode] = bytes;
-  return e;
-}
-
-cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int smem, int* out) {
+cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int* out) {
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(cluster * sm_count, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = smem;
+  lc.dynamicSmemBytes = kRingBytes;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = cluster;
@@ -1739,11 +1672,11 @@ cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int smem, int
   return cudaOccupancyMaxActiveClusters(out, reinterpret_cast<const void*>(fn), &lc);
 }
 
-cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, int smem, cudaStream_t stream) {
+cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, cudaStream_t stream) {
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * cluster, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = smem;
+  lc.dynamicSmemBytes = kRingBytes;
   lc.stream = stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
@@ -1803,10 +1736,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   }
   ctx->sm_count = prop.multiProcessorCount;
   KernelFn fn = pick_kernel(config->dtype, mode_of(*config));
-  ctx->draw_nv_cap = resident_nv_cap(*config, ctx->cluster_draw);
-  ctx->draw_smem = ctx->draw_nv_cap > 0 ? ctx->draw_nv_cap * 16 * config->n : kRingBytes;
-  if (ctx->draw_smem < kRingBytes) ctx->draw_smem = kRingBytes;
-  e = raise_dynamic_smem(fn, config->device, config->dtype, mode_of(*config), ctx->draw_smem);
+  e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
   if (e != cudaSuccess) {
     delete ctx;
     return cuda_fail(nullptr, "cudaFuncSetAttribute(shared memory)", e);
@@ -1823,23 +1753,12 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     ctx->max_clusters[k] = 0;
     if (cs == 16 && config->cluster_size != 16) continue;
     int nc = 0;
-    e = query_clusters(fn, cs, ctx->sm_count, kRingBytes, &nc);
+    e = query_clusters(fn, cs, ctx->sm_count, &nc);
     if (e != cudaSuccess) {
       (void)cudaGetLastError();
       nc = 0;
     }
     ctx->max_clusters[k] = nc;
-  }
-  ctx->draw_max_clusters = 0;
-  if (ctx->draw_nv_cap > 0) {
-    int nc = 0;
-    e = query_clusters(fn, ctx->cluster_draw, ctx->sm_count, ctx->draw_smem, &nc);
-    if (e != cudaSuccess || nc < 1) {
-      (void)cudaGetLastError();
-      ctx->draw_nv_cap = 0;  // fall back to streaming
-    } else {
-      ctx->draw_max_clusters = nc;
-    }
   }
   {
     const int need = config->cluster_size > 0 ? config->cluster_size : 1;
@@ -1985,19 +1904,17 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.stage = 0;
   p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
   ctx->scratch_dirty = true;  // cleared below once the launches are known to be queued
-  e = launch_stage(fn, p, c0, kRingBytes, stream);
+  e = launch_stage(fn, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (draws) {
     // stage 1: the units listed by stage 0 (one per row, or all of them under the test hooks)
     const int c1 = ctx->cluster_draw;
-    p.resident = (ctx->draw_nv_cap > 0 && p.vec_ok) ? 1 : 0;
-    p.nv_cap = ctx->draw_nv_cap;
-    const int mc1 = p.resident ? ctx->draw_max_clusters : ctx->max_clusters[log2i(c1)];
+    const int mc1 = ctx->max_clusters[log2i(c1)];
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
     p.stage = 1;
     p.num_clusters = most < mc1 ? most : mc1;
-    e = launch_stage(fn, p, c1, p.resident ? ctx->draw_smem : kRingBytes, stream);
+    e = launch_stage(fn, p, c1, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 1)", e);
   }
   // every cluster starts on the unit of its own index and draws once after each unit it finishes,
@@ -2167,7 +2084,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     g_static_addr[c.device] = static_cast<unsigned char*>(addr);
     g_static_ready[c.device] = true;
   }
-  e = raise_dynamic_smem(fn, c.device, c.dtype, mode_of(c), kRingBytes);
+  e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
   if (e == cudaSuccess && c.cluster_size > 8)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaFuncSetAttribute", e);
@@ -2177,8 +2094,8 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   const int c0 = choose_stream_cluster(c, static_cast<int>(units), sm_count);
   const int c1 = choose_cluster(c);
   int mc0 = 0, mc1 = 0;
-  e = query_clusters(fn, c0, sm_count, kRingBytes, &mc0);
-  if (e == cudaSuccess) e = query_clusters(fn, c1, sm_count, kRingBytes, &mc1);
+  e = query_clusters(fn, c0, sm_count, &mc0);
+  if (e == cudaSuccess) e = query_clusters(fn, c1, sm_count, &mc1);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaOccupancyMaxActiveClusters", e);
   if (mc0 < 1 || mc1 < 1) return static_fail(COS_ERR_UNSUPPORTED, "no cluster of the requested size fits on the device");
 
@@ -2247,14 +2164,14 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
 
   p.stage = 0;
   p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
-  e = launch_stage(fn, p, c0, kRingBytes, stream);
+  e = launch_stage(fn, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (stage 0)", e);
   if (mode_of(c) == kEnsembleSample || mode_of(c) == kLogitSample) {
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
     p.stage = 1;
     p.num_clusters = most < mc1 ? most : mc1;
-    e = launch_stage(fn, p, c1, kRingBytes, stream);
+    e = launch_stage(fn, p, c1, stream);
     if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (stage 1)", e);
   }
   return COS_OK;
