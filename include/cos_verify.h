@@ -108,7 +108,7 @@ typedef struct {
   int32_t threads_per_block;
   int32_t max_clusters;      /* clusters that can be resident at once on the device                   */
   int32_t sm_count;
-  int32_t launches_per_run;  /* kernels cos_verify_run enqueues per call (2 when T > 0, else 1)        */
+  int32_t launches_per_run;  /* kernels cos_verify_run enqueues per call (4 when T > 0, else 1)        */
   int32_t reserved[3];
 } cos_verify_info;
 
@@ -149,8 +149,8 @@ cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args,
  * the whole device to its own memory pool, or a serving loop in which the device-wide
  * synchronisation that cudaMalloc / cudaFree imply would stall every other stream.  This call
  * needs no context: the kernels' scratch (work and job counters, per-row arrival counters,
- * per-position results and statistics, the list of positions that draw a token) lives in an
- * array that is part of the
+ * per-position results, statistics and partial sums, the list of positions that draw a token)
+ * lives in an array that is part of the
  * library image, COS_STATIC_SCRATCH_BYTES long, resident on every device that loads the
  * library until the process exits.  The call performs no cudaMalloc, cudaFree or other
  * device allocation; `config` is read on every call (max_batch and host_staging are ignored).
@@ -170,9 +170,10 @@ cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args,
  */
 #define COS_STATIC_MAX_BATCH 1024
 #define COS_STATIC_MAX_POSITIONS 8192
-#define COS_STATIC_SCRATCH_BYTES \
-  (256 + 4 * COS_STATIC_MAX_BATCH + 16 * COS_STATIC_MAX_POSITIONS + 8 * (COS_STATIC_MAX_POSITIONS + COS_STATIC_MAX_BATCH) + \
-   112 * COS_STATIC_MAX_POSITIONS)
+#define COS_STATIC_SCRATCH_BYTES                                                                          \
+  (256 + 4 * COS_STATIC_MAX_BATCH + 16 * COS_STATIC_MAX_POSITIONS +                                      \
+   8 * (COS_STATIC_MAX_POSITIONS + COS_STATIC_MAX_BATCH) + 112 * COS_STATIC_MAX_POSITIONS +              \
+   8 * 8 * COS_STATIC_MAX_POSITIONS + 8 * 16 * COS_STATIC_MAX_POSITIONS + 8 * 16 * 16 * COS_STATIC_MAX_BATCH)
 cos_status cos_verify_run_static(const cos_verify_config* config, const cos_verify_args* args, void* cuda_stream);
 
 /* Launch geometry chosen at creation. */

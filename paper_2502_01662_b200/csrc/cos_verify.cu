@@ -40,11 +40,12 @@ namespace {
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxSlots = COS_MAX_MODELS + 2;
-constexpr int kMaxCluster = 16;
 constexpr int kNoReject = 0x7fffffff;
 constexpr double kBigShare = 1.0 / 1024.0;  // probabilities above 2^-10 get fp64 treatment in sweep 2
 constexpr int kRingVecs = 8;                 // 16-byte vectors per lane staged ahead in sweep 2 (4 KB per warp)
 constexpr int kRingBytes = kWarps * kRingVecs * 32 * 16;
+constexpr int kRecG = 16;                    // running totals per warp kept in global memory between the drawing stages
+constexpr int kMaxParts = 16;                // blocks that share one unit in the drawing stages
 constexpr int kRec = 64;                     // running totals recorded per warp in sweep 2
 
 enum Mode { kEnsembleSample = 0, kLogitSample = 1, kEnsembleGreedy = 2, kLogitGreedy = 3 };
@@ -67,7 +68,9 @@ struct KParams {
   int nsteps;   // ceil(V / (32 * E))
   int flags;
   int num_units, num_clusters;
-  int stage;     // 0: statistics, decisions, row scan (every unit); 1: draw tokens for the listed units
+  int stage;     // 0: statistics, decisions, row scan (every unit); then for the listed units only:
+                 // 1: normalisers again with fp64 care, 2: token masses and their running totals, 3: locate the token
+  int parts;     // blocks that share one unit in stages 1 and 2
   int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
   double w64[COS_MAX_MODELS];
@@ -89,7 +92,10 @@ struct KParams {
   int* job_count;          // units that stage 1 must process (this run's counter)
   int* job_reset;          // the other run parity's counter, cleared by stage 0
   int2* jobs;              // x = b * P + j, y = 1 if the drawn token is the row's output at position j
-  UnitStats* ustats;       // [B*P]: merged statistics of sweep 1, read back by stage 1
+  UnitStats* ustats;       // [B*P]: merged statistics of sweep 1, read back by the later stages
+  double* zpart;           // [B*P][parts][8]: stage 1's partial normalisers
+  double* wtotg;           // [B*P][parts*16]: stage 2's mass of every warp run
+  double* srung;           // [B][parts*16][kRecG]: running totals inside the runs of the row's drawing unit
 };
 
 // ------------------------------------------------------------------------------------
@@ -252,6 +258,8 @@ struct Shared {
   double wtot[kWarps];        // this block's per-warp totals of sweep 2
   double wincl[kWarps];       // their running sum
   double srun[kWarps][kRec];  // a warp's running total after each group of steps
+  double gw[kMaxParts * kWarps];  // stage 3: mass of every warp run of the unit
+  int win_g;
   SoftPart fsoft[kMaxSlots];  // merged over the cluster
   ArgPart farg[kMaxSlots];
   double pdraft[kMaxSlots];   // probability of the draft token under each merged softmax
@@ -572,8 +580,11 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   constexpr int E = Elem<DT>::E;
   constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
   cg::cluster_group cluster = cg::this_cluster();
-  const int C = cluster.num_blocks();
-  const int rank = cluster.block_rank();
+  // stage 0 shares a unit among the blocks of a cluster; stages 1 and 2 among `parts` independent
+  // blocks (they meet only through global memory between launches); stage 3 uses one block per unit
+  const int lparts = (p.stage == 1 || p.stage == 2) ? p.parts : 1;  // blocks per unit in this launch
+  const int C = (p.stage == 0) ? static_cast<int>(cluster.num_blocks()) : p.parts;
+  const int rank = (p.stage == 0) ? static_cast<int>(cluster.block_rank()) : static_cast<int>(blockIdx.x % lparts);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gwarp = rank * kWarps + warp, G = C * kWarps;
   __shared__ Shared sh;
@@ -590,7 +601,8 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   // this block's slice of every row in sweep 1
   const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
 
-  const int cluster_id = blockIdx.x / C;
+  const int cluster_id = (p.stage == 0) ? blockIdx.x / C : blockIdx.x / lparts;
+  const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
   if (p.stage == 0) {
     if (blockIdx.x == 0 && tid == 0) *p.job_reset = 0;  // the list of the next run starts empty
@@ -605,7 +617,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       j = unit / p.B;  // earlier positions of every row come first
       b = unit % p.B;
     } else {
-      const int job = cluster_id + job_it * p.num_clusters;
+      const int job = cluster_id + job_it * job_stride;
       if (job >= njobs) break;
       const int2 jb = p.jobs[job];
       ++job_it;
@@ -980,7 +992,12 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       if (tid < nkeep) {
         sh.fsoft[tid].s = p.ustats[uidx].s[tid];
         sh.fsoft[tid].ref = p.ustats[uidx].ref[tid];
-        sh.big_thr[tid] = static_cast<float>(sh.fsoft[tid].s * kBigShare);
+        sh.big_thr[tid] = static_cast<float>(sh.fsoft[tid].s * kBigShare);  // from the first estimate, in every stage
+        if (p.stage >= 2) {
+          double z = 0.0;
+          for (int q = 0; q < p.parts; ++q) z += p.zpart[(static_cast<size_t>(uidx) * p.parts + q) * 8 + tid];
+          sh.fsoft[tid].s = z;
+        }
       }
       if (tid == 32) {
         const int4 ur = __ldcg(&p.unit_res[uidx]);
@@ -1019,16 +1036,14 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
     }
 
     // ================================ sweep 2: draw a token ================================
-    bool published = false;
     if (kSample && need2) {
-      bool from_r = is_bonus;  // the bonus is drawn from r itself; a rejected draft from max(0, r - q)
       const float thr = masked ? sh.thr32 : -INFINITY;
-      double S_report = kNaN;
       const int nsoft2 = (MODE == kEnsembleSample) ? p.n : 2;
 
       // ---- 2a: normalisers again, now that the references are known: terms holding more
       // than 2^-14 of a normaliser are evaluated in fp64 and kept out of the fp32 sums, so
       // a dominant token neither absorbs the small ones nor carries the fast exp's error
+      if (p.stage == 1) {
       if (MODE == kEnsembleSample) {
         for (int i = 0; i < p.n; ++i) {
           const void* row = row_of(i);
@@ -1180,7 +1195,15 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
         }
       }
-      cluster_merge(sh, cluster, phase, nsoft2, 0, 0);  // refined normalisers replace sh.fsoft[*].s
+      // this block's share of every normaliser goes to global memory; stage 2 adds the shares up
+      __syncthreads();
+      if (warp < nsoft2) {
+        float ref = (lane < kWarps) ? sh.wsoft[lane][warp].ref : -INFINITY;
+        double sum = (lane < kWarps) ? sh.wsoft[lane][warp].s : 0.0;
+        SoftPart o = warp_reduce_soft(ref, sum);
+        if (lane == 0) p.zpart[(static_cast<size_t>(uidx) * p.parts + rank) * 8 + warp] = o.s;
+      }
+      } else {
       if (MODE == kEnsembleSample && tid < p.n) {
         // r - q = sum_i (w_i/Z_i - [i = proposer]/Z_i) e_i, and r = sum_i (w_i/Z_i) e_i
         const double a = p.w64[tid] / sh.fsoft[tid].s;
@@ -1303,31 +1326,27 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         return own;
       };
 
-      // running totals are recorded every gsz steps; the search below re-reads one such group
-      const int nst = s_end - s_begin;
-      const int gsz = (nst + kRec - 1) / kRec > 4 ? (nst + kRec - 1) / kRec : 4;
-      const int ngrp = (nst + gsz - 1) / gsz;
-      for (int attempt = 0; attempt < 2; ++attempt) {
-        const bool dump = (p.dump_r != nullptr) && attempt == 0;
-        double wrun = 0.0;   // this warp's total, accumulated group by group
-        double lacc = 0.0;   // this lane's mass within the current group
-        // vectors of the coming steps are staged in shared memory with cp.async so that a warp
-        // keeps several loads in flight although it consumes its run in token order
+      uint4* myring = ring + static_cast<size_t>(warp) * kRingVecs * 32 + lane;
+      // Mass of one warp run [sb, se) in token order; the running total after every gszv steps goes to
+      // rec[] (lane 0 writes; rec may be null).  Vectors of the coming steps are staged in shared memory
+      // with cp.async so that a warp keeps several loads in flight although it consumes its run in order.
+      auto run_totals = [&](int sb, int se, int gszv, bool use_r, bool dump, double* rec) -> double {
+        double wrun = 0.0;  // the run's total, accumulated group by group
+        double lacc = 0.0;  // this lane's mass within the current group
         const int depth = (p.n <= 2) ? 4 : (p.n <= 4 ? 2 : 1);
         const int nfull = vec_ok ? p.V / (32 * E) : 0;
-        const int fe = (s_end < nfull) ? s_end : nfull;  // steps [s_begin, fe) go through the ring
-        uint4* myring = ring + static_cast<size_t>(warp) * kRingVecs * 32 + lane;
-        auto stage = [&](int s) {  // issue the loads of step s into its ring slot
-          const int slot = ((s - s_begin) % depth) * p.n;
+        const int fe = (se < nfull) ? se : nfull;  // steps [sb, fe) go through the ring
+        auto stage_in = [&](int s) {  // issue the loads of step s into its ring slot
+          const int slot = ((s - sb) % depth) * p.n;
           for (int i = 0; i < p.n; ++i)
             cp_async16(&myring[(slot + i) * 32],
                        reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(s * 32 + lane) * 16);
         };
         for (int t = 0; t < depth; ++t) {
-          if (s_begin + t < fe) stage(s_begin + t);
+          if (sb + t < fe) stage_in(sb + t);
           cp_async_commit();
         }
-        for (int s = s_begin; s < s_end; ++s) {
+        for (int s = sb; s < se; ++s) {
           float mass32[E];
           unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
@@ -1338,126 +1357,55 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               cp_async_wait<1>();
             else
               cp_async_wait<0>();
-            const int slot = ((s - s_begin) % depth) * p.n;
-            chunk_mass(e0, from_r, dump, mass32, bigbits, &myring[slot * 32]);
-            if (s + depth < fe) stage(s + depth);
+            const int slot = ((s - sb) % depth) * p.n;
+            chunk_mass(e0, use_r, dump, mass32, bigbits, &myring[slot * 32]);
+            if (s + depth < fe) stage_in(s + depth);
             cp_async_commit();
           } else {
-            chunk_mass(e0, from_r, dump, mass32, bigbits, nullptr);
+            chunk_mass(e0, use_r, dump, mass32, bigbits, nullptr);
           }
-          lacc += lane_mass(e0, mass32, bigbits, from_r, dump);
-          const int done = s - s_begin + 1;
-          if (done % gsz == 0 || s + 1 == s_end) {
+          lacc += lane_mass(e0, mass32, bigbits, use_r, dump);
+          const int done = s - sb + 1;
+          if (done % gszv == 0 || s + 1 == se) {
             double t = lacc;
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
             wrun += t;
-            if (lane == 0) sh.srun[warp][(done - 1) / gsz] = wrun;
+            if (lane == 0 && rec != nullptr) rec[(done - 1) / gszv] = wrun;
             lacc = 0.0;
           }
         }
         cp_async_wait<0>();
-        if (lane == 0) sh.wtot[warp] = wrun;
-        __syncthreads();
-        if (tid == 0) {
-          double run = 0.0;
-          for (int w = 0; w < kWarps; ++w) {
-            run += sh.wtot[w];
-            sh.wincl[w] = run;
-          }
-          sh.x[phase & 1].cta_total = run;
-        }
-        cluster.sync();
-        if (tid == 0) {
-          double tot[kMaxCluster];
-          for (int r = 0; r < C; ++r) tot[r] = cluster.map_shared_rank(&sh.x[phase & 1], r)->cta_total;
-          double S = 0.0;
-          for (int r = 0; r < C; ++r) S += tot[r];
-          const double target = sh.u_smp * S;
-          double cp = 0.0;
-          int wr = -1, ww = -1;
-          double wbase = 0.0;
-          for (int r = 0; r < C && wr < 0; ++r) {
-            if (cp + tot[r] >= target && tot[r] > 0.0) {
-              wr = r;
-              wbase = cp;
-            }
-            cp += tot[r];
-          }
-          if (wr < 0 && S > 0.0) {  // rounding corner: last block with mass
-            cp = 0.0;
-            for (int r = 0; r < C; ++r) {
-              if (tot[r] > 0.0) {
-                wr = r;
-                wbase = cp;
-              }
-              cp += tot[r];
-            }
-          }
-          if (wr == rank) {
-            for (int w = 0; w < kWarps; ++w) {
-              if (wbase + sh.wincl[w] >= target && sh.wtot[w] > 0.0) {
-                ww = w;
-                break;
-              }
-            }
-            if (ww < 0) {  // rounding corner: last warp with mass
-              for (int w = kWarps - 1; w >= 0; --w)
-                if (sh.wtot[w] > 0.0) {
-                  ww = w;
-                  break;
-                }
-            }
-          }
-          sh.dec.S = S;
-          sh.target = target;
-          sh.base = wbase;
-          sh.win_rank = (S > 0.0) ? wr : -2;
-          sh.win_warp = ww;
-        }
-        __syncthreads();
-        ++phase;
-        if (attempt == 0 && !from_r) S_report = sh.dec.S;
-        if (sh.win_rank == -2 && !from_r) {
-          // no residual mass although a token is needed: draw from r instead
-          from_r = true;
-          __syncthreads();
-          if (tid == 0 && !sh.dec.accept) sh.dec.status |= COS_ROW_RESIDUAL_EMPTY;
-          __syncthreads();
-          continue;
-        }
-        break;
-      }
-
-      // the winning warp finds the group of steps from the recorded totals, then walks that group
-      // again step by step with an fp64 prefix over the lanes and a walk over the lane's tokens
-      if (sh.win_rank == rank && sh.win_warp == warp) {
-        const double target = sh.target;
-        const double lex = (warp > 0) ? sh.wincl[warp - 1] : 0.0;
-        const double cbase = sh.base;
+        return wrun;
+      };
+      // One warp finds the token inside the run [sb, se): `base` is the mass before the run, rec[] its
+      // recorded running totals.  It picks the group of steps from rec[], walks that group again step
+      // by step with an fp64 prefix over the lanes, then walks the lane's tokens.
+      auto walk = [&](int sb, int se, int gszv, double base, const double* rec, double target, bool use_r) -> int {
+        const int ngrp = (se - sb + gszv - 1) / gszv;
         int grp = -1;
         for (int g0 = 0; g0 < ngrp && grp < 0; g0 += 32) {
           const int g = g0 + lane;
-          const double prev = (g > 0 && g < ngrp) ? sh.srun[warp][g - 1] : 0.0;
-          const bool ok = (g < ngrp) && (sh.srun[warp][g < ngrp ? g : 0] > prev) &&
-                          (cbase + (lex + sh.srun[warp][g < ngrp ? g : 0]) >= target);
+          const double cur = (g < ngrp) ? rec[g] : 0.0;
+          const double prev = (g > 0 && g < ngrp) ? rec[g - 1] : 0.0;
+          const bool ok = (g < ngrp) && (cur > prev) && (base + cur >= target);
           const unsigned m = __ballot_sync(0xffffffffu, ok);
           if (m) grp = g0 + __ffs(m) - 1;
         }
         if (grp < 0) {  // rounding corner: last group with mass
           for (int g = ngrp - 1; g >= 0 && grp < 0; --g)
-            if (sh.srun[warp][g] > (g > 0 ? sh.srun[warp][g - 1] : 0.0)) grp = g;
+            if (rec[g] > (g > 0 ? rec[g - 1] : 0.0)) grp = g;
           if (grp < 0) grp = 0;
         }
-        double R = (grp > 0) ? sh.srun[warp][grp - 1] : 0.0;
+        double R = (grp > 0) ? rec[grp - 1] : 0.0;
         int token = -1, last_pos = -1;
-        const int rs_begin = s_begin + grp * gsz;
-        const int rs_end = (rs_begin + gsz < s_end) ? rs_begin + gsz : s_end;
+        const int rs_begin = sb + grp * gszv;
+        const int rs_end = (rs_begin + gszv < se) ? rs_begin + gszv : se;
         for (int s = rs_begin; s < rs_end && token < 0; ++s) {
           float mass32[E];
           unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
-          chunk_mass(e0, from_r, false, mass32, bigbits, nullptr);
+          chunk_mass(e0, use_r, false, mass32, bigbits, nullptr);
           // per-token masses of this lane in fp64 (big tokens from their fp64 evaluation)
           double m64[E];
 #pragma unroll
@@ -1465,9 +1413,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           if (bigbits) {
 #pragma unroll
             for (int k = 0; k < E; ++k)
-              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, from_r, false);
+              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, false);
           }
-          const double own = lane_mass(e0, mass32, bigbits, from_r, false);
+          const double own = lane_mass(e0, mass32, bigbits, use_r, false);
           double inc = own;
 #pragma unroll
           for (int d = 1; d < 32; d <<= 1) {
@@ -1478,7 +1426,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           if (lane == 0) excl = 0.0;
           const double incl = excl + own;
           const double step_total = shfl_double(incl, 31);
-          const bool hit = (own > 0.0) && (cbase + (lex + (R + incl)) >= target);
+          const bool hit = (own > 0.0) && (base + (R + incl) >= target);
           unsigned hits = __ballot_sync(0xffffffffu, hit);
           unsigned pos_lanes = __ballot_sync(0xffffffffu, own > 0.0);
           const bool last_chance = (s + 1 == rs_end);
@@ -1493,7 +1441,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
                 part += m64[k];
                 if (m64[k] > 0.0) {
                   lastk = k;
-                  if (found < 0 && cbase + (lex + (R + (excl + part))) >= target) found = e0 + k;
+                  if (found < 0 && base + (R + (excl + part)) >= target) found = e0 + k;
                 }
               }
               if (found < 0) found = e0 + lastk;
@@ -1509,27 +1457,93 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           }
           R += step_total;
         }
-        if (token < 0) token = last_pos;
-        if (lane == 0) {
-          // stage 1 result: the row's token at its first rejection (or bonus), and the residual mass
-          if (emit) {
-            p.out_tokens[uidx] = token;
-            if (sh.dec.status & COS_ROW_RESIDUAL_EMPTY) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_RESIDUAL_EMPTY));
+        return (token < 0) ? last_pos : token;
+      };
+      // sequential sums over the runs in token order: picks the first run whose inclusive sum reaches
+      // u * S and has mass; thread 0 only.  Results in sh.dec.S, sh.target, sh.base, sh.win_g (-1: no mass).
+      auto pick_run = [&](const double* tot, int count) {
+        double S = 0.0;
+        for (int g = 0; g < count; ++g) S += tot[g];
+        const double target = sh.u_smp * S;
+        double run = 0.0, wbase = 0.0;
+        int win = -1;
+        for (int g = 0; g < count && win < 0; ++g) {
+          if (tot[g] > 0.0 && run + tot[g] >= target) {
+            win = g;
+            wbase = run;
           }
-          if (p.diag) p.diag[static_cast<long long>(uidx) * 4 + 3] = static_cast<float>(S_report);
+          run += tot[g];
+        }
+        if (win < 0 && S > 0.0) {  // rounding corner: last run with mass
+          run = 0.0;
+          for (int g = 0; g < count; ++g) {
+            if (tot[g] > 0.0) {
+              win = g;
+              wbase = run;
+            }
+            run += tot[g];
+          }
+        }
+        sh.dec.S = S;
+        sh.target = target;
+        sh.base = wbase;
+        sh.win_g = (S > 0.0) ? win : -1;
+      };
+      auto run_gsz = [&](int nst, int nrec) { return (nst + nrec - 1) / nrec > 1 ? (nst + nrec - 1) / nrec : 1; };
+
+      if (p.stage == 2) {
+        // ---- masses of this block's runs, for stage 3 to add up and search
+        const int gszv = run_gsz(s_end - s_begin, kRecG);
+        double* rec = emit ? p.srung + (static_cast<size_t>(b) * G + gwarp) * kRecG : nullptr;
+        const double t = run_totals(s_begin, s_end, gszv, is_bonus, p.dump_r != nullptr, rec);
+        if (lane == 0) p.wtotg[static_cast<size_t>(uidx) * G + gwarp] = t;
+      } else {
+        // ---- stage 3, one block per unit: add the runs up, find the run, walk it
+        for (int g = tid; g < G; g += kThreads) sh.gw[g] = p.wtotg[static_cast<size_t>(uidx) * G + g];
+        __syncthreads();
+        if (tid == 0) pick_run(sh.gw, G);
+        __syncthreads();
+        // the residual mass S (Eq. 7: 1 - alpha) is reported wherever it was computed
+        if (tid == 0 && p.diag) p.diag[static_cast<long long>(uidx) * 4 + 3] = is_bonus ? __int_as_float(0x7fc00000) : static_cast<float>(sh.dec.S);
+        if (sh.win_g >= 0) {
+          if (emit && warp == 0) {
+            const int g = sh.win_g;
+            const int sb = static_cast<int>(static_cast<long long>(g) * p.nsteps / G);
+            const int se = static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
+            const int token = walk(sb, se, run_gsz(se - sb, kRecG), sh.base,
+                                   p.srung + (static_cast<size_t>(b) * G + g) * kRecG, sh.target, is_bonus);
+            if (lane == 0) p.out_tokens[uidx] = token;  // the row's token at its first rejection, or the bonus
+          }
+        } else if (!is_bonus && emit) {
+          // no residual mass although a token is needed: this block draws from r instead, over the whole
+          // vocabulary (sixteen runs, totals in shared memory)
+          const int sb = static_cast<int>(static_cast<long long>(warp) * p.nsteps / kWarps);
+          const int se = static_cast<int>(static_cast<long long>(warp + 1) * p.nsteps / kWarps);
+          const int gszv = run_gsz(se - sb, kRec);
+          const double t = run_totals(sb, se, gszv, true, false, &sh.srun[warp][0]);
+          if (lane == 0) sh.wtot[warp] = t;
+          __syncthreads();
+          if (tid == 0) {
+            pick_run(sh.wtot, kWarps);
+            if (!sh.dec.accept) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_RESIDUAL_EMPTY));
+          }
+          __syncthreads();
+          if (sh.win_g == warp) {
+            const int token = walk(sb, se, gszv, sh.base, &sh.srun[warp][0], sh.target, true);
+            if (lane == 0) p.out_tokens[uidx] = token;
+          }
         }
       }
-      published = (sh.win_rank >= 0);  // otherwise nothing had mass: rank 0 reports token -1 below
+      }  // stages 2 and 3
     }
     if (p.stage == 0 && rank == 0 && tid == 0) {
       const Decision& d = sh.dec;
       publish_unit(p, b, j, d.accept, d.status, d.cand, d.drawable, d.ratio, d.r_d, d.q_d, d.S);
     }
-    (void)published;
     // No barrier here: everything the next unit writes before its first block barrier
     // (ldraft, next_local, u_acc/u_smp, warp partials) is read only before this point; stage 1
     // starts every unit with a block barrier of its own.
-    if (p.stage == 1) __syncthreads();
+    if (p.stage >= 1) __syncthreads();
     unit = next_unit;
   }
   cluster.sync();  // no block leaves while a peer may still read its shared memory
@@ -1544,7 +1558,7 @@ thread_local std::string g_create_error;
 
 struct cos_verify_ctx {
   cos_verify_config cfg;
-  int cluster_draw;     // blocks per unit in stage 1
+  int parts;            // blocks per unit in the drawing stages
   int max_clusters[5];  // resident clusters for cluster sizes 1, 2, 4, 8, 16 (0 = not available)
   int sm_count;
   unsigned work_base;
@@ -1557,6 +1571,9 @@ struct cos_verify_ctx {
   int* d_job_count;  // two counters, used alternately by successive runs
   int2* d_jobs;
   UnitStats* d_ustats;
+  double* d_zpart;
+  double* d_wtotg;
+  double* d_srung;
   // optional staging for host-pointer runs
   void* d_logits;
   int* d_drafts;
@@ -1645,6 +1662,18 @@ int choose_cluster(const cos_verify_config& c) {
   return cs;
 }
 
+// Blocks per unit in the drawing stages: enough blocks to occupy the device several times over,
+// at least two steps per warp.
+int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
+  const int cap = choose_cluster(c) * 2 > kMaxParts ? kMaxParts : choose_cluster(c) * 2;
+  int parts = 1;
+  while (parts < cap && rows * parts < 4 * sm_count) parts <<= 1;
+  const int E = entries_per_vec(c.dtype);
+  const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
+  while (parts > 1 && nsteps / (parts * kWarps) < 2) parts >>= 1;
+  return parts;
+}
+
 int log2i(int c) { return c >= 16 ? 4 : (c >= 8 ? 3 : (c >= 4 ? 2 : (c >= 2 ? 1 : 0))); }
 
 // Stage 0 streams best with one block per unit (long contiguous reads, no cluster barrier);
@@ -1727,7 +1756,6 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     return COS_ERR_NOMEM;
   }
   ctx->cfg = *config;
-  ctx->cluster_draw = choose_cluster(*config);
   cudaDeviceProp prop;
   e = cudaGetDeviceProperties(&prop, config->device);
   if (e != cudaSuccess) {
@@ -1735,6 +1763,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     return cuda_fail(nullptr, "cudaGetDeviceProperties", e);
   }
   ctx->sm_count = prop.multiProcessorCount;
+  ctx->parts = choose_parts(*config, config->max_batch, ctx->sm_count);
   KernelFn fn = pick_kernel(config->dtype, mode_of(*config));
   e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
   if (e != cudaSuccess) {
@@ -1762,7 +1791,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   }
   {
     const int need = config->cluster_size > 0 ? config->cluster_size : 1;
-    if (ctx->max_clusters[log2i(need)] < 1 || ctx->max_clusters[log2i(ctx->cluster_draw)] < 1) {
+    if (ctx->max_clusters[log2i(need)] < 1 || ctx->max_clusters[0] < 1) {
       delete ctx;
       g_create_error = "no cluster of the requested size fits on the device";
       return COS_ERR_UNSUPPORTED;
@@ -1776,6 +1805,9 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   ok = ok && cudaMalloc(&ctx->d_job_count, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_jobs, (rows * P + rows) * sizeof(int2)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_ustats, rows * P * sizeof(UnitStats)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_zpart, rows * P * ctx->parts * 8 * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_wtotg, rows * P * ctx->parts * kWarps * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_srung, rows * ctx->parts * kWarps * kRecG * sizeof(double)) == cudaSuccess;
   if (ok && config->host_staging) {
     const size_t V = static_cast<size_t>(config->vocab);
     ok = ok && cudaMalloc(&ctx->d_logits, static_cast<size_t>(config->n) * rows * P * V * elem_bytes(config->dtype)) == cudaSuccess;
@@ -1889,6 +1921,10 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.job_reset = ctx->d_job_count + ((ctx->run_parity & 1u) ^ 1u);
   p.jobs = ctx->d_jobs;
   p.ustats = ctx->d_ustats;
+  p.zpart = ctx->d_zpart;
+  p.wtotg = ctx->d_wtotg;
+  p.srung = ctx->d_srung;
+  p.parts = ctx->parts;
   p.max_jobs = p.num_units + a->batch;
 
   KernelFn fn = pick_kernel(c.dtype, mode_of(c));
@@ -1907,15 +1943,17 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   e = launch_stage(fn, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (draws) {
-    // stage 1: the units listed by stage 0 (one per row, or all of them under the test hooks)
-    const int c1 = ctx->cluster_draw;
-    const int mc1 = ctx->max_clusters[log2i(c1)];
+    // stages 1-3: the units listed by stage 0 (one per row, or all of them under the test hooks);
+    // blocks of a launch are independent, the launches themselves order the three steps
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
-    p.stage = 1;
-    p.num_clusters = most < mc1 ? most : mc1;
-    e = launch_stage(fn, p, c1, stream);
-    if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 1)", e);
+    const int cap = 4096;  // a block walks the job list with a stride, so the grid may be smaller than the list
+    for (int st = 1; st <= 3; ++st) {
+      p.stage = st;
+      p.num_clusters = (most < cap ? most : cap) * (st == 3 ? 1 : p.parts);  // blocks of this launch
+      e = launch_stage(fn, p, 1, stream);
+      if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stages)", e);
+    }
   }
   // every cluster starts on the unit of its own index and draws once after each unit it finishes,
   // so a run draws exactly num_units numbers from the counter
@@ -1992,8 +2030,8 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
   info->threads_per_block = kThreads;
   info->max_clusters = ctx->max_clusters[log2i(info->cluster_size)];
   info->sm_count = ctx->sm_count;
-  info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? 2 : 1;
-  info->reserved[0] = ctx->cluster_draw;
+  info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? 4 : 1;
+  info->reserved[0] = ctx->parts;
   return COS_OK;
 }
 
@@ -2006,6 +2044,9 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_job_count);
   cudaFree(ctx->d_jobs);
   cudaFree(ctx->d_ustats);
+  cudaFree(ctx->d_zpart);
+  cudaFree(ctx->d_wtotg);
+  cudaFree(ctx->d_srung);
   cudaFree(ctx->d_unit_res);
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_drafts);
@@ -2030,7 +2071,8 @@ namespace {
 
 // Scratch of the context-free entry point.  It is part of the library image: every device
 // that loads the library holds these COS_STATIC_SCRATCH_BYTES until the process exits.
-// Layout: [0, 256) work and job counters | row arrival counters | unit results | job list | unit statistics.
+// Layout: [0, 256) work and job counters | row arrival counters | unit results | job list | unit statistics |
+// partial normalisers | run masses | running totals of the drawing unit of each row.
 static __device__ __align__(256) unsigned char g_static_scratch[COS_STATIC_SCRATCH_BYTES];
 
 constexpr int kStaticMaxDevices = 64;
@@ -2092,12 +2134,10 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c.device);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaDeviceGetAttribute", e);
   const int c0 = choose_stream_cluster(c, static_cast<int>(units), sm_count);
-  const int c1 = choose_cluster(c);
-  int mc0 = 0, mc1 = 0;
+  int mc0 = 0;
   e = query_clusters(fn, c0, sm_count, &mc0);
-  if (e == cudaSuccess) e = query_clusters(fn, c1, sm_count, &mc1);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaOccupancyMaxActiveClusters", e);
-  if (mc0 < 1 || mc1 < 1) return static_fail(COS_ERR_UNSUPPORTED, "no cluster of the requested size fits on the device");
+  if (mc0 < 1) return static_fail(COS_ERR_UNSUPPORTED, "no cluster of the requested size fits on the device");
 
   // carve the array; what must start clean is cleared on the caller's stream before the kernels
   unsigned char* basep = g_static_addr[c.device];
@@ -2109,6 +2149,11 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   UnitStats* d_ustats = reinterpret_cast<UnitStats*>(reinterpret_cast<unsigned char*>(d_jobs) +
                                                       8 * (COS_STATIC_MAX_POSITIONS + COS_STATIC_MAX_BATCH));
   static_assert(sizeof(UnitStats) == 112, "COS_STATIC_SCRATCH_BYTES assumes 112 bytes of statistics per position");
+  // one block per unit in the drawing stages here (parts = 1), which keeps the built-in array small
+  double* d_zpart = reinterpret_cast<double*>(reinterpret_cast<unsigned char*>(d_ustats) + 112 * COS_STATIC_MAX_POSITIONS);
+  double* d_wtotg = d_zpart + 8 * COS_STATIC_MAX_POSITIONS;
+  double* d_srung = d_wtotg + 16 * COS_STATIC_MAX_POSITIONS;
+  static_assert(kWarps == 16 && kRecG == 16, "COS_STATIC_SCRATCH_BYTES assumes 16 runs and 16 recorded totals per run");
   e = cudaMemsetAsync(basep, 0, 256, stream);  // work counter and both job counters
   if (e == cudaSuccess) e = cudaMemsetAsync(d_arrivals, 0, static_cast<size_t>(a->batch) * sizeof(int), stream);
   if (e != cudaSuccess) return cuda_fail(nullptr, "clearing the built-in scratch", e);
@@ -2160,6 +2205,10 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.job_reset = d_job_count + 1;
   p.jobs = d_jobs;
   p.ustats = d_ustats;
+  p.zpart = d_zpart;
+  p.wtotg = d_wtotg;
+  p.srung = d_srung;
+  p.parts = 1;
   p.max_jobs = p.num_units + a->batch;
 
   p.stage = 0;
@@ -2169,10 +2218,12 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   if (mode_of(c) == kEnsembleSample || mode_of(c) == kLogitSample) {
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
-    p.stage = 1;
-    p.num_clusters = most < mc1 ? most : mc1;
-    e = launch_stage(fn, p, c1, stream);
-    if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (stage 1)", e);
+    for (int st = 1; st <= 3; ++st) {
+      p.stage = st;
+      p.num_clusters = most < 4096 ? most : 4096;
+      e = launch_stage(fn, p, 1, stream);
+      if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (drawing stages)", e);
+    }
   }
   return COS_OK;
 }
