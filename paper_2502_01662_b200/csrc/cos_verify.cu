@@ -1662,12 +1662,11 @@ int choose_cluster(const cos_verify_config& c) {
   return cs;
 }
 
-// Blocks per unit in the drawing stages: enough blocks to occupy the device several times over,
-// at least two steps per warp.
+// Blocks per unit in the drawing stages: as many as fit on the device in one wave (two blocks per
+// multiprocessor), at least two steps per warp.
 int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
-  const int cap = choose_cluster(c) * 2 > kMaxParts ? kMaxParts : choose_cluster(c) * 2;
   int parts = 1;
-  while (parts < cap && rows * parts < 4 * sm_count) parts <<= 1;
+  while (parts < kMaxParts && rows * parts * 2 <= 2 * sm_count) parts <<= 1;
   const int E = entries_per_vec(c.dtype);
   const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
   while (parts > 1 && nsteps / (parts * kWarps) < 2) parts >>= 1;
