@@ -1227,10 +1227,11 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             uint4 raw = staged[i * 32];
             Elem<DT>::unpack(raw, v);
           } else {
-            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
+            load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);  // entries beyond V read as -inf: mass 0
           }
         };
         float acc[E], rr[E];
+        bool anybig = false;
         bigbits = 0u;
 #pragma unroll
         for (int k = 0; k < E; ++k) {
@@ -1241,15 +1242,17 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           for (int i = 0; i < p.n; ++i) {
             float v[E];
             fetch(i, v);
-            const float co = use_r ? sh.a_scale[i] : sh.a_resid[i], rf = sh.a_ref[i], bt = sh.big_thr[i];
+            const float co = use_r ? sh.a_scale[i] : sh.a_resid[i], rf = sh.a_ref[i];
             const float cr = sh.a_scale[i];
+            float emax = 0.f;
 #pragma unroll
             for (int k = 0; k < E; ++k) {
               const float e = ex2_approx(fmaf(v[k], p.cT, rf));
-              bigbits |= (e > bt) ? (1u << k) : 0u;
+              emax = fmaxf(emax, e);
               acc[k] = fmaf(co, e, acc[k]);
               if (dump) rr[k] = fmaf(cr, e, rr[k]);
             }
+            anybig |= emax > sh.big_thr[i];
           }
         } else {
           float cmb[E], ve[E], eq[E];
@@ -1270,19 +1273,47 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               if (i == pis) eq[k] = ex2_approx(fmaf(v[k], p.cT, ref_q));
             }
           }
+          const float qco = use_r ? 0.f : inv_zq;
+          const bool tail = (staged == nullptr);
+          float emq = 0.f, emc = 0.f;
 #pragma unroll
           for (int k = 0; k < E; ++k) {
-            const bool in = (e0 + k < p.V) && (!masked || ve[k] >= thr);
+            bool in = !masked || ve[k] >= thr;
+            if (tail) in = in && (e0 + k < p.V);
             const float ec = in ? ex2_approx(fmaf(cmb[k], p.cT, ref_c)) : 0.f;
-            bigbits |= (ec > sh.big_thr[1] || eq[k] > sh.big_thr[0]) ? (1u << k) : 0u;
+            emc = fmaxf(emc, ec);
+            emq = fmaxf(emq, eq[k]);
             rr[k] = ec * inv_zc;
-            acc[k] = use_r ? rr[k] : fmaf(-eq[k], inv_zq, rr[k]);
+            acc[k] = fmaf(-eq[k], qco, rr[k]);
           }
+          anybig = (emc > sh.big_thr[1]) || (emq > sh.big_thr[0]);
         }
 #pragma unroll
-        for (int k = 0; k < E; ++k) {
-          const bool keep = (e0 + k < p.V) && !(bigbits & (1u << k));
-          mass32[k] = keep ? (use_r ? acc[k] : fmaxf(0.f, acc[k])) : 0.f;
+        for (int k = 0; k < E; ++k) mass32[k] = fmaxf(0.f, acc[k]);  // r - q clipped at zero; r itself is never negative
+        if (anybig) {
+          // rare: find which tokens are big under some distribution; big_mass evaluates those in fp64
+          if (MODE == kEnsembleSample) {
+            for (int i = 0; i < p.n; ++i) {
+              float v[E];
+              fetch(i, v);
+              const float rf = sh.a_ref[i], bt = sh.big_thr[i];
+#pragma unroll
+              for (int k = 0; k < E; ++k) bigbits |= (ex2_approx(fmaf(v[k], p.cT, rf)) > bt) ? (1u << k) : 0u;
+            }
+          } else {
+            const float zc = static_cast<float>(sh.fsoft[1].s);
+#pragma unroll
+            for (int k = 0; k < E; ++k) {
+              const float ec = rr[k] * zc;  // rr = ec / Z_c
+              const bool inside = (e0 + k < p.V);
+              const float lq = Elem<DT>::load1(row_of(pis), inside ? e0 + k : p.V - 1);
+              const float eqk = inside ? ex2_approx(fmaf(lq, p.cT, ref_q)) : 0.f;
+              bigbits |= (ec > sh.big_thr[1] || eqk > sh.big_thr[0]) ? (1u << k) : 0u;
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < E; ++k)
+            if (bigbits & (1u << k)) mass32[k] = 0.f;
         }
         if (dump) {
           float* out = p.dump_r + (static_cast<long long>(b) * p.P + j) * p.V;
@@ -1336,16 +1367,20 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         const int depth = (p.n <= 2) ? 4 : (p.n <= 4 ? 2 : 1);
         const int nfull = vec_ok ? p.V / (32 * E) : 0;
         const int fe = (se < nfull) ? se : nfull;  // steps [sb, fe) go through the ring
-        auto stage_in = [&](int s) {  // issue the loads of step s into its ring slot
-          const int slot = ((s - sb) % depth) * p.n;
-          for (int i = 0; i < p.n; ++i)
-            cp_async16(&myring[(slot + i) * 32],
-                       reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(s * 32 + lane) * 16);
+        const char* row0 = reinterpret_cast<const char*>(row_of(0));
+        const long long row_step = p.s_model * Elem<DT>::bytes;
+        auto stage_in = [&](int s, int to_slot) {  // issue the loads of step s into a ring slot
+          const char* src = row0 + static_cast<long long>(s * 32 + lane) * 16;
+          uint4* dst = &myring[to_slot * p.n * 32];
+          for (int i = 0; i < p.n; ++i) cp_async16(dst + i * 32, src + i * row_step);
         };
+        int fill = 0;  // ring slot the next staged step goes to
         for (int t = 0; t < depth; ++t) {
-          if (sb + t < fe) stage_in(sb + t);
+          if (sb + t < fe) stage_in(sb + t, fill);
+          fill = (fill + 1 == depth) ? 0 : fill + 1;
           cp_async_commit();
         }
+        int slot = 0, in_group = 0, grp = 0;
         for (int s = sb; s < se; ++s) {
           float mass32[E];
           unsigned bigbits;
@@ -1357,21 +1392,22 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               cp_async_wait<1>();
             else
               cp_async_wait<0>();
-            const int slot = ((s - sb) % depth) * p.n;
-            chunk_mass(e0, use_r, dump, mass32, bigbits, &myring[slot * 32]);
-            if (s + depth < fe) stage_in(s + depth);
+            chunk_mass(e0, use_r, dump, mass32, bigbits, &myring[slot * p.n * 32]);
+            if (s + depth < fe) stage_in(s + depth, slot);
+            slot = (slot + 1 == depth) ? 0 : slot + 1;
             cp_async_commit();
           } else {
             chunk_mass(e0, use_r, dump, mass32, bigbits, nullptr);
           }
           lacc += lane_mass(e0, mass32, bigbits, use_r, dump);
-          const int done = s - sb + 1;
-          if (done % gszv == 0 || s + 1 == se) {
+          if (++in_group == gszv || s + 1 == se) {
             double t = lacc;
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
             wrun += t;
-            if (lane == 0 && rec != nullptr) rec[(done - 1) / gszv] = wrun;
+            if (lane == 0 && rec != nullptr) rec[grp] = wrun;
+            ++grp;
+            in_group = 0;
             lacc = 0.0;
           }
         }
