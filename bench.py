@@ -321,7 +321,7 @@ def main():
                    "mean_accept_count": mean_accept},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_kind": peak_kind, "bytes_per_launch": bytes_per_launch,
-                     "kernel": "cos_verify_kernel"},
+                     "kernel": "cos_verify_kernel (all launches of one call)"},
         "gpu_launches": args.steps * info["launches_per_run"],
         "clocks": sampler.summary() if sampler else None,
     }
