@@ -108,7 +108,7 @@ typedef struct {
   int32_t threads_per_block;
   int32_t max_clusters;      /* clusters that can be resident at once on the device                   */
   int32_t sm_count;
-  int32_t launches_per_run;  /* kernels cos_verify_run enqueues per call (4 when T > 0, else 1)        */
+  int32_t launches_per_run;  /* kernels cos_verify_run enqueues per call (3 when T > 0, else 1)        */
   int32_t reserved[3];
 } cos_verify_info;
 
@@ -173,7 +173,8 @@ cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args,
 #define COS_STATIC_SCRATCH_BYTES                                                                          \
   (256 + 4 * COS_STATIC_MAX_BATCH + 16 * COS_STATIC_MAX_POSITIONS +                                      \
    8 * (COS_STATIC_MAX_POSITIONS + COS_STATIC_MAX_BATCH) + 112 * COS_STATIC_MAX_POSITIONS +              \
-   8 * 8 * COS_STATIC_MAX_POSITIONS + 8 * 16 * COS_STATIC_MAX_POSITIONS + 8 * 16 * 16 * COS_STATIC_MAX_BATCH)
+   8 * 8 * COS_STATIC_MAX_POSITIONS + 8 * 16 * COS_STATIC_MAX_POSITIONS + 8 * 16 * 16 * COS_STATIC_MAX_BATCH +   \
+   4 * COS_STATIC_MAX_POSITIONS)
 cos_status cos_verify_run_static(const cos_verify_config* config, const cos_verify_args* args, void* cuda_stream);
 
 /* Launch geometry chosen at creation. */

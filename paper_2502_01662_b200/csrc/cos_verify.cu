@@ -69,7 +69,7 @@ struct KParams {
   int flags;
   int num_units, num_clusters;
   int stage;     // 0: statistics, decisions, row scan (every unit); then for the listed units only:
-                 // 1: normalisers again with fp64 care, 2: token masses and their running totals, 3: locate the token
+                 // 1: normalisers again with fp64 care, 2: token masses, running totals, and the token
   int parts;     // blocks that share one unit in stages 1 and 2
   int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
@@ -91,11 +91,12 @@ struct KParams {
   int4* unit_res;          // [B*P]: x = accept flag, y = status bits, z = candidate token, w = a token can be drawn
   int* job_count;          // units that stage 1 must process (this run's counter)
   int* job_reset;          // the other run parity's counter, cleared by stage 0
-  int2* jobs;              // x = b * P + j, y = 1 if the drawn token is the row's output at position j
+  int2* jobs;              // x = b * P + j of a unit that draws a token (y unused)
   UnitStats* ustats;       // [B*P]: merged statistics of sweep 1, read back by the later stages
   double* zpart;           // [B*P][parts][8]: stage 1's partial normalisers
   double* wtotg;           // [B*P][parts*16]: stage 2's mass of every warp run
   double* srung;           // [B][parts*16][kRecG]: running totals inside the runs of the row's drawing unit
+  int* part_arrivals;      // [B*P]: blocks of the unit that finished stage 2; zero between runs
 };
 
 // ------------------------------------------------------------------------------------
@@ -494,7 +495,9 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
   for (int k = 0; k < p.P; ++k) o[k] = (k < a) ? p.drafts[b * p.gamma + k] : (k == a ? tok : -1);
   p.row_status[b] = st;
   p.row_arrivals[b] = 0;  // leave the scratch ready for the next run
-  if (draw) push_job(p, b * p.P + a, 1);
+  // under the test hooks the unit may already be on the list: every unit is listed once at most
+  const bool listed = (p.dump_r != nullptr) || ((p.flags & COS_RUN_ALL_RESIDUALS) && a < p.gamma);
+  if (draw && !listed) push_job(p, b * p.P + a, 1);
 }
 
 // ------------------------------------------------------------------------------------
@@ -621,9 +624,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       if (job >= njobs) break;
       const int2 jb = p.jobs[job];
       ++job_it;
-      emit = jb.y;
       b = jb.x / p.P;
       j = jb.x % p.P;
+      emit = (p.accept_count[b] == j) ? 1 : 0;  // the token drawn here is the row's output
     }
     const int uidx = b * p.P + j;
     const int pi = p.proposer[b];
@@ -1527,15 +1530,31 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       };
       auto run_gsz = [&](int nst, int nrec) { return (nst + nrec - 1) / nrec > 1 ? (nst + nrec - 1) / nrec : 1; };
 
+      bool do_locate = false;
       if (p.stage == 2) {
-        // ---- masses of this block's runs, for stage 3 to add up and search
+        // ---- masses of this block's runs, to be added up and searched by the last block of the unit
         const int gszv = run_gsz(s_end - s_begin, kRecG);
         double* rec = emit ? p.srung + (static_cast<size_t>(b) * G + gwarp) * kRecG : nullptr;
         const double t = run_totals(s_begin, s_end, gszv, is_bonus, p.dump_r != nullptr, rec);
         if (lane == 0) p.wtotg[static_cast<size_t>(uidx) * G + gwarp] = t;
-      } else {
-        // ---- stage 3, one block per unit: add the runs up, find the run, walk it
-        for (int g = tid; g < G; g += kThreads) sh.gw[g] = p.wtotg[static_cast<size_t>(uidx) * G + g];
+        // the last block of the unit to get here goes on to locate the token (fence + counter, no waiting)
+        __syncthreads();
+        if (tid == 0) {
+          __threadfence();
+          const int prev = atomicAdd(&p.part_arrivals[uidx], 1);
+          sh.win_g = (prev == p.parts - 1) ? 1 : 0;
+          if (prev == p.parts - 1) {
+            p.part_arrivals[uidx] = 0;  // ready for the next run
+            __threadfence();
+          }
+        }
+        __syncthreads();
+        do_locate = (sh.win_g != 0);
+        __syncthreads();
+      }
+      if (do_locate) {
+        // ---- one block per unit: add the runs up, find the run, walk it
+        for (int g = tid; g < G; g += kThreads) sh.gw[g] = __ldcg(&p.wtotg[static_cast<size_t>(uidx) * G + g]);
         __syncthreads();
         if (tid == 0) pick_run(sh.gw, G);
         __syncthreads();
@@ -1610,6 +1629,7 @@ struct cos_verify_ctx {
   double* d_zpart;
   double* d_wtotg;
   double* d_srung;
+  int* d_part_arrivals;
   // optional staging for host-pointer runs
   void* d_logits;
   int* d_drafts;
@@ -1767,6 +1787,8 @@ cos_status init_scratch(cos_verify_ctx* ctx, cudaStream_t stream) {
   cudaError_t e = cudaMemsetAsync(ctx->d_work_counter, 0, sizeof(unsigned), stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_row_arrivals, 0, rows * sizeof(int), stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_job_count, 0, 2 * sizeof(int), stream);
+  if (e == cudaSuccess)
+    e = cudaMemsetAsync(ctx->d_part_arrivals, 0, rows * (static_cast<size_t>(ctx->cfg.gamma) + 1) * sizeof(int), stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "scratch reset", e);
   ctx->work_base = 0;
   ctx->run_parity = 0;
@@ -1843,6 +1865,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   ok = ok && cudaMalloc(&ctx->d_zpart, rows * P * ctx->parts * 8 * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_wtotg, rows * P * ctx->parts * kWarps * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_srung, rows * ctx->parts * kWarps * kRecG * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_part_arrivals, rows * P * sizeof(int)) == cudaSuccess;
   if (ok && config->host_staging) {
     const size_t V = static_cast<size_t>(config->vocab);
     ok = ok && cudaMalloc(&ctx->d_logits, static_cast<size_t>(config->n) * rows * P * V * elem_bytes(config->dtype)) == cudaSuccess;
@@ -1959,6 +1982,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.zpart = ctx->d_zpart;
   p.wtotg = ctx->d_wtotg;
   p.srung = ctx->d_srung;
+  p.part_arrivals = ctx->d_part_arrivals;
   p.parts = ctx->parts;
   p.max_jobs = p.num_units + a->batch;
 
@@ -1978,14 +2002,14 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   e = launch_stage(fn, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (draws) {
-    // stages 1-3: the units listed by stage 0 (one per row, or all of them under the test hooks);
-    // blocks of a launch are independent, the launches themselves order the three steps
+    // stages 1 and 2: the units listed by stage 0 (one per row, or all of them under the test hooks);
+    // blocks of a launch are independent, the launches themselves order the steps
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
     const int cap = 4096;  // a block walks the job list with a stride, so the grid may be smaller than the list
-    for (int st = 1; st <= 3; ++st) {
+    for (int st = 1; st <= 2; ++st) {
       p.stage = st;
-      p.num_clusters = (most < cap ? most : cap) * (st == 3 ? 1 : p.parts);  // blocks of this launch
+      p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of this launch
       e = launch_stage(fn, p, 1, stream);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stages)", e);
     }
@@ -2065,7 +2089,7 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
   info->threads_per_block = kThreads;
   info->max_clusters = ctx->max_clusters[log2i(info->cluster_size)];
   info->sm_count = ctx->sm_count;
-  info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? 4 : 1;
+  info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? 3 : 1;
   info->reserved[0] = ctx->parts;
   return COS_OK;
 }
@@ -2082,6 +2106,7 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_zpart);
   cudaFree(ctx->d_wtotg);
   cudaFree(ctx->d_srung);
+  cudaFree(ctx->d_part_arrivals);
   cudaFree(ctx->d_unit_res);
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_drafts);
@@ -2188,9 +2213,11 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   double* d_zpart = reinterpret_cast<double*>(reinterpret_cast<unsigned char*>(d_ustats) + 112 * COS_STATIC_MAX_POSITIONS);
   double* d_wtotg = d_zpart + 8 * COS_STATIC_MAX_POSITIONS;
   double* d_srung = d_wtotg + 16 * COS_STATIC_MAX_POSITIONS;
+  int* d_part_arrivals = reinterpret_cast<int*>(d_srung + 16 * 16 * COS_STATIC_MAX_BATCH);
   static_assert(kWarps == 16 && kRecG == 16, "COS_STATIC_SCRATCH_BYTES assumes 16 runs and 16 recorded totals per run");
   e = cudaMemsetAsync(basep, 0, 256, stream);  // work counter and both job counters
   if (e == cudaSuccess) e = cudaMemsetAsync(d_arrivals, 0, static_cast<size_t>(a->batch) * sizeof(int), stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_part_arrivals, 0, static_cast<size_t>(units) * sizeof(int), stream);
   if (e != cudaSuccess) return cuda_fail(nullptr, "clearing the built-in scratch", e);
 
   KParams p;
@@ -2243,6 +2270,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.zpart = d_zpart;
   p.wtotg = d_wtotg;
   p.srung = d_srung;
+  p.part_arrivals = d_part_arrivals;
   p.parts = 1;
   p.max_jobs = p.num_units + a->batch;
 
@@ -2253,7 +2281,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   if (mode_of(c) == kEnsembleSample || mode_of(c) == kLogitSample) {
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
-    for (int st = 1; st <= 3; ++st) {
+    for (int st = 1; st <= 2; ++st) {
       p.stage = st;
       p.num_clusters = most < 4096 ? most : 4096;
       e = launch_stage(fn, p, 1, stream);
