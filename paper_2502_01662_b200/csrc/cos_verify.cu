@@ -1252,7 +1252,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             for (int k = 0; k < E; ++k) {
               const float e = ex2_approx(fmaf(v[k], p.cT, rf));
               emax = fmaxf(emax, e);
-              acc[k] = fmaf(co, e, acc[k]);
+              // products rounded one by one (no fused multiply-add): when r and q coincide the terms
+              // cancel exactly, as they do in exact arithmetic
+              acc[k] = __fadd_rn(acc[k], __fmul_rn(co, e));
               if (dump) rr[k] = fmaf(cr, e, rr[k]);
             }
             anybig |= emax > sh.big_thr[i];
@@ -1287,7 +1289,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             emc = fmaxf(emc, ec);
             emq = fmaxf(emq, eq[k]);
             rr[k] = ec * inv_zc;
-            acc[k] = fmaf(-eq[k], qco, rr[k]);
+            acc[k] = __fsub_rn(rr[k], __fmul_rn(eq[k], qco));  // rounded product: r == q cancels exactly
           }
           anybig = (emc > sh.big_thr[1]) || (emq > sh.big_thr[0]);
         }

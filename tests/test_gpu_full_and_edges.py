@@ -1,0 +1,162 @@
+"""GPU parity at the full benchmark sizes (sampled rows) and on the edge cases of the method."""
+import numpy as np
+import pytest
+import torch
+
+import helpers
+from paper_2502_01662_b200 import (COS_ROW_BAD_DRAFT, COS_ROW_NONFINITE, COS_ROW_Q_ZERO, COS_ROW_RESIDUAL_EMPTY,
+                                   COS_RUN_ALL_RESIDUALS, CosVerifier, CosVerifyError, synth)
+from oracle import cos_oracle as orc
+
+pytestmark = pytest.mark.gpu
+C = synth.CONFIGS
+
+
+@pytest.mark.parametrize("name,nrows", [("cfg1", 1), ("cfg2", 8), ("cfg3", 10), ("cfg4", 8), ("cfg5", 8), ("cfg5_greedy", 8)])
+def test_full_size_workloads_on_sampled_rows(name, nrows):
+    """The launch configuration bench.py times (default cluster choice, full batch), compared with the
+    oracle on a seeded sample of rows; a row's result does not depend on the other rows."""
+    w = C[name]
+    inputs = synth.make_inputs(w, "cuda")
+    rows = sorted(np.random.default_rng(7).choice(w.batch, size=min(nrows, w.batch), replace=False).tolist())
+    gpu = helpers.run_gpu(w, inputs, diag=True)
+    ref = helpers.run_oracle(w, inputs, rows=rows)
+    stats = helpers.check_parity(w, gpu, ref, rows=rows)
+    assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
+    # the sampled rows are not degenerate: some rows reject, and sampling modes do not reject everything at 0
+    acc = gpu["accept_count"]
+    assert acc.min() >= 0 and acc.max() <= w.gamma
+    assert np.all(gpu["out_tokens"][np.arange(w.batch), acc] >= 0)
+    # second run with the same arguments is bit-identical (no dependence on scheduling)
+    again = helpers.run_gpu(w, inputs, diag=True)
+    for k in ("accept_count", "out_tokens", "row_status"):
+        assert np.array_equal(gpu[k], again[k]), k
+    del inputs
+    torch.cuda.empty_cache()
+
+
+def _small(cfg, **kw):
+    return C[cfg].scaled(**kw)
+
+
+def test_statistics_of_acceptance_match_eq7():
+    """Mean accept flag against mean alpha_j = 1 - sum max(0, r - q) (Eq. 7) from the kernel's own S."""
+    w = _small("cfg4", batch=32, vocab=12808, gamma=6, name="stat")
+    inputs = synth.make_inputs(w, "cuda")
+    gpu = helpers.run_gpu(w, inputs, diag=True, flags=COS_RUN_ALL_RESIDUALS)
+    ref = helpers.run_oracle(w, inputs)
+    S = gpu["diag"][:, : w.gamma, 3]
+    assert np.all(np.isfinite(S))
+    np.testing.assert_allclose(S, ref["S"][:, : w.gamma], rtol=1e-5, atol=1e-7)
+    alpha = 1.0 - S
+    assert np.all(alpha >= np.asarray(w.weights)[inputs["proposer"].cpu().numpy()][:, None] - 1e-6)   # Thm 3.2
+
+
+def test_row_base_and_partial_batches_and_strides():
+    w = _small("cfg3", batch=6, vocab=4096, gamma=3, name="layout")
+    inputs = synth.make_inputs(w, "cuda")
+    full = helpers.run_gpu(w, inputs)
+    # rows 2..5 as a shard: same numbers when row_base = 2; context sized for a larger batch
+    v = helpers.make_verifier(w, max_batch=16)
+    try:
+        part = v.run(inputs["logits"][:, 2:], inputs["drafts"][2:].contiguous(), inputs["proposer"][2:].contiguous(),
+                     inputs["seed"], inputs["offset"], row_base=2)
+        torch.cuda.synchronize()
+        for k in ("accept_count", "out_tokens", "row_status"):
+            assert np.array_equal(part[k].cpu().numpy(), full[k][2:]), k
+        # a padded layout (row pitch larger than V, still 16-byte aligned) and an unaligned one (scalar loads)
+        for pad in (8, 3):
+            big = torch.zeros((w.n, w.batch, w.gamma + 1, w.vocab + pad), dtype=inputs["logits"].dtype, device="cuda")
+            big[..., : w.vocab] = inputs["logits"]
+            view = big[..., : w.vocab]
+            got = v.run(view, inputs["drafts"], inputs["proposer"], inputs["seed"], inputs["offset"])
+            torch.cuda.synchronize()
+            for k in ("accept_count", "out_tokens", "row_status"):
+                assert np.array_equal(got[k].cpu().numpy(), full[k]), (pad, k)
+    finally:
+        v.close()
+
+
+def test_host_pointer_entry_matches_device_entry():
+    w = _small("cfg2", batch=5, vocab=8000, gamma=3, name="host")
+    dev_in = synth.make_inputs(w, "cuda")
+    want = helpers.run_gpu(w, dev_in, diag=True)
+    v = helpers.make_verifier(w, host_staging=True)
+    try:
+        got = v.run_host(dev_in["logits"].cpu().contiguous().pin_memory(), dev_in["drafts"].cpu().pin_memory(),
+                         dev_in["proposer"].cpu().pin_memory(), dev_in["seed"], dev_in["offset"], diag=True)
+        for k in ("accept_count", "out_tokens", "row_status"):
+            assert np.array_equal(got[k].numpy(), want[k]), k
+        np.testing.assert_array_equal(got["diag"].numpy()[..., :3], want["diag"][..., :3])
+    finally:
+        v.close()
+
+
+def test_data_dependent_problems_are_flagged_not_trapped():
+    w = _small("cfg3", batch=6, vocab=2048, gamma=3, name="flags")
+    inputs = synth.make_inputs(w, "cuda")
+    logits = inputs["logits"].clone()
+    drafts = inputs["drafts"].clone()
+    logits[1, 0, 0, 77] = float("nan")          # row 0: NaN at position 0
+    logits[0, 1, 1, 5] = float("inf")           # row 1: +inf at position 1
+    logits[1, 2, 0, 9] = float("-inf")          # row 2: a token one model rules out (legal)
+    drafts[3, 0] = w.vocab                      # row 3: draft outside the vocabulary
+    drafts[4, 1] = -1                           # row 4: negative draft at position 1
+    bad = dict(inputs, logits=logits, drafts=drafts)
+    gpu = helpers.run_gpu(w, bad, diag=True)
+    ref = helpers.run_oracle(w, bad)
+    helpers.check_parity(w, gpu, ref, check_diag=False)
+    assert gpu["row_status"][0] & COS_ROW_NONFINITE and gpu["accept_count"][0] == 0 and gpu["out_tokens"][0, 0] == -1
+    assert gpu["row_status"][3] & COS_ROW_BAD_DRAFT and gpu["accept_count"][3] == 0
+    assert gpu["row_status"][2] == ref["row_status"][2]
+
+
+def test_identical_models_accept_everything_and_empty_residual_falls_back_to_r():
+    w = _small("cfg3", batch=4, vocab=3000, gamma=2, name="same")
+    inputs = synth.make_inputs(w, "cuda")
+    logits = inputs["logits"].clone()
+    logits[1] = logits[0]                        # r == q exactly
+    drafts = inputs["drafts"].clone()
+    drafts[2, 0] = w.vocab + 5                   # an invalid draft is rejected although the residual is empty
+    same = dict(inputs, logits=logits, drafts=drafts)
+    gpu = helpers.run_gpu(w, same, diag=True)
+    ref = helpers.run_oracle(w, same)
+    helpers.check_parity(w, gpu, ref, check_diag=False)
+    assert np.all(gpu["accept_count"][[0, 1, 3]] == w.gamma)
+    assert gpu["accept_count"][2] == 0
+    assert gpu["row_status"][2] == (COS_ROW_BAD_DRAFT | COS_ROW_RESIDUAL_EMPTY)
+    assert 0 <= gpu["out_tokens"][2, 0] < w.vocab
+
+
+def test_greedy_ensemble_atoms_and_q_zero():
+    w = synth.Workload("we_greedy", 3, 0, (0.5, 0.3, 0.2), 0.0, 8, 3, 5000, "f32", "gauss", sigma=2.0, rho=0.5,
+                       proposer_rule="cycle")
+    inputs = synth.make_inputs(w, "cuda")
+    drafts = inputs["drafts"].clone()
+    drafts[0, 0] = (int(drafts[0, 0]) + 1) % w.vocab     # not the proposer's argmax: q(draft) = 0
+    mod = dict(inputs, drafts=drafts)
+    gpu = helpers.run_gpu(w, mod, diag=True, dump_r=True)
+    ref = helpers.run_oracle(w, mod, return_r=True)
+    helpers.check_parity(w, gpu, ref, check_diag=False)
+    helpers.check_combined_probabilities(w, gpu["r"], ref["r"])
+    assert gpu["row_status"][0] & COS_ROW_Q_ZERO
+
+
+def test_invalid_arguments_return_errors():
+    w = _small("cfg3", batch=2, vocab=1024, gamma=2, name="args")
+    inputs = synth.make_inputs(w, "cuda")
+    v = helpers.make_verifier(w)
+    try:
+        with pytest.raises(CosVerifyError):        # batch larger than max_batch
+            big = torch.zeros((w.n, 3, w.gamma + 1, w.vocab), dtype=inputs["logits"].dtype, device="cuda")
+            v.run(big, torch.zeros((3, w.gamma), dtype=torch.int32, device="cuda"),
+                  torch.zeros(3, dtype=torch.int32, device="cuda"), 1, 0)
+        with pytest.raises(ValueError):            # wrong vocabulary
+            v.run(inputs["logits"][..., :-8], inputs["drafts"], inputs["proposer"], 1, 0)
+        with pytest.raises(CosVerifyError):        # host-pointer call without staging
+            v.run_host(inputs["logits"].cpu(), inputs["drafts"].cpu(), inputs["proposer"].cpu(), 1, 0)
+        ok = v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], 1, 0)   # the context still works
+        torch.cuda.synchronize()
+        assert ok["accept_count"].min() >= 0
+    finally:
+        v.close()
