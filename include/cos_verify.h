@@ -177,6 +177,16 @@ cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args,
    4 * COS_STATIC_MAX_POSITIONS)
 cos_status cos_verify_run_static(const cos_verify_config* config, const cos_verify_args* args, void* cuda_stream);
 
+/*
+ * Measurement aid: with `enable` non-zero, every later cos_verify_run records CUDA events on its
+ * stream around each of its launches (stage 0: every position, Eq. 3-6 and the row scan; then the
+ * launches that draw the tokens).  cos_verify_get_stage_ms waits for the last timed run and
+ * returns the duration of each of its launches in milliseconds (at most 3 values) and their
+ * number.  Timing adds a few event records per run and changes no result.
+ */
+cos_status cos_verify_set_stage_timing(cos_verify_ctx* ctx, int enable);
+cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, int32_t* count);
+
 /* Launch geometry chosen at creation. */
 cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info);
 

@@ -26,7 +26,8 @@ _STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR
                  4: "COS_ERR_CUDA", 5: "COS_ERR_NOMEM"}
 
 EXPORTS = ("cos_verify_create", "cos_verify_run", "cos_verify_run_host", "cos_verify_get_info",
-           "cos_verify_destroy", "cos_verify_last_error")
+           "cos_verify_destroy", "cos_verify_last_error", "cos_verify_set_stage_timing", "cos_verify_get_stage_ms",
+           "cos_verify_run_static")
 
 
 class CosVerifyError(RuntimeError):
@@ -81,6 +82,10 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.cos_verify_run_host.restype = ctypes.c_int
     lib.cos_verify_get_info.argtypes = [ctypes.c_void_p, ctypes.POINTER(cos_verify_info)]
     lib.cos_verify_get_info.restype = ctypes.c_int
+    lib.cos_verify_set_stage_timing.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    lib.cos_verify_set_stage_timing.restype = ctypes.c_int
+    lib.cos_verify_get_stage_ms.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
+    lib.cos_verify_get_stage_ms.restype = ctypes.c_int
     lib.cos_verify_destroy.argtypes = [ctypes.c_void_p]
     lib.cos_verify_destroy.restype = ctypes.c_int
     lib.cos_verify_last_error.argtypes = [ctypes.c_void_p]
@@ -157,6 +162,17 @@ class CosVerifier:
         a.diag = outs["diag"].data_ptr() if "diag" in outs else None
         a.dump_r = outs["r"].data_ptr() if "r" in outs else None
         return a
+
+    def set_stage_timing(self, enable: bool):
+        """cos_verify_set_stage_timing: record events around every launch of later runs."""
+        self._check(self._lib.cos_verify_set_stage_timing(self._ctx, int(bool(enable))))
+
+    def stage_ms(self):
+        """cos_verify_get_stage_ms: durations (ms) of the launches of the last timed run."""
+        ms = (ctypes.c_float * 4)()
+        count = ctypes.c_int32(0)
+        self._check(self._lib.cos_verify_get_stage_ms(self._ctx, ms, ctypes.byref(count)))
+        return [float(ms[k]) for k in range(count.value)]
 
     @staticmethod
     def _alloc_outs(B, P, V, device, diag, dump_r, pin=False):

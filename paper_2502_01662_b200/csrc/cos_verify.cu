@@ -1632,6 +1632,10 @@ struct cos_verify_ctx {
   double* d_wtotg;
   double* d_srung;
   int* d_part_arrivals;
+  // optional per-stage timing (cos_verify_set_stage_timing)
+  bool timing;
+  cudaEvent_t ev[4];
+  int ev_used;  // events recorded by the last run
   // optional staging for host-pointer runs
   void* d_logits;
   int* d_drafts;
@@ -2001,8 +2005,11 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.stage = 0;
   p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
   ctx->scratch_dirty = true;  // cleared below once the launches are known to be queued
+  if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
   e = launch_stage(fn, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
+  if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
+  ctx->ev_used = 2;
   if (draws) {
     // stages 1 and 2: the units listed by stage 0 (one per row, or all of them under the test hooks);
     // blocks of a launch are independent, the launches themselves order the steps
@@ -2014,6 +2021,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
       p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of this launch
       e = launch_stage(fn, p, 1, stream);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stages)", e);
+      if (ctx->timing) cudaEventRecord(ctx->ev[st + 1], stream);
+      ctx->ev_used = st + 2;
     }
   }
   // every cluster starts on the unit of its own index and draws once after each unit it finishes,
@@ -2084,6 +2093,33 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
   return COS_OK;
 }
 
+extern "C" cos_status cos_verify_set_stage_timing(cos_verify_ctx* ctx, int enable) {
+  if (!ctx) return COS_ERR_INVALID_ARG;
+  if (enable && !ctx->ev[0]) {
+    for (int k = 0; k < 4; ++k) {
+      cudaError_t e = cudaEventCreate(&ctx->ev[k]);
+      if (e != cudaSuccess) return cuda_fail(ctx, "cudaEventCreate", e);
+    }
+  }
+  ctx->timing = enable != 0;
+  ctx->ev_used = 0;
+  return COS_OK;
+}
+
+extern "C" cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, int32_t* count) {
+  if (!ctx || !ms || !count) return COS_ERR_INVALID_ARG;
+  *count = 0;
+  if (!ctx->timing || ctx->ev_used < 2) {
+    ctx->err = "no timed run to report";
+    return COS_ERR_INVALID_ARG;
+  }
+  cudaError_t e = cudaEventSynchronize(ctx->ev[ctx->ev_used - 1]);
+  for (int k = 0; e == cudaSuccess && k + 1 < ctx->ev_used; ++k) e = cudaEventElapsedTime(&ms[k], ctx->ev[k], ctx->ev[k + 1]);
+  if (e != cudaSuccess) return cuda_fail(ctx, "stage timing", e);
+  *count = ctx->ev_used - 1;
+  return COS_OK;
+}
+
 extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info) {
   if (!ctx || !info) return COS_ERR_INVALID_ARG;
   memset(info, 0, sizeof(*info));
@@ -2109,6 +2145,8 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_wtotg);
   cudaFree(ctx->d_srung);
   cudaFree(ctx->d_part_arrivals);
+  for (int k = 0; k < 4; ++k)
+    if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   cudaFree(ctx->d_unit_res);
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_drafts);
