@@ -725,55 +725,98 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       const float thr = masked ? sh.thr32 : -INFINITY;
       if (MODE == kLogitSample) {
         LaneSoft accq, accc;
-        accq.init();
-        accc.init();
-        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
-          float cmb[E], vq[E], ve[E];
+        const char* row0 = reinterpret_cast<const char*>(row_of(0));
+        const long long row_step = p.s_model * Elem<DT>::bytes;
+        // fixed reference exponents seeded from the thread's first vector; overflow or a non-finite input
+        // falls back to the running-maximum form (second pass)
+        for (int pass = 0; pass < 2; ++pass) {
+          const bool fixed = (pass == 0);
+          accq.init();
+          accc.init();
+          bool seeded_q = false, seeded_c = false;
+          // one model's vector: add to the combined logits; the proposer's row also feeds its own softmax,
+          // the expert's row yields the mask bits
+          auto take = [&](int i, const uint4& raw, float (&cmb)[E], unsigned& inbits) {
+            float x[E];
+            Elem<DT>::unpack(raw, x);
+            const float wi = p.w[i];
 #pragma unroll
-          for (int k = 0; k < E; ++k) {
-            cmb[k] = 0.f;
-            vq[k] = -INFINITY;
-            ve[k] = 0.f;
-          }
-          for (int i = 0; i < p.n; i += 2) {
-            const bool two = (i + 1 < p.n);
-            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
-            uint4 rb = ra;
-            if (two) rb = ldg_stream16(reinterpret_cast<const char*>(row_of(i + 1)) + static_cast<long long>(v) * 16);
-            float va[E], vb[E];
-            Elem<DT>::unpack(ra, va);
-            Elem<DT>::unpack(rb, vb);
-            const float wa = p.w[i], wb = two ? p.w[i + 1] : 0.f;
-#pragma unroll
-            for (int k = 0; k < E; ++k) {
-              cmb[k] = fmaf(wa, va[k], cmb[k]);
-              if (i == pis) vq[k] = va[k];
-              if (i == p.mask_model) ve[k] = va[k];
-              if (two) {
-                cmb[k] = fmaf(wb, vb[k], cmb[k]);
-                if (i + 1 == pis) vq[k] = vb[k];
-                if (i + 1 == p.mask_model) ve[k] = vb[k];
+            for (int k = 0; k < E; ++k) cmb[k] = fmaf(wi, x[k], cmb[k]);
+            if (i == pis) {
+              if (fixed) {
+                if (!seeded_q) {
+                  accq.seed(x, p.cT);
+                  seeded_q = true;
+                }
+                accq.add_fixed(x, p.cT);
+              } else {
+                accq.add_online(x, p.cT);
               }
             }
-          }
-          if (masked) {
+            if (masked && i == p.mask_model) {
+              inbits = 0u;
 #pragma unroll
-            for (int k = 0; k < E; ++k) cmb[k] = (ve[k] >= thr) ? cmb[k] : -INFINITY;
+              for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
+            }
+          };
+          auto finish = [&](float (&cmb)[E], unsigned inbits) {
+            if (masked) {
+#pragma unroll
+              for (int k = 0; k < E; ++k) cmb[k] = (inbits & (1u << k)) ? cmb[k] : -INFINITY;
+            }
+            if (fixed) {
+              if (!seeded_c) {
+                accc.seed(cmb, p.cT);
+                seeded_c = true;
+              }
+              accc.add_fixed(cmb, p.cT);
+            } else {
+              accc.add_online(cmb, p.cT);
+            }
+          };
+          for (int v = sl.v_lo + tid; v < sl.v_hi; v += 2 * kThreads) {
+            const bool have_b = (v + kThreads < sl.v_hi);
+            const long long oa = static_cast<long long>(v) * 16;
+            const long long ob = have_b ? oa + static_cast<long long>(kThreads) * 16 : oa;
+            float ca[E], cb[E];
+            unsigned ba = 0xffffffffu, bb = 0xffffffffu;
+#pragma unroll
+            for (int k = 0; k < E; ++k) ca[k] = cb[k] = 0.f;
+            int i = 0;
+            for (; i + 1 < p.n; i += 2) {  // two models, two vectors: four loads in flight
+              const char* r0 = row0 + i * row_step;
+              const char* r1 = r0 + row_step;
+              const uint4 a0 = ldg_stream16(r0 + oa), b0 = ldg_stream16(r0 + ob);
+              const uint4 a1 = ldg_stream16(r1 + oa), b1 = ldg_stream16(r1 + ob);
+              take(i, a0, ca, ba);
+              take(i + 1, a1, ca, ba);
+              if (have_b) {
+                take(i, b0, cb, bb);
+                take(i + 1, b1, cb, bb);
+              }
+            }
+            if (i < p.n) {
+              const char* r0 = row0 + i * row_step;
+              const uint4 a0 = ldg_stream16(r0 + oa), b0 = ldg_stream16(r0 + ob);
+              take(i, a0, ca, ba);
+              if (have_b) take(i, b0, cb, bb);
+            }
+            finish(ca, ba);
+            if (have_b) finish(cb, bb);
           }
-          accq.add_online(vq, p.cT);
-          accc.add_online(cmb, p.cT);
-        }
-        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
-          float cmb = 0.f, xq = -INFINITY, xe = 0.f;
-          for (int i = 0; i < p.n; ++i) {
-            float x = Elem<DT>::load1(row_of(i), e);
-            cmb = fmaf(p.w[i], x, cmb);
-            if (i == pis) xq = x;
-            if (i == p.mask_model) xe = x;
+          for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+            float cmb = 0.f, xq = -INFINITY, xe = 0.f;
+            for (int i = 0; i < p.n; ++i) {
+              float x = Elem<DT>::load1(row_of(i), e);
+              cmb = fmaf(p.w[i], x, cmb);
+              if (i == pis) xq = x;
+              if (i == p.mask_model) xe = x;
+            }
+            if (masked && !(xe >= thr)) cmb = -INFINITY;
+            accq.add_online1(xq, p.cT);
+            accc.add_online1(cmb, p.cT);
           }
-          if (masked && !(xe >= thr)) cmb = -INFINITY;
-          accq.add_online1(xq, p.cT);
-          accc.add_online1(cmb, p.cT);
+          if ((accq.s < INFINITY) && (accc.s < INFINITY)) break;
         }
         warp_merge_soft(accq, &sh.wsoft[warp][0], lane);
         warp_merge_soft(accc, &sh.wsoft[warp][1], lane);
