@@ -41,7 +41,7 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxSlots = COS_MAX_MODELS + 2;
 constexpr int kNoReject = 0x7fffffff;
-constexpr double kBigShare = 1.0 / 1024.0;  // probabilities above 2^-10 get fp64 treatment in sweep 2
+constexpr double kBigShare = 1.0 / 256.0;  // probabilities above 2^-8 get fp64 treatment when tokens are drawn
 constexpr int kRingVecs = 8;                 // 16-byte vectors per lane staged ahead in sweep 2 (4 KB per warp)
 constexpr int kRingBytes = kWarps * kRingVecs * 32 * 16;
 constexpr int kRecG = 16;                    // running totals per warp kept in global memory between the drawing stages
@@ -141,6 +141,9 @@ struct Elem<COS_DTYPE_F32> {
   static __device__ __forceinline__ float load1(const void* row, long long x) {
     return __ldg(reinterpret_cast<const float*>(row) + x);
   }
+  static __device__ __forceinline__ float pick(const uint4* vec, int k) {  // entry k of a vector in shared memory
+    return reinterpret_cast<const float*>(vec)[k];
+  }
 };
 template <>
 struct Elem<COS_DTYPE_BF16> {
@@ -159,6 +162,9 @@ struct Elem<COS_DTYPE_BF16> {
   static __device__ __forceinline__ float load1(const void* row, long long x) {
     unsigned short h = __ldg(reinterpret_cast<const unsigned short*>(row) + x);
     return __uint_as_float(static_cast<unsigned>(h) << 16);
+  }
+  static __device__ __forceinline__ float pick(const uint4* vec, int k) {  // entry k of a vector in shared memory
+    return __uint_as_float(static_cast<unsigned>(reinterpret_cast<const unsigned short*>(vec)[k]) << 16);
   }
 };
 
@@ -1370,11 +1376,16 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             if (e0 + k < p.V && !(bigbits & (1u << k))) out[e0 + k] = rr[k];
         }
       };
-      auto big_mass = [&](int e, bool use_r, bool dump) -> double {
+      // `staged`/`k`: where the token's logits sit in shared memory (null: read them from global memory)
+      auto big_mass = [&](int e, bool use_r, bool dump, const uint4* staged, int k) -> double {
         if (e >= p.V) return 0.0;
         double r64 = 0.0, q64 = 0.0;
         float lv[COS_MAX_MODELS];
-        for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::load1(row_of(i), e);  // all loads first
+        if (staged != nullptr) {
+          for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::pick(staged + i * 32, k);
+        } else {
+          for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::load1(row_of(i), e);  // all loads first
+        }
         if (MODE == kEnsembleSample) {
           for (int i = 0; i < p.n; ++i) {
             double pr = exp2(static_cast<double>(lv[i]) * p.cT64 - static_cast<double>(sh.fsoft[i].ref)) / sh.fsoft[i].s;
@@ -1392,15 +1403,16 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         return use_r ? r64 : fmax(0.0, r64 - q64);
       };
       // a lane's mass of one step: fp32 sum of the small tokens in token order plus the big ones in fp64
-      auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, bool dump) -> double {
+      auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, bool dump,
+                           const uint4* staged) -> double {
         float ls = 0.f;
 #pragma unroll
         for (int k = 0; k < E; ++k) ls += mass32[k];
         double own = static_cast<double>(ls);
-        if (bigbits) {
-#pragma unroll
-          for (int k = 0; k < E; ++k)
-            if (bigbits & (1u << k)) own += big_mass(e0 + k, use_r, dump);
+        while (bigbits) {  // big tokens in token order
+          const int k = __ffs(bigbits) - 1;
+          bigbits &= bigbits - 1;
+          own += big_mass(e0 + k, use_r, dump, staged, k);
         }
         return own;
       };
@@ -1441,13 +1453,14 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             else
               cp_async_wait<0>();
             chunk_mass(e0, use_r, dump, mass32, bigbits, &myring[slot * p.n * 32]);
+            lacc += lane_mass(e0, mass32, bigbits, use_r, dump, &myring[slot * p.n * 32]);
             if (s + depth < fe) stage_in(s + depth, slot);
             slot = (slot + 1 == depth) ? 0 : slot + 1;
             cp_async_commit();
           } else {
             chunk_mass(e0, use_r, dump, mass32, bigbits, nullptr);
+            lacc += lane_mass(e0, mass32, bigbits, use_r, dump, nullptr);
           }
-          lacc += lane_mass(e0, mass32, bigbits, use_r, dump);
           if (++in_group == gszv || s + 1 == se) {
             double t = lacc;
 #pragma unroll
@@ -1497,9 +1510,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           if (bigbits) {
 #pragma unroll
             for (int k = 0; k < E; ++k)
-              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, false);
+              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, false, nullptr, k);
           }
-          const double own = lane_mass(e0, mass32, bigbits, use_r, false);
+          const double own = lane_mass(e0, mass32, bigbits, use_r, false, nullptr);
           double inc = own;
 #pragma unroll
           for (int d = 1; d < 32; d <<= 1) {
