@@ -1273,7 +1273,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       // tokens holding more than 2^-10 of any normaliser are flagged in `bigbits`, get mass32 = 0
       // and are evaluated by big_mass() in fp64 from the stored logits.
       // `staged` points at this lane's staged vector of model 0 (models 32 vectors apart), or is null.
-      auto chunk_mass = [&](int e0, bool use_r, bool dump, float (&mass32)[E], unsigned& bigbits, const uint4* staged) {
+      auto chunk_mass = [&](int e0, bool use_r, float (&mass32)[E], unsigned& bigbits, const uint4* staged) {
         auto fetch = [&](int i, float (&v)[E]) {
           if (staged != nullptr) {
             uint4 raw = staged[i * 32];
@@ -1285,6 +1285,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         float acc[E], rr[E];
         bool anybig = false;
         bigbits = 0u;
+        const float* coef = use_r ? sh.a_scale : sh.a_resid;
 #pragma unroll
         for (int k = 0; k < E; ++k) {
           acc[k] = 0.f;
@@ -1294,8 +1295,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           for (int i = 0; i < p.n; ++i) {
             float v[E];
             fetch(i, v);
-            const float co = use_r ? sh.a_scale[i] : sh.a_resid[i], rf = sh.a_ref[i];
-            const float cr = sh.a_scale[i];
+            const float co = coef[i], rf = sh.a_ref[i];
             float emax = 0.f;
 #pragma unroll
             for (int k = 0; k < E; ++k) {
@@ -1304,7 +1304,6 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               // products rounded one by one (no fused multiply-add): when r and q coincide the terms
               // cancel exactly, as they do in exact arithmetic
               acc[k] = __fadd_rn(acc[k], __fmul_rn(co, e));
-              if (dump) rr[k] = fmaf(cr, e, rr[k]);
             }
             anybig |= emax > sh.big_thr[i];
           }
@@ -1369,15 +1368,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           for (int k = 0; k < E; ++k)
             if (bigbits & (1u << k)) mass32[k] = 0.f;
         }
-        if (dump) {
-          float* out = p.dump_r + (static_cast<long long>(b) * p.P + j) * p.V;
-#pragma unroll
-          for (int k = 0; k < E; ++k)
-            if (e0 + k < p.V && !(bigbits & (1u << k))) out[e0 + k] = rr[k];
-        }
       };
       // `staged`/`k`: where the token's logits sit in shared memory (null: read them from global memory)
-      auto big_mass = [&](int e, bool use_r, bool dump, const uint4* staged, int k) -> double {
+      auto big_mass = [&](int e, bool use_r, const uint4* staged, int k) -> double {
         if (e >= p.V) return 0.0;
         double r64 = 0.0, q64 = 0.0;
         float lv[COS_MAX_MODELS];
@@ -1399,12 +1392,10 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           r64 = in ? exp2(cd * p.cT64 - static_cast<double>(sh.fsoft[1].ref)) / sh.fsoft[1].s : 0.0;
           q64 = exp2(static_cast<double>(lv[pis]) * p.cT64 - static_cast<double>(sh.fsoft[0].ref)) / sh.fsoft[0].s;
         }
-        if (dump) p.dump_r[(static_cast<long long>(b) * p.P + j) * p.V + e] = static_cast<float>(r64);
         return use_r ? r64 : fmax(0.0, r64 - q64);
       };
       // a lane's mass of one step: fp32 sum of the small tokens in token order plus the big ones in fp64
-      auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, bool dump,
-                           const uint4* staged) -> double {
+      auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, const uint4* staged) -> double {
         float ls = 0.f;
 #pragma unroll
         for (int k = 0; k < E; ++k) ls += mass32[k];
@@ -1412,7 +1403,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         while (bigbits) {  // big tokens in token order
           const int k = __ffs(bigbits) - 1;
           bigbits &= bigbits - 1;
-          own += big_mass(e0 + k, use_r, dump, staged, k);
+          own += big_mass(e0 + k, use_r, staged, k);
         }
         return own;
       };
@@ -1421,7 +1412,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       // Mass of one warp run [sb, se) in token order; the running total after every gszv steps goes to
       // rec[] (lane 0 writes; rec may be null).  Vectors of the coming steps are staged in shared memory
       // with cp.async so that a warp keeps several loads in flight although it consumes its run in order.
-      auto run_totals = [&](int sb, int se, int gszv, bool use_r, bool dump, double* rec) -> double {
+      auto run_totals = [&](int sb, int se, int gszv, bool use_r, double* rec) -> double {
         double wrun = 0.0;  // the run's total, accumulated group by group
         double lacc = 0.0;  // this lane's mass within the current group
         const int depth = (p.n <= 2) ? 4 : (p.n <= 4 ? 2 : 1);
@@ -1452,14 +1443,14 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               cp_async_wait<1>();
             else
               cp_async_wait<0>();
-            chunk_mass(e0, use_r, dump, mass32, bigbits, &myring[slot * p.n * 32]);
-            lacc += lane_mass(e0, mass32, bigbits, use_r, dump, &myring[slot * p.n * 32]);
+            chunk_mass(e0, use_r, mass32, bigbits, &myring[slot * p.n * 32]);
+            lacc += lane_mass(e0, mass32, bigbits, use_r, &myring[slot * p.n * 32]);
             if (s + depth < fe) stage_in(s + depth, slot);
             slot = (slot + 1 == depth) ? 0 : slot + 1;
             cp_async_commit();
           } else {
-            chunk_mass(e0, use_r, dump, mass32, bigbits, nullptr);
-            lacc += lane_mass(e0, mass32, bigbits, use_r, dump, nullptr);
+            chunk_mass(e0, use_r, mass32, bigbits, nullptr);
+            lacc += lane_mass(e0, mass32, bigbits, use_r, nullptr);
           }
           if (++in_group == gszv || s + 1 == se) {
             double t = lacc;
@@ -1502,7 +1493,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           float mass32[E];
           unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
-          chunk_mass(e0, use_r, false, mass32, bigbits, nullptr);
+          chunk_mass(e0, use_r, mass32, bigbits, nullptr);
           // per-token masses of this lane in fp64 (big tokens from their fp64 evaluation)
           double m64[E];
 #pragma unroll
@@ -1510,9 +1501,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           if (bigbits) {
 #pragma unroll
             for (int k = 0; k < E; ++k)
-              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, false, nullptr, k);
+              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, nullptr, k);
           }
-          const double own = lane_mass(e0, mass32, bigbits, use_r, false, nullptr);
+          const double own = lane_mass(e0, mass32, bigbits, use_r, nullptr);
           double inc = own;
 #pragma unroll
           for (int d = 1; d < 32; d <<= 1) {
@@ -1593,7 +1584,44 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         // ---- masses of this block's runs, to be added up and searched by the last block of the unit
         const int gszv = run_gsz(s_end - s_begin, kRecG);
         double* rec = emit ? p.srung + (static_cast<size_t>(b) * G + gwarp) * kRecG : nullptr;
-        const double t = run_totals(s_begin, s_end, gszv, is_bonus, p.dump_r != nullptr, rec);
+        if (p.dump_r != nullptr) {
+          // test hook: the combined distribution of this block's runs, token by token
+          float* out = p.dump_r + (static_cast<long long>(b) * p.P + j) * p.V;
+          for (int s = s_begin; s < s_end; ++s) {
+            const int e0 = (s * 32 + lane) * E;
+            float r[E];
+#pragma unroll
+            for (int k = 0; k < E; ++k) r[k] = 0.f;
+            if (MODE == kEnsembleSample) {
+              for (int i = 0; i < p.n; ++i) {
+                float v[E];
+                load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
+#pragma unroll
+                for (int k = 0; k < E; ++k) r[k] = fmaf(sh.a_scale[i], ex2_approx(fmaf(v[k], p.cT, sh.a_ref[i])), r[k]);
+              }
+            } else {
+              float cmb[E], ve[E];
+#pragma unroll
+              for (int k = 0; k < E; ++k) cmb[k] = ve[k] = 0.f;
+              for (int i = 0; i < p.n; ++i) {
+                float v[E];
+                load_chunk<DT>(row_of(i), e0, p.V, vec_ok, v);
+#pragma unroll
+                for (int k = 0; k < E; ++k) {
+                  cmb[k] = fmaf(p.w[i], v[k], cmb[k]);
+                  if (i == p.mask_model) ve[k] = v[k];
+                }
+              }
+#pragma unroll
+              for (int k = 0; k < E; ++k)
+                r[k] = (!masked || ve[k] >= thr) ? ex2_approx(fmaf(cmb[k], p.cT, ref_c)) * inv_zc : 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < E; ++k)
+              if (e0 + k < p.V) out[e0 + k] = r[k];
+          }
+        }
+        const double t = run_totals(s_begin, s_end, gszv, is_bonus, rec);
         if (lane == 0) p.wtotg[static_cast<size_t>(uidx) * G + gwarp] = t;
         // the last block of the unit to get here goes on to locate the token (fence + counter, no waiting)
         __syncthreads();
@@ -1633,7 +1661,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
           const int sb = static_cast<int>(static_cast<long long>(warp) * p.nsteps / kWarps);
           const int se = static_cast<int>(static_cast<long long>(warp + 1) * p.nsteps / kWarps);
           const int gszv = run_gsz(se - sb, kRec);
-          const double t = run_totals(sb, se, gszv, true, false, &sh.srun[warp][0]);
+          const double t = run_totals(sb, se, gszv, true, &sh.srun[warp][0]);
           if (lane == 0) sh.wtot[warp] = t;
           __syncthreads();
           if (tid == 0) {
