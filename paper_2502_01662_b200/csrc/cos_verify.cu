@@ -581,6 +581,37 @@ __device__ __forceinline__ LaneSoft soft_slice(const void* row, const Slice& sl,
   return acc;
 }
 
+// Mass of one "big" token (more than 2^-8 of some normaliser) in fp64 from the stored logits: r - q
+// clipped at zero, or r.  Rare; kept out of line so that the mass loop stays small.
+// `staged`/`k`: where the token's logits sit in shared memory (null: read them from global memory).
+template <int DT, int MODE>
+__device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* fsoft, const char* base, int e, bool use_r,
+                                              const uint4* staged, int k, bool masked, float thr, int pis) {
+  if (e >= p.V) return 0.0;
+  double r64 = 0.0, q64 = 0.0;
+  float lv[COS_MAX_MODELS];
+  if (staged != nullptr) {
+    for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::pick(staged + i * 32, k);
+  } else {
+    for (int i = 0; i < p.n; ++i)
+      lv[i] = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);  // all loads first
+  }
+  if (MODE == kEnsembleSample) {
+    for (int i = 0; i < p.n; ++i) {
+      double pr = exp2(static_cast<double>(lv[i]) * p.cT64 - static_cast<double>(fsoft[i].ref)) / fsoft[i].s;
+      r64 += p.w64[i] * pr;
+      if (i == pis) q64 = pr;
+    }
+  } else {
+    double cd = 0.0;
+    for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(lv[i]), cd);
+    bool in = !masked || (lv[p.mask_model] >= thr);
+    r64 = in ? exp2(cd * p.cT64 - static_cast<double>(fsoft[1].ref)) / fsoft[1].s : 0.0;
+    q64 = exp2(static_cast<double>(lv[pis]) * p.cT64 - static_cast<double>(fsoft[0].ref)) / fsoft[0].s;
+  }
+  return use_r ? r64 : fmax(0.0, r64 - q64);
+}
+
 // ------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------
@@ -1369,30 +1400,8 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             if (bigbits & (1u << k)) mass32[k] = 0.f;
         }
       };
-      // `staged`/`k`: where the token's logits sit in shared memory (null: read them from global memory)
       auto big_mass = [&](int e, bool use_r, const uint4* staged, int k) -> double {
-        if (e >= p.V) return 0.0;
-        double r64 = 0.0, q64 = 0.0;
-        float lv[COS_MAX_MODELS];
-        if (staged != nullptr) {
-          for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::pick(staged + i * 32, k);
-        } else {
-          for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::load1(row_of(i), e);  // all loads first
-        }
-        if (MODE == kEnsembleSample) {
-          for (int i = 0; i < p.n; ++i) {
-            double pr = exp2(static_cast<double>(lv[i]) * p.cT64 - static_cast<double>(sh.fsoft[i].ref)) / sh.fsoft[i].s;
-            r64 += p.w64[i] * pr;
-            if (i == pis) q64 = pr;
-          }
-        } else {
-          double cd = 0.0;
-          for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(lv[i]), cd);
-          bool in = !masked || (lv[p.mask_model] >= thr);
-          r64 = in ? exp2(cd * p.cT64 - static_cast<double>(sh.fsoft[1].ref)) / sh.fsoft[1].s : 0.0;
-          q64 = exp2(static_cast<double>(lv[pis]) * p.cT64 - static_cast<double>(sh.fsoft[0].ref)) / sh.fsoft[0].s;
-        }
-        return use_r ? r64 : fmax(0.0, r64 - q64);
+        return big_token_mass<DT, MODE>(p, sh.fsoft, base, e, use_r, staged, k, masked, thr, pis);
       };
       // a lane's mass of one step: fp32 sum of the small tokens in token order plus the big ones in fp64
       auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, const uint4* staged) -> double {
