@@ -642,6 +642,9 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
 
   const int cluster_id = (p.stage == 0) ? blockIdx.x / C : blockIdx.x / lparts;
+  // later stages are launched while the previous one drains (programmatic dependent launch);
+  // nothing it wrote is read before this point
+  if (p.stage >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
   const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
   if (p.stage == 0) {
@@ -1855,19 +1858,21 @@ cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int* out) {
   return cudaOccupancyMaxActiveClusters(out, reinterpret_cast<const void*>(fn), &lc);
 }
 
-cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, cudaStream_t stream) {
+cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, cudaStream_t stream, bool overlap_prev = false) {
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * cluster, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
   lc.dynamicSmemBytes = kRingBytes;
   lc.stream = stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = cluster;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = overlap_prev ? 2 : 1;
   return cudaLaunchKernelEx(&lc, fn, p);
 }
 
@@ -2112,7 +2117,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     for (int st = 1; st <= 2; ++st) {
       p.stage = st;
       p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of this launch
-      e = launch_stage(fn, p, 1, stream);
+      e = launch_stage(fn, p, 1, stream, true);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stages)", e);
       if (ctx->timing) cudaEventRecord(ctx->ev[st + 1], stream);
       ctx->ev_used = st + 2;
