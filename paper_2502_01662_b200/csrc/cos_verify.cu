@@ -861,60 +861,103 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         warp_merge_soft(accq, &sh.wsoft[warp][0], lane);
         warp_merge_soft(accc, &sh.wsoft[warp][1], lane);
         cluster_merge(sh, cluster, phase, 2, 0, 0);
-      } else {  // kLogitGreedy: combined logits in fp64, the same chain of fused multiply-adds on every token
+      } else {  // kLogitGreedy
+        // The argmax of the combined logits must be the fp64 one (the same chain of fused multiply-adds
+        // on every token, lowest index among equals).  Every token gets an fp32 value and a bound on its
+        // distance from the fp64 value; only tokens that could reach the best fp64 value seen so far are
+        // evaluated in fp64.
         double cbest = -INFINITY;
+        float cbest_lo = -INFINITY;  // a lower bound of the maximum in fp32: the best fp64 value seen by the warp, rounded down
         int cidx = kNoReject, bad = 0;
         float qbest = -INFINITY;
         int qidx = kNoReject;
-        auto see = [&](double cm, float xq, float xe, int e) {
-          if (xq > qbest) {
-            qbest = xq;
-            qidx = e;
-          }
-          if (!masked || xe >= thr) {
-            bad |= (cm != cm);
-            if (cm > cbest) {
+        const char* row0 = reinterpret_cast<const char*>(row_of(0));
+        const long long row_step = p.s_model * Elem<DT>::bytes;
+        const float kSlack = static_cast<float>(p.n) * 1.1920929e-07f;  // n * 2^-23: rounding of the fp32 chain
+        auto exact = [&](int e) {  // fp64 value of one token from the stored logits
+          double cm = 0.0;
+          for (int i = 0; i < p.n; ++i) cm = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e)), cm);
+          return cm;
+        };
+        auto consider = [&](float c32, float bnd, int e) {  // token inside the mask
+          bad |= (c32 != c32);
+          if (__fadd_ru(c32, __fmul_ru(bnd, kSlack)) >= cbest_lo) {
+            const double cm = exact(e);
+            if (cm > cbest) {  // tokens come in increasing order within a thread: ties keep the earlier one
               cbest = cm;
               cidx = e;
+              const float lo = __double2float_rd(cm);
+              if (lo > cbest_lo) cbest_lo = lo;
             }
           }
         };
         for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
-          double cmb[E];
-          float vq[E], ve[E];
+          float c32[E], bnd[E];
+          unsigned inbits = 0xffffffffu;
 #pragma unroll
-          for (int k = 0; k < E; ++k) {
-            cmb[k] = 0.0;
-            vq[k] = -INFINITY;
-            ve[k] = 0.f;
-          }
-          for (int i = 0; i < p.n; ++i) {
-            float va[E];
-            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
-            Elem<DT>::unpack(ra, va);
-            const double wa = p.w64[i];
+          for (int k = 0; k < E; ++k) c32[k] = bnd[k] = 0.f;
+          auto take = [&](int i, const uint4& raw) {
+            float x[E];
+            Elem<DT>::unpack(raw, x);
+            const float wi = p.w[i], wa = fabsf(wi);
 #pragma unroll
             for (int k = 0; k < E; ++k) {
-              bad |= !(va[k] < INFINITY);
-              cmb[k] = fma(wa, static_cast<double>(va[k]), cmb[k]);
-              if (i == p.mask_model) ve[k] = va[k];
-              if (i == pis) vq[k] = va[k];
+              bad |= !(x[k] < INFINITY);
+              c32[k] = fmaf(wi, x[k], c32[k]);
+              bnd[k] = fmaf(wa, fabsf(x[k]), bnd[k]);
             }
-          }
+            if (i == pis) {
 #pragma unroll
-          for (int k = 0; k < E; ++k) see(cmb[k], vq[k], ve[k], v * E + k);
+              for (int k = 0; k < E; ++k) {
+                if (x[k] > qbest) {
+                  qbest = x[k];
+                  qidx = v * E + k;
+                }
+              }
+            }
+            if (masked && i == p.mask_model) {
+              inbits = 0u;
+#pragma unroll
+              for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
+            }
+          };
+          const long long off = static_cast<long long>(v) * 16;
+          int i = 0;
+          for (; i + 1 < p.n; i += 2) {
+            const uint4 a0 = ldg_stream16(row0 + i * row_step + off);
+            const uint4 a1 = ldg_stream16(row0 + (i + 1) * row_step + off);
+            take(i, a0);
+            take(i + 1, a1);
+          }
+          if (i < p.n) take(i, ldg_stream16(row0 + i * row_step + off));
+#pragma unroll
+          for (int k = 0; k < E; ++k)
+            if (inbits & (1u << k)) consider(c32[k], bnd[k], v * E + k);
+          // any exact value found by a lane of the warp is a lower bound of the maximum for all of them:
+          // share the largest (floats ordered as unsigned integers, one warp-wide max)
+          {
+            const unsigned bits = __float_as_uint(cbest_lo);
+            const unsigned key = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
+            const unsigned top = __reduce_max_sync(__activemask(), key);
+            const unsigned back = top ^ ((top >> 31) ? 0x80000000u : 0xffffffffu);
+            const float shared_lo = __uint_as_float(back);
+            if (shared_lo > cbest_lo) cbest_lo = shared_lo;
+          }
         }
         for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
-          double cm = 0.0;
-          float xq = -INFINITY, xe = 0.f;
+          float c32 = 0.f, bnd = 0.f, xe = 0.f;
           for (int i = 0; i < p.n; ++i) {
             float x = Elem<DT>::load1(row_of(i), e);
             bad |= !(x < INFINITY);
-            cm = fma(p.w64[i], static_cast<double>(x), cm);
-            if (i == pis) xq = x;
+            c32 = fmaf(p.w[i], x, c32);
+            bnd = fmaf(fabsf(p.w[i]), fabsf(x), bnd);
+            if (i == pis && x > qbest) {
+              qbest = x;
+              qidx = e;
+            }
             if (i == p.mask_model) xe = x;
           }
-          see(cm, xq, xe, e);
+          if (!masked || xe >= thr) consider(c32, bnd, e);
         }
         warp_merge_arg(static_cast<double>(qbest), qidx, bad, &sh.warg[warp][1], lane);
         warp_merge_arg(cbest, cidx, bad, &sh.warg[warp][2], lane);
