@@ -68,8 +68,6 @@ struct KParams {
   int nsteps;   // ceil(V / (32 * E))
   int flags;
   int num_units, num_clusters;
-  int stage;     // 0: statistics, decisions, row scan (every unit); then for the listed units only:
-                 // 1: normalisers again with fp64 care, 2: token masses, running totals, and the token
   int parts;     // blocks that share one unit in stages 1 and 2
   int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
@@ -615,16 +613,16 @@ __device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* 
 // ------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------
-template <int DT, int MODE>
+template <int DT, int MODE, int STAGE>
 __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_constant__ KParams p) {
   constexpr int E = Elem<DT>::E;
   constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
   cg::cluster_group cluster = cg::this_cluster();
   // stage 0 shares a unit among the blocks of a cluster; stages 1 and 2 among `parts` independent
   // blocks (they meet only through global memory between launches); stage 3 uses one block per unit
-  const int lparts = (p.stage == 1 || p.stage == 2) ? p.parts : 1;  // blocks per unit in this launch
-  const int C = (p.stage == 0) ? static_cast<int>(cluster.num_blocks()) : p.parts;
-  const int rank = (p.stage == 0) ? static_cast<int>(cluster.block_rank()) : static_cast<int>(blockIdx.x % lparts);
+  const int lparts = (STAGE == 1 || STAGE == 2) ? p.parts : 1;  // blocks per unit in this launch
+  const int C = (STAGE == 0) ? static_cast<int>(cluster.num_blocks()) : p.parts;
+  const int rank = (STAGE == 0) ? static_cast<int>(cluster.block_rank()) : static_cast<int>(blockIdx.x % lparts);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gwarp = rank * kWarps + warp, G = C * kWarps;
   __shared__ Shared sh;
@@ -641,13 +639,13 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   // this block's slice of every row in sweep 1
   const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
 
-  const int cluster_id = (p.stage == 0) ? blockIdx.x / C : blockIdx.x / lparts;
+  const int cluster_id = (STAGE == 0) ? blockIdx.x / C : blockIdx.x / lparts;
   // later stages are launched while the previous one drains (programmatic dependent launch);
   // nothing it wrote is read before this point
-  if (p.stage >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (STAGE >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
   const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
-  if (p.stage == 0) {
+  if (STAGE == 0) {
     if (blockIdx.x == 0 && tid == 0) *p.job_reset = 0;  // the list of the next run starts empty
   } else {
     njobs = *p.job_count;
@@ -655,7 +653,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   }
   while (true) {
     int j, b;
-    if (p.stage == 0) {
+    if (STAGE == 0) {
       if (unit >= p.num_units) break;
       j = unit / p.B;  // earlier positions of every row come first
       b = unit % p.B;
@@ -679,7 +677,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
     const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
     const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
 
-    if (p.stage == 0) {
+    if (STAGE == 0) {
     // ---- small jobs issued before the sweep so that their latency hides behind it
     if (tid < p.n && !is_bonus && draft_ok) sh.ldraft[tid] = Elem<DT>::load1(row_of(tid), draft);
     if (warp == kWarps - 1) {
@@ -1122,7 +1120,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         sh.fsoft[tid].s = p.ustats[uidx].s[tid];
         sh.fsoft[tid].ref = p.ustats[uidx].ref[tid];
         sh.big_thr[tid] = static_cast<float>(sh.fsoft[tid].s * kBigShare);  // from the first estimate, in every stage
-        if (p.stage >= 2) {
+        if (STAGE >= 2) {
           double z = 0.0;
           for (int q = 0; q < p.parts; ++q) z += p.zpart[(static_cast<size_t>(uidx) * p.parts + q) * 8 + tid];
           sh.fsoft[tid].s = z;
@@ -1172,7 +1170,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       // ---- 2a: normalisers again, now that the references are known: terms holding more
       // than 2^-14 of a normaliser are evaluated in fp64 and kept out of the fp32 sums, so
       // a dominant token neither absorbs the small ones nor carries the fast exp's error
-      if (p.stage == 1) {
+      if (STAGE == 1) {
       if (MODE == kEnsembleSample) {
         for (int i = 0; i < p.n; ++i) {
           const void* row = row_of(i);
@@ -1635,7 +1633,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       auto run_gsz = [&](int nst, int nrec) { return (nst + nrec - 1) / nrec > 1 ? (nst + nrec - 1) / nrec : 1; };
 
       bool do_locate = false;
-      if (p.stage == 2) {
+      if (STAGE == 2) {
         // ---- masses of this block's runs, to be added up and searched by the last block of the unit
         const int gszv = run_gsz(s_end - s_begin, kRecG);
         double* rec = emit ? p.srung + (static_cast<size_t>(b) * G + gwarp) * kRecG : nullptr;
@@ -1732,14 +1730,14 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       }
       }  // stages 2 and 3
     }
-    if (p.stage == 0 && rank == 0 && tid == 0) {
+    if (STAGE == 0 && rank == 0 && tid == 0) {
       const Decision& d = sh.dec;
       publish_unit(p, b, j, d.accept, d.status, d.cand, d.drawable, d.ratio, d.r_d, d.q_d, d.S);
     }
     // No barrier here: everything the next unit writes before its first block barrier
     // (ldraft, next_local, u_acc/u_smp, warp partials) is read only before this point; stage 1
     // starts every unit with a block barrier of its own.
-    if (p.stage >= 1) __syncthreads();
+    if (STAGE >= 1) __syncthreads();
     unit = next_unit;
   }
   cluster.sync();  // no block leaves while a peer may still read its shared memory
@@ -1790,17 +1788,20 @@ namespace {
 
 using KernelFn = void (*)(const KParams);
 
-KernelFn pick_kernel(int dtype, int mode) {
-#define COS_CASE(DT, M) \
-  if (dtype == DT && mode == M) return cos_verify_kernel<DT, M>;
-  COS_CASE(COS_DTYPE_F32, kEnsembleSample)
-  COS_CASE(COS_DTYPE_F32, kLogitSample)
-  COS_CASE(COS_DTYPE_F32, kEnsembleGreedy)
-  COS_CASE(COS_DTYPE_F32, kLogitGreedy)
-  COS_CASE(COS_DTYPE_BF16, kEnsembleSample)
-  COS_CASE(COS_DTYPE_BF16, kLogitSample)
-  COS_CASE(COS_DTYPE_BF16, kEnsembleGreedy)
-  COS_CASE(COS_DTYPE_BF16, kLogitGreedy)
+KernelFn pick_kernel(int dtype, int mode, int stage) {
+  // one instantiation per stage, so that each gets its own register allocation; greedy modes have stage 0 only
+#define COS_CASE(DT, M, S) \
+  if (dtype == DT && mode == M && stage == S) return cos_verify_kernel<DT, M, S>;
+#define COS_SAMPLING(DT, M) COS_CASE(DT, M, 0) COS_CASE(DT, M, 1) COS_CASE(DT, M, 2)
+  COS_SAMPLING(COS_DTYPE_F32, kEnsembleSample)
+  COS_SAMPLING(COS_DTYPE_F32, kLogitSample)
+  COS_CASE(COS_DTYPE_F32, kEnsembleGreedy, 0)
+  COS_CASE(COS_DTYPE_F32, kLogitGreedy, 0)
+  COS_SAMPLING(COS_DTYPE_BF16, kEnsembleSample)
+  COS_SAMPLING(COS_DTYPE_BF16, kLogitSample)
+  COS_CASE(COS_DTYPE_BF16, kEnsembleGreedy, 0)
+  COS_CASE(COS_DTYPE_BF16, kLogitGreedy, 0)
+#undef COS_SAMPLING
 #undef COS_CASE
   return nullptr;
 }
@@ -1890,7 +1891,7 @@ cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int* out) {
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(cluster * sm_count, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = kRingBytes;
+  lc.dynamicSmemBytes = 0;  // only stage 0 runs in clusters, and it stages nothing
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = cluster;
@@ -1901,11 +1902,19 @@ cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int* out) {
   return cudaOccupancyMaxActiveClusters(out, reinterpret_cast<const void*>(fn), &lc);
 }
 
-cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, cudaStream_t stream, bool overlap_prev = false) {
+// attributes the kernels of one (dtype, mode) need before their first launch
+cudaError_t prepare_kernels(int dtype, int mode, int cluster_size);
+
+int stage_smem(int stage) { return stage == 2 ? kRingBytes : 0; }  // the staging ring of the token-mass sweep
+
+cudaError_t launch_stage(int dtype, int mode, int stage, const KParams& p, int cluster, cudaStream_t stream,
+                         bool overlap_prev = false) {
+  KernelFn fn = pick_kernel(dtype, mode, stage);
+  if (fn == nullptr) return cudaErrorInvalidDeviceFunction;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(p.num_clusters) * cluster, 1, 1);
   lc.blockDim = dim3(kThreads, 1, 1);
-  lc.dynamicSmemBytes = kRingBytes;
+  lc.dynamicSmemBytes = stage_smem(stage);
   lc.stream = stream;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
@@ -1917,6 +1926,18 @@ cudaError_t launch_stage(KernelFn fn, const KParams& p, int cluster, cudaStream_
   lc.attrs = at;
   lc.numAttrs = overlap_prev ? 2 : 1;
   return cudaLaunchKernelEx(&lc, fn, p);
+}
+
+cudaError_t prepare_kernels(int dtype, int mode, int cluster_size) {
+  const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
+  cudaError_t e = cudaSuccess;
+  if (draws)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, 2)),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+  if (e == cudaSuccess && cluster_size > 8)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, 0)),
+                             cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  return e;
 }
 
 cos_status cuda_fail(cos_verify_ctx* ctx, const char* what, cudaError_t e) {
@@ -1968,18 +1989,11 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   }
   ctx->sm_count = prop.multiProcessorCount;
   ctx->parts = choose_parts(*config, config->max_batch, ctx->sm_count);
-  KernelFn fn = pick_kernel(config->dtype, mode_of(*config));
-  e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+  KernelFn fn = pick_kernel(config->dtype, mode_of(*config), 0);
+  e = prepare_kernels(config->dtype, mode_of(*config), config->cluster_size);
   if (e != cudaSuccess) {
     delete ctx;
-    return cuda_fail(nullptr, "cudaFuncSetAttribute(shared memory)", e);
-  }
-  if (config->cluster_size > 8) {
-    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-    if (e != cudaSuccess) {
-      delete ctx;
-      return cuda_fail(nullptr, "cluster size above 8 not available", e);
-    }
+    return cuda_fail(nullptr, "cudaFuncSetAttribute (shared memory or cluster size)", e);
   }
   for (int k = 0; k < 5; ++k) {
     const int cs = 1 << k;
@@ -2133,7 +2147,6 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.parts = ctx->parts;
   p.max_jobs = p.num_units + a->batch;
 
-  KernelFn fn = pick_kernel(c.dtype, mode_of(c));
   const int mode = mode_of(c);
   const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
   // stage 0: every unit once (statistics, accept tests, row scans)
@@ -2143,11 +2156,10 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     ctx->err = "no cluster of the chosen size fits on the device";
     return COS_ERR_UNSUPPORTED;
   }
-  p.stage = 0;
   p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
   ctx->scratch_dirty = true;  // cleared below once the launches are known to be queued
   if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
-  e = launch_stage(fn, p, c0, stream);
+  e = launch_stage(c.dtype, mode, 0, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
   ctx->ev_used = 2;
@@ -2158,9 +2170,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     const int most = all ? p.max_jobs : a->batch;
     const int cap = 4096;  // a block walks the job list with a stride, so the grid may be smaller than the list
     for (int st = 1; st <= 2; ++st) {
-      p.stage = st;
       p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of this launch
-      e = launch_stage(fn, p, 1, stream, true);
+      e = launch_stage(c.dtype, mode, st, p, 1, stream, true);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stages)", e);
       if (ctx->timing) cudaEventRecord(ctx->ev[st + 1], stream);
       ctx->ev_used = st + 2;
@@ -2358,7 +2369,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e = cudaSetDevice(c.device);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaSetDevice", e);
-  KernelFn fn = pick_kernel(c.dtype, mode_of(c));
+  KernelFn fn = pick_kernel(c.dtype, mode_of(c), 0);
   if (!g_static_ready[c.device]) {
     // once per device, with that device current: the device address of the built-in array
     void* addr = nullptr;
@@ -2367,9 +2378,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     g_static_addr[c.device] = static_cast<unsigned char*>(addr);
     g_static_ready[c.device] = true;
   }
-  e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
-  if (e == cudaSuccess && c.cluster_size > 8)
-    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  e = prepare_kernels(c.dtype, mode_of(c), c.cluster_size);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaFuncSetAttribute", e);
   int sm_count = 0;
   e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, c.device);
@@ -2455,17 +2464,15 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.parts = 1;
   p.max_jobs = p.num_units + a->batch;
 
-  p.stage = 0;
   p.num_clusters = p.num_units < mc0 ? p.num_units : mc0;
-  e = launch_stage(fn, p, c0, stream);
+  e = launch_stage(c.dtype, mode_of(c), 0, p, c0, stream);
   if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (stage 0)", e);
   if (mode_of(c) == kEnsembleSample || mode_of(c) == kLogitSample) {
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
     for (int st = 1; st <= 2; ++st) {
-      p.stage = st;
       p.num_clusters = most < 4096 ? most : 4096;
-      e = launch_stage(fn, p, 1, stream);
+      e = launch_stage(c.dtype, mode_of(c), st, p, 1, stream);
       if (e != cudaSuccess) return cuda_fail(nullptr, "kernel launch (drawing stages)", e);
     }
   }
