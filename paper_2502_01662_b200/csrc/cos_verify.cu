@@ -610,6 +610,18 @@ __device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* 
   return use_r ? r64 : fmax(0.0, r64 - q64);
 }
 
+// Combined logit of one token in fp64, from the stored logits: the chain of fused multiply-adds that
+// defines the greedy argmax (Eq. 5 at T = 0).  Out of line: the sweep calls it for a handful of tokens.
+template <int DT>
+__device__ __noinline__ double exact_combined(const KParams& p, const char* base, int e) {
+  double cm = 0.0;
+  for (int i = 0; i < p.n; ++i) {
+    const void* row = base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes;
+    cm = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row, e)), cm);
+  }
+  return cm;
+}
+
 // ------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------
@@ -872,15 +884,10 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
         const char* row0 = reinterpret_cast<const char*>(row_of(0));
         const long long row_step = p.s_model * Elem<DT>::bytes;
         const float kSlack = static_cast<float>(p.n) * 1.1920929e-07f;  // n * 2^-23: rounding of the fp32 chain
-        auto exact = [&](int e) {  // fp64 value of one token from the stored logits
-          double cm = 0.0;
-          for (int i = 0; i < p.n; ++i) cm = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e)), cm);
-          return cm;
-        };
         auto consider = [&](float c32, float bnd, int e) {  // token inside the mask
           bad |= (c32 != c32);
-          if (__fadd_ru(c32, __fmul_ru(bnd, kSlack)) >= cbest_lo) {
-            const double cm = exact(e);
+          if (__fmaf_ru(bnd, kSlack, c32) >= cbest_lo) {
+            const double cm = exact_combined<DT>(p, base, e);
             if (cm > cbest) {  // tokens come in increasing order within a thread: ties keep the earlier one
               cbest = cm;
               cidx = e;
@@ -889,7 +896,25 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
             }
           }
         };
+        // the vectors of the first two models are fetched one trip ahead: four loads in flight per thread
+        const bool pair = (p.n >= 2);
+        uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+        {
+          const int v0 = sl.v_lo + tid;
+          if (v0 < sl.v_hi) {
+            nx0 = ldg_stream16(row0 + static_cast<long long>(v0) * 16);
+            if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(v0) * 16);
+          }
+        }
         for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+          const uint4 a0 = nx0, a1 = nx1;
+          {
+            const int vn = v + kThreads;
+            if (vn < sl.v_hi) {
+              nx0 = ldg_stream16(row0 + static_cast<long long>(vn) * 16);
+              if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(vn) * 16);
+            }
+          }
           float c32[E], bnd[E];
           unsigned inbits = 0xffffffffu;
 #pragma unroll
@@ -905,12 +930,14 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               bnd[k] = fmaf(wa, fabsf(x[k]), bnd[k]);
             }
             if (i == pis) {
+              float xm = x[0];
 #pragma unroll
-              for (int k = 0; k < E; ++k) {
-                if (x[k] > qbest) {
-                  qbest = x[k];
-                  qidx = v * E + k;
-                }
+              for (int k = 1; k < E; ++k) xm = fmaxf(xm, x[k]);
+              if (xm > qbest) {  // rare after the first few vectors; the first of equal entries wins
+                qbest = xm;
+#pragma unroll
+                for (int k = E - 1; k >= 0; --k)
+                  if (x[k] == xm) qidx = v * E + k;
               }
             }
             if (masked && i == p.mask_model) {
@@ -919,18 +946,24 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
               for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
             }
           };
+          take(0, a0);
+          if (pair) take(1, a1);
           const long long off = static_cast<long long>(v) * 16;
-          int i = 0;
-          for (; i + 1 < p.n; i += 2) {
-            const uint4 a0 = ldg_stream16(row0 + i * row_step + off);
-            const uint4 a1 = ldg_stream16(row0 + (i + 1) * row_step + off);
-            take(i, a0);
-            take(i + 1, a1);
-          }
-          if (i < p.n) take(i, ldg_stream16(row0 + i * row_step + off));
+          for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + off));
+          // upper bounds of the fp64 values; one comparison decides whether any entry of the vector can matter.
+          // The sum only carries a NaN (or an infinity of each sign) to the check below.
+          float tmax = -INFINITY, tsum = 0.f;
 #pragma unroll
-          for (int k = 0; k < E; ++k)
-            if (inbits & (1u << k)) consider(c32[k], bnd[k], v * E + k);
+          for (int k = 0; k < E; ++k) {
+            const float t = (inbits & (1u << k)) ? __fmaf_ru(bnd[k], kSlack, c32[k]) : -INFINITY;
+            tmax = fmaxf(tmax, t);
+            tsum += t;
+          }
+          if (tmax >= cbest_lo || tsum != tsum) {
+#pragma unroll
+            for (int k = 0; k < E; ++k)
+              if (inbits & (1u << k)) consider(c32[k], bnd[k], v * E + k);
+          }
           // any exact value found by a lane of the warp is a lower bound of the maximum for all of them:
           // share the largest (floats ordered as unsigned integers, one warp-wide max)
           {
