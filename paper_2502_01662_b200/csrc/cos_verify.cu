@@ -622,6 +622,411 @@ __device__ __noinline__ double exact_combined(const KParams& p, const char* base
   return cm;
 }
 
+// Sweep 1 of one (row, position): this thread's share of the slice `sl` of every model's row, merged
+// over the warp into the warp's slots.  Ensemble sampling: soft slot i = softmax statistics of model i.
+// Ensemble greedy: arg slot i = argmax of model i.  Logit-level sampling: soft slot 0 = proposer,
+// soft slot 1 = combined logits.  Logit-level greedy: arg slot 1 = proposer argmax, arg slot 2 =
+// combined argmax.  `thr` is the plausibility threshold (logit-level modes with a mask).
+template <int DT, int MODE>
+__device__ __forceinline__ void sweep_unit(const KParams& p, const char* base, const Slice& sl, int pis, bool masked,
+                                           float thr, SoftPart* wsoft, ArgPart* warg) {
+  constexpr int E = Elem<DT>::E;
+  const int tid = threadIdx.x, lane = tid & 31;
+  auto row_of = [&](int i) -> const void* { return base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes; };
+  if (MODE == kEnsembleSample) {
+    for (int i = 0; i < p.n; ++i) {
+      LaneSoft acc = soft_slice<DT>(row_of(i), sl, tid, p.cT);
+      warp_merge_soft(acc, &wsoft[i], lane);
+    }
+  } else if (MODE == kEnsembleGreedy) {
+    for (int i = 0; i < p.n; ++i) {
+      const void* row = row_of(i);
+      float best = -INFINITY;
+      int bidx = kNoReject, bad = 0;
+      auto see = [&](float x, int e) {
+        bad |= !(x < INFINITY);
+        if (x > best) {
+          best = x;
+          bidx = e;
+        }
+      };
+      for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+        float x[E];
+        uint4 raw = ldg_stream16(reinterpret_cast<const char*>(row) + static_cast<long long>(v) * 16);
+        Elem<DT>::unpack(raw, x);
+#pragma unroll
+        for (int k = 0; k < E; ++k) see(x[k], v * E + k);
+      }
+      for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) see(Elem<DT>::load1(row, e), e);
+      warp_merge_arg(static_cast<double>(best), bidx, bad, &warg[i], lane);
+    }
+  } else if (MODE == kLogitSample) {
+    LaneSoft accq, accc;
+    const char* row0 = reinterpret_cast<const char*>(row_of(0));
+    const long long row_step = p.s_model * Elem<DT>::bytes;
+    // fixed reference exponents seeded from the thread's first vector; overflow or a non-finite input
+    // falls back to the running-maximum form (second pass)
+    for (int pass = 0; pass < 2; ++pass) {
+      const bool fixed = (pass == 0);
+      accq.init();
+      accc.init();
+      bool seeded_q = false, seeded_c = false;
+      // one model's vector: add to the combined logits; the proposer's row also feeds its own softmax,
+      // the expert's row yields the mask bits
+      auto take = [&](int i, const uint4& raw, float (&cmb)[E], unsigned& inbits) {
+        float x[E];
+        Elem<DT>::unpack(raw, x);
+        const float wi = p.w[i];
+#pragma unroll
+        for (int k = 0; k < E; ++k) cmb[k] = fmaf(wi, x[k], cmb[k]);
+        if (i == pis) {
+          if (fixed) {
+            if (!seeded_q) {
+              accq.seed(x, p.cT);
+              seeded_q = true;
+            }
+            accq.add_fixed(x, p.cT);
+          } else {
+            accq.add_online(x, p.cT);
+          }
+        }
+        if (masked && i == p.mask_model) {
+          inbits = 0u;
+#pragma unroll
+          for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
+        }
+      };
+      auto finish = [&](float (&cmb)[E], unsigned inbits) {
+        if (masked) {
+#pragma unroll
+          for (int k = 0; k < E; ++k) cmb[k] = (inbits & (1u << k)) ? cmb[k] : -INFINITY;
+        }
+        if (fixed) {
+          if (!seeded_c) {
+            accc.seed(cmb, p.cT);
+            seeded_c = true;
+          }
+          accc.add_fixed(cmb, p.cT);
+        } else {
+          accc.add_online(cmb, p.cT);
+        }
+      };
+      for (int v = sl.v_lo + tid; v < sl.v_hi; v += 2 * kThreads) {
+        const bool have_b = (v + kThreads < sl.v_hi);
+        const long long oa = static_cast<long long>(v) * 16;
+        const long long ob = have_b ? oa + static_cast<long long>(kThreads) * 16 : oa;
+        float ca[E], cb[E];
+        unsigned ba = 0xffffffffu, bb = 0xffffffffu;
+#pragma unroll
+        for (int k = 0; k < E; ++k) ca[k] = cb[k] = 0.f;
+        int i = 0;
+        for (; i + 1 < p.n; i += 2) {  // two models, two vectors: four loads in flight
+          const char* r0 = row0 + i * row_step;
+          const char* r1 = r0 + row_step;
+          const uint4 a0 = ldg_stream16(r0 + oa), b0 = ldg_stream16(r0 + ob);
+          const uint4 a1 = ldg_stream16(r1 + oa), b1 = ldg_stream16(r1 + ob);
+          take(i, a0, ca, ba);
+          take(i + 1, a1, ca, ba);
+          if (have_b) {
+            take(i, b0, cb, bb);
+            take(i + 1, b1, cb, bb);
+          }
+        }
+        if (i < p.n) {
+          const char* r0 = row0 + i * row_step;
+          const uint4 a0 = ldg_stream16(r0 + oa), b0 = ldg_stream16(r0 + ob);
+          take(i, a0, ca, ba);
+          if (have_b) take(i, b0, cb, bb);
+        }
+        finish(ca, ba);
+        if (have_b) finish(cb, bb);
+      }
+      for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+        float cmb = 0.f, xq = -INFINITY, xe = 0.f;
+        for (int i = 0; i < p.n; ++i) {
+          float x = Elem<DT>::load1(row_of(i), e);
+          cmb = fmaf(p.w[i], x, cmb);
+          if (i == pis) xq = x;
+          if (i == p.mask_model) xe = x;
+        }
+        if (masked && !(xe >= thr)) cmb = -INFINITY;
+        accq.add_online1(xq, p.cT);
+        accc.add_online1(cmb, p.cT);
+      }
+      if ((accq.s < INFINITY) && (accc.s < INFINITY)) break;
+    }
+    warp_merge_soft(accq, &wsoft[0], lane);
+    warp_merge_soft(accc, &wsoft[1], lane);
+  } else {
+    // The argmax of the combined logits must be the fp64 one (the same chain of fused multiply-adds
+    // on every token, lowest index among equals).  Every token gets an fp32 value and a bound on its
+    // distance from the fp64 value; only tokens that could reach the best fp64 value seen so far are
+    // evaluated in fp64.
+    double cbest = -INFINITY;
+    float cbest_lo = -INFINITY;  // a lower bound of the maximum in fp32: the best fp64 value seen by the warp, rounded down
+    int cidx = kNoReject, bad = 0;
+    float qbest = -INFINITY;
+    int qidx = kNoReject;
+    const char* row0 = reinterpret_cast<const char*>(row_of(0));
+    const long long row_step = p.s_model * Elem<DT>::bytes;
+    const float kSlack = static_cast<float>(p.n) * 1.1920929e-07f;  // n * 2^-23: rounding of the fp32 chain
+    auto consider = [&](float c32, float bnd, int e) {  // token inside the mask
+      bad |= (c32 != c32);
+      if (__fmaf_ru(bnd, kSlack, c32) >= cbest_lo) {
+        const double cm = exact_combined<DT>(p, base, e);
+        if (cm > cbest) {  // tokens come in increasing order within a thread: ties keep the earlier one
+          cbest = cm;
+          cidx = e;
+          const float lo = __double2float_rd(cm);
+          if (lo > cbest_lo) cbest_lo = lo;
+        }
+      }
+    };
+    // the vectors of the first two models are fetched one trip ahead: four loads in flight per thread
+    const bool pair = (p.n >= 2);
+    uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+    {
+      const int v0 = sl.v_lo + tid;
+      if (v0 < sl.v_hi) {
+        nx0 = ldg_stream16(row0 + static_cast<long long>(v0) * 16);
+        if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(v0) * 16);
+      }
+    }
+    for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+      const uint4 a0 = nx0, a1 = nx1;
+      {
+        const int vn = v + kThreads;
+        if (vn < sl.v_hi) {
+          nx0 = ldg_stream16(row0 + static_cast<long long>(vn) * 16);
+          if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(vn) * 16);
+        }
+      }
+      float c32[E], bnd[E];
+      unsigned inbits = 0xffffffffu;
+#pragma unroll
+      for (int k = 0; k < E; ++k) c32[k] = bnd[k] = 0.f;
+      auto take = [&](int i, const uint4& raw) {
+        float x[E];
+        Elem<DT>::unpack(raw, x);
+        const float wi = p.w[i], wa = fabsf(wi);
+#pragma unroll
+        for (int k = 0; k < E; ++k) {
+          bad |= !(x[k] < INFINITY);
+          c32[k] = fmaf(wi, x[k], c32[k]);
+          bnd[k] = fmaf(wa, fabsf(x[k]), bnd[k]);
+        }
+        if (i == pis) {
+          float xm = x[0];
+#pragma unroll
+          for (int k = 1; k < E; ++k) xm = fmaxf(xm, x[k]);
+          if (xm > qbest) {  // rare after the first few vectors; the first of equal entries wins
+            qbest = xm;
+#pragma unroll
+            for (int k = E - 1; k >= 0; --k)
+              if (x[k] == xm) qidx = v * E + k;
+          }
+        }
+        if (masked && i == p.mask_model) {
+          inbits = 0u;
+#pragma unroll
+          for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
+        }
+      };
+      take(0, a0);
+      if (pair) take(1, a1);
+      const long long off = static_cast<long long>(v) * 16;
+      for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + off));
+      // upper bounds of the fp64 values; one comparison decides whether any entry of the vector can matter.
+      // The sum only carries a NaN (or an infinity of each sign) to the check below.
+      float tmax = -INFINITY, tsum = 0.f;
+#pragma unroll
+      for (int k = 0; k < E; ++k) {
+        const float t = (inbits & (1u << k)) ? __fmaf_ru(bnd[k], kSlack, c32[k]) : -INFINITY;
+        tmax = fmaxf(tmax, t);
+        tsum += t;
+      }
+      if (tmax >= cbest_lo || tsum != tsum) {
+#pragma unroll
+        for (int k = 0; k < E; ++k)
+          if (inbits & (1u << k)) consider(c32[k], bnd[k], v * E + k);
+      }
+      // any exact value found by a lane of the warp is a lower bound of the maximum for all of them:
+      // share the largest (floats ordered as unsigned integers, one warp-wide max)
+      {
+        const unsigned bits = __float_as_uint(cbest_lo);
+        const unsigned key = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
+        const unsigned top = __reduce_max_sync(__activemask(), key);
+        const unsigned back = top ^ ((top >> 31) ? 0x80000000u : 0xffffffffu);
+        const float shared_lo = __uint_as_float(back);
+        if (shared_lo > cbest_lo) cbest_lo = shared_lo;
+      }
+    }
+    for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+      float c32 = 0.f, bnd = 0.f, xe = 0.f;
+      for (int i = 0; i < p.n; ++i) {
+        float x = Elem<DT>::load1(row_of(i), e);
+        bad |= !(x < INFINITY);
+        c32 = fmaf(p.w[i], x, c32);
+        bnd = fmaf(fabsf(p.w[i]), fabsf(x), bnd);
+        if (i == pis && x > qbest) {
+          qbest = x;
+          qidx = e;
+        }
+        if (i == p.mask_model) xe = x;
+      }
+      if (!masked || xe >= thr) consider(c32, bnd, e);
+    }
+    warp_merge_arg(static_cast<double>(qbest), qidx, bad, &warg[1], lane);
+    warp_merge_arg(cbest, cidx, bad, &warg[2], lane);
+  }
+}
+
+// The accept test of one (row, position) from the merged statistics in shared memory (Eq. 6), taken
+// by one thread in fp64; greedy modes also settle the replacement token here.  Reads fsoft / farg /
+// pdraft / ldraft / u_acc / u_smp / thr32, writes dec and big_thr.
+template <int DT, int MODE>
+__device__ __forceinline__ void decide_unit(const KParams& p, Shared& sh, bool is_bonus, int draft, bool draft_ok,
+                                            int pi, bool pi_ok, int pis, bool masked) {
+  constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
+  const double kNaN = __longlong_as_double(0x7ff8000000000000LL);
+  const double kInf = __longlong_as_double(0x7ff0000000000000LL);
+  Decision& d = sh.dec;
+  const double u_acc = sh.u_acc;
+  d.accept = 0;
+  d.status = 0;
+  d.want_sample = 0;
+  d.cand = -1;
+  d.natoms = 0;
+  d.ratio = d.r_d = d.q_d = d.S = kNaN;
+  bool finite = pi_ok;
+  if (kSample) {
+    const int nsoft = (MODE == kEnsembleSample) ? p.n : 2;
+    for (int k = 0; k < nsoft; ++k) {
+      const SoftPart& f = sh.fsoft[k];
+      finite = finite && isfinite(f.ref) && isfinite(f.s) && (f.s > 0.0);
+    }
+    if (masked && sh.farg[0].bad) finite = false;
+    if (!finite) {
+      d.status |= COS_ROW_NONFINITE;
+    } else {
+      for (int k = 0; k < nsoft; ++k) sh.big_thr[k] = static_cast<float>(sh.fsoft[k].s * kBigShare);
+      if (!is_bonus) {
+        if (draft_ok) {
+          double r_d = 0.0, q_d = 0.0;
+          if (MODE == kEnsembleSample) {
+            for (int i = 0; i < p.n; ++i) {
+              r_d += p.w64[i] * sh.pdraft[i];
+              if (i == pi) q_d = sh.pdraft[i];
+            }
+          } else {
+            double cd = 0.0;
+            for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(sh.ldraft[i]), cd);
+            bool in = !masked || (sh.ldraft[p.mask_model] >= sh.thr32);
+            r_d = in ? exp2(cd * p.cT64 - static_cast<double>(sh.fsoft[1].ref)) / sh.fsoft[1].s : 0.0;
+            double lq = static_cast<double>(sh.ldraft[pi]);
+            q_d = exp2(lq * p.cT64 - static_cast<double>(sh.fsoft[0].ref)) / sh.fsoft[0].s;
+          }
+          d.r_d = r_d;
+          d.q_d = q_d;
+          if (q_d > 0.0) {
+            d.ratio = r_d / q_d;
+          } else {
+            d.status |= COS_ROW_Q_ZERO;
+            d.ratio = (r_d > 0.0) ? kInf : 0.0;
+          }
+          d.accept = (u_acc <= fmin(1.0, d.ratio)) ? 1 : 0;
+        } else {
+          d.status |= COS_ROW_BAD_DRAFT;
+        }
+      }
+      d.want_sample = is_bonus || !d.accept;
+    }
+  } else {
+    // greedy: distributions are atoms at lowest-index argmaxes
+    int qtok;
+    if (MODE == kEnsembleGreedy) {
+      for (int i = 0; i < p.n; ++i) finite = finite && !sh.farg[i].bad && isfinite(sh.farg[i].val);
+      qtok = sh.farg[pis].idx;
+    } else {
+      finite = finite && !sh.farg[1].bad && !sh.farg[2].bad && isfinite(sh.farg[1].val) && isfinite(sh.farg[2].val);
+      if (masked && sh.farg[0].bad) finite = false;
+      qtok = sh.farg[1].idx;
+    }
+    if (!finite) {
+      d.status |= COS_ROW_NONFINITE;
+    } else {
+      // atoms of r, sorted by token, masses accumulated in model order
+      if (MODE == kEnsembleGreedy) {
+        for (int i = 0; i < p.n; ++i) {
+          int t = sh.farg[i].idx, pos = 0;
+          while (pos < d.natoms && d.atom_tok[pos] < t) ++pos;
+          if (pos < d.natoms && d.atom_tok[pos] == t) {
+            d.atom_mass[pos] += p.w64[i];
+          } else {
+            for (int k = d.natoms; k > pos; --k) {
+              d.atom_tok[k] = d.atom_tok[k - 1];
+              d.atom_mass[k] = d.atom_mass[k - 1];
+            }
+            d.atom_tok[pos] = t;
+            d.atom_mass[pos] = 0.0 + p.w64[i];
+            ++d.natoms;
+          }
+        }
+      } else {
+        d.natoms = 1;
+        d.atom_tok[0] = sh.farg[2].idx;
+        d.atom_mass[0] = 1.0;
+      }
+      auto r_at = [&](int t) {
+        for (int k = 0; k < d.natoms; ++k)
+          if (d.atom_tok[k] == t) return d.atom_mass[k];
+        return 0.0;
+      };
+      bool use_r = is_bonus;
+      if (!is_bonus) {
+        if (draft_ok) {
+          d.r_d = r_at(draft);
+          d.q_d = (draft == qtok) ? 1.0 : 0.0;
+          if (d.q_d > 0.0) {
+            d.ratio = d.r_d / d.q_d;
+          } else {
+            d.status |= COS_ROW_Q_ZERO;
+            d.ratio = (d.r_d > 0.0) ? kInf : 0.0;
+          }
+          d.accept = (u_acc <= fmin(1.0, d.ratio)) ? 1 : 0;
+        } else {
+          d.status |= COS_ROW_BAD_DRAFT;
+        }
+        // residual max(0, r - q) over the atoms, summed in token order
+        double S = 0.0;
+        for (int k = 0; k < d.natoms; ++k) S += fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
+        d.S = S;
+        if (!(S > 0.0)) {
+          use_r = true;
+          if (!d.accept) d.status |= COS_ROW_RESIDUAL_EMPTY;
+        }
+      }
+      // inverse CDF over the atoms (token order): smallest k with running sum >= u * total
+      double total = 0.0;
+      for (int k = 0; k < d.natoms; ++k)
+        total += use_r ? d.atom_mass[k] : fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
+      const double target = sh.u_smp * total;
+      double run = 0.0;
+      int lastpos = -1;
+      d.cand = -1;
+      for (int k = 0; k < d.natoms; ++k) {
+        double m = use_r ? d.atom_mass[k] : fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
+        run += m;
+        if (m > 0.0) lastpos = d.atom_tok[k];
+        if (d.cand < 0 && m > 0.0 && run >= target) d.cand = d.atom_tok[k];
+      }
+      if (d.cand < 0) d.cand = lastpos;
+    }
+  }
+  d.need2 = 0;  // tokens are drawn by stage 1, for the one position per row that needs it
+  d.drawable = (kSample && finite) ? 1 : 0;
+}
+
 // ------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------
@@ -708,10 +1113,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
 
     // ================================ sweep 1: statistics ================================
     if (MODE == kEnsembleSample) {
-      for (int i = 0; i < p.n; ++i) {
-        LaneSoft acc = soft_slice<DT>(row_of(i), sl, tid, p.cT);
-        warp_merge_soft(acc, &sh.wsoft[warp][i], lane);
-      }
+      sweep_unit<DT, MODE>(p, base, sl, pis, false, 0.f, &sh.wsoft[warp][0], &sh.warg[warp][0]);
       cluster_merge(sh, cluster, phase, p.n, 0, 0);
       if (tid < p.n && !is_bonus && draft_ok) {
         // probability of the draft under model tid, with the constant the sweep used
@@ -719,27 +1121,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
                          sh.fsoft[tid].s;
       }
     } else if (MODE == kEnsembleGreedy) {
-      for (int i = 0; i < p.n; ++i) {
-        const void* row = row_of(i);
-        float best = -INFINITY;
-        int bidx = kNoReject, bad = 0;
-        auto see = [&](float x, int e) {
-          bad |= !(x < INFINITY);
-          if (x > best) {
-            best = x;
-            bidx = e;
-          }
-        };
-        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
-          float x[E];
-          uint4 raw = ldg_stream16(reinterpret_cast<const char*>(row) + static_cast<long long>(v) * 16);
-          Elem<DT>::unpack(raw, x);
-#pragma unroll
-          for (int k = 0; k < E; ++k) see(x[k], v * E + k);
-        }
-        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) see(Elem<DT>::load1(row, e), e);
-        warp_merge_arg(static_cast<double>(best), bidx, bad, &sh.warg[warp][i], lane);
-      }
+      sweep_unit<DT, MODE>(p, base, sl, pis, false, 0.f, &sh.wsoft[warp][0], &sh.warg[warp][0]);
       cluster_merge(sh, cluster, phase, 0, 0, p.n);
     } else {
       // logit-level combine.  soft slot 0 = proposer, soft slot 1 = combined logits;
@@ -774,224 +1156,10 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
       }
       const float thr = masked ? sh.thr32 : -INFINITY;
       if (MODE == kLogitSample) {
-        LaneSoft accq, accc;
-        const char* row0 = reinterpret_cast<const char*>(row_of(0));
-        const long long row_step = p.s_model * Elem<DT>::bytes;
-        // fixed reference exponents seeded from the thread's first vector; overflow or a non-finite input
-        // falls back to the running-maximum form (second pass)
-        for (int pass = 0; pass < 2; ++pass) {
-          const bool fixed = (pass == 0);
-          accq.init();
-          accc.init();
-          bool seeded_q = false, seeded_c = false;
-          // one model's vector: add to the combined logits; the proposer's row also feeds its own softmax,
-          // the expert's row yields the mask bits
-          auto take = [&](int i, const uint4& raw, float (&cmb)[E], unsigned& inbits) {
-            float x[E];
-            Elem<DT>::unpack(raw, x);
-            const float wi = p.w[i];
-#pragma unroll
-            for (int k = 0; k < E; ++k) cmb[k] = fmaf(wi, x[k], cmb[k]);
-            if (i == pis) {
-              if (fixed) {
-                if (!seeded_q) {
-                  accq.seed(x, p.cT);
-                  seeded_q = true;
-                }
-                accq.add_fixed(x, p.cT);
-              } else {
-                accq.add_online(x, p.cT);
-              }
-            }
-            if (masked && i == p.mask_model) {
-              inbits = 0u;
-#pragma unroll
-              for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
-            }
-          };
-          auto finish = [&](float (&cmb)[E], unsigned inbits) {
-            if (masked) {
-#pragma unroll
-              for (int k = 0; k < E; ++k) cmb[k] = (inbits & (1u << k)) ? cmb[k] : -INFINITY;
-            }
-            if (fixed) {
-              if (!seeded_c) {
-                accc.seed(cmb, p.cT);
-                seeded_c = true;
-              }
-              accc.add_fixed(cmb, p.cT);
-            } else {
-              accc.add_online(cmb, p.cT);
-            }
-          };
-          for (int v = sl.v_lo + tid; v < sl.v_hi; v += 2 * kThreads) {
-            const bool have_b = (v + kThreads < sl.v_hi);
-            const long long oa = static_cast<long long>(v) * 16;
-            const long long ob = have_b ? oa + static_cast<long long>(kThreads) * 16 : oa;
-            float ca[E], cb[E];
-            unsigned ba = 0xffffffffu, bb = 0xffffffffu;
-#pragma unroll
-            for (int k = 0; k < E; ++k) ca[k] = cb[k] = 0.f;
-            int i = 0;
-            for (; i + 1 < p.n; i += 2) {  // two models, two vectors: four loads in flight
-              const char* r0 = row0 + i * row_step;
-              const char* r1 = r0 + row_step;
-              const uint4 a0 = ldg_stream16(r0 + oa), b0 = ldg_stream16(r0 + ob);
-              const uint4 a1 = ldg_stream16(r1 + oa), b1 = ldg_stream16(r1 + ob);
-              take(i, a0, ca, ba);
-              take(i + 1, a1, ca, ba);
-              if (have_b) {
-                take(i, b0, cb, bb);
-                take(i + 1, b1, cb, bb);
-              }
-            }
-            if (i < p.n) {
-              const char* r0 = row0 + i * row_step;
-              const uint4 a0 = ldg_stream16(r0 + oa), b0 = ldg_stream16(r0 + ob);
-              take(i, a0, ca, ba);
-              if (have_b) take(i, b0, cb, bb);
-            }
-            finish(ca, ba);
-            if (have_b) finish(cb, bb);
-          }
-          for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
-            float cmb = 0.f, xq = -INFINITY, xe = 0.f;
-            for (int i = 0; i < p.n; ++i) {
-              float x = Elem<DT>::load1(row_of(i), e);
-              cmb = fmaf(p.w[i], x, cmb);
-              if (i == pis) xq = x;
-              if (i == p.mask_model) xe = x;
-            }
-            if (masked && !(xe >= thr)) cmb = -INFINITY;
-            accq.add_online1(xq, p.cT);
-            accc.add_online1(cmb, p.cT);
-          }
-          if ((accq.s < INFINITY) && (accc.s < INFINITY)) break;
-        }
-        warp_merge_soft(accq, &sh.wsoft[warp][0], lane);
-        warp_merge_soft(accc, &sh.wsoft[warp][1], lane);
+        sweep_unit<DT, MODE>(p, base, sl, pis, masked, thr, &sh.wsoft[warp][0], &sh.warg[warp][0]);
         cluster_merge(sh, cluster, phase, 2, 0, 0);
       } else {  // kLogitGreedy
-        // The argmax of the combined logits must be the fp64 one (the same chain of fused multiply-adds
-        // on every token, lowest index among equals).  Every token gets an fp32 value and a bound on its
-        // distance from the fp64 value; only tokens that could reach the best fp64 value seen so far are
-        // evaluated in fp64.
-        double cbest = -INFINITY;
-        float cbest_lo = -INFINITY;  // a lower bound of the maximum in fp32: the best fp64 value seen by the warp, rounded down
-        int cidx = kNoReject, bad = 0;
-        float qbest = -INFINITY;
-        int qidx = kNoReject;
-        const char* row0 = reinterpret_cast<const char*>(row_of(0));
-        const long long row_step = p.s_model * Elem<DT>::bytes;
-        const float kSlack = static_cast<float>(p.n) * 1.1920929e-07f;  // n * 2^-23: rounding of the fp32 chain
-        auto consider = [&](float c32, float bnd, int e) {  // token inside the mask
-          bad |= (c32 != c32);
-          if (__fmaf_ru(bnd, kSlack, c32) >= cbest_lo) {
-            const double cm = exact_combined<DT>(p, base, e);
-            if (cm > cbest) {  // tokens come in increasing order within a thread: ties keep the earlier one
-              cbest = cm;
-              cidx = e;
-              const float lo = __double2float_rd(cm);
-              if (lo > cbest_lo) cbest_lo = lo;
-            }
-          }
-        };
-        // the vectors of the first two models are fetched one trip ahead: four loads in flight per thread
-        const bool pair = (p.n >= 2);
-        uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
-        {
-          const int v0 = sl.v_lo + tid;
-          if (v0 < sl.v_hi) {
-            nx0 = ldg_stream16(row0 + static_cast<long long>(v0) * 16);
-            if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(v0) * 16);
-          }
-        }
-        for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
-          const uint4 a0 = nx0, a1 = nx1;
-          {
-            const int vn = v + kThreads;
-            if (vn < sl.v_hi) {
-              nx0 = ldg_stream16(row0 + static_cast<long long>(vn) * 16);
-              if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(vn) * 16);
-            }
-          }
-          float c32[E], bnd[E];
-          unsigned inbits = 0xffffffffu;
-#pragma unroll
-          for (int k = 0; k < E; ++k) c32[k] = bnd[k] = 0.f;
-          auto take = [&](int i, const uint4& raw) {
-            float x[E];
-            Elem<DT>::unpack(raw, x);
-            const float wi = p.w[i], wa = fabsf(wi);
-#pragma unroll
-            for (int k = 0; k < E; ++k) {
-              bad |= !(x[k] < INFINITY);
-              c32[k] = fmaf(wi, x[k], c32[k]);
-              bnd[k] = fmaf(wa, fabsf(x[k]), bnd[k]);
-            }
-            if (i == pis) {
-              float xm = x[0];
-#pragma unroll
-              for (int k = 1; k < E; ++k) xm = fmaxf(xm, x[k]);
-              if (xm > qbest) {  // rare after the first few vectors; the first of equal entries wins
-                qbest = xm;
-#pragma unroll
-                for (int k = E - 1; k >= 0; --k)
-                  if (x[k] == xm) qidx = v * E + k;
-              }
-            }
-            if (masked && i == p.mask_model) {
-              inbits = 0u;
-#pragma unroll
-              for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
-            }
-          };
-          take(0, a0);
-          if (pair) take(1, a1);
-          const long long off = static_cast<long long>(v) * 16;
-          for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + off));
-          // upper bounds of the fp64 values; one comparison decides whether any entry of the vector can matter.
-          // The sum only carries a NaN (or an infinity of each sign) to the check below.
-          float tmax = -INFINITY, tsum = 0.f;
-#pragma unroll
-          for (int k = 0; k < E; ++k) {
-            const float t = (inbits & (1u << k)) ? __fmaf_ru(bnd[k], kSlack, c32[k]) : -INFINITY;
-            tmax = fmaxf(tmax, t);
-            tsum += t;
-          }
-          if (tmax >= cbest_lo || tsum != tsum) {
-#pragma unroll
-            for (int k = 0; k < E; ++k)
-              if (inbits & (1u << k)) consider(c32[k], bnd[k], v * E + k);
-          }
-          // any exact value found by a lane of the warp is a lower bound of the maximum for all of them:
-          // share the largest (floats ordered as unsigned integers, one warp-wide max)
-          {
-            const unsigned bits = __float_as_uint(cbest_lo);
-            const unsigned key = bits ^ ((bits >> 31) ? 0xffffffffu : 0x80000000u);
-            const unsigned top = __reduce_max_sync(__activemask(), key);
-            const unsigned back = top ^ ((top >> 31) ? 0x80000000u : 0xffffffffu);
-            const float shared_lo = __uint_as_float(back);
-            if (shared_lo > cbest_lo) cbest_lo = shared_lo;
-          }
-        }
-        for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
-          float c32 = 0.f, bnd = 0.f, xe = 0.f;
-          for (int i = 0; i < p.n; ++i) {
-            float x = Elem<DT>::load1(row_of(i), e);
-            bad |= !(x < INFINITY);
-            c32 = fmaf(p.w[i], x, c32);
-            bnd = fmaf(fabsf(p.w[i]), fabsf(x), bnd);
-            if (i == pis && x > qbest) {
-              qbest = x;
-              qidx = e;
-            }
-            if (i == p.mask_model) xe = x;
-          }
-          if (!masked || xe >= thr) consider(c32, bnd, e);
-        }
-        warp_merge_arg(static_cast<double>(qbest), qidx, bad, &sh.warg[warp][1], lane);
-        warp_merge_arg(cbest, cidx, bad, &sh.warg[warp][2], lane);
+        sweep_unit<DT, MODE>(p, base, sl, pis, masked, thr, &sh.wsoft[warp][0], &sh.warg[warp][0]);
         cluster_merge(sh, cluster, phase, 0, 1, 2);
       }
     }
@@ -999,143 +1167,7 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
 
     // ================================ decision (Eq. 6) ================================
     // every block takes the same decision from the same merged numbers
-    if (tid == 0) {
-      Decision& d = sh.dec;
-      const double u_acc = sh.u_acc;
-      d.accept = 0;
-      d.status = 0;
-      d.want_sample = 0;
-      d.cand = -1;
-      d.natoms = 0;
-      d.ratio = d.r_d = d.q_d = d.S = kNaN;
-      bool finite = pi_ok;
-      if (kSample) {
-        const int nsoft = (MODE == kEnsembleSample) ? p.n : 2;
-        for (int k = 0; k < nsoft; ++k) {
-          const SoftPart& f = sh.fsoft[k];
-          finite = finite && isfinite(f.ref) && isfinite(f.s) && (f.s > 0.0);
-        }
-        if (masked && sh.farg[0].bad) finite = false;
-        if (!finite) {
-          d.status |= COS_ROW_NONFINITE;
-        } else {
-          for (int k = 0; k < nsoft; ++k) sh.big_thr[k] = static_cast<float>(sh.fsoft[k].s * kBigShare);
-          if (!is_bonus) {
-            if (draft_ok) {
-              double r_d = 0.0, q_d = 0.0;
-              if (MODE == kEnsembleSample) {
-                for (int i = 0; i < p.n; ++i) {
-                  r_d += p.w64[i] * sh.pdraft[i];
-                  if (i == pi) q_d = sh.pdraft[i];
-                }
-              } else {
-                double cd = 0.0;
-                for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(sh.ldraft[i]), cd);
-                bool in = !masked || (sh.ldraft[p.mask_model] >= sh.thr32);
-                r_d = in ? exp2(cd * p.cT64 - static_cast<double>(sh.fsoft[1].ref)) / sh.fsoft[1].s : 0.0;
-                double lq = static_cast<double>(sh.ldraft[pi]);
-                q_d = exp2(lq * p.cT64 - static_cast<double>(sh.fsoft[0].ref)) / sh.fsoft[0].s;
-              }
-              d.r_d = r_d;
-              d.q_d = q_d;
-              if (q_d > 0.0) {
-                d.ratio = r_d / q_d;
-              } else {
-                d.status |= COS_ROW_Q_ZERO;
-                d.ratio = (r_d > 0.0) ? kInf : 0.0;
-              }
-              d.accept = (u_acc <= fmin(1.0, d.ratio)) ? 1 : 0;
-            } else {
-              d.status |= COS_ROW_BAD_DRAFT;
-            }
-          }
-          d.want_sample = is_bonus || !d.accept;
-        }
-      } else {
-        // greedy: distributions are atoms at lowest-index argmaxes
-        int qtok;
-        if (MODE == kEnsembleGreedy) {
-          for (int i = 0; i < p.n; ++i) finite = finite && !sh.farg[i].bad && isfinite(sh.farg[i].val);
-          qtok = sh.farg[pis].idx;
-        } else {
-          finite = finite && !sh.farg[1].bad && !sh.farg[2].bad && isfinite(sh.farg[1].val) && isfinite(sh.farg[2].val);
-          if (masked && sh.farg[0].bad) finite = false;
-          qtok = sh.farg[1].idx;
-        }
-        if (!finite) {
-          d.status |= COS_ROW_NONFINITE;
-        } else {
-          // atoms of r, sorted by token, masses accumulated in model order
-          if (MODE == kEnsembleGreedy) {
-            for (int i = 0; i < p.n; ++i) {
-              int t = sh.farg[i].idx, pos = 0;
-              while (pos < d.natoms && d.atom_tok[pos] < t) ++pos;
-              if (pos < d.natoms && d.atom_tok[pos] == t) {
-                d.atom_mass[pos] += p.w64[i];
-              } else {
-                for (int k = d.natoms; k > pos; --k) {
-                  d.atom_tok[k] = d.atom_tok[k - 1];
-                  d.atom_mass[k] = d.atom_mass[k - 1];
-                }
-                d.atom_tok[pos] = t;
-                d.atom_mass[pos] = 0.0 + p.w64[i];
-                ++d.natoms;
-              }
-            }
-          } else {
-            d.natoms = 1;
-            d.atom_tok[0] = sh.farg[2].idx;
-            d.atom_mass[0] = 1.0;
-          }
-          auto r_at = [&](int t) {
-            for (int k = 0; k < d.natoms; ++k)
-              if (d.atom_tok[k] == t) return d.atom_mass[k];
-            return 0.0;
-          };
-          bool use_r = is_bonus;
-          if (!is_bonus) {
-            if (draft_ok) {
-              d.r_d = r_at(draft);
-              d.q_d = (draft == qtok) ? 1.0 : 0.0;
-              if (d.q_d > 0.0) {
-                d.ratio = d.r_d / d.q_d;
-              } else {
-                d.status |= COS_ROW_Q_ZERO;
-                d.ratio = (d.r_d > 0.0) ? kInf : 0.0;
-              }
-              d.accept = (u_acc <= fmin(1.0, d.ratio)) ? 1 : 0;
-            } else {
-              d.status |= COS_ROW_BAD_DRAFT;
-            }
-            // residual max(0, r - q) over the atoms, summed in token order
-            double S = 0.0;
-            for (int k = 0; k < d.natoms; ++k) S += fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
-            d.S = S;
-            if (!(S > 0.0)) {
-              use_r = true;
-              if (!d.accept) d.status |= COS_ROW_RESIDUAL_EMPTY;
-            }
-          }
-          // inverse CDF over the atoms (token order): smallest k with running sum >= u * total
-          double total = 0.0;
-          for (int k = 0; k < d.natoms; ++k)
-            total += use_r ? d.atom_mass[k] : fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
-          const double target = sh.u_smp * total;
-          double run = 0.0;
-          int lastpos = -1;
-          d.cand = -1;
-          for (int k = 0; k < d.natoms; ++k) {
-            double m = use_r ? d.atom_mass[k] : fmax(0.0, d.atom_mass[k] - (d.atom_tok[k] == qtok ? 1.0 : 0.0));
-            run += m;
-            if (m > 0.0) lastpos = d.atom_tok[k];
-            if (d.cand < 0 && m > 0.0 && run >= target) d.cand = d.atom_tok[k];
-          }
-          if (d.cand < 0) d.cand = lastpos;
-        }
-      }
-      d.need2 = 0;  // tokens are drawn by stage 1, for the one position per row that needs it
-      d.drawable = (kSample && finite) ? 1 : 0;
-    }
+    if (tid == 0) decide_unit<DT, MODE>(p, sh, is_bonus, draft, draft_ok, pi, pi_ok, pis, masked);
     __syncthreads();
     // rank 0 keeps the merged statistics for stage 1 and reports the unit
     if (rank == 0) {
