@@ -53,7 +53,10 @@ enum {
   COS_ROW_NONFINITE = 1,      /* a distribution was NaN/Inf: that position counts as rejected, token -1 */
   COS_ROW_BAD_DRAFT = 2,      /* draft token outside [0, vocab): rejected, residual still sampled       */
   COS_ROW_Q_ZERO = 4,         /* q(draft) == 0: ratio taken as +inf if r(draft) > 0, else 0             */
-  COS_ROW_RESIDUAL_EMPTY = 8  /* rejected but max(0, r - q) == 0 everywhere: token drawn from r         */
+  COS_ROW_RESIDUAL_EMPTY = 8, /* rejected but max(0, r - q) == 0 everywhere: token drawn from r         */
+  COS_ROW_FAULT = 16          /* an internal wait of the kernel gave up (a defect, never the data): the */
+                              /* call's outputs are undefined and the context must not be used again;   */
+                              /* set on every row, reported whatever the row's first rejection          */
 };
 
 /* bits of cos_verify_args.flags */

@@ -256,8 +256,21 @@ struct Decision {  // written by thread 0 of every block, identically
   double ratio, r_d, q_d, S;
 };
 
+// Stage 0 without block barriers: every warp streams its share of unit after unit; what the warps of
+// a block tell each other goes through these words (volatile accesses, fences, bounded waits).
+struct FreeRun {
+  SoftPart wsoft[2][kWarps][kMaxSlots];  // warp partials, two units deep
+  ArgPart warg[2][kWarps][kMaxSlots];
+  int unit_of[4];   // the unit this block processes as its seq-th, at [seq & 3]
+  int unit_tag[4];  // seq + 1 once unit_of[seq & 3] is valid
+  int arrive[2];    // warps that have finished the unit of that parity
+  int epi_done;     // units whose merge and decision are complete
+  int fault;        // a wait gave up
+};
+
 struct Shared {
   Xchg x[2];
+  FreeRun fr;
   SoftPart wsoft[kWarps][kMaxSlots];
   ArgPart warg[kWarps][kMaxSlots];
   double wtot[kWarps];        // this block's per-warp totals of sweep 2
@@ -1028,6 +1041,172 @@ __device__ __forceinline__ void decide_unit(const KParams& p, Shared& sh, bool i
 }
 
 // ------------------------------------------------------------------------------------
+// stage 0, one block per unit, no block barriers
+// ------------------------------------------------------------------------------------
+constexpr int kWaitSpins = 1 << 20;  // polls before a wait gives up (each at least 100 ns apart)
+
+// Wait until *flag >= want.  False when the wait gave up or another warp did.
+__device__ __forceinline__ bool wait_reach(const volatile int* flag, int want, const volatile int* fault, int lane) {
+  int ok = 0;
+  if (lane == 0) {
+    for (int it = 0; it < kWaitSpins; ++it) {
+      if (*flag >= want) {
+        ok = 1;
+        break;
+      }
+      if (*fault) break;
+      __nanosleep(100);
+    }
+    __threadfence_block();
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+// A wait gave up (a defect, never the data): mark every row and let the other warps of the block leave.
+__device__ __noinline__ void raise_fault(const KParams& p, FreeRun& fr, int lane) {
+  if (lane == 0) *reinterpret_cast<volatile int*>(&fr.fault) = 1;
+  for (int b = lane; b < p.B; b += 32) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_FAULT));
+}
+
+// Every warp sweeps its share of the block's current unit and moves straight on to the next one.
+// The last warp to finish a unit merges the sixteen partials, takes the decision (Eq. 6) and publishes
+// it while the others are already streaming; the first warp to finish draws the unit after the next
+// from the work counter.  Partials are kept two units deep; a warp may run at most one unit ahead.
+template <int DT, int MODE>
+__device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh) {
+  constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  FreeRun& fr = sh.fr;
+  volatile int* unit_of = fr.unit_of;
+  volatile int* unit_tag = fr.unit_tag;
+  volatile int* epi_done = &fr.epi_done;
+  volatile int* fault = &fr.fault;
+  const Slice sl = slice_of<DT>(0, 1, p.V, p.vec_ok != 0);
+  if (tid == 0) {
+    for (int k = 0; k < 4; ++k) {
+      fr.unit_of[k] = p.num_units;
+      fr.unit_tag[k] = 0;
+    }
+    fr.unit_of[0] = blockIdx.x;
+    fr.unit_tag[0] = 1;
+    fr.arrive[0] = fr.arrive[1] = 0;
+    fr.epi_done = 0;
+    fr.fault = 0;
+  }
+  __syncthreads();
+  if (tid == kThreads - 32) {  // the block's first unit is valid: one draw settles its second
+    const int nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
+    unit_of[1] = nx;
+    __threadfence_block();
+    unit_tag[1] = 2;
+  }
+  for (int seq = 0;; ++seq) {
+    const int par = seq & 1;
+    if (!wait_reach(&unit_tag[seq & 3], seq + 1, fault, lane)) {
+      raise_fault(p, fr, lane);
+      return;
+    }
+    const int unit = unit_of[seq & 3];
+    if (unit >= p.num_units) break;
+    const int j = unit / p.B, b = unit % p.B;  // earlier positions of every row come first
+    const int pi = p.proposer[b];
+    const bool pi_ok = (pi >= 0 && pi < p.n);
+    const int pis = pi_ok ? pi : 0;
+    const char* base = reinterpret_cast<const char*>(p.logits) +
+                       (static_cast<long long>(b) * p.s_row + static_cast<long long>(j) * p.s_pos) * Elem<DT>::bytes;
+    // the partials of this parity are free once the unit two back has been merged
+    if (seq >= 2 && !wait_reach(epi_done, seq - 1, fault, lane)) {
+      raise_fault(p, fr, lane);
+      return;
+    }
+    sweep_unit<DT, MODE>(p, base, sl, pis, false, -INFINITY, &fr.wsoft[par][warp][0], &fr.warg[par][warp][0]);
+    int prev = 0;
+    if (lane == 0) {
+      __threadfence_block();
+      prev = atomicAdd(&fr.arrive[par], 1);
+      __threadfence_block();
+    }
+    prev = __shfl_sync(0xffffffffu, prev, 0);
+    __syncwarp();
+    if (prev == 0) {
+      // first to finish: one draw per valid unit, made one unit ahead of its use
+      if (!wait_reach(&unit_tag[(seq + 1) & 3], seq + 2, fault, lane)) {
+        raise_fault(p, fr, lane);
+        return;
+      }
+      if (lane == 0) {
+        int nx = p.num_units;
+        if (unit_of[(seq + 1) & 3] < p.num_units)
+          nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
+        unit_of[(seq + 2) & 3] = nx;
+        __threadfence_block();
+        unit_tag[(seq + 2) & 3] = seq + 3;
+      }
+    }
+    if (prev == kWarps - 1) {
+      // last to finish: merge, decide, publish
+      const int uidx = b * p.P + j;
+      const bool is_bonus = (j == p.gamma);
+      const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
+      const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
+      if (lane < p.n && !is_bonus && draft_ok)
+        sh.ldraft[lane] = Elem<DT>::load1(base + static_cast<long long>(lane) * p.s_model * Elem<DT>::bytes, draft);
+      if (lane == 31) {
+        unsigned rnd[4];
+        const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
+        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi,
+                      rnd);
+        sh.u_acc = word_to_uniform(rnd[0]);
+        sh.u_smp = word_to_uniform(rnd[1]);
+      }
+      const int nsoft = (MODE == kEnsembleSample) ? p.n : (MODE == kLogitSample ? 2 : 0);
+      const int arg_lo = (MODE == kLogitGreedy) ? 1 : 0;
+      const int narg = (MODE == kEnsembleGreedy) ? p.n : (MODE == kLogitGreedy ? 2 : 0);
+      for (int k = 0; k < nsoft; ++k) {
+        const float ref = (lane < kWarps) ? fr.wsoft[par][lane][k].ref : -INFINITY;
+        const double sum = (lane < kWarps) ? fr.wsoft[par][lane][k].s : 0.0;
+        const SoftPart o = warp_reduce_soft(ref, sum);
+        if (lane == 0) sh.fsoft[k] = o;
+      }
+      for (int k = arg_lo; k < arg_lo + narg; ++k) {
+        ArgPart in;
+        if (lane < kWarps) {
+          in = fr.warg[par][lane][k];
+        } else {
+          in.val = -INFINITY;
+          in.idx = kNoReject;
+          in.bad = 0;
+        }
+        const ArgPart o = warp_reduce_arg(in.val, in.idx, in.bad, lane);
+        if (lane == 0) sh.farg[k] = o;
+      }
+      __syncwarp();
+      if (MODE == kEnsembleSample && lane < p.n && !is_bonus && draft_ok) {
+        // probability of the draft under model `lane`, with the constant the sweep used
+        sh.pdraft[lane] = exp2(static_cast<double>(sh.ldraft[lane]) * p.cT64 - static_cast<double>(sh.fsoft[lane].ref)) /
+                          sh.fsoft[lane].s;
+      }
+      __syncwarp();
+      if (lane == 0) decide_unit<DT, MODE>(p, sh, is_bonus, draft, draft_ok, pi, pi_ok, pis, false);
+      __syncwarp();
+      if (kSample && lane < nsoft) {  // kept for the drawing stages
+        p.ustats[uidx].s[lane] = sh.fsoft[lane].s;
+        p.ustats[uidx].ref[lane] = sh.fsoft[lane].ref;
+      }
+      if (kSample && lane == 31) p.ustats[uidx].thr32 = 0.f;
+      if (lane == 0) {
+        const Decision& d = sh.dec;
+        publish_unit(p, b, j, d.accept, d.status, d.cand, d.drawable, d.ratio, d.r_d, d.q_d, d.S);
+        fr.arrive[par] = 0;
+        __threadfence_block();
+        *epi_done = seq + 1;
+      }
+      __syncwarp();
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------
 template <int DT, int MODE, int STAGE>
@@ -1064,6 +1243,12 @@ __global__ void __launch_bounds__(kThreads, 2) cos_verify_kernel(const __grid_co
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
   if (STAGE == 0) {
     if (blockIdx.x == 0 && tid == 0) *p.job_reset = 0;  // the list of the next run starts empty
+    // One block per unit and no step that needs the whole block twice (the plausibility mask does, and so
+    // does the greedy form of the combined-distribution test hook): the warps run without block barriers.
+    if (C == 1 && !masked && (kSample || p.dump_r == nullptr)) {
+      stage0_free_running<DT, MODE>(p, sh);
+      return;
+    }
   } else {
     njobs = *p.job_count;
     njobs = njobs < p.max_jobs ? njobs : p.max_jobs;
