@@ -1807,7 +1807,17 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             for (int k = 0; k < E; ++k)
               if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, nullptr, k);
           }
-          const double own = lane_mass(e0, mass32, bigbits, use_r, nullptr);
+          // the lane's mass exactly as lane_mass() forms it (fp32 sum of the small tokens, then the big ones
+          // in token order), from the values already at hand
+          float ls = 0.f;
+#pragma unroll
+          for (int k = 0; k < E; ++k) ls += mass32[k];
+          double own = static_cast<double>(ls);
+          if (bigbits) {
+#pragma unroll
+            for (int k = 0; k < E; ++k)
+              if (bigbits & (1u << k)) own += m64[k];
+          }
           double inc = own;
 #pragma unroll
           for (int d = 1; d < 32; d <<= 1) {
