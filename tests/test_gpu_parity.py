@@ -41,3 +41,26 @@ def test_small_cases_match_oracle(w):
     plain = helpers.run_gpu(w, inputs)
     for k in ("accept_count", "out_tokens", "row_status"):
         assert np.array_equal(plain[k], gpu[k]), k
+
+
+# Both forms of the streaming stage at small sizes: cluster_size 1 runs it without block barriers (one block
+# per position, unless a plausibility mask is set), larger sizes split a position across a cluster.
+FORMS = [SMALL[i] for i in (1, 3, 4, 6, 7, 8)]
+
+
+@pytest.mark.parametrize("cs", [1, 2, 4, 8])
+@pytest.mark.parametrize("w", FORMS, ids=[w.name for w in FORMS])
+def test_every_cluster_size_gives_the_oracles_rows(w, cs):
+    inputs = synth.make_inputs(w, "cuda")
+    ref = helpers.run_oracle(w, inputs)
+    v = helpers.make_verifier(w, cluster_size=cs)
+    try:
+        gpu = helpers.run_gpu(w, inputs, verifier=v, diag=True, flags=COS_RUN_ALL_RESIDUALS)
+        stats = helpers.check_parity(w, gpu, ref)
+        assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
+        # a second call on the same context (its scratch was left clean) gives the same rows
+        again = helpers.run_gpu(w, inputs, verifier=v)
+        for k in ("accept_count", "out_tokens", "row_status"):
+            assert np.array_equal(again[k], gpu[k]), k
+    finally:
+        v.close()
