@@ -1491,7 +1491,27 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e)), cd);
           return exp2(cd * p.cT64 - dref_c);
         };
+        // the vectors of the first two models are fetched one trip ahead: four loads in flight per thread
+        const char* row0 = reinterpret_cast<const char*>(row_of(0));
+        const long long row_step = p.s_model * Elem<DT>::bytes;
+        const bool pair = (p.n >= 2);
+        uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+        {
+          const int v0 = sl.v_lo + tid;
+          if (v0 < sl.v_hi) {
+            nx0 = ldg_stream16(row0 + static_cast<long long>(v0) * 16);
+            if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(v0) * 16);
+          }
+        }
         for (int v = sl.v_lo + tid; v < sl.v_hi; v += kThreads) {
+          const uint4 a0 = nx0, a1 = nx1;
+          {
+            const int vn = v + kThreads;
+            if (vn < sl.v_hi) {
+              nx0 = ldg_stream16(row0 + static_cast<long long>(vn) * 16);
+              if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(vn) * 16);
+            }
+          }
           float cmb[E], vq[E], ve[E];
 #pragma unroll
           for (int k = 0; k < E; ++k) {
@@ -1499,27 +1519,20 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             vq[k] = -INFINITY;
             ve[k] = 0.f;
           }
-          for (int i = 0; i < p.n; i += 2) {
-            const bool two = (i + 1 < p.n);
-            uint4 ra = ldg_stream16(reinterpret_cast<const char*>(row_of(i)) + static_cast<long long>(v) * 16);
-            uint4 rb = ra;
-            if (two) rb = ldg_stream16(reinterpret_cast<const char*>(row_of(i + 1)) + static_cast<long long>(v) * 16);
-            float va[E], vb[E];
-            Elem<DT>::unpack(ra, va);
-            Elem<DT>::unpack(rb, vb);
-            const float wa = p.w[i], wb = two ? p.w[i + 1] : 0.f;
+          auto take = [&](int i, const uint4& raw) {
+            float x[E];
+            Elem<DT>::unpack(raw, x);
+            const float wi = p.w[i];
 #pragma unroll
             for (int k = 0; k < E; ++k) {
-              cmb[k] = fmaf(wa, va[k], cmb[k]);
-              if (i == pis) vq[k] = va[k];
-              if (i == p.mask_model) ve[k] = va[k];
-              if (two) {
-                cmb[k] = fmaf(wb, vb[k], cmb[k]);
-                if (i + 1 == pis) vq[k] = vb[k];
-                if (i + 1 == p.mask_model) ve[k] = vb[k];
-              }
+              cmb[k] = fmaf(wi, x[k], cmb[k]);
+              if (i == pis) vq[k] = x[k];
+              if (i == p.mask_model) ve[k] = x[k];
             }
-          }
+          };
+          take(0, a0);
+          if (pair) take(1, a1);
+          for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(v) * 16));
           bool any = false;
           float eq[E], ec[E];
 #pragma unroll
