@@ -29,7 +29,7 @@ from paper_2502_01662_b200 import synth  # noqa: E402
 
 HEADLINE = "cfg3"
 # dram read + write bytes of one stage-0 launch from the ncu capture summarised under profiles/
-TRAFFIC_BYTES = {"cfg3": 356224000}
+TRAFFIC_BYTES = {"cfg3": 355220480}
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
 
@@ -164,9 +164,13 @@ def oracle_sample(w, target_seconds=15.0, max_rows=None):
     one row first, then as many more as fit the time budget."""
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     import helpers
+    made = {}
     def timed(rows, first_row):
         small = w.scaled(batch=first_row + rows, name=w.name)
-        inputs = synth.make_inputs(small, "cpu")
+        if small.batch not in made:
+            made.clear()
+            made[small.batch] = synth.make_inputs(small, "cpu")
+        inputs = made[small.batch]
         t0 = time.perf_counter()
         helpers.run_oracle(small, inputs, rows=range(first_row, first_row + rows))
         return time.perf_counter() - t0
@@ -177,7 +181,13 @@ def oracle_sample(w, target_seconds=15.0, max_rows=None):
     if more > 0:
         total_t += timed(more, 1)
         rows += more
-    return rows * (w.gamma + 1) / total_t, rows, total_t
+    # a batch the oracle finishes in a second or two is verified again (whole) until about ten seconds are spent
+    passes = 1
+    if rows == w.batch:
+        while total_t < 10.0 and passes < 64:
+            total_t += timed(w.batch, 0)
+            passes += 1
+    return passes * rows * (w.gamma + 1) / total_t, rows, total_t, passes
 
 
 def run_reference(args, w):
@@ -352,9 +362,9 @@ def main():
     if extra:
         line["all_configs"] = extra
     if not args.skip_cpu:
-        v, rows, dt = oracle_sample(w)
+        v, rows, dt, passes = oracle_sample(w)
         line["cpu_baseline"] = {"value": v, "unit": "positions/s", "cores": 1, "kind": "oracle",
-                                "sample": f"first {rows} rows x {w.gamma + 1} positions of {w.name}, {dt:.1f} s"}
+                                "sample": f"first {rows} rows x {w.gamma + 1} positions of {w.name}, {passes} pass(es), {dt:.1f} s"}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
