@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     COS_DTYPE_BF16,
     COS_DTYPE_F32,
     COS_ROW_BAD_DRAFT,
+    COS_ROW_FAULT,
     COS_ROW_NONFINITE,
     COS_ROW_Q_ZERO,
     COS_ROW_RESIDUAL_EMPTY,

@@ -20,6 +20,7 @@ COS_ROW_NONFINITE = 1
 COS_ROW_BAD_DRAFT = 2
 COS_ROW_Q_ZERO = 4
 COS_ROW_RESIDUAL_EMPTY = 8
+COS_ROW_FAULT = 16   # an internal wait of the kernel gave up: the call's outputs are undefined
 COS_RUN_ALL_RESIDUALS = 1
 
 _STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR_ALIGNMENT",
