@@ -123,6 +123,9 @@ class OracleConfig:
     vocab: int
     mask_model: int = -1              # logit-linear only; -1 = no plausibility mask
     mask_alpha: float = 1.0           # keep x with l_e(x) >= max l_e + ln(alpha)
+    bonus_model: int = -1             # -1: the token after gamma acceptances follows the combined r;
+                                      # i >= 0: it follows model i's own distribution (Sec. 3.3: the
+                                      # verifier's bonus token, later treated as that model's proposal)
     w64: np.ndarray = field(init=False, repr=False)
 
     def __post_init__(self):
@@ -131,6 +134,8 @@ class OracleConfig:
         self.mask_alpha = float(np.float32(self.mask_alpha))
         if len(self.w64) != self.n:
             raise ValueError("need n weights")
+        if not (-1 <= self.bonus_model < self.n):
+            raise ValueError("bonus_model must be -1 or a model index")
         if self.combine == COMBINE_PROB_ENSEMBLE:
             if self.mask_model >= 0:
                 raise ValueError("mask only with the logit-level combine")
@@ -256,6 +261,7 @@ class PositionResult:
     r_d: float = float("nan")
     q_d: float = float("nan")
     S: float = float("nan")       # residual mass sum_x max(0, r - q)  (j < gamma)
+    prob: float = float("nan")    # bonus position only: probability of cand under the law it was drawn from
     status: int = 0
     boundary_accept: bool = False
     boundary_sample: bool = False
@@ -266,15 +272,22 @@ def verify_position(l: np.ndarray, cfg: OracleConfig, proposer: int, draft: Opti
     """Eq. 6 at a draft position (draft is an int) or the bonus sample (draft is None).
 
     `dist` may carry the (r, q, ok) triple of position_distributions for these same
-    arguments, so that many trials on one position need not recompute it."""
+    arguments (with proposer = cfg.bonus_model at a bonus position that names a model), so
+    that many trials on one position need not recompute it."""
     res = PositionResult()
+    if draft is None and cfg.bonus_model >= 0 and dist is None:
+        proposer = cfg.bonus_model               # q below is then that model's own distribution
     r, q, ok = position_distributions(l, cfg, proposer) if dist is None else dist
     if not ok:
         res.status |= STATUS_NONFINITE           # defined fallback: rejected, no candidate
         return (res, r) if return_r else res
     if draft is None:
-        k, _, lo, hi = inverse_cdf(r, u_smp)
+        # Sec. 3.1: after gamma acceptances one more token is drawn; from r, or (Sec. 3.3, Algorithm 2's
+        # Score) from the named model's own distribution, whose probability of it is reported
+        law = q if cfg.bonus_model >= 0 else r
+        k, _, lo, hi = inverse_cdf(law, u_smp)
         res.cand = k
+        res.prob = float(law[k])
         res.boundary_sample = min(abs(lo - u_smp), abs(hi - u_smp)) < BOUNDARY_CDF
         return (res, r) if return_r else res
     V = l.shape[1]
@@ -312,20 +325,24 @@ def verify(logits, dtype: str, drafts, proposer, cfg: OracleConfig, seed: int, o
            row_base: int = 0, rows: Optional[Sequence[int]] = None, return_r: bool = False,
            uniforms=None):
     """logits: array [n, B, gamma+1, V] (raw uint16 patterns when dtype == 'bf16').
-    drafts [B, gamma] int, proposer [B] int.  `rows` restricts the work to some rows
+    drafts [B, gamma] int; proposer [B] int, or [B, gamma+1] int naming the model that proposed each
+    draft (Algorithm 2: the cached sequence holds tokens of several proposers; the entry of the bonus
+    position is not read).  `rows` restricts the work to some rows
     (the others are left at their fill values), which is how full-size cases are sampled.
     `uniforms` = (u_acc, u_smp), each [B, gamma+1], replaces the Philox draws (used by the
     enumeration tests, which need to place the uniforms themselves).
 
     Returns a dict of arrays: accept_count [B], out_tokens [B, gamma+1] (-1 padded),
-    row_status [B], and per-position diagnostics (accept, cand, ratio, r_d, q_d, S,
+    row_status [B], bonus_prob [B] (NaN unless every draft passed), and per-position diagnostics (accept, cand, ratio, r_d, q_d, S,
     boundary_accept, boundary_sample, u_acc, u_smp), optionally r [B, gamma+1, V].
     """
     n, B, P, V = logits.shape
     g = cfg.gamma
     assert P == g + 1 and n == cfg.n and V == cfg.vocab
     drafts = np.asarray(drafts).reshape(B, g) if g > 0 else np.zeros((B, 0), np.int64)
-    proposer = np.asarray(proposer).reshape(B)
+    proposer = np.asarray(proposer)
+    proposer = np.repeat(proposer.reshape(B, 1), P, axis=1) if proposer.size == B and proposer.ndim <= 1 \
+        else proposer.reshape(B, P)
     if uniforms is None:
         u_acc, u_smp = position_uniforms(seed, offset, B, P, row_base)
     else:
@@ -340,16 +357,17 @@ def verify(logits, dtype: str, drafts, proposer, cfg: OracleConfig, seed: int, o
         "q_d": np.full((B, P), np.nan), "S": np.full((B, P), np.nan),
         "boundary_accept": np.zeros((B, P), bool), "boundary_sample": np.zeros((B, P), bool),
         "pos_status": np.zeros((B, P), np.uint32),
+        "bonus_prob": np.full(B, np.nan),
         "u_acc": u_acc, "u_smp": u_smp,
     }
     if return_r:
         out["r"] = np.full((B, P, V), np.nan)
     for b in (range(B) if rows is None else rows):
-        pi = int(proposer[b])
         pos = []
         for j in range(P):
             l = to_float64(logits[:, b, j, :], dtype)
             d = int(drafts[b, j]) if j < g else None
+            pi = int(proposer[b, j])
             got = verify_position(l, cfg, pi, d, float(u_acc[b, j]), float(u_smp[b, j]), return_r)
             if return_r:
                 got, r = got
@@ -368,6 +386,8 @@ def verify(logits, dtype: str, drafts, proposer, cfg: OracleConfig, seed: int, o
         out["accept_count"][b] = a
         out["out_tokens"][b, :a] = drafts[b, :a]
         out["out_tokens"][b, a] = pos[a].cand
+        if a == g:
+            out["bonus_prob"][b] = pos[g].prob
         st = 0
         for j in range(a + 1):                    # positions after the first rejection are discarded
             st |= pos[j].status

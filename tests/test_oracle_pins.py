@@ -484,3 +484,94 @@ def test_greedy_verification_is_deterministic_argmax_comparison():
         assert a["accept_count"][row] == k
         assert a["out_tokens"][row, k] == target[row, k]
     assert 0 < a["accept_count"].mean() < g                       # both outcomes occur
+
+
+# --------------------------------------------------------------------------------------
+# alternate proposals (Sec. 3.3, Algorithm 2): bonus token from a named model, proposer per position
+# --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,mk,n,pi", LAW_CASES, ids=[c[0] for c in LAW_CASES])
+@pytest.mark.parametrize("T0", [False, True])
+def test_named_bonus_model_draws_from_that_models_own_law(name, mk, n, pi, T0):
+    """Sec. 3.3: the token after gamma acceptances "is drawn from p" of the verifier, not from the
+    combined law; Algorithm 2's Score returns it with its probability.  Counted over the uniform lattice
+    against scipy's softmax of that model alone; at T = 0 it is that model's lowest-index argmax."""
+    V = 8
+    l = rng_logits(300 + n, n, V, scale=1.5)
+    base = mk(V)
+    for m in range(n):
+        cfg = orc.OracleConfig(n=n, combine=base.combine, weights=list(base.w64), gamma=1, vocab=V,
+                               temperature=0.0 if T0 else base.temperature, mask_model=base.mask_model,
+                               mask_alpha=base.mask_alpha, bonus_model=m)
+        if T0:
+            res = orc.verify_position(l, cfg, pi, None, 0.3, 0.77)
+            assert res.cand == int(np.argmax(l[m])) and res.prob == 1.0
+            continue
+        p_m = sp_softmax(l[m] / cfg.temperature)
+        counts = _count_sampled_u(l, cfg, pi, None, V, None)
+        assert np.all(np.abs(counts - p_m * LATTICE) <= 1.0 + 1e-6)
+        for u in (0.01, 0.4, 0.93):
+            res = orc.verify_position(l, cfg, pi, None, 0.5, u)
+            assert abs(res.prob - p_m[res.cand]) < 1e-15
+        # the draft positions are untouched by the choice of bonus model
+        a = orc.verify_position(l, cfg, pi, 2, 0.4, 0.6)
+        b = orc.verify_position(l, base, pi, 2, 0.4, 0.6)
+        assert (a.accept, a.cand, a.ratio, a.S) == (b.accept, b.cand, b.ratio, b.S)
+
+
+def test_bonus_probability_is_reported_only_after_gamma_acceptances():
+    n, B, V, g = 2, 30, 11, 2
+    gen = np.random.default_rng(5)
+    logits = gen.normal(size=(n, B, g + 1, V)).astype(np.float32)
+    drafts = gen.integers(0, V, size=(B, g))
+    for m in (-1, 0, 1):
+        cfg = orc.OracleConfig(n=n, combine=WE, weights=[0.5, 0.5], temperature=1.0, gamma=g, vocab=V, bonus_model=m)
+        out = orc.verify(logits, "f32", drafts, np.zeros(B, int), cfg, seed=9, offset=3)
+        full = out["accept_count"] == g
+        assert full.any() and (~full).any()
+        assert np.all(np.isnan(out["bonus_prob"][~full]))
+        for b in np.nonzero(full)[0]:
+            l = logits[:, b, g, :].astype(np.float64)
+            law = 0.5 * sp_softmax(l[0]) + 0.5 * sp_softmax(l[1]) if m < 0 else sp_softmax(l[m])
+            assert abs(out["bonus_prob"][b] - law[out["out_tokens"][b, g]]) < 1e-14
+
+
+def test_proposer_per_position_changes_q_position_by_position():
+    """Algorithm 2: the cached sequence mixes tokens proposed by different models, so q at position j is
+    the law of the model that proposed draft j.  P(accept draft d at j) = min(1, r_j(d) / p_{pi_j, j}(d)),
+    counted over the uniform lattice with the laws rebuilt from scipy's softmax."""
+    n, V, g = 3, 6, 3
+    gen = np.random.default_rng(12)
+    logits = (gen.normal(size=(n, 1, g + 1, V)) * 1.5).astype(np.float32)
+    w = [0.5, 0.3, 0.2]
+    cfg = cfg_we(n, V, w, T=0.9, gamma=g)
+    prop = np.array([[2, 0, 1, 0]])
+    drafts = np.array([[1, 4, 2]])
+    for j in range(g):
+        l = logits[:, 0, j, :].astype(np.float64)
+        ps = [sp_softmax(l[i] / cfg.temperature) for i in range(n)]
+        r = sum(cfg.w64[i] * ps[i] for i in range(n))
+        want = min(1.0, r[drafts[0, j]] / ps[prop[0, j]][drafts[0, j]])
+        # bisection over the accept decision of the whole-batch entry point at position j
+        def accepted(mi):
+            ua = np.full((1, g + 1), 2.0 ** -24)     # every other position accepts
+            ua[0, j] = lattice_u(mi)
+            out = orc.verify(logits, "f32", drafts, prop, cfg, 0, 0, uniforms=(ua, np.full((1, g + 1), 0.5)))
+            return bool(out["accept"][0, j])
+        lo, hi = 0, LATTICE - 1
+        assert accepted(lo)
+        if accepted(hi):
+            count = LATTICE
+        else:
+            while hi - lo > 1:
+                mid = (lo + hi) // 2
+                if accepted(mid):
+                    lo = mid
+                else:
+                    hi = mid
+            count = lo + 1
+        assert abs(count / LATTICE - want) <= 2.0 ** -22
+    # a constant table is the per-row form
+    a = orc.verify(logits, "f32", drafts, np.array([[1, 1, 1, 1]]), cfg, 3, 1)
+    b = orc.verify(logits, "f32", drafts, np.array([1]), cfg, 3, 1)
+    for k in ("accept_count", "out_tokens", "row_status"):
+        assert np.array_equal(a[k], b[k])
