@@ -61,8 +61,18 @@ enum {
 
 /* bits of cos_verify_args.flags */
 enum {
-  COS_RUN_ALL_RESIDUALS = 1 /* compute the residual mass S = sum max(0, r - q) = 1 - alpha (Eq. 7) at  */
-                            /* every draft position and report it in diag, not only where it is needed */
+  COS_RUN_ALL_RESIDUALS = 1,         /* compute the residual mass S = sum max(0, r - q) = 1 - alpha      */
+                                     /* (Eq. 7) at every draft position and report it in diag, not only  */
+                                     /* where it is needed                                               */
+  COS_RUN_PROPOSER_PER_POSITION = 2, /* `proposer` is [B][gamma+1]: entry (b, j), j < gamma, is the model */
+                                     /* that proposed draft j of row b, so q changes from position to    */
+                                     /* position (Algorithm 2 verifies a cached sequence that holds      */
+                                     /* tokens of several proposers).  Entry (b, gamma) must be a valid  */
+                                     /* index; its distribution decides nothing.                         */
+  COS_RUN_BONUS_FROM_MODEL = 4       /* the token after gamma acceptances is drawn from model            */
+                                     /* `bonus_model`'s own distribution instead of the combined one     */
+                                     /* (Sec. 3.3: the verifier's bonus token, to be treated as that     */
+                                     /* model's next proposal)                                           */
 };
 
 typedef struct {
@@ -90,6 +100,7 @@ typedef struct {
   int64_t stride_model, stride_row, stride_pos;
   const int32_t* draft_tokens; /* [B][gamma]; may be NULL when gamma == 0                               */
   const int32_t* proposer;     /* [B], index in [0, n) of the model that proposed the row's drafts      */
+                               /* ([B][gamma+1] with COS_RUN_PROPOSER_PER_POSITION)                     */
   int32_t batch;               /* B, 1..max_batch                                                       */
   int32_t flags;               /* COS_RUN_* bits                                                        */
   int64_t row_base;            /* global index of row 0 (for row-sharded batches); enters the RNG only  */
@@ -104,6 +115,10 @@ typedef struct {
                                /* draft, and S where it was computed (NaN elsewhere); may be NULL       */
   float* dump_r;               /* optional test hook, out [B][gamma+1][V]: the combined distribution;   */
                                /* forces the full second sweep everywhere; may be NULL                  */
+  float* bonus_prob;           /* optional out [B]: where accept_count == gamma, the probability of the */
+                               /* bonus token under the distribution it was drawn from (what Score of   */
+                               /* Algorithm 2 returns beside the token); NaN elsewhere; may be NULL     */
+  int32_t bonus_model;         /* read only with COS_RUN_BONUS_FROM_MODEL: index in [0, n)              */
 } cos_verify_args;
 
 typedef struct {

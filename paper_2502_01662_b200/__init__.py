@@ -15,6 +15,8 @@ from .binding import (  # noqa: F401
     COS_ROW_Q_ZERO,
     COS_ROW_RESIDUAL_EMPTY,
     COS_RUN_ALL_RESIDUALS,
+    COS_RUN_BONUS_FROM_MODEL,
+    COS_RUN_PROPOSER_PER_POSITION,
     CosVerifier,
     CosVerifyError,
     load_library,

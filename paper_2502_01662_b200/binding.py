@@ -22,6 +22,8 @@ COS_ROW_Q_ZERO = 4
 COS_ROW_RESIDUAL_EMPTY = 8
 COS_ROW_FAULT = 16   # an internal wait of the kernel gave up: the call's outputs are undefined
 COS_RUN_ALL_RESIDUALS = 1
+COS_RUN_PROPOSER_PER_POSITION = 2   # proposer is [B, gamma+1]: the model that proposed each draft (Algorithm 2)
+COS_RUN_BONUS_FROM_MODEL = 4        # the bonus token follows one named model's own distribution (Sec. 3.3)
 
 _STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR_ALIGNMENT",
                  4: "COS_ERR_CUDA", 5: "COS_ERR_NOMEM"}
@@ -54,7 +56,7 @@ class cos_verify_args(ctypes.Structure):
         ("batch", ctypes.c_int32), ("flags", ctypes.c_int32), ("row_base", ctypes.c_int64),
         ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64), ("accept_count", ctypes.c_void_p),
         ("out_tokens", ctypes.c_void_p), ("row_status", ctypes.c_void_p), ("diag", ctypes.c_void_p),
-        ("dump_r", ctypes.c_void_p),
+        ("dump_r", ctypes.c_void_p), ("bonus_prob", ctypes.c_void_p), ("bonus_model", ctypes.c_int32),
     ]
 
 
@@ -142,8 +144,18 @@ class CosVerifier:
         return {k: getattr(inf, k) for k in ("cluster_size", "threads_per_block", "max_clusters", "sm_count",
                                              "launches_per_run")}
 
-    def _fill_args(self, logits, drafts, proposer, seed, offset, row_base, flags, outs) -> cos_verify_args:
+    def _fill_args(self, logits, drafts, proposer, seed, offset, row_base, flags, outs,
+                   bonus_model=None) -> cos_verify_args:
         n, B, P, V = logits.shape
+        # a [B, gamma+1] proposer table selects the per-position form; a bonus model selects its flag
+        if proposer.dim() == 2:
+            if tuple(proposer.shape) != (B, P):
+                raise ValueError("a per-position proposer table must be [B, gamma+1]")
+            flags |= COS_RUN_PROPOSER_PER_POSITION
+        elif proposer.numel() != B:
+            raise ValueError("proposer must be [B] or [B, gamma+1]")
+        if bonus_model is not None and bonus_model >= 0:
+            flags |= COS_RUN_BONUS_FROM_MODEL
         if n != self.cfg.n or P != self.cfg.gamma + 1 or V != self.cfg.vocab:
             raise ValueError(f"logits shape {tuple(logits.shape)} does not match the context")
         if logits.stride(3) != 1:
@@ -162,6 +174,8 @@ class CosVerifier:
         a.row_status = outs["row_status"].data_ptr()
         a.diag = outs["diag"].data_ptr() if "diag" in outs else None
         a.dump_r = outs["r"].data_ptr() if "r" in outs else None
+        a.bonus_prob = outs["bonus_prob"].data_ptr() if "bonus_prob" in outs else None
+        a.bonus_model = bonus_model if (bonus_model is not None and bonus_model >= 0) else 0
         return a
 
     def set_stage_timing(self, enable: bool):
@@ -185,6 +199,7 @@ class CosVerifier:
             "accept_count": torch.empty(B, dtype=torch.int32, **kw),
             "out_tokens": torch.empty((B, P), dtype=torch.int32, **kw),
             "row_status": torch.empty(B, dtype=torch.int32, **kw),
+            "bonus_prob": torch.empty(B, dtype=torch.float32, **kw),
         }
         if diag:
             outs["diag"] = torch.empty((B, P, 4), dtype=torch.float32, **kw)
@@ -194,8 +209,13 @@ class CosVerifier:
 
     # -- the calls -------------------------------------------------------------------
     def run(self, logits, drafts, proposer, seed: int, offset: int, row_base: int = 0, flags: int = 0,
-            diag: bool = False, dump_r: bool = False, outs: Optional[dict] = None, stream=None) -> dict:
-        """cos_verify_run on device tensors; asynchronous on `stream` (default: torch's current stream)."""
+            diag: bool = False, dump_r: bool = False, outs: Optional[dict] = None, stream=None,
+            bonus_model: Optional[int] = None) -> dict:
+        """cos_verify_run on device tensors; asynchronous on `stream` (default: torch's current stream).
+
+        `proposer` is [B], or [B, gamma+1] to name the proposer of every draft (Algorithm 2); `bonus_model`
+        draws the token after gamma acceptances from that model's own distribution (Sec. 3.3).  The outputs
+        include "bonus_prob" [B]: the bonus token's probability under the law it was drawn from."""
         import torch
         if not logits.is_cuda:
             raise ValueError("run() needs device tensors; use run_host() for host tensors")
@@ -205,13 +225,14 @@ class CosVerifier:
         n, B, P, V = logits.shape
         if outs is None:
             outs = self._alloc_outs(B, P, V, logits.device, diag, dump_r)
-        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs)
+        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs, bonus_model)
         s = torch.cuda.current_stream(logits.device) if stream is None else stream
         self._check(self._lib.cos_verify_run(self._ctx, ctypes.byref(a), ctypes.c_void_p(s.cuda_stream)))
         return outs
 
     def run_host(self, logits, drafts, proposer, seed: int, offset: int, row_base: int = 0, flags: int = 0,
-                 diag: bool = False, outs: Optional[dict] = None, stream=None) -> dict:
+                 diag: bool = False, outs: Optional[dict] = None, stream=None,
+                 bonus_model: Optional[int] = None) -> dict:
         """cos_verify_run_host on host tensors: copies in, runs, copies out, waits."""
         import torch
         if logits.is_cuda or not logits.is_contiguous():
@@ -222,7 +243,7 @@ class CosVerifier:
         n, B, P, V = logits.shape
         if outs is None:
             outs = self._alloc_outs(B, P, V, "cpu", diag, False, pin=True)
-        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs)
+        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs, bonus_model)
         s = torch.cuda.current_stream(self.cfg.device) if stream is None else stream
         self._check(self._lib.cos_verify_run_host(self._ctx, ctypes.byref(a), ctypes.c_void_p(s.cuda_stream)))
         return outs
@@ -285,6 +306,8 @@ def run_static(n: int, combine: int, weights: Sequence[float], temperature: floa
     a.row_status = outs["row_status"].data_ptr()
     a.diag = outs["diag"].data_ptr() if "diag" in outs else None
     a.dump_r = None
+    a.bonus_prob = outs["bonus_prob"].data_ptr() if "bonus_prob" in outs else None
+    a.bonus_model = 0
     s = torch.cuda.current_stream(logits.device) if stream is None else stream
     st = lib.cos_verify_run_static(ctypes.byref(cfg), ctypes.byref(a), ctypes.c_void_p(s.cuda_stream))
     if st != COS_OK:

@@ -41,6 +41,7 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxSlots = COS_MAX_MODELS + 2;
 constexpr int kNoReject = 0x7fffffff;
+constexpr int kDrawResidual = 0, kDrawR = 1, kDrawQ = 2;  // what a token is drawn from: max(0, r - q), r, or q
 constexpr double kBigShare = 1.0 / 256.0;  // probabilities above 2^-8 get fp64 treatment when tokens are drawn
 constexpr int kRingVecs = 8;                 // 16-byte vectors per lane staged ahead in sweep 2 (4 KB per warp)
 constexpr int kRingBytes = kWarps * kRingVecs * 32 * 16;
@@ -68,6 +69,9 @@ struct KParams {
   int nsteps;   // ceil(V / (32 * E))
   int flags;
   int num_units, num_clusters;
+  int per_pos;      // proposer is [B][gamma+1] (the model that proposed each draft) instead of [B]
+  int greedy;       // T = 0: no drawing stages; the fourth word of a unit's result carries the bonus probability
+  int bonus_model;  // >= 0: the token after gamma acceptances follows this model's own distribution; -1: the combined one
   int parts;     // blocks that share one unit in stages 1 and 2
   int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
@@ -82,6 +86,7 @@ struct KParams {
   unsigned* row_status;
   float* diag;
   float* dump_r;
+  float* bonus_prob;
   // scratch owned by the context
   unsigned* work_counter;  // units are handed out from here; grows by num_units every run
   unsigned work_base;      // its value when this run starts
@@ -254,6 +259,7 @@ struct Decision {  // written by thread 0 of every block, identically
   int atom_tok[COS_MAX_MODELS];
   double atom_mass[COS_MAX_MODELS];
   double ratio, r_d, q_d, S;
+  double prob;  // greedy, bonus position: probability of cand under the law it came from
 };
 
 // Stage 0 without block barriers: every warp streams its share of unit after unit; what the warps of
@@ -284,6 +290,7 @@ struct Shared {
   float a_scale[COS_MAX_MODELS];  // w_i / Z_i (ensemble) for sweep 2
   float a_ref[COS_MAX_MODELS];
   float a_resid[COS_MAX_MODELS];  // coefficient of e_i in r - q
+  float a_draw[COS_MAX_MODELS];   // coefficient of e_i in the law a bonus token is drawn from (r, or the named model's)
   Decision dec;
   double u_acc, u_smp;
   double target, base;  // sweep-2 search: u*S and the mass before the winning block
@@ -464,6 +471,15 @@ __device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& clu
   ++phase;
 }
 
+// The model whose distribution is q at position j of row b: the row's proposer, or the proposer of that draft
+// when the caller gave one per position (Algorithm 2 verifies tokens of several proposers in one sequence).
+// At the bonus position of a call that names a bonus model, q is that model's distribution: the token is
+// then drawn from q (Sec. 3.3) by the machinery that otherwise draws from r.
+__device__ __forceinline__ int proposer_of(const KParams& p, int b, int j) {
+  if (j == p.gamma && p.bonus_model >= 0) return p.bonus_model;
+  return p.proposer[p.per_pos ? b * p.P + j : b];
+}
+
 // ------------------------------------------------------------------------------------
 // publishing a unit and the per-row first-rejection scan (Sec. 3.1)
 // ------------------------------------------------------------------------------------
@@ -475,8 +491,11 @@ __device__ __forceinline__ void push_job(const KParams& p, int idx, int emit) {
 // Stage 0: record a unit's decision; the last unit of a row to arrive scans for the first
 // rejection, writes the row's outputs and, where a token has to be drawn, lists that unit
 // for stage 1 (which fills in out_tokens[b][a]).
-__device__ void publish_unit(const KParams& p, int b, int j, int accept, int status, int cand, int drawable,
+// `word4`: sampling modes: whether a token can be drawn at this unit; greedy modes: the bits of the bonus
+// token's probability (a float), NaN away from the bonus position.
+__device__ void publish_unit(const KParams& p, int b, int j, int accept, int status, int cand, int word4,
                              double ratio, double r_d, double q_d, double S) {
+  const int drawable = p.greedy ? 0 : word4;
   const int idx = b * p.P + j;
   if (p.diag) {
     float* d = p.diag + static_cast<long long>(idx) * 4;
@@ -485,7 +504,7 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
     d[2] = static_cast<float>(q_d);
     d[3] = static_cast<float>(S);
   }
-  int4 res = make_int4(accept, status, cand, drawable);
+  int4 res = make_int4(accept, status, cand, word4);
   __stcg(&p.unit_res[idx], res);
   // test hooks: the combined distribution everywhere, or the residual mass at every draft position
   if (drawable && (p.dump_r != nullptr || ((p.flags & COS_RUN_ALL_RESIDUALS) && j < p.gamma))) push_job(p, idx, 0);
@@ -507,6 +526,12 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
       break;
     }
   }
+  if (p.bonus_prob != nullptr) {
+    // sampling modes: the drawing stage fills it in after a full acceptance; greedy modes know it here
+    const bool known = p.greedy && a == p.gamma && tok >= 0;
+    p.bonus_prob[b] = known ? __int_as_float(draw) : __int_as_float(0x7fc00000);
+  }
+  if (p.greedy) draw = 0;
   p.accept_count[b] = a;
   int* o = p.out_tokens + static_cast<long long>(b) * p.P;
   for (int k = 0; k < p.P; ++k) o[k] = (k < a) ? p.drafts[b * p.gamma + k] : (k == a ? tok : -1);
@@ -596,7 +621,7 @@ __device__ __forceinline__ LaneSoft soft_slice(const void* row, const Slice& sl,
 // clipped at zero, or r.  Rare; kept out of line so that the mass loop stays small.
 // `staged`/`k`: where the token's logits sit in shared memory (null: read them from global memory).
 template <int DT, int MODE>
-__device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* fsoft, const char* base, int e, bool use_r,
+__device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* fsoft, const char* base, int e, int draw,
                                               const uint4* staged, int k, bool masked, float thr, int pis) {
   if (e >= p.V) return 0.0;
   double r64 = 0.0, q64 = 0.0;
@@ -620,7 +645,7 @@ __device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* 
     r64 = in ? exp2(cd * p.cT64 - static_cast<double>(fsoft[1].ref)) / fsoft[1].s : 0.0;
     q64 = exp2(static_cast<double>(lv[pis]) * p.cT64 - static_cast<double>(fsoft[0].ref)) / fsoft[0].s;
   }
-  return use_r ? r64 : fmax(0.0, r64 - q64);
+  return draw == kDrawR ? r64 : (draw == kDrawQ ? q64 : fmax(0.0, r64 - q64));
 }
 
 // Combined logit of one token in fp64, from the stored logits: the chain of fused multiply-adds that
@@ -910,7 +935,7 @@ __device__ __forceinline__ void decide_unit(const KParams& p, Shared& sh, bool i
   d.want_sample = 0;
   d.cand = -1;
   d.natoms = 0;
-  d.ratio = d.r_d = d.q_d = d.S = kNaN;
+  d.ratio = d.r_d = d.q_d = d.S = d.prob = kNaN;
   bool finite = pi_ok;
   if (kSample) {
     const int nsoft = (MODE == kEnsembleSample) ? p.n : 2;
@@ -1034,6 +1059,14 @@ __device__ __forceinline__ void decide_unit(const KParams& p, Shared& sh, bool i
         if (d.cand < 0 && m > 0.0 && run >= target) d.cand = d.atom_tok[k];
       }
       if (d.cand < 0) d.cand = lastpos;
+      if (is_bonus) {
+        if (p.bonus_model >= 0) {  // the named model's one-hot law (its argmax sits in the proposer's slot)
+          d.cand = qtok;
+          d.prob = 1.0;
+        } else {
+          d.prob = r_at(d.cand);
+        }
+      }
     }
   }
   d.need2 = 0;  // tokens are drawn by stage 1, for the one position per row that needs it
@@ -1109,7 +1142,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
     const int unit = unit_of[seq & 3];
     if (unit >= p.num_units) break;
     const int j = unit / p.B, b = unit % p.B;  // earlier positions of every row come first
-    const int pi = p.proposer[b];
+    const int pi = proposer_of(p, b, j);
     const bool pi_ok = (pi >= 0 && pi < p.n);
     const int pis = pi_ok ? pi : 0;
     const char* base = reinterpret_cast<const char*>(p.logits) +
@@ -1196,7 +1229,8 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       if (kSample && lane == 31) p.ustats[uidx].thr32 = 0.f;
       if (lane == 0) {
         const Decision& d = sh.dec;
-        publish_unit(p, b, j, d.accept, d.status, d.cand, d.drawable, d.ratio, d.r_d, d.q_d, d.S);
+        publish_unit(p, b, j, d.accept, d.status, d.cand, kSample ? d.drawable : __float_as_int(static_cast<float>(d.prob)),
+                     d.ratio, d.r_d, d.q_d, d.S);
         fr.arrive[par] = 0;
         __threadfence_block();
         *epi_done = seq + 1;
@@ -1270,13 +1304,14 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       emit = (p.accept_count[b] == j) ? 1 : 0;  // the token drawn here is the row's output
     }
     const int uidx = b * p.P + j;
-    const int pi = p.proposer[b];
+    const int pi = proposer_of(p, b, j);
     const bool pi_ok = (pi >= 0 && pi < p.n);
     const int pis = pi_ok ? pi : 0;
     const char* base = reinterpret_cast<const char*>(p.logits) +
                        (static_cast<long long>(b) * p.s_row + static_cast<long long>(j) * p.s_pos) * Elem<DT>::bytes;
     auto row_of = [&](int i) -> const void* { return base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes; };
     const bool is_bonus = (j == p.gamma);
+    const bool draw_q = is_bonus && p.bonus_model >= 0;  // the bonus token follows the named model's own law
     const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
     const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
 
@@ -1600,6 +1635,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         const double a = p.w64[tid] / sh.fsoft[tid].s;
         sh.a_scale[tid] = static_cast<float>(a);
         sh.a_resid[tid] = static_cast<float>(a - (tid == pis ? 1.0 / sh.fsoft[tid].s : 0.0));
+        sh.a_draw[tid] = draw_q ? static_cast<float>(tid == pis ? 1.0 / sh.fsoft[tid].s : 0.0) : sh.a_scale[tid];
         sh.a_ref[tid] = -sh.fsoft[tid].ref;
       }
       __syncthreads();
@@ -1624,7 +1660,8 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         float acc[E], rr[E];
         bool anybig = false;
         bigbits = 0u;
-        const float* coef = use_r ? sh.a_scale : sh.a_resid;
+        const float* coef = use_r ? sh.a_draw : sh.a_resid;
+        const bool from_q = use_r && draw_q;
 #pragma unroll
         for (int k = 0; k < E; ++k) {
           acc[k] = 0.f;
@@ -1676,7 +1713,8 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             emc = fmaxf(emc, ec);
             emq = fmaxf(emq, eq[k]);
             rr[k] = ec * inv_zc;
-            acc[k] = __fsub_rn(rr[k], __fmul_rn(eq[k], qco));  // rounded product: r == q cancels exactly
+            // rounded product: r == q cancels exactly
+            acc[k] = from_q ? __fmul_rn(eq[k], inv_zq) : __fsub_rn(rr[k], __fmul_rn(eq[k], qco));
           }
           anybig = (emc > sh.big_thr[1]) || (emq > sh.big_thr[0]);
         }
@@ -1709,7 +1747,8 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         }
       };
       auto big_mass = [&](int e, bool use_r, const uint4* staged, int k) -> double {
-        return big_token_mass<DT, MODE>(p, sh.fsoft, base, e, use_r, staged, k, masked, thr, pis);
+        const int draw = use_r ? (draw_q ? kDrawQ : kDrawR) : kDrawResidual;
+        return big_token_mass<DT, MODE>(p, sh.fsoft, base, e, draw, staged, k, masked, thr, pis);
       };
       // a lane's mass of one step: fp32 sum of the small tokens in token order plus the big ones in fp64
       auto lane_mass = [&](int e0, const float (&mass32)[E], unsigned bigbits, bool use_r, const uint4* staged) -> double {
@@ -1980,7 +2019,12 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             const int se = static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
             const int token = walk(sb, se, run_gsz(se - sb, kRecG), sh.base,
                                    p.srung + (static_cast<size_t>(b) * G + g) * kRecG, sh.target, is_bonus);
-            if (lane == 0) p.out_tokens[uidx] = token;  // the row's token at its first rejection, or the bonus
+            if (lane == 0) {
+              p.out_tokens[uidx] = token;  // the row's token at its first rejection, or the bonus
+              // Algorithm 2's Score returns the bonus token with its probability under the law it came from
+              if (is_bonus && p.bonus_prob != nullptr && token >= 0)
+                p.bonus_prob[b] = static_cast<float>(big_mass(token, true, nullptr, 0));
+            }
           }
         } else if (!is_bonus && emit) {
           // no residual mass although a token is needed: this block draws from r instead, over the whole
@@ -2006,7 +2050,8 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     }
     if (STAGE == 0 && rank == 0 && tid == 0) {
       const Decision& d = sh.dec;
-      publish_unit(p, b, j, d.accept, d.status, d.cand, d.drawable, d.ratio, d.r_d, d.q_d, d.S);
+      publish_unit(p, b, j, d.accept, d.status, d.cand, kSample ? d.drawable : __float_as_int(static_cast<float>(d.prob)),
+                   d.ratio, d.r_d, d.q_d, d.S);
     }
     // No barrier here: everything the next unit writes before its first block barrier
     // (ldraft, next_local, u_acc/u_smp, warp partials) is read only before this point; stage 1
@@ -2052,6 +2097,7 @@ struct cos_verify_ctx {
   void* d_logits;
   int* d_drafts;
   int* d_proposer;
+  float* d_bonus;
   int* d_accept;
   int* d_tokens;
   unsigned* d_status;
@@ -2323,7 +2369,8 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
     const size_t V = static_cast<size_t>(config->vocab);
     ok = ok && cudaMalloc(&ctx->d_logits, static_cast<size_t>(config->n) * rows * P * V * elem_bytes(config->dtype)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_drafts, rows * (P > 1 ? P - 1 : 1) * sizeof(int)) == cudaSuccess;
-    ok = ok && cudaMalloc(&ctx->d_proposer, rows * sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_proposer, rows * P * sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_bonus, rows * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_accept, rows * sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_tokens, rows * P * sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&ctx->d_status, rows * sizeof(unsigned)) == cudaSuccess;
@@ -2364,7 +2411,13 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   if (!a->logits || !a->proposer || !a->accept_count || !a->out_tokens || !a->row_status) return bad("null device pointer");
   if (c.gamma > 0 && !a->draft_tokens) return bad("draft_tokens is null although gamma > 0");
   if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return bad("negative stride");
-  if (a->flags & ~COS_RUN_ALL_RESIDUALS) return bad("unknown flag bits");
+  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL)) return bad("unknown flag bits");
+  if ((a->flags & COS_RUN_BONUS_FROM_MODEL) && (a->bonus_model < 0 || a->bonus_model >= c.n))
+    return bad("bonus_model outside [0, n)");
+  if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4) {
+    ctx->err = "bonus_prob is not 4-byte aligned";
+    return COS_ERR_ALIGNMENT;
+  }
   const int eb = elem_bytes(c.dtype);
   if (reinterpret_cast<uintptr_t>(a->logits) % eb) {
     ctx->err = "logits pointer not aligned to its element type";
@@ -2424,6 +2477,10 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.row_status = a->row_status;
   p.diag = a->diag;
   p.dump_r = a->dump_r;
+  p.bonus_prob = a->bonus_prob;
+  p.per_pos = (a->flags & COS_RUN_PROPOSER_PER_POSITION) ? 1 : 0;
+  p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
+  p.greedy = (c.temperature == 0.0f) ? 1 : 0;
   p.work_counter = ctx->d_work_counter;
   p.work_base = ctx->work_base;
   p.row_arrivals = ctx->d_row_arrivals;
@@ -2515,7 +2572,8 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
   e = cudaMemcpyAsync(ctx->d_logits, a->logits, lbytes, cudaMemcpyHostToDevice, stream);
   if (e == cudaSuccess && c.gamma > 0)
     e = cudaMemcpyAsync(ctx->d_drafts, a->draft_tokens, B * c.gamma * sizeof(int), cudaMemcpyHostToDevice, stream);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_proposer, a->proposer, B * sizeof(int), cudaMemcpyHostToDevice, stream);
+  const size_t nprop = (a->flags & COS_RUN_PROPOSER_PER_POSITION) ? static_cast<size_t>(B * P) : static_cast<size_t>(B);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_proposer, a->proposer, nprop * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "host to device copy", e);
   cos_verify_args d = *a;
   d.logits = ctx->d_logits;
@@ -2525,6 +2583,7 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
   d.out_tokens = ctx->d_tokens;
   d.row_status = ctx->d_status;
   d.diag = a->diag ? ctx->d_diag : nullptr;
+  d.bonus_prob = a->bonus_prob ? ctx->d_bonus : nullptr;
   cos_status st = cos_verify_run(ctx, &d, stream);
   if (st != COS_OK) return st;
   e = cudaMemcpyAsync(a->accept_count, ctx->d_accept, B * sizeof(int), cudaMemcpyDeviceToHost, stream);
@@ -2532,6 +2591,8 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
   if (e == cudaSuccess) e = cudaMemcpyAsync(a->row_status, ctx->d_status, B * sizeof(unsigned), cudaMemcpyDeviceToHost, stream);
   if (e == cudaSuccess && a->diag)
     e = cudaMemcpyAsync(a->diag, ctx->d_diag, B * P * 4 * sizeof(float), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess && a->bonus_prob)
+    e = cudaMemcpyAsync(a->bonus_prob, ctx->d_bonus, B * sizeof(float), cudaMemcpyDeviceToHost, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
   if (e != cudaSuccess) {
     ctx->scratch_dirty = true;
@@ -2598,6 +2659,7 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_drafts);
   cudaFree(ctx->d_proposer);
+  cudaFree(ctx->d_bonus);
   cudaFree(ctx->d_accept);
   cudaFree(ctx->d_tokens);
   cudaFree(ctx->d_status);
@@ -2652,7 +2714,11 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     return static_fail(COS_ERR_INVALID_ARG, "null device pointer");
   if (c.gamma > 0 && !a->draft_tokens) return static_fail(COS_ERR_INVALID_ARG, "draft_tokens is null although gamma > 0");
   if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return static_fail(COS_ERR_INVALID_ARG, "negative stride");
-  if (a->flags & ~COS_RUN_ALL_RESIDUALS) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
+  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL)) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
+  if ((a->flags & COS_RUN_BONUS_FROM_MODEL) && (a->bonus_model < 0 || a->bonus_model >= c.n))
+    return static_fail(COS_ERR_INVALID_ARG, "bonus_model outside [0, n)");
+  if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4)
+    return static_fail(COS_ERR_ALIGNMENT, "bonus_prob is not 4-byte aligned");
   const int eb = elem_bytes(c.dtype);
   if (reinterpret_cast<uintptr_t>(a->logits) % eb) return static_fail(COS_ERR_ALIGNMENT, "logits pointer not aligned to its element type");
   if (reinterpret_cast<uintptr_t>(a->proposer) % 4 || reinterpret_cast<uintptr_t>(a->accept_count) % 4 ||
@@ -2744,6 +2810,10 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.row_status = a->row_status;
   p.diag = a->diag;
   p.dump_r = a->dump_r;
+  p.bonus_prob = a->bonus_prob;
+  p.per_pos = (a->flags & COS_RUN_PROPOSER_PER_POSITION) ? 1 : 0;
+  p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
+  p.greedy = (c.temperature == 0.0f) ? 1 : 0;
   p.work_counter = d_counter;
   p.work_base = 0;  // the counter was just cleared
   p.row_arrivals = d_arrivals;

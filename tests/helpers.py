@@ -16,12 +16,13 @@ TOL_R = {"f32": 1e-5, "bf16": 2e-3}      # relative tolerance on combined probab
 FLOOR_R = 1e-30                          # fp32 cannot hold probabilities far below this
 
 
-def oracle_config(w: synth.Workload) -> orc.OracleConfig:
+def oracle_config(w: synth.Workload, bonus_model: int = -1) -> orc.OracleConfig:
     return orc.OracleConfig(n=w.n, combine=w.combine, weights=list(w.weights), temperature=w.temperature,
-                            gamma=w.gamma, vocab=w.vocab, mask_model=w.mask_model, mask_alpha=w.mask_alpha)
+                            gamma=w.gamma, vocab=w.vocab, mask_model=w.mask_model, mask_alpha=w.mask_alpha,
+                            bonus_model=bonus_model)
 
 
-def run_oracle(w: synth.Workload, inputs: dict, rows=None, return_r=False, row_base=0) -> dict:
+def run_oracle(w: synth.Workload, inputs: dict, rows=None, return_r=False, row_base=0, bonus_model: int = -1) -> dict:
     logits = inputs["logits"]
     if rows is not None:
         # copy only the sampled rows to the host (full-size cases hold gigabytes)
@@ -33,7 +34,7 @@ def run_oracle(w: synth.Workload, inputs: dict, rows=None, return_r=False, row_b
     else:
         host = synth.logits_as_numpy(logits)
     return orc.verify(host, w.dtype, inputs["drafts"].cpu().numpy(), inputs["proposer"].cpu().numpy(),
-                      oracle_config(w), inputs["seed"], inputs["offset"], row_base=row_base, rows=rows,
+                      oracle_config(w, bonus_model), inputs["seed"], inputs["offset"], row_base=row_base, rows=rows,
                       return_r=return_r)
 
 
@@ -94,6 +95,18 @@ def check_parity(w: synth.Workload, gpu: dict, ref: dict, rows=None, check_diag=
                 if np.isfinite(s_got):
                     assert abs(s_got - ref["S"][b, j]) <= 1e-5 * max(ref["S"][b, j], 1e-3) + 1e-7, \
                         (b, j, "S", s_got, ref["S"][b, j])
+    if "bonus_prob" in gpu and "bonus_prob" in ref:
+        # probability of the bonus token under the law it was drawn from; NaN unless every draft passed
+        tol = TOL_R[w.dtype]
+        for b in rows:
+            if int(gpu["accept_count"][b]) != int(ref["accept_count"][b]) or \
+                    not np.array_equal(gpu["out_tokens"][b], ref["out_tokens"][b]):
+                continue  # an excused boundary row
+            want, got = ref["bonus_prob"][b], gpu["bonus_prob"][b]
+            if np.isnan(want):
+                assert np.isnan(got), (b, "bonus_prob", got)
+            else:
+                assert abs(got - want) <= tol * abs(want) + FLOOR_R, (b, "bonus_prob", got, want)
     return {"rows": len(list(rows)), "excused_accept": excused_accept, "excused_sample": excused_sample}
 
 

@@ -64,3 +64,42 @@ def test_every_cluster_size_gives_the_oracles_rows(w, cs):
             assert np.array_equal(again[k], gpu[k]), k
     finally:
         v.close()
+
+
+# Alternate proposals (Sec. 3.3, Algorithm 2): the proposer of every draft given position by position, and
+# the bonus token drawn from one named model's own distribution, with its probability returned.
+from dataclasses import replace as _replace
+
+ALT = [SMALL[i] for i in (0, 2, 4, 6, 7, 8)] + [
+    C["cfg2"].scaled(batch=16, vocab=9001, gamma=1, name="cfg2_gamma1"),     # masked, many rows reach the bonus
+    _replace(C["cfg4"].scaled(batch=6, vocab=12808, gamma=3, name="cfg4_greedy_small"), temperature=0.0),
+]
+
+
+@pytest.mark.parametrize("cs", [0, 1, 2])
+@pytest.mark.parametrize("w", ALT, ids=[w.name for w in ALT])
+def test_proposer_per_position_and_named_bonus_model(w, cs):
+    inputs = synth.make_inputs(w, "cuda")
+    B, P = w.batch, w.gamma + 1
+    gen = np.random.default_rng(77)
+    table = gen.integers(0, w.n, size=(B, P)).astype(np.int32)
+    if w.temperature == 0.0:
+        # make some rows pass every draft: their drafts are the argmax of the model named at each position
+        lg = inputs["logits"].float()
+        for b in range(0, B, 2):
+            for j in range(w.gamma):
+                inputs["drafts"][b, j] = int(torch.argmax(lg[int(table[b, j]), b, j]))
+    inputs = dict(inputs, proposer=torch.as_tensor(table, device="cuda"))
+    for m in range(-1, w.n):
+        ref = helpers.run_oracle(w, inputs, bonus_model=m)
+        v = helpers.make_verifier(w, cluster_size=cs)
+        try:
+            gpu = helpers.run_gpu(w, inputs, verifier=v, diag=True, bonus_model=m)
+        finally:
+            v.close()
+        stats = helpers.check_parity(w, gpu, ref)
+        assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
+    # the table is read: with another one some row changes
+    other = helpers.run_oracle(w, dict(inputs, proposer=torch.as_tensor((table + 1) % w.n)), bonus_model=-1)
+    assert w.n == 1 or not np.array_equal(other["accept_count"], ref["accept_count"]) or \
+        not np.array_equal(other["out_tokens"], ref["out_tokens"])
