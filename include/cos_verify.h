@@ -46,7 +46,7 @@ enum {
                                  /*     interpolation of an aligned / base model pair)             */
 };
 
-enum { COS_DTYPE_F32 = 0, COS_DTYPE_BF16 = 1 };
+enum { COS_DTYPE_F32 = 0, COS_DTYPE_BF16 = 1, COS_DTYPE_F16 = 2 };
 
 /* bits of row_status[b]; only positions up to and including the row's first rejection report */
 enum {

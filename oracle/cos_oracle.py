@@ -150,6 +150,11 @@ def to_float64(a, dtype: str) -> np.ndarray:
         return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
     if dtype == "f32":
         return np.asarray(a, dtype=np.float32).astype(np.float64)
+    if dtype == "f16":
+        a = np.asarray(a)
+        if a.dtype != np.float16:
+            raise ValueError("f16 logits must be passed as a float16 array")
+        return a.astype(np.float64)
     if dtype == "f64":
         return np.asarray(a, dtype=np.float64)
     raise ValueError(dtype)

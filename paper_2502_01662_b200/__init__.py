@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     COS_COMBINE_LOGIT_LINEAR,
     COS_COMBINE_PROB_ENSEMBLE,
     COS_DTYPE_BF16,
+    COS_DTYPE_F16,
     COS_DTYPE_F32,
     COS_ROW_BAD_DRAFT,
     COS_ROW_FAULT,

@@ -16,6 +16,7 @@ COS_COMBINE_PROB_ENSEMBLE = 0
 COS_COMBINE_LOGIT_LINEAR = 1
 COS_DTYPE_F32 = 0
 COS_DTYPE_BF16 = 1
+COS_DTYPE_F16 = 2
 COS_ROW_NONFINITE = 1
 COS_ROW_BAD_DRAFT = 2
 COS_ROW_Q_ZERO = 4
@@ -103,7 +104,9 @@ def _dtype_code(torch_dtype) -> int:
         return COS_DTYPE_F32
     if torch_dtype == torch.bfloat16:
         return COS_DTYPE_BF16
-    raise ValueError(f"logits must be float32 or bfloat16, not {torch_dtype}")
+    if torch_dtype == torch.float16:
+        return COS_DTYPE_F16
+    raise ValueError(f"logits must be float32, bfloat16 or float16, not {torch_dtype}")
 
 
 class CosVerifier:

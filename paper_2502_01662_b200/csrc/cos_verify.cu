@@ -21,6 +21,7 @@
 // Nothing in the kernel spins on memory: blocks meet only at hardware cluster barriers.
 
 #include <cooperative_groups.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdarg.h>
@@ -146,6 +147,26 @@ struct Elem<COS_DTYPE_F32> {
   }
   static __device__ __forceinline__ float pick(const uint4* vec, int k) {  // entry k of a vector in shared memory
     return reinterpret_cast<const float*>(vec)[k];
+  }
+};
+template <>
+struct Elem<COS_DTYPE_F16> {  // IEEE half: 8 entries per 16-byte vector, widened exactly
+  static constexpr int E = 8;
+  static constexpr int bytes = 2;
+  static __device__ __forceinline__ void unpack(const uint4& r, float (&v)[8]) {
+    const unsigned w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[k]));
+      v[2 * k] = f.x;
+      v[2 * k + 1] = f.y;
+    }
+  }
+  static __device__ __forceinline__ float load1(const void* row, long long x) {
+    return __half2float(__ldg(reinterpret_cast<const __half*>(row) + x));
+  }
+  static __device__ __forceinline__ float pick(const uint4* vec, int k) {  // entry k of a vector in shared memory
+    return __half2float(reinterpret_cast<const __half*>(vec)[k]);
   }
 };
 template <>
@@ -2117,6 +2138,7 @@ KernelFn pick_kernel(int dtype, int mode, int stage, bool dense = false) {
   if (dense && stage == 0 && mode == kEnsembleSample) {
     if (dtype == COS_DTYPE_F32) return cos_verify_kernel<COS_DTYPE_F32, kEnsembleSample, 0, 4>;
     if (dtype == COS_DTYPE_BF16) return cos_verify_kernel<COS_DTYPE_BF16, kEnsembleSample, 0, 4>;
+    if (dtype == COS_DTYPE_F16) return cos_verify_kernel<COS_DTYPE_F16, kEnsembleSample, 0, 4>;
   }
 #define COS_CASE(DT, M, S) \
   if (dtype == DT && mode == M && stage == S) return cos_verify_kernel<DT, M, S>;
@@ -2129,6 +2151,10 @@ KernelFn pick_kernel(int dtype, int mode, int stage, bool dense = false) {
   COS_SAMPLING(COS_DTYPE_BF16, kLogitSample)
   COS_CASE(COS_DTYPE_BF16, kEnsembleGreedy, 0)
   COS_CASE(COS_DTYPE_BF16, kLogitGreedy, 0)
+  COS_SAMPLING(COS_DTYPE_F16, kEnsembleSample)
+  COS_SAMPLING(COS_DTYPE_F16, kLogitSample)
+  COS_CASE(COS_DTYPE_F16, kEnsembleGreedy, 0)
+  COS_CASE(COS_DTYPE_F16, kLogitGreedy, 0)
 #undef COS_SAMPLING
 #undef COS_CASE
   return nullptr;
@@ -2140,8 +2166,8 @@ int mode_of(const cos_verify_config& c) {
   return greedy ? kLogitGreedy : kLogitSample;
 }
 
-int entries_per_vec(int dtype) { return dtype == COS_DTYPE_BF16 ? 8 : 4; }
-int elem_bytes(int dtype) { return dtype == COS_DTYPE_BF16 ? 2 : 4; }
+int entries_per_vec(int dtype) { return dtype == COS_DTYPE_F32 ? 4 : 8; }
+int elem_bytes(int dtype) { return dtype == COS_DTYPE_F32 ? 4 : 2; }
 
 bool fail(std::string* dst, const char* fmt, ...) {
   char buf[512];
@@ -2157,7 +2183,8 @@ bool validate_config(const cos_verify_config& c, std::string* err) {
   if (c.n < 1 || c.n > COS_MAX_MODELS) return fail(err, "n = %d outside 1..%d", c.n, COS_MAX_MODELS);
   if (c.combine != COS_COMBINE_PROB_ENSEMBLE && c.combine != COS_COMBINE_LOGIT_LINEAR)
     return fail(err, "unknown combine %d", c.combine);
-  if (c.dtype != COS_DTYPE_F32 && c.dtype != COS_DTYPE_BF16) return fail(err, "unknown dtype %d", c.dtype);
+  if (c.dtype != COS_DTYPE_F32 && c.dtype != COS_DTYPE_BF16 && c.dtype != COS_DTYPE_F16)
+    return fail(err, "unknown dtype %d", c.dtype);
   if (!(c.temperature >= 0.0f) || !isfinite(c.temperature)) return fail(err, "temperature must be finite and >= 0");
   if (c.gamma < 0) return fail(err, "gamma = %d must be >= 0", c.gamma);
   if (c.vocab < 1) return fail(err, "vocab = %d must be >= 1", c.vocab);

@@ -38,7 +38,7 @@ class Workload:
     batch: int
     gamma: int
     vocab: int
-    dtype: str                  # "f32" or "bf16"
+    dtype: str                  # "f32", "bf16" or "f16"
     generator: str              # "gauss" or "gumbel_zipf"
     sigma: float = 1.0          # gauss only
     rho: float = 0.8
@@ -55,7 +55,7 @@ class Workload:
 
     @property
     def elem_bytes(self) -> int:
-        return 2 if self.dtype == "bf16" else 4
+        return 4 if self.dtype == "f32" else 2
 
     @property
     def bytes_per_position(self) -> int:
@@ -64,7 +64,7 @@ class Workload:
 
     @property
     def torch_dtype(self):
-        return torch.bfloat16 if self.dtype == "bf16" else torch.float32
+        return {"bf16": torch.bfloat16, "f16": torch.float16}.get(self.dtype, torch.float32)
 
     def scaled(self, batch: Optional[int] = None, vocab: Optional[int] = None, gamma: Optional[int] = None,
                name: Optional[str] = None) -> "Workload":
@@ -91,6 +91,9 @@ CONFIGS: Dict[str, Workload] = {
     # 5: logit interpolation 1.5 * aligned - 0.5 * base, sampling and greedy
     "cfg5": Workload("cfg5", 2, COMBINE_LOGIT_LINEAR, (1.5, -0.5), 1.0, 256, 8, 256000, "bf16", "gumbel_zipf",
                      rho=0.9, proposer_rule="zero"),
+    # workload 3 with the logits stored as IEEE half (a variant; not one of the five baseline workloads)
+    "cfg3_f16": Workload("cfg3_f16", 2, COMBINE_PROB_ENSEMBLE, (0.5, 0.5), 0.7, 64, 8, 151936, "f16", "gumbel_zipf",
+                         rho=0.85, proposer_rule="bernoulli"),
     "cfg5_greedy": Workload("cfg5_greedy", 2, COMBINE_LOGIT_LINEAR, (1.5, -0.5), 0.0, 256, 8, 256000, "bf16",
                             "gumbel_zipf", rho=0.9, proposer_rule="zero"),
 }
@@ -180,7 +183,7 @@ def make_inputs(w: Workload, device="cpu") -> dict:
 
 
 def logits_as_numpy(logits: torch.Tensor) -> np.ndarray:
-    """Host copy for a CPU consumer: float32 array, or the raw 16-bit patterns of bf16."""
+    """Host copy for a CPU consumer: float32 or float16 array, or the raw 16-bit patterns of bf16."""
     t = logits.detach().cpu().contiguous()
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view(np.uint16)

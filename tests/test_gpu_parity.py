@@ -1,4 +1,6 @@
 """GPU parity: the CUDA path through the C ABI against the float64 oracle, element by element."""
+from dataclasses import replace as _replace
+
 import numpy as np
 import pytest
 import torch
@@ -26,6 +28,13 @@ SMALL = [
     C["cfg3"].scaled(batch=4, vocab=64, gamma=2, name="tiny_v64"),
     C["cfg3"].scaled(batch=4, vocab=5, gamma=1, name="tiny_v5"),
     C["cfg5"].scaled(batch=3, vocab=1000, gamma=0, name="gamma0"),
+]
+# the same recipes stored as IEEE half
+SMALL += [
+    _replace(C["cfg3"].scaled(batch=6, vocab=20008, gamma=4, name="cfg3_f16"), dtype="f16"),
+    _replace(C["cfg2"].scaled(batch=4, vocab=9001, name="cfg2_ragged_f16"), dtype="f16"),
+    _replace(C["cfg5"].scaled(batch=5, vocab=50000, gamma=3, name="cfg5_f16"), dtype="f16"),
+    _replace(C["cfg5_greedy"].scaled(batch=6, vocab=50000, gamma=3, name="cfg5_greedy_f16"), dtype="f16"),
 ]
 
 
@@ -68,8 +77,6 @@ def test_every_cluster_size_gives_the_oracles_rows(w, cs):
 
 # Alternate proposals (Sec. 3.3, Algorithm 2): the proposer of every draft given position by position, and
 # the bonus token drawn from one named model's own distribution, with its probability returned.
-from dataclasses import replace as _replace
-
 ALT = [SMALL[i] for i in (0, 2, 4, 6, 7, 8)] + [
     C["cfg2"].scaled(batch=16, vocab=9001, gamma=1, name="cfg2_gamma1"),     # masked, many rows reach the bonus
     _replace(C["cfg4"].scaled(batch=6, vocab=12808, gamma=3, name="cfg4_greedy_small"), temperature=0.0),

@@ -113,6 +113,14 @@ def test_bf16_and_f32_upcasts_are_exact():
     assert np.isposinf(v[5]) and np.isneginf(v[6]) and v[7] == 2.0 ** -133
     f = np.array([0.1, 1e-20, 3.5], dtype=np.float32)
     assert np.array_equal(orc.to_float64(f, "f32"), f.astype(np.float64))
+    # IEEE half, decoded here from the bit fields (1 sign, 5 exponent, 10 fraction bits)
+    hb = np.array([0x3C00, 0xC000, 0x3555, 0x0001, 0x03FF, 0x7BFF, 0x7C00, 0xFC00, 0x8000], dtype=np.uint16)
+    want = []
+    for x in hb.tolist():
+        sgn, ex, fr = -1.0 if x >> 15 else 1.0, (x >> 10) & 31, x & 1023
+        want.append(sgn * (math.inf if ex == 31 else (fr * 2.0 ** -24 if ex == 0 else (1 + fr / 1024) * 2.0 ** (ex - 15))))
+    got = orc.to_float64(hb.view(np.float16), "f16")
+    assert np.array_equal(got, np.array(want)) and np.signbit(got[8])
 
 
 # --------------------------------------------------------------------------------------
