@@ -1,4 +1,5 @@
-"""The alternate proposal framework (Sec. 3.3, Algorithm 1) around the verification step.
+"""The schedulers of the paper around the verification step: the alternate proposal framework for two
+models (Sec. 3.3, Algorithm 1) and its n-model form (App. B, Algorithm 2).
 
 Two models take turns.  In a cycle the proposer extends the cached token (if any) to its proposal
 length, the verifier scores the proposal, and one verification call decides: the accepted prefix is
@@ -20,9 +21,11 @@ from typing import Callable, List, Optional, Sequence, Tuple
 
 import numpy as np
 
-# verify(logits[2, 1, g+1, V] float32, drafts[1, g] int32, proposer, bonus_model, seed, offset)
+# verify(logits[n, 1, g+1, V] float32, drafts[1, g] int32, proposer, bonus_model, seed, offset)
 #   -> (accept_count, out_tokens[g+1], bonus_prob)
-VerifyFn = Callable[[np.ndarray, np.ndarray, int, int, int, int], Tuple[int, np.ndarray, float]]
+# proposer: one model index for the row, or an int32 table [1, g+1] naming the proposer of every draft;
+# bonus_model: -1 (bonus from the combined distribution) or the model whose own distribution it follows
+VerifyFn = Callable[[np.ndarray, np.ndarray, object, int, int, int], Tuple[int, np.ndarray, float]]
 
 
 class TableModel:
@@ -144,21 +147,137 @@ class AlternateProposal:
         return S[len(prefix):], st
 
 
+@dataclass
+class Event:
+    kind: str              # "propose", "score", "verify"
+    model: int             # the model that proposed / scored; -1 for verify
+    count: int             # tokens proposed, cached tokens scored, or tokens verified
+    accepted: int = -1     # verify only
+
+
+class CollaborativeSpeculation:
+    """Algorithm 2: n models, proposal lengths gamma_1..gamma_n, model 0 the default proposer.
+
+    S_c is the cached sequence, `owner[k]` the model that produced its k-th token, `scored[i]` how many
+    of its tokens model i has probabilities for (its own proposals count).  The model with the fewest
+    scores the whole cache, which also yields its bonus token (drawn from its own distribution, with its
+    probability); every cached token that all models have scored is then verified against the combined
+    distribution, its proposer's distribution being q -- one verification call for the whole verifiable
+    prefix, which stops at the first rejection exactly as the token-by-token loop of the listing does.
+    After a rejection everything cached is dropped and the default proposer starts over (the reading of
+    Sec. 3.3 and of the walk-through in App. B; the listing would let the scoring model propose first)."""
+
+    def __init__(self, models: Sequence[TableModel], gammas: Sequence[int], temperature: float, verify: VerifyFn,
+                 propose_seed: int = 1, verify_seed: int = 2, keep_events: bool = False):
+        if len(models) < 2 or len(models) != len(gammas) or min(gammas) < 1:
+            raise ValueError("n >= 2 models and one proposal length >= 1 for each")
+        self.models, self.gammas, self.T = list(models), list(gammas), float(temperature)
+        self.n, self.V = len(models), models[0].vocab
+        self.verify, self.verify_seed = verify, verify_seed
+        self._u = np.random.Generator(np.random.Philox(key=propose_seed))
+        self.keep_events = keep_events
+        self.events: List[Event] = []
+        self.calls = 0         # verification calls so far: the counter offset of the next one
+
+    def _log(self, *a):
+        if self.keep_events:
+            self.events.append(Event(*a))
+
+    def _sample(self, i: int, prefix: Sequence[int]) -> int:
+        m = self.models[i]
+        m.calls += 1
+        l = m.logits(prefix).astype(np.float64)
+        if self.T == 0.0:
+            return int(np.argmax(l))
+        z = l / self.T
+        p = np.exp(z - z.max())
+        cdf = np.cumsum(p)
+        return min(int(np.searchsorted(cdf, self._u.random() * cdf[-1], side="left")), self.V - 1)
+
+    def generate(self, prefix: Sequence[int], max_new_tokens: int) -> Tuple[List[int], Stats]:
+        n, V = self.n, self.V
+        S: List[int] = list(prefix)
+        Sc: List[int] = []
+        owner: List[int] = []
+        scored = [0] * n
+        st = Stats()
+        start = len(prefix)
+
+        def propose(i: int, count: int):
+            for _ in range(count):
+                Sc.append(self._sample(i, S + Sc))
+                owner.append(i)
+                st.proposed += 1
+            scored[i] = len(Sc)      # a model knows its own probabilities along everything it has seen
+            self._log("propose", i, count)
+
+        while len(S) - start < max_new_tokens:
+            if not Sc:
+                propose(0, self.gammas[0])
+                continue
+            i = int(np.argmin(scored))                    # fewest cached probabilities; lowest index on ties
+            # Score: model i reads the whole cache (one forward pass) and draws its bonus token from its own
+            # distribution after it; the probability comes back with the token
+            self.models[i].calls += 1
+            st.scored += 1
+            self._log("score", i, len(Sc))
+            row = self.models[i].logits(S + Sc)
+            lg = np.broadcast_to(row, (n, 1, 1, V)).astype(np.float32).copy()
+            _, out, prob = self.verify(lg, np.zeros((1, 0), np.int32), 0, i, self.verify_seed, self.calls)
+            self.calls += 1
+            Sc.append(int(out[0]))
+            owner.append(i)
+            scored[i] = len(Sc)
+            # Verify every cached token that all models have scored
+            L = min(scored)
+            rejected = False
+            if L > 0:
+                lg = np.empty((n, 1, L + 1, V), dtype=np.float32)
+                for j in range(L + 1):                    # position L only fills the call's bonus slot, unused here
+                    ctx = S + Sc[:j]
+                    for k in range(n):
+                        lg[k, 0, j] = self.models[k].logits(ctx)
+                table = np.asarray(owner[:L] + [0], dtype=np.int32).reshape(1, L + 1)
+                a, out, _ = self.verify(lg, np.asarray(Sc[:L], np.int32).reshape(1, L), table, -1, self.verify_seed,
+                                        self.calls)
+                self.calls += 1
+                self._log("verify", -1, L, int(a))
+                st.cycles += 1
+                if a == L:
+                    S += Sc[:L]
+                    del Sc[:L], owner[:L]
+                    scored = [c - L for c in scored]
+                    st.full_accepts += 1
+                else:
+                    S += Sc[:a] + [int(out[a])]           # the resampled token replaces the rejected one
+                    Sc.clear()
+                    owner.clear()
+                    scored = [0] * n
+                    rejected = True
+            if not rejected:
+                propose(i, self.gammas[i] - 1)            # the bonus token was the first of model i's proposal
+        st.tokens = len(S) - start
+        return S[start:], st
+
+
 def gpu_verify(combine: int, weights: Sequence[float], temperature: float, vocab: int, mask_model: int = -1,
                mask_alpha: float = 1.0, device: int = 0) -> VerifyFn:
-    """The verification call of the CUDA library for the scheduler: one context per proposal length,
+    """The verification call of the CUDA library for the schedulers: one context per proposal length,
     made on first use, host tensors in and out (cos_verify_run_host)."""
     import torch
     from .binding import CosVerifier
     ctxs = {}
+    n = len(list(weights))
 
     def verify(logits, drafts, proposer, bonus_model, seed, offset):
         g = logits.shape[2] - 1
         if g not in ctxs:
-            ctxs[g] = CosVerifier(2, combine, weights, temperature, g, vocab, 1, torch.float32, mask_model=mask_model,
+            ctxs[g] = CosVerifier(n, combine, weights, temperature, g, vocab, 1, torch.float32, mask_model=mask_model,
                                   mask_alpha=mask_alpha, device=device, host_staging=True)
-        outs = ctxs[g].run_host(torch.from_numpy(logits), torch.from_numpy(drafts),
-                                torch.tensor([proposer], dtype=torch.int32), seed, offset, bonus_model=bonus_model)
+        prop = torch.tensor([proposer], dtype=torch.int32) if np.isscalar(proposer) else \
+            torch.from_numpy(np.ascontiguousarray(proposer, dtype=np.int32))
+        outs = ctxs[g].run_host(torch.from_numpy(logits), torch.from_numpy(drafts) if g > 0 else None,
+                                prop, seed, offset, bonus_model=bonus_model)
         return int(outs["accept_count"][0]), outs["out_tokens"][0].numpy().copy(), float(outs["bonus_prob"][0])
 
     verify.close = lambda: [c.close() for c in ctxs.values()]

@@ -103,3 +103,62 @@ def test_greedy_run_is_the_argmax_chain_of_the_combined_model():
         # token order, an accepted one is either atom; both are atoms of r
         assert t in (a0, a1)
         S.append(t)
+
+
+# --------------------------------------------------------------------------------------
+# n models (Algorithm 2)
+# --------------------------------------------------------------------------------------
+def oracle_verify_n(n, combine, weights, T, V):
+    def verify(logits, drafts, proposer, bonus_model, seed, offset):
+        g = logits.shape[2] - 1
+        cfg = orc.OracleConfig(n=n, combine=combine, weights=list(weights), temperature=T, gamma=g, vocab=V,
+                               bonus_model=bonus_model)
+        prop = np.array([proposer]) if np.isscalar(proposer) else np.asarray(proposer)
+        out = orc.verify(logits, "f32", drafts, prop, cfg, seed, offset)
+        return int(out["accept_count"][0]), out["out_tokens"][0], float(out["bonus_prob"][0])
+    return verify
+
+
+def test_three_models_follow_the_walk_through_of_the_paper():
+    """App. B, proposal lengths (3, 2, 1): M1 proposes x1..x3; M2 scores them, draws x4 and proposes x5; M3
+    scores x1..x5 and draws x6; now x1..x3 have been scored by all three and are verified together.  If they
+    pass, M1 (which holds no probabilities for x4..x6) scores those three and proposes x7..x9, after which x4
+    and x5 are verifiable."""
+    V, T = 50, 1.0
+    models = sch.make_table_models(3, V, contexts=32, seed=4, sigma=0.3, rho=0.95)   # near-identical: drafts pass
+    run = sch.CollaborativeSpeculation(models, (3, 2, 1), T, oracle_verify_n(3, WE, (0.4, 0.3, 0.3), T, V), keep_events=True)
+    run.generate([7], 12)
+    ev = [(e.kind, e.model, e.count) for e in run.events]
+    assert ev[:5] == [("propose", 0, 3), ("score", 1, 3), ("propose", 1, 1), ("score", 2, 5), ("verify", -1, 3)]
+    first = run.events[4]
+    if first.accepted == 3:
+        assert ev[5:10] == [("propose", 2, 0), ("score", 0, 3), ("verify", -1, 2), ("propose", 0, 2), ("score", 1, 4)] or \
+            ev[5:8] == [("propose", 2, 0), ("score", 0, 3), ("verify", -1, 2)]
+    else:
+        assert ev[5] == ("propose", 0, 3)       # everything cached was dropped: the default proposer again
+
+
+@pytest.mark.parametrize("n,weights,gammas", [(3, (0.5, 0.3, 0.2), (3, 2, 1)), (2, (0.5, 0.5), (2, 2)),
+                                              (4, (0.25, 0.25, 0.25, 0.25), (1, 2, 1, 3))])
+def test_n_model_output_follows_the_combined_law(n, weights, gammas):
+    """Every emitted token passed the accept test against r = sum_i w_i p_i with the law of its own proposer
+    as q (or was resampled from the residual), whichever model produced it and whether it began as a bonus
+    token: with context-free models the output is an i.i.d. sample of r."""
+    V, T, N = 10, 1.1, 12000
+    models = sch.make_table_models(n, V, contexts=1, seed=17, sigma=1.0, rho=0.5)
+    run = sch.CollaborativeSpeculation(models, gammas, T, oracle_verify_n(n, WE, weights, T, V), propose_seed=5,
+                                       verify_seed=6, keep_events=True)
+    tokens, st = run.generate([0], N)
+    w = np.asarray(np.asarray(weights, dtype=np.float32), dtype=np.float64)
+    r = sum(w[i] * sp_softmax(models[i].table[0].astype(np.float64) / T) for i in range(n))
+    counts = np.bincount(np.asarray(tokens[:N]), minlength=V)
+    chi2 = float(np.sum((counts - N * r) ** 2 / (N * r)))
+    assert chi2_dist.sf(chi2, V - 1) > 1e-4, (chi2, counts, N * r)
+    # every model proposed and scored; forward passes are all accounted for
+    kinds = {(e.kind, e.model) for e in run.events}
+    assert all(("score", i) in kinds for i in range(1, n)) and ("propose", 0) in kinds
+    assert sum(m.calls for m in models) == st.proposed + st.scored
+    # a verification never covers more tokens than the cache held, and after a rejection the default proposer restarts
+    for prev, cur in zip(run.events, run.events[1:]):
+        if prev.kind == "verify" and prev.accepted < prev.count:
+            assert (cur.kind, cur.model, cur.count) == ("propose", 0, gammas[0])
