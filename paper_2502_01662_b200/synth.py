@@ -91,7 +91,7 @@ CONFIGS: Dict[str, Workload] = {
     # 5: logit interpolation 1.5 * aligned - 0.5 * base, sampling and greedy
     "cfg5": Workload("cfg5", 2, COMBINE_LOGIT_LINEAR, (1.5, -0.5), 1.0, 256, 8, 256000, "bf16", "gumbel_zipf",
                      rho=0.9, proposer_rule="zero"),
-    # workload 3 with the logits stored as IEEE half (a variant; not one of the five baseline workloads)
+    # workload 3 with the logits stored as IEEE half (a variant beside the five workloads the benchmark reports)
     "cfg3_f16": Workload("cfg3_f16", 2, COMBINE_PROB_ENSEMBLE, (0.5, 0.5), 0.7, 64, 8, 151936, "f16", "gumbel_zipf",
                          rho=0.85, proposer_rule="bernoulli"),
     "cfg5_greedy": Workload("cfg5_greedy", 2, COMBINE_LOGIT_LINEAR, (1.5, -0.5), 0.0, 256, 8, 256000, "bf16",
