@@ -69,10 +69,16 @@ enum {
                                      /* position (Algorithm 2 verifies a cached sequence that holds      */
                                      /* tokens of several proposers).  Entry (b, gamma) must be a valid  */
                                      /* index; its distribution decides nothing.                         */
-  COS_RUN_BONUS_FROM_MODEL = 4       /* the token after gamma acceptances is drawn from model            */
+  COS_RUN_BONUS_FROM_MODEL = 4,      /* the token after gamma acceptances is drawn from model            */
                                      /* `bonus_model`'s own distribution instead of the combined one     */
                                      /* (Sec. 3.3: the verifier's bonus token, to be treated as that     */
                                      /* model's next proposal)                                           */
+  COS_RUN_EARLY_EXIT = 8             /* a hint: positions behind a rejection that their row has already  */
+                                     /* reported may be left unread (Sec. 3.1 discards them anyway).     */
+                                     /* accept_count, out_tokens, row_status and bonus_prob are those of */
+                                     /* the full run; diag is NaN at a position that was left unread,    */
+                                     /* and which positions those are depends on timing.  Taken by       */
+                                     /* cos_verify_run when no cluster size and no mask is configured.   */
 };
 
 typedef struct {

@@ -71,6 +71,7 @@ struct KParams {
   int flags;
   int num_units, num_clusters;
   int per_pos;      // proposer is [B][gamma+1] (the model that proposed each draft) instead of [B]
+  int early_exit;   // positions after a row's known first rejection may be left unread (barrier-free form only)
   int greedy;       // T = 0: no drawing stages; the fourth word of a unit's result carries the bonus probability
   int bonus_model;  // >= 0: the token after gamma acceptances follows this model's own distribution; -1: the combined one
   int parts;     // blocks that share one unit in stages 1 and 2
@@ -92,6 +93,7 @@ struct KParams {
   unsigned* work_counter;  // units are handed out from here; grows by num_units every run
   unsigned work_base;      // its value when this run starts
   int* row_arrivals;       // [B], zero between runs
+  int* row_reject;         // [B]: earliest rejected position published so far; kNoReject between runs
   int4* unit_res;          // [B*P]: x = accept flag, y = status bits, z = candidate token, w = a token can be drawn
   int* job_count;          // units that stage 1 must process (this run's counter)
   int* job_reset;          // the other run parity's counter, cleared by stage 0
@@ -293,6 +295,7 @@ struct FreeRun {
   int arrive[2];    // warps that have finished the unit of that parity
   int epi_done;     // units whose merge and decision are complete
   int fault;        // a wait gave up
+  int skip_state[2];  // unit of that parity: 0 undecided, 1 swept, 2 left unread (its row is already rejected earlier)
 };
 
 struct Shared {
@@ -527,6 +530,7 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
   }
   int4 res = make_int4(accept, status, cand, word4);
   __stcg(&p.unit_res[idx], res);
+  if (p.early_exit && !accept && j < p.gamma) atomicMin(&p.row_reject[b], j);  // later positions may be left unread
   // test hooks: the combined distribution everywhere, or the residual mass at every draft position
   if (drawable && (p.dump_r != nullptr || ((p.flags & COS_RUN_ALL_RESIDUALS) && j < p.gamma))) push_job(p, idx, 0);
   __threadfence();
@@ -558,6 +562,7 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
   for (int k = 0; k < p.P; ++k) o[k] = (k < a) ? p.drafts[b * p.gamma + k] : (k == a ? tok : -1);
   p.row_status[b] = st;
   p.row_arrivals[b] = 0;  // leave the scratch ready for the next run
+  if (p.early_exit) p.row_reject[b] = kNoReject;
   // under the test hooks the unit may already be on the list: every unit is listed once at most
   const bool listed = (p.dump_r != nullptr) || ((p.flags & COS_RUN_ALL_RESIDUALS) && a < p.gamma);
   if (draw && !listed) push_job(p, b * p.P + a, 1);
@@ -1144,6 +1149,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
     fr.unit_of[0] = blockIdx.x;
     fr.unit_tag[0] = 1;
     fr.arrive[0] = fr.arrive[1] = 0;
+    fr.skip_state[0] = fr.skip_state[1] = 0;
     fr.epi_done = 0;
     fr.fault = 0;
   }
@@ -1173,7 +1179,22 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       raise_fault(p, fr, lane);
       return;
     }
-    sweep_unit<DT, MODE>(p, base, sl, pis, false, -INFINITY, &fr.wsoft[par][warp][0], &fr.warg[par][warp][0]);
+    // Early exit: a position behind a rejection that its row has already published decides nothing
+    // (Sec. 3.1: the tokens after the first rejection are discarded).  The first warp to get here settles
+    // it for the block, so that all sixteen do the same.  (Letting every warp look for itself during its
+    // sweep was tried: the polls slowed the ordinary path by 4-6 % and gained nothing over this.)
+    bool skipped = false;
+    if (p.early_exit) {
+      int st = 0;
+      if (lane == 0) {
+        const int mine = (*reinterpret_cast<volatile int*>(&p.row_reject[b]) < j) ? 2 : 1;
+        st = atomicCAS(&fr.skip_state[par], 0, mine);
+        if (st == 0) st = mine;
+      }
+      skipped = (__shfl_sync(0xffffffffu, st, 0) == 2);
+    }
+    if (!skipped)
+      sweep_unit<DT, MODE>(p, base, sl, pis, false, -INFINITY, &fr.wsoft[par][warp][0], &fr.warg[par][warp][0]);
     int prev = 0;
     if (lane == 0) {
       __threadfence_block();
@@ -1197,7 +1218,18 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
         unit_tag[(seq + 2) & 3] = seq + 3;
       }
     }
-    if (prev == kWarps - 1) {
+    if (prev == kWarps - 1 && skipped) {
+      // nothing was read: the unit reports "not accepted, no candidate", which the row's scan never reaches
+      if (lane == 0) {
+        const double nan = __longlong_as_double(0x7ff8000000000000LL);
+        publish_unit(p, b, j, 0, 0, -1, kSample ? 0 : __float_as_int(__int_as_float(0x7fc00000)), nan, nan, nan, nan);
+        fr.arrive[par] = 0;
+        fr.skip_state[par] = 0;
+        __threadfence_block();
+        *epi_done = seq + 1;
+      }
+      __syncwarp();
+    } else if (prev == kWarps - 1) {
       // last to finish: merge, decide, publish
       const int uidx = b * p.P + j;
       const bool is_bonus = (j == p.gamma);
@@ -1253,6 +1285,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
         publish_unit(p, b, j, d.accept, d.status, d.cand, kSample ? d.drawable : __float_as_int(static_cast<float>(d.prob)),
                      d.ratio, d.r_d, d.q_d, d.S);
         fr.arrive[par] = 0;
+        fr.skip_state[par] = 0;
         __threadfence_block();
         *epi_done = seq + 1;
       }
@@ -2102,6 +2135,7 @@ struct cos_verify_ctx {
   bool scratch_dirty;
   // device scratch
   int* d_row_arrivals;
+  int* d_row_reject;
   int4* d_unit_res;
   int* d_job_count;  // two counters, used alternately by successive runs
   int2* d_jobs;
@@ -2309,6 +2343,7 @@ cos_status init_scratch(cos_verify_ctx* ctx, cudaStream_t stream) {
   const size_t rows = static_cast<size_t>(ctx->cfg.max_batch);
   cudaError_t e = cudaMemsetAsync(ctx->d_work_counter, 0, sizeof(unsigned), stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_row_arrivals, 0, rows * sizeof(int), stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_row_reject, 0x7f, rows * sizeof(int), stream);  // "none yet"
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_job_count, 0, 2 * sizeof(int), stream);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->d_part_arrivals, 0, rows * (static_cast<size_t>(ctx->cfg.gamma) + 1) * sizeof(int), stream);
@@ -2384,6 +2419,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   bool ok = true;
   ok = ok && cudaMalloc(&ctx->d_work_counter, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_row_arrivals, rows * sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_row_reject, rows * sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_unit_res, rows * P * sizeof(int4)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_job_count, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_jobs, (rows * P + rows) * sizeof(int2)) == cudaSuccess;
@@ -2438,7 +2474,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   if (!a->logits || !a->proposer || !a->accept_count || !a->out_tokens || !a->row_status) return bad("null device pointer");
   if (c.gamma > 0 && !a->draft_tokens) return bad("draft_tokens is null although gamma > 0");
   if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return bad("negative stride");
-  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL)) return bad("unknown flag bits");
+  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL | COS_RUN_EARLY_EXIT)) return bad("unknown flag bits");
   if ((a->flags & COS_RUN_BONUS_FROM_MODEL) && (a->bonus_model < 0 || a->bonus_model >= c.n))
     return bad("bonus_model outside [0, n)");
   if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4) {
@@ -2511,6 +2547,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.work_counter = ctx->d_work_counter;
   p.work_base = ctx->work_base;
   p.row_arrivals = ctx->d_row_arrivals;
+  p.row_reject = ctx->d_row_reject;
+  p.early_exit = (a->flags & COS_RUN_EARLY_EXIT) ? 1 : 0;
   p.unit_res = ctx->d_unit_res;
   p.job_count = ctx->d_job_count + (ctx->run_parity & 1u);
   p.job_reset = ctx->d_job_count + ((ctx->run_parity & 1u) ^ 1u);
@@ -2673,6 +2711,7 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   (void)cudaDeviceSynchronize();
   cudaFree(ctx->d_work_counter);
   cudaFree(ctx->d_row_arrivals);
+  cudaFree(ctx->d_row_reject);
   cudaFree(ctx->d_job_count);
   cudaFree(ctx->d_jobs);
   cudaFree(ctx->d_ustats);
@@ -2741,7 +2780,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     return static_fail(COS_ERR_INVALID_ARG, "null device pointer");
   if (c.gamma > 0 && !a->draft_tokens) return static_fail(COS_ERR_INVALID_ARG, "draft_tokens is null although gamma > 0");
   if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return static_fail(COS_ERR_INVALID_ARG, "negative stride");
-  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL)) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
+  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL | COS_RUN_EARLY_EXIT)) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
   if ((a->flags & COS_RUN_BONUS_FROM_MODEL) && (a->bonus_model < 0 || a->bonus_model >= c.n))
     return static_fail(COS_ERR_INVALID_ARG, "bonus_model outside [0, n)");
   if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4)
@@ -2844,6 +2883,8 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.work_counter = d_counter;
   p.work_base = 0;  // the counter was just cleared
   p.row_arrivals = d_arrivals;
+  p.row_reject = nullptr;  // the hint to leave positions unread is not taken here
+  p.early_exit = 0;
   p.unit_res = d_unit_res;
   p.job_count = d_job_count;
   p.job_reset = d_job_count + 1;
