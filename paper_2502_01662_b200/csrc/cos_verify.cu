@@ -1,24 +1,23 @@
-// CoS verification step for sm_100a: fused combine + accept test + residual / bonus sample
-// + first-rejection scan, one persistent kernel of thread-block clusters.
+// CoS verification step for sm_100a: combine (Eq. 3-5), accept test (Eq. 6), residual / bonus sample and
+// first-rejection scan (Sec. 3.1) for every row of a batch and every one of its gamma + 1 positions.
 //
-// Work unit = one (row b, position j).  A cluster of C thread blocks owns a unit; every
-// warp of the cluster owns a contiguous run of the vocabulary, so prefix order equals
-// token order.  Per unit:
-//   sweep 1  stream the n logit rows once from HBM (128-bit loads), keep per-lane online
-//            softmax statistics (reference exponent, sum of 2^(l*c - ref)) or argmaxes,
-//            merge lane -> warp -> block -> cluster (the last two in fp64, across blocks
-//            through distributed shared memory);
-//   decide   the accept test of Eq. 6 in fp64 from the merged statistics and the logits at
-//            the draft token;
-//   sweep 2  only where a token must be drawn (first rejected position of a row, or the
-//            bonus position when nothing earlier was rejected): re-read the unit (it is
-//            still in L2), form r and q per token, residual max(0, r - q), warp-ordered
-//            fp64 prefix sums, locate u * S, rescan one warp's run for the token;
-//   publish  per-unit result, and the last unit of a row to arrive runs the
-//            first-rejection scan and writes the row's outputs.
-// Units are handed out from a global counter (a cluster draws its next unit while it sweeps
-// the current one), because units that must draw a token take several times longer.
-// Nothing in the kernel spins on memory: blocks meet only at hardware cluster barriers.
+// Work unit = one (row b, position j).  One kernel template, instantiated per stage:
+//   stage 0  every unit: stream the n logit rows once from HBM (128-bit streaming loads), keep per-lane
+//            softmax statistics (reference exponent, sum of 2^(l*c - ref)) or argmaxes, merge them, take
+//            the accept test in fp64 from the merged statistics and the logits at the draft token, publish
+//            the unit; the last unit of a row to arrive scans for the first rejection, writes the row's
+//            outputs and lists the one unit of the row that must draw a token.  Two forms of the unit loop:
+//            a barrier-free one (a block owns a unit, its warps run from unit to unit and meet through
+//            volatile words in shared memory) and a cluster form (the blocks of a thread-block cluster
+//            split the vocabulary and exchange partial results through distributed shared memory);
+//   stage 1  listed units only: the normalisers again, terms above 2^-8 of a normaliser in fp64;
+//   stage 2  listed units only: token masses max(0, r - q) (or the law of the bonus token), every warp on
+//            a contiguous run of the vocabulary so that prefix order is token order, fp64 running totals;
+//            the last block of a unit to finish locates u * S and walks to the token.
+// Units are handed out from a global counter.  Between blocks there are only fences and arrival counters;
+// the three launches of a run order the stages.  Waits exist only inside a block of the barrier-free form,
+// and they are bounded: a wait that gave up marks every row with COS_ROW_FAULT and the block leaves.
+// At T = 0 stage 0 is the whole run.
 
 #include <cooperative_groups.h>
 #include <cuda_fp16.h>
