@@ -305,7 +305,7 @@ struct Shared {
   double wtot[kWarps];        // this block's per-warp totals of sweep 2
   double wincl[kWarps];       // their running sum
   double srun[kWarps][kRec];  // a warp's running total after each group of steps
-  double gw[kMaxParts * kWarps];  // stage 3: mass of every warp run of the unit
+  double gw[kMaxParts * kWarps];  // locating the token: mass of every warp run of the unit
   int win_g;
   SoftPart fsoft[kMaxSlots];  // merged over the cluster
   ArgPart farg[kMaxSlots];
@@ -513,7 +513,7 @@ __device__ __forceinline__ void push_job(const KParams& p, int idx, int emit) {
 
 // Stage 0: record a unit's decision; the last unit of a row to arrive scans for the first
 // rejection, writes the row's outputs and, where a token has to be drawn, lists that unit
-// for stage 1 (which fills in out_tokens[b][a]).
+// for the drawing stages (stage 2 fills in out_tokens[b][a]).
 // `word4`: sampling modes: whether a token can be drawn at this unit; greedy modes: the bits of the bonus
 // token's probability (a float), NaN away from the bonus position.
 __device__ void publish_unit(const KParams& p, int b, int j, int accept, int status, int cand, int word4,
@@ -1094,7 +1094,7 @@ __device__ __forceinline__ void decide_unit(const KParams& p, Shared& sh, bool i
       }
     }
   }
-  d.need2 = 0;  // tokens are drawn by stage 1, for the one position per row that needs it
+  d.need2 = 0;  // tokens are drawn by the later stages, for the one position per row that needs it
   d.drawable = (kSample && finite) ? 1 : 0;
 }
 
@@ -1303,7 +1303,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
   cg::cluster_group cluster = cg::this_cluster();
   // stage 0 shares a unit among the blocks of a cluster; stages 1 and 2 among `parts` independent
-  // blocks (they meet only through global memory between launches); stage 3 uses one block per unit
+  // blocks (they meet only through global memory: partial sums between the launches, an arrival counter within stage 2)
   const int lparts = (STAGE == 1 || STAGE == 2) ? p.parts : 1;  // blocks per unit in this launch
   const int C = (STAGE == 0) ? static_cast<int>(cluster.num_blocks()) : p.parts;
   const int rank = (STAGE == 0) ? static_cast<int>(cluster.block_rank()) : static_cast<int>(blockIdx.x % lparts);
@@ -1443,7 +1443,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     // every block takes the same decision from the same merged numbers
     if (tid == 0) decide_unit<DT, MODE>(p, sh, is_bonus, draft, draft_ok, pi, pi_ok, pis, masked);
     __syncthreads();
-    // rank 0 keeps the merged statistics for stage 1 and reports the unit
+    // rank 0 keeps the merged statistics for the drawing stages and reports the unit
     if (rank == 0) {
       const int nkeep = (MODE == kEnsembleSample) ? p.n : (MODE == kLogitSample ? 2 : 0);
       if (tid < nkeep) {
@@ -1507,7 +1507,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       const int nsoft2 = (MODE == kEnsembleSample) ? p.n : 2;
 
       // ---- 2a: normalisers again, now that the references are known: terms holding more
-      // than 2^-14 of a normaliser are evaluated in fp64 and kept out of the fp32 sums, so
+      // than 2^-8 of a normaliser are evaluated in fp64 and kept out of the fp32 sums, so
       // a dominant token neither absorbs the small ones nor carries the fast exp's error
       if (STAGE == 1) {
       if (MODE == kEnsembleSample) {
@@ -1698,7 +1698,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       const float ref_c = (MODE == kLogitSample) ? -sh.fsoft[1].ref : 0.f;
 
       // ---- 2b: token masses.  mass32[k] is max(0, r - q) (or r) of the lane's k-th token in fp32;
-      // tokens holding more than 2^-10 of any normaliser are flagged in `bigbits`, get mass32 = 0
+      // tokens holding more than 2^-8 of any normaliser are flagged in `bigbits`, get mass32 = 0
       // and are evaluated by big_mass() in fp64 from the stored logits.
       // `staged` points at this lane's staged vector of model 0 (models 32 vectors apart), or is null.
       auto chunk_mass = [&](int e0, bool use_r, float (&mass32)[E], unsigned& bigbits, const uint4* staged) {
