@@ -326,7 +326,27 @@ def main():
             t2, _ = time_device(ww, v2, s2, k2, 5, 0)
             # a variant, not the metric: with the early-exit hint positions behind a reported rejection go unread
             t3, _ = time_device(ww, v2, s2, k2, 5, 0, flags=COS_RUN_EARLY_EXIT)
+            # the same calls captured once in a CUDA graph and replayed (one call per input copy, 64 at most)
+            outs2 = v2._alloc_outs(ww.batch, ww.gamma + 1, ww.vocab, dev, False, False)
+            ncap = min(len(s2), 64)
+            graph = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize(dev)
+            with torch.cuda.graph(graph):
+                for q in range(ncap):
+                    v2.run(s2[q]["logits"], s2[q]["drafts"], s2[q]["proposer"], s2[q]["seed"], s2[q]["offset"], outs=outs2)
+            reps = max(3, k2 // ncap)
+            for _ in range(2):
+                graph.replay()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            for _ in range(reps):
+                graph.replay()
+            ev1.record()
+            torch.cuda.synchronize(dev)
+            t4 = ev0.elapsed_time(ev1) / 1e3
+            del graph
             extra[name] = {"us_per_call": 1e6 * t2 / k2, "positions_per_s": ww.positions * k2 / t2,
+                           "us_per_call_graph": 1e6 * t4 / (reps * ncap),
                            "GBps": ww.positions * ww.bytes_per_position * k2 / t2 / 1e9,
                            "cluster": v2.info()["cluster_size"], "buffers": len(s2),
                            "us_per_call_early_exit": 1e6 * t3 / k2}

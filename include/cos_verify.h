@@ -125,6 +125,9 @@ typedef struct {
                                /* bonus token under the distribution it was drawn from (what Score of   */
                                /* Algorithm 2 returns beside the token); NaN elsewhere; may be NULL     */
   int32_t bonus_model;         /* read only with COS_RUN_BONUS_FROM_MODEL: index in [0, n)              */
+  const uint64_t* offset_device; /* optional: device address of the counter offset, read by the kernels */
+                               /* in place of `offset` (8-byte aligned); lets a captured run be         */
+                               /* replayed with fresh uniforms; may be NULL                             */
 } cos_verify_args;
 
 typedef struct {
@@ -151,6 +154,9 @@ cos_status cos_verify_create(const cos_verify_config* config, cos_verify_ctx** o
  * Host-detected problems return an error code and enqueue nothing; data-dependent
  * problems are reported per row in row_status and never trap the device.
  * Runs that share a context must be ordered on one stream.
+ * The launches of a run depend on its arguments only (the kernels leave the context's scratch as they
+ * found it), so a run may be captured into a CUDA graph and replayed; keep the counter offset in device
+ * memory (offset_device) to give every replay its own uniforms.
  */
 cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* args, void* cuda_stream);
 

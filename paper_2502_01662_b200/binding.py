@@ -59,6 +59,7 @@ class cos_verify_args(ctypes.Structure):
         ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64), ("accept_count", ctypes.c_void_p),
         ("out_tokens", ctypes.c_void_p), ("row_status", ctypes.c_void_p), ("diag", ctypes.c_void_p),
         ("dump_r", ctypes.c_void_p), ("bonus_prob", ctypes.c_void_p), ("bonus_model", ctypes.c_int32),
+        ("offset_device", ctypes.c_void_p),
     ]
 
 
@@ -149,7 +150,7 @@ class CosVerifier:
                                              "launches_per_run")}
 
     def _fill_args(self, logits, drafts, proposer, seed, offset, row_base, flags, outs,
-                   bonus_model=None) -> cos_verify_args:
+                   bonus_model=None, offset_device=None) -> cos_verify_args:
         n, B, P, V = logits.shape
         # a [B, gamma+1] proposer table selects the per-position form; a bonus model selects its flag
         if proposer.dim() == 2:
@@ -180,6 +181,7 @@ class CosVerifier:
         a.dump_r = outs["r"].data_ptr() if "r" in outs else None
         a.bonus_prob = outs["bonus_prob"].data_ptr() if "bonus_prob" in outs else None
         a.bonus_model = bonus_model if (bonus_model is not None and bonus_model >= 0) else 0
+        a.offset_device = offset_device.data_ptr() if offset_device is not None else None
         return a
 
     def set_stage_timing(self, enable: bool):
@@ -214,12 +216,14 @@ class CosVerifier:
     # -- the calls -------------------------------------------------------------------
     def run(self, logits, drafts, proposer, seed: int, offset: int, row_base: int = 0, flags: int = 0,
             diag: bool = False, dump_r: bool = False, outs: Optional[dict] = None, stream=None,
-            bonus_model: Optional[int] = None) -> dict:
+            bonus_model: Optional[int] = None, offset_device=None) -> dict:
         """cos_verify_run on device tensors; asynchronous on `stream` (default: torch's current stream).
 
         `proposer` is [B], or [B, gamma+1] to name the proposer of every draft (Algorithm 2); `bonus_model`
         draws the token after gamma acceptances from that model's own distribution (Sec. 3.3).  The outputs
-        include "bonus_prob" [B]: the bonus token's probability under the law it was drawn from."""
+        include "bonus_prob" [B]: the bonus token's probability under the law it was drawn from.
+        `offset_device` (a one-element int64 device tensor) replaces `offset`: the kernels read it, so a
+        run captured in a CUDA graph can be replayed with a new offset each time."""
         import torch
         if not logits.is_cuda:
             raise ValueError("run() needs device tensors; use run_host() for host tensors")
@@ -229,7 +233,9 @@ class CosVerifier:
         n, B, P, V = logits.shape
         if outs is None:
             outs = self._alloc_outs(B, P, V, logits.device, diag, dump_r)
-        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs, bonus_model)
+        if offset_device is not None and (offset_device.dtype != torch.int64 or not offset_device.is_cuda):
+            raise ValueError("offset_device must be an int64 device tensor")
+        a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs, bonus_model, offset_device)
         s = torch.cuda.current_stream(logits.device) if stream is None else stream
         self._check(self._lib.cos_verify_run(self._ctx, ctypes.byref(a), ctypes.c_void_p(s.cuda_stream)))
         return outs

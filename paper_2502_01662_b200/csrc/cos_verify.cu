@@ -81,6 +81,7 @@ struct KParams {
   double cT64;    // the same value widened: the decision uses the constant the sweeps used
   double ln_alpha;
   unsigned seed_lo, seed_hi, off_lo, off_hi;
+  const unsigned long long* off_dev;  // when set, the counter offset is read from device memory instead
   long long row_base;
   int* accept_count;
   int* out_tokens;
@@ -90,12 +91,11 @@ struct KParams {
   float* bonus_prob;
   // scratch owned by the context
   unsigned* work_counter;  // units are handed out from here; grows by num_units every run
-  unsigned work_base;      // its value when this run starts
+  unsigned* exit_count;    // [2]: blocks of stage 0 / stage 2 that have left; the last one clears the counters
   int* row_arrivals;       // [B], zero between runs
   int* row_reject;         // [B]: earliest rejected position published so far; kNoReject between runs
   int4* unit_res;          // [B*P]: x = accept flag, y = status bits, z = candidate token, w = a token can be drawn
-  int* job_count;          // units that stage 1 must process (this run's counter)
-  int* job_reset;          // the other run parity's counter, cleared by stage 0
+  int* job_count;          // units the drawing stages must process; cleared by the last block of stage 2
   int2* jobs;              // x = b * P + j of a unit that draws a token (y unused)
   UnitStats* ustats;       // [B*P]: merged statistics of sweep 1, read back by the later stages
   double* zpart;           // [B*P][parts][8]: stage 1's partial normalisers
@@ -294,6 +294,7 @@ struct FreeRun {
   int arrive[2];    // warps that have finished the unit of that parity
   int epi_done;     // units whose merge and decision are complete
   int fault;        // a wait gave up
+  int left;         // warps that have left the loop
   int skip_state[2];  // unit of that parity: 0 undecided, 1 swept, 2 left unread (its row is already rejected earlier)
 };
 
@@ -501,6 +502,32 @@ __device__ __forceinline__ void cluster_merge(Shared& sh, cg::cluster_group& clu
 __device__ __forceinline__ int proposer_of(const KParams& p, int b, int j) {
   if (j == p.gamma && p.bonus_model >= 0) return p.bonus_model;
   return p.proposer[p.per_pos ? b * p.P + j : b];
+}
+
+// Counter words 2 and 3 of the Philox call: from the arguments, or from device memory when the caller keeps
+// the offset there (so that a captured graph can be replayed with fresh uniforms).
+__device__ __forceinline__ unsigned offset_lo(const KParams& p) {
+  return p.off_dev ? static_cast<unsigned>(__ldcg(p.off_dev)) : p.off_lo;
+}
+__device__ __forceinline__ unsigned offset_hi(const KParams& p) {
+  return p.off_dev ? static_cast<unsigned>(__ldcg(p.off_dev) >> 32) : p.off_hi;
+}
+
+// A block leaves stage 0 of a greedy run (which = 0) or stage 2 (which = 1).  The last block of the launch to
+// leave puts the counter of that stage back to zero, so that every run starts from the same state with the same
+// arguments (a run can then be captured in a graph and replayed).  One thread per block calls it, after the
+// block's last use of the counter has returned its value; the end of the launch publishes the reset.
+// (When stages follow, the work counter is cleared by stage 1 instead, which costs nothing.)
+__device__ __forceinline__ void stage_exit(const KParams& p, int which) {
+  const unsigned prev = atomicAdd(&p.exit_count[which], 1u);
+  if (prev == gridDim.x - 1) {
+    p.exit_count[which] = 0u;
+    if (which == 0)
+      *p.work_counter = 0u;
+    else
+      *p.job_count = 0;
+    __threadfence();
+  }
 }
 
 // ------------------------------------------------------------------------------------
@@ -1148,13 +1175,14 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
     fr.unit_of[0] = blockIdx.x;
     fr.unit_tag[0] = 1;
     fr.arrive[0] = fr.arrive[1] = 0;
+    fr.left = 0;
     fr.skip_state[0] = fr.skip_state[1] = 0;
     fr.epi_done = 0;
     fr.fault = 0;
   }
   __syncthreads();
   if (tid == kThreads - 32) {  // the block's first unit is valid: one draw settles its second
-    const int nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
+    const int nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u));
     unit_of[1] = nx;
     __threadfence_block();
     unit_tag[1] = 2;
@@ -1211,7 +1239,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       if (lane == 0) {
         int nx = p.num_units;
         if (unit_of[(seq + 1) & 3] < p.num_units)
-          nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
+          nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u));
         unit_of[(seq + 2) & 3] = nx;
         __threadfence_block();
         unit_tag[(seq + 2) & 3] = seq + 3;
@@ -1239,7 +1267,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       if (lane == 31) {
         unsigned rnd[4];
         const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
-        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi,
+        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), offset_lo(p), offset_hi(p), p.seed_lo, p.seed_hi,
                       rnd);
         sh.u_acc = word_to_uniform(rnd[0]);
         sh.u_smp = word_to_uniform(rnd[1]);
@@ -1291,6 +1319,8 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       __syncwarp();
     }
   }
+  // the last warp of the block to run out of units reports the block's departure
+  if (p.greedy && lane == 0 && atomicAdd(&fr.left, 1) == kWarps - 1) stage_exit(p, 0);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1327,10 +1357,10 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   // later stages are launched while the previous one drains (programmatic dependent launch);
   // nothing it wrote is read before this point
   if (STAGE >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (STAGE == 1 && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
   const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
   if (STAGE == 0) {
-    if (blockIdx.x == 0 && tid == 0) *p.job_reset = 0;  // the list of the next run starts empty
     // One block per unit and no step that needs the whole block twice (the plausibility mask does, and so
     // does the greedy form of the combined-distribution test hook): the warps run without block barriers.
     if (C == 1 && !masked && (kSample || p.dump_r == nullptr)) {
@@ -1374,11 +1404,11 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     if (warp == kWarps - 1) {
       if (lane == 2) {
         // rank 0 draws the cluster's next unit now; every block learns it with the merged statistics
-        if (rank == 0) sh.next_local = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u) - p.work_base);
+        if (rank == 0) sh.next_local = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u));
       } else if (lane == 1) {
         unsigned rnd[4];
         const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
-        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi,
+        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), offset_lo(p), offset_hi(p), p.seed_lo, p.seed_hi,
                       rnd);
         sh.u_acc = word_to_uniform(rnd[0]);
         sh.u_smp = word_to_uniform(rnd[1]);
@@ -1479,7 +1509,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         sh.thr32 = p.ustats[uidx].thr32;
         unsigned rnd[4];
         const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
-        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), p.off_lo, p.off_hi, p.seed_lo, p.seed_hi,
+        philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), offset_lo(p), offset_hi(p), p.seed_lo, p.seed_hi,
                       rnd);
         sh.u_smp = word_to_uniform(rnd[1]);
         sh.next = 0;
@@ -2113,6 +2143,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     unit = next_unit;
   }
   cluster.sync();  // no block leaves while a peer may still read its shared memory
+  if (((STAGE == 0 && p.greedy) || STAGE == 2) && tid == 0) stage_exit(p, STAGE == 0 ? 0 : 1);
 }
 
 // ------------------------------------------------------------------------------------
@@ -2128,15 +2159,13 @@ struct cos_verify_ctx {
   int max_clusters[5];  // resident clusters for cluster sizes 1, 2, 4, 8, 16 (0 = not available)
   int dense_blocks;     // resident blocks of the four-per-multiprocessor build of stage 0 (0 = there is none)
   int sm_count;
-  unsigned work_base;
-  unsigned run_parity;
   unsigned* d_work_counter;
   bool scratch_dirty;
   // device scratch
   int* d_row_arrivals;
   int* d_row_reject;
   int4* d_unit_res;
-  int* d_job_count;  // two counters, used alternately by successive runs
+  int* d_job_count;
   int2* d_jobs;
   UnitStats* d_ustats;
   double* d_zpart;
@@ -2340,15 +2369,13 @@ cos_status cuda_fail(cos_verify_ctx* ctx, const char* what, cudaError_t e) {
 
 cos_status init_scratch(cos_verify_ctx* ctx, cudaStream_t stream) {
   const size_t rows = static_cast<size_t>(ctx->cfg.max_batch);
-  cudaError_t e = cudaMemsetAsync(ctx->d_work_counter, 0, sizeof(unsigned), stream);
+  cudaError_t e = cudaMemsetAsync(ctx->d_work_counter, 0, 4 * sizeof(unsigned), stream);  // counter and the two exit counts
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_row_arrivals, 0, rows * sizeof(int), stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_row_reject, 0x7f, rows * sizeof(int), stream);  // "none yet"
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_job_count, 0, 2 * sizeof(int), stream);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->d_part_arrivals, 0, rows * (static_cast<size_t>(ctx->cfg.gamma) + 1) * sizeof(int), stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "scratch reset", e);
-  ctx->work_base = 0;
-  ctx->run_parity = 0;
   ctx->scratch_dirty = false;
   return COS_OK;
 }
@@ -2480,6 +2507,10 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     ctx->err = "bonus_prob is not 4-byte aligned";
     return COS_ERR_ALIGNMENT;
   }
+  if (a->offset_device && reinterpret_cast<uintptr_t>(a->offset_device) % 8) {
+    ctx->err = "offset_device is not 8-byte aligned";
+    return COS_ERR_ALIGNMENT;
+  }
   const int eb = elem_bytes(c.dtype);
   if (reinterpret_cast<uintptr_t>(a->logits) % eb) {
     ctx->err = "logits pointer not aligned to its element type";
@@ -2533,6 +2564,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.seed_hi = static_cast<unsigned>(a->seed >> 32);
   p.off_lo = static_cast<unsigned>(a->offset);
   p.off_hi = static_cast<unsigned>(a->offset >> 32);
+  p.off_dev = reinterpret_cast<const unsigned long long*>(a->offset_device);
   p.row_base = a->row_base;
   p.accept_count = a->accept_count;
   p.out_tokens = a->out_tokens;
@@ -2544,13 +2576,12 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
   p.greedy = (c.temperature == 0.0f) ? 1 : 0;
   p.work_counter = ctx->d_work_counter;
-  p.work_base = ctx->work_base;
+  p.exit_count = ctx->d_work_counter + 1;
   p.row_arrivals = ctx->d_row_arrivals;
   p.row_reject = ctx->d_row_reject;
   p.early_exit = (a->flags & COS_RUN_EARLY_EXIT) ? 1 : 0;
   p.unit_res = ctx->d_unit_res;
-  p.job_count = ctx->d_job_count + (ctx->run_parity & 1u);
-  p.job_reset = ctx->d_job_count + ((ctx->run_parity & 1u) ^ 1u);
+  p.job_count = ctx->d_job_count;
   p.jobs = ctx->d_jobs;
   p.ustats = ctx->d_ustats;
   p.zpart = ctx->d_zpart;
@@ -2593,10 +2624,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
       ctx->ev_used = st + 2;
     }
   }
-  // every cluster starts on the unit of its own index and draws once after each unit it finishes,
-  // so a run draws exactly num_units numbers from the counter
-  ctx->work_base += static_cast<unsigned>(p.num_units);
-  ctx->run_parity ^= 1u;
+  // the last block of stage 0 to leave clears the work counter, the last of stage 2 the job counter: every
+  // run starts from the same scratch state with the same arguments, whatever ran before it
   ctx->scratch_dirty = false;
   return COS_OK;
 }
@@ -2648,6 +2677,10 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
   d.row_status = ctx->d_status;
   d.diag = a->diag ? ctx->d_diag : nullptr;
   d.bonus_prob = a->bonus_prob ? ctx->d_bonus : nullptr;
+  if (a->offset_device) {  // a host address here, like every other pointer of this call
+    d.offset = *a->offset_device;
+    d.offset_device = nullptr;
+  }
   cos_status st = cos_verify_run(ctx, &d, stream);
   if (st != COS_OK) return st;
   e = cudaMemcpyAsync(a->accept_count, ctx->d_accept, B * sizeof(int), cudaMemcpyDeviceToHost, stream);
@@ -2869,6 +2902,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.seed_hi = static_cast<unsigned>(a->seed >> 32);
   p.off_lo = static_cast<unsigned>(a->offset);
   p.off_hi = static_cast<unsigned>(a->offset >> 32);
+  p.off_dev = reinterpret_cast<const unsigned long long*>(a->offset_device);
   p.row_base = a->row_base;
   p.accept_count = a->accept_count;
   p.out_tokens = a->out_tokens;
@@ -2880,13 +2914,12 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
   p.greedy = (c.temperature == 0.0f) ? 1 : 0;
   p.work_counter = d_counter;
-  p.work_base = 0;  // the counter was just cleared
+  p.exit_count = d_counter + 1;
   p.row_arrivals = d_arrivals;
   p.row_reject = nullptr;  // the hint to leave positions unread is not taken here
   p.early_exit = 0;
   p.unit_res = d_unit_res;
   p.job_count = d_job_count;
-  p.job_reset = d_job_count + 1;
   p.jobs = d_jobs;
   p.ustats = d_ustats;
   p.zpart = d_zpart;

@@ -195,3 +195,44 @@ def test_early_exit_hint_gives_the_rows_of_the_full_run(name):
     assert unread > 0 or name == "cfg3"
     del inputs
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name,kw", [("cfg3", dict(batch=40, vocab=20008, gamma=8)), ("cfg5", dict(batch=6, vocab=50000, gamma=3)),
+                                     ("cfg2", dict(batch=8, vocab=9001, gamma=5)), ("cfg5_greedy", dict(batch=6, vocab=50000, gamma=3))])
+def test_a_run_can_be_captured_in_a_graph_and_replayed(name, kw):
+    """The launches of a run depend on its arguments only, and the kernels leave the scratch as they found it:
+    a captured run, replayed with the counter offset kept in device memory, gives what an ordinary run with
+    that offset gives."""
+    w = C[name].scaled(**kw)
+    inputs = synth.make_inputs(w, "cuda")
+    B, P = w.batch, w.gamma + 1
+    v, ref_v = helpers.make_verifier(w), helpers.make_verifier(w)
+    try:
+        off = torch.zeros(1, dtype=torch.int64, device="cuda")
+        outs = v._alloc_outs(B, P, w.vocab, torch.device("cuda"), True, False)
+        args = (inputs["logits"], inputs["drafts"], inputs["proposer"], inputs["seed"], 0)
+        v.run(*args, outs=outs, offset_device=off)          # an ordinary run first
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            v.run(*args, outs=outs, offset_device=off)
+        for k in (3, 4, 1 << 40):
+            off.fill_(k)
+            for t in outs.values():
+                t.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            want = ref_v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], inputs["seed"], k, diag=True)
+            torch.cuda.synchronize()
+            for key in ("accept_count", "out_tokens", "row_status"):
+                assert torch.equal(outs[key], want[key]), (k, key)
+            assert torch.equal(torch.nan_to_num(outs["diag"], nan=-7.0), torch.nan_to_num(want["diag"], nan=-7.0))
+            assert torch.equal(torch.nan_to_num(outs["bonus_prob"], nan=-7.0), torch.nan_to_num(want["bonus_prob"], nan=-7.0))
+        # an ordinary run after the replays still works on the same context
+        again = v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], inputs["seed"], 3)
+        want = ref_v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], inputs["seed"], 3)
+        torch.cuda.synchronize()
+        assert torch.equal(again["out_tokens"], want["out_tokens"])
+    finally:
+        v.close()
+        ref_v.close()
