@@ -754,9 +754,80 @@ __device__ __forceinline__ void sweep_unit(const KParams& p, const char* base, c
     LaneSoft accq, accc;
     const char* row0 = reinterpret_cast<const char*>(row_of(0));
     const long long row_step = p.s_model * Elem<DT>::bytes;
-    // fixed reference exponents seeded from the thread's first vector; overflow or a non-finite input
-    // falls back to the running-maximum form (second pass)
-    for (int pass = 0; pass < 2; ++pass) {
+    // Fast form: fixed reference exponents seeded from the thread's first vector, one vector of every model
+    // per trip, the first two models fetched one trip ahead (four loads in flight per thread).
+    bool settled = false;
+    {
+      accq.init();
+      accc.init();
+      const bool pair = (p.n >= 2);
+      uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+      const int v0 = sl.v_lo + tid;
+      if (v0 < sl.v_hi) {
+        nx0 = ldg_stream16(row0 + static_cast<long long>(v0) * 16);
+        if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(v0) * 16);
+      }
+      bool first = true;
+      for (int v = v0; v < sl.v_hi; v += kThreads) {
+        const uint4 a0 = nx0, a1 = nx1;
+        {
+          const int vn = v + kThreads;
+          if (vn < sl.v_hi) {
+            nx0 = ldg_stream16(row0 + static_cast<long long>(vn) * 16);
+            if (pair) nx1 = ldg_stream16(row0 + row_step + static_cast<long long>(vn) * 16);
+          }
+        }
+        float cmb[E], xq[E];
+        unsigned inbits = 0xffffffffu;
+#pragma unroll
+        for (int k = 0; k < E; ++k) cmb[k] = 0.f;
+        auto take = [&](int i, const uint4& raw) {
+          float x[E];
+          Elem<DT>::unpack(raw, x);
+          const float wi = p.w[i];
+#pragma unroll
+          for (int k = 0; k < E; ++k) cmb[k] = fmaf(wi, x[k], cmb[k]);
+          if (i == pis) {
+#pragma unroll
+            for (int k = 0; k < E; ++k) xq[k] = x[k];
+          }
+          if (masked && i == p.mask_model) {
+            inbits = 0u;
+#pragma unroll
+            for (int k = 0; k < E; ++k) inbits |= (x[k] >= thr) ? (1u << k) : 0u;
+          }
+        };
+        take(0, a0);
+        if (pair) take(1, a1);
+        for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(v) * 16));
+        if (masked) {
+#pragma unroll
+          for (int k = 0; k < E; ++k) cmb[k] = (inbits & (1u << k)) ? cmb[k] : -INFINITY;
+        }
+        if (first) {
+          accq.seed(xq, p.cT);
+          accc.seed(cmb, p.cT);
+          first = false;
+        }
+        accq.add_fixed(xq, p.cT);
+        accc.add_fixed(cmb, p.cT);
+      }
+      for (int e = sl.e_lo + tid; e < sl.e_hi; e += kThreads) {
+        float cmb = 0.f, xq = -INFINITY, xe = 0.f;
+        for (int i = 0; i < p.n; ++i) {
+          float x = Elem<DT>::load1(row_of(i), e);
+          cmb = fmaf(p.w[i], x, cmb);
+          if (i == pis) xq = x;
+          if (i == p.mask_model) xe = x;
+        }
+        if (masked && !(xe >= thr)) cmb = -INFINITY;
+        accq.add_online1(xq, p.cT);
+        accc.add_online1(cmb, p.cT);
+      }
+      settled = (accq.s < INFINITY) && (accc.s < INFINITY);
+    }
+    // overflow or a non-finite input: the running-maximum form (two vectors of two models per trip)
+    for (int pass = 1; pass < 2 && !settled; ++pass) {
       const bool fixed = (pass == 0);
       accq.init();
       accc.init();
