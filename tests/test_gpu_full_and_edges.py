@@ -155,6 +155,15 @@ def test_invalid_arguments_return_errors():
             v.run(inputs["logits"][..., :-8], inputs["drafts"], inputs["proposer"], 1, 0)
         with pytest.raises(CosVerifyError):        # host-pointer call without staging
             v.run_host(inputs["logits"].cpu(), inputs["drafts"].cpu(), inputs["proposer"].cpu(), 1, 0)
+        with pytest.raises(CosVerifyError):        # bonus model outside [0, n)
+            v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], 1, 0, bonus_model=w.n)
+        with pytest.raises(CosVerifyError):        # unknown flag bit
+            v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], 1, 0, flags=1 << 9)
+        with pytest.raises(ValueError):            # a proposer table of the wrong shape
+            v.run(inputs["logits"], inputs["drafts"], torch.zeros((2, w.gamma), dtype=torch.int32, device="cuda"), 1, 0)
+        with pytest.raises(ValueError):            # the device-resident offset must be an int64 device tensor
+            v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], 1, 0,
+                  offset_device=torch.zeros(1, dtype=torch.int32, device="cuda"))
         ok = v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], 1, 0)   # the context still works
         torch.cuda.synchronize()
         assert ok["accept_count"].min() >= 0
