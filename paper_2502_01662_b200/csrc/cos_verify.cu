@@ -41,6 +41,7 @@ constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxSlots = COS_MAX_MODELS + 2;
 constexpr int kNoReject = 0x7fffffff;
+constexpr int kPackedP = 13;  // rows of up to this many positions keep their accept flags in the arrival word
 constexpr int kDrawResidual = 0, kDrawR = 1, kDrawQ = 2;  // what a token is drawn from: max(0, r - q), r, or q
 constexpr double kBigShare = 1.0 / 256.0;  // probabilities above 2^-8 get fp64 treatment when tokens are drawn
 constexpr int kRingVecs = 8;                 // 16-byte vectors per lane staged ahead in sweep 2 (4 KB per warp)
@@ -560,21 +561,44 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
   // test hooks: the combined distribution everywhere, or the residual mass at every draft position
   if (drawable && (p.dump_r != nullptr || ((p.flags & COS_RUN_ALL_RESIDUALS) && j < p.gamma))) push_job(p, idx, 0);
   __threadfence();
-  int prev = atomicAdd(&p.row_arrivals[b], 1);
-  if (prev != p.P - 1) return;
+  // The row's word counts its published positions (low six bits) and, for rows of up to kPackedP positions,
+  // also carries one "not accepted" bit and one "has status bits" bit per position: the last position to
+  // arrive then knows the first rejection from the value the atomic returns, without reading the others.
+  const bool packed = (p.P <= kPackedP);
+  int mine = 1;
+  if (packed) {
+    if (!accept || j == p.gamma) mine |= 1 << (6 + j);
+    if (status) mine |= 1 << (6 + kPackedP + j);
+  }
+  const int prev = atomicAdd(&p.row_arrivals[b], mine);
+  if ((prev & 63) != p.P - 1) return;
   // last unit of the row: every other unit's result is visible after the fence below
   __threadfence();
   int a = p.gamma;
   unsigned st = 0;
   int tok = -1, draw = 0;
-  for (int k = 0; k < p.P; ++k) {
-    int4 u = __ldcg(&p.unit_res[b * p.P + k]);
-    st |= static_cast<unsigned>(u.y);
-    if (k == p.gamma || !u.x) {
-      a = k;
-      tok = u.z;
-      draw = u.w;
-      break;
+  if (packed) {
+    const int total = prev + mine;  // every position added its own bits once: no carries
+    a = __ffs((total >> 6) & ((1 << kPackedP) - 1)) - 1;
+    const int4 u = __ldcg(&p.unit_res[b * p.P + a]);
+    tok = u.z;
+    draw = u.w;
+    int with_status = (total >> (6 + kPackedP)) & ((2 << a) - 1);
+    while (with_status) {  // rare: some position up to the first rejection reported status bits
+      const int k = __ffs(with_status) - 1;
+      with_status &= with_status - 1;
+      st |= static_cast<unsigned>(__ldcg(&p.unit_res[b * p.P + k]).y);
+    }
+  } else {
+    for (int k = 0; k < p.P; ++k) {
+      int4 u = __ldcg(&p.unit_res[b * p.P + k]);
+      st |= static_cast<unsigned>(u.y);
+      if (k == p.gamma || !u.x) {
+        a = k;
+        tok = u.z;
+        draw = u.w;
+        break;
+      }
     }
   }
   if (p.bonus_prob != nullptr) {
