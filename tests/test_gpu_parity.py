@@ -28,6 +28,7 @@ SMALL = [
     C["cfg3"].scaled(batch=4, vocab=64, gamma=2, name="tiny_v64"),
     C["cfg3"].scaled(batch=4, vocab=5, gamma=1, name="tiny_v5"),
     C["cfg5"].scaled(batch=3, vocab=1000, gamma=0, name="gamma0"),
+    C["cfg4"].scaled(batch=5, vocab=3000, gamma=14, name="gamma14"),      # more positions than the arrival word packs
 ]
 # the same recipes stored as IEEE half
 SMALL += [
