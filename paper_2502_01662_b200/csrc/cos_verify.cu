@@ -366,7 +366,7 @@ struct LaneSoft {
 #pragma unroll
     for (int k = 1; k < E; ++k) vmax = fmaxf(vmax, v[k]);
     float cand = vmax * c;
-    ref = (fabsf(cand) < INFINITY) ? cand : 0.f;
+    ref = (fabsf(cand) < INFINITY) ? floorf(cand) : 0.f;  // a whole number: sums with such references rescale exactly
     s = 0.f;
   }
   template <int E>
@@ -387,7 +387,15 @@ __device__ __forceinline__ SoftPart warp_reduce_soft(float ref, double s) {
   float R = ref;
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) R = fmaxf(R, __shfl_xor_sync(0xffffffffu, R, d));
-  double t = (ref == R) ? s : s * exp2(static_cast<double>(ref) - static_cast<double>(R));
+  // references seeded by the sweep are whole numbers: the factor is then an exact power of two and cheap
+  const float d = ref - R;
+  double t;
+  if (ref == R)
+    t = s;
+  else if (d == floorf(d) && d > -1000.f)
+    t = s * __hiloint2double((1023 + static_cast<int>(d)) << 20, 0);
+  else
+    t = s * exp2(static_cast<double>(ref) - static_cast<double>(R));
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) {
     int lo = __shfl_xor_sync(0xffffffffu, __double2loint(t), d);
