@@ -103,6 +103,8 @@ struct KParams {
   double* wtotg;           // [B*P][parts*16]: stage 2's mass of every warp run
   double* srung;           // [B][parts*16][kRecG]: running totals inside the runs of the row's drawing unit
   int* part_arrivals;      // [B*P]: blocks of the unit that finished stage 2; zero between runs
+  double* wtotgB;          // the one-sweep drawing stage: second channel of wtotg (null where that stage is not used)
+  double* srungB;          // and of srung
 };
 
 // ------------------------------------------------------------------------------------
@@ -299,6 +301,13 @@ struct FreeRun {
   int skip_state[2];  // unit of that parity: 0 undecided, 1 swept, 2 left unread (its row is already rejected earlier)
 };
 
+struct OneSweep {  // constants of the one-sweep drawing stage, for its out-of-line part
+  float ctA, ctB;        // k / first-estimate normaliser of each channel: decides the sign of a mass
+  float nrefA, nrefB;    // minus the reference exponents
+  float btA, btB;        // terms above these are big
+  double ctA64, ctB64, drefA, drefB;
+};
+
 struct Shared {
   Xchg x[2];
   FreeRun fr;
@@ -323,6 +332,8 @@ struct Shared {
   int next_local, next;
   float thr32;  // plausibility threshold rounded up to fp32
   float big_thr[kMaxSlots];  // sweep 2: terms above this share of a normaliser are redone in fp64
+  double chan_c[2];          // one-sweep drawing stage: exact coefficients of the two channel sums in a mass
+  OneSweep one;
   float ldraft[COS_MAX_MODELS];  // the n logits at the draft token, fetched before sweep 1
 };
 
@@ -730,6 +741,59 @@ __device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* 
     q64 = exp2(static_cast<double>(lv[pis]) * p.cT64 - static_cast<double>(fsoft[0].ref)) / fsoft[0].s;
   }
   return draw == kDrawR ? r64 : (draw == kDrawQ ? q64 : fmax(0.0, r64 - q64));
+}
+
+// One-sweep drawing stage, a vector that holds a big entry (more than 2^-8 of a normaliser), done again
+// entry by entry from the stored logits: big entries in fp64 into the thread's slots `bigacc` ([0] Z_A,
+// [kThreads] Z_B, [2 kThreads] and [3 kThreads] the sums over entries with a positive mass), the others as the
+// sweep does them, returned as (Z_A, Z_B, sum A, sum B) of this vector.  Rare; out of line.
+template <int DT, int MODE>
+__device__ __noinline__ float4 one_sweep_big_vector(const KParams& p, const OneSweep& c, const char* base, int e0, int pis,
+                                                    bool masked, float thr, double* bigacc) {
+  constexpr int E = Elem<DT>::E;
+  float4 out = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k = 0; k < E; ++k) {
+    const int e = e0 + k;
+    if (e >= p.V) break;
+    float xa, xb;
+    double cb;
+    bool in = true;
+    if (MODE == kEnsembleSample) {
+      xa = Elem<DT>::load1(base, e);
+      xb = Elem<DT>::load1(base + p.s_model * Elem<DT>::bytes, e);
+      cb = static_cast<double>(xb);
+    } else {
+      xb = 0.f;
+      cb = 0.0;
+      xa = 0.f;
+      for (int i = 0; i < p.n; ++i) {
+        const float x = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
+        xb = fmaf(p.w[i], x, xb);
+        cb = fma(p.w64[i], static_cast<double>(x), cb);
+        if (i == pis) xa = x;
+        if (masked && i == p.mask_model) in = (x >= thr);
+      }
+    }
+    const float eA = ex2_approx(fmaf(xa, p.cT, c.nrefA));
+    const float eB = in ? ex2_approx(fmaf(xb, p.cT, c.nrefB)) : 0.f;
+    if (eA > c.btA || eB > c.btB) {
+      const double dA = exp2(static_cast<double>(xa) * p.cT64 - c.drefA);
+      const double dB = in ? exp2(cb * p.cT64 - c.drefB) : 0.0;
+      bigacc[0] += dA;
+      bigacc[kThreads] += dB;
+      if (c.ctA64 * dA + c.ctB64 * dB > 0.0) {
+        bigacc[2 * kThreads] += dA;
+        bigacc[3 * kThreads] += dB;
+      }
+    } else {
+      const bool pos = __fadd_rn(__fmul_rn(c.ctA, eA), __fmul_rn(c.ctB, eB)) > 0.f;
+      out.x += eA;
+      out.y += eB;
+      out.z += pos ? eA : 0.f;
+      out.w += pos ? eB : 0.f;
+    }
+  }
+  return out;
 }
 
 // Combined logit of one token in fp64, from the stored logits: the chain of fused multiply-adds that
@@ -1437,7 +1501,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   cg::cluster_group cluster = cg::this_cluster();
   // stage 0 shares a unit among the blocks of a cluster; stages 1 and 2 among `parts` independent
   // blocks (they meet only through global memory: partial sums between the launches, an arrival counter within stage 2)
-  const int lparts = (STAGE == 1 || STAGE == 2) ? p.parts : 1;  // blocks per unit in this launch
+  const int lparts = (STAGE >= 1) ? p.parts : 1;  // blocks per unit in this launch
   const int C = (STAGE == 0) ? static_cast<int>(cluster.num_blocks()) : p.parts;
   const int rank = (STAGE == 0) ? static_cast<int>(cluster.block_rank()) : static_cast<int>(blockIdx.x % lparts);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1460,7 +1524,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   // later stages are launched while the previous one drains (programmatic dependent launch);
   // nothing it wrote is read before this point
   if (STAGE >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (STAGE == 1 && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
+  if ((STAGE == 1 || STAGE == 3) && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
   const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
   if (STAGE == 0) {
@@ -1592,7 +1656,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         sh.fsoft[tid].s = p.ustats[uidx].s[tid];
         sh.fsoft[tid].ref = p.ustats[uidx].ref[tid];
         sh.big_thr[tid] = static_cast<float>(sh.fsoft[tid].s * kBigShare);  // from the first estimate, in every stage
-        if (STAGE >= 2) {
+        if (STAGE == 2) {
           double z = 0.0;
           for (int q = 0; q < p.parts; ++q) z += p.zpart[(static_cast<size_t>(uidx) * p.parts + q) * 8 + tid];
           sh.fsoft[tid].s = z;
@@ -1816,6 +1880,244 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         if (lane == 0) p.zpart[(static_cast<size_t>(uidx) * p.parts + rank) * 8 + warp] = o.s;
       }
       } else {
+      bool do_locate = false;
+      if (STAGE == 3) {
+        // ---- the drawing stages in one sweep.  A token's mass is k_A e_A / Z_A + k_B e_B / Z_B clipped at zero,
+        // where the two channels are the two models (ensemble, n = 2) or the proposer's and the combined logits
+        // (logit level), and (k_A, k_B) says what is drawn: max(0, r - q), r, or q.  The set of tokens with a
+        // positive mass is decided with the normalisers stage 0 left (they are good to 1e-7, and a token whose sign
+        // that could change carries no mass to speak of); over that set the mass is LINEAR in 1/Z_A and 1/Z_B,
+        // so this sweep only adds up e_A and e_B per group of steps, and with them the refined normalisers of
+        // stage 1.  Whoever locates the token turns the sums into masses once the normalisers are complete.
+        // Terms above 2^-8 of a normaliser go through fp64, as in stage 1.
+        double kA, kB;
+        if (MODE == kEnsembleSample) {
+          const double selA = (pis == 0) ? 1.0 : 0.0, selB = (pis == 1) ? 1.0 : 0.0;
+          kA = !is_bonus ? p.w64[0] - selA : (draw_q ? selA : p.w64[0]);
+          kB = !is_bonus ? p.w64[1] - selB : (draw_q ? selB : p.w64[1]);
+        } else {
+          kA = !is_bonus ? -1.0 : (draw_q ? 1.0 : 0.0);
+          kB = (is_bonus && draw_q) ? 0.0 : 1.0;
+        }
+        const double ctA64 = kA / sh.fsoft[0].s, ctB64 = kB / sh.fsoft[1].s;  // with the first estimates: signs only
+        const float ctA = static_cast<float>(ctA64), ctB = static_cast<float>(ctB64);
+        const float nrefA = -sh.fsoft[0].ref, nrefB = -sh.fsoft[1].ref;
+        const float btA = sh.big_thr[0], btB = sh.big_thr[1];
+        const double drefA = static_cast<double>(sh.fsoft[0].ref), drefB = static_cast<double>(sh.fsoft[1].ref);
+        const char* row0 = reinterpret_cast<const char*>(row_of(0));
+        const long long row_step = p.s_model * Elem<DT>::bytes;
+        const int nst = s_end - s_begin;
+        const int gszv = (nst + kRecG - 1) / kRecG > 1 ? (nst + kRecG - 1) / kRecG : 1;
+        const size_t rec_at = (static_cast<size_t>(b) * G + gwarp) * kRecG;
+        const int nfull = vec_ok ? p.V / (32 * E) : 0;
+        const int fe = (s_end < nfull) ? s_end : nfull;  // steps [s_begin, fe) are whole aligned vectors
+        float zsA = 0.f, zsB = 0.f, aA = 0.f, aB = 0.f;  // small terms: normalisers (whole run), group sums
+        // the big terms of the same four sums sit in shared memory (the staging ring is idle during this sweep),
+        // one slot per thread and sum: [0] Z_A, [1] Z_B, [2] group sum A, [3] group sum B
+        double* bigacc = reinterpret_cast<double*>(ring) + tid;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) bigacc[q * kThreads] = 0.0;
+        bool hasbig = false;
+        if (tid == 0) {
+          OneSweep& c = sh.one;
+          c.ctA = ctA;
+          c.ctB = ctB;
+          c.nrefA = nrefA;
+          c.nrefB = nrefB;
+          c.btA = btA;
+          c.btB = btB;
+          c.ctA64 = ctA64;
+          c.ctB64 = ctB64;
+          c.drefA = drefA;
+          c.drefB = drefB;
+        }
+        if (lane == 0) sh.wtot[warp] = sh.wincl[warp] = 0.0;  // the run's sums, group by group (lane 0 only)
+        __syncthreads();
+        // one vector of entries: channel arguments xa (proposer's or model 0's logits) and xb (model 1's or the
+        // combined logits), `inb` = inside the plausibility mask (bit per entry)
+        auto eat = [&](const float (&xa)[E], const float (&xb)[E], unsigned inb, int e0) {
+          float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f, mA = 0.f, mB = 0.f;
+#pragma unroll
+          for (int k = 0; k < E; ++k) {
+            const float eA = ex2_approx(fmaf(xa[k], p.cT, nrefA));
+            float eB = ex2_approx(fmaf(xb[k], p.cT, nrefB));
+            if (MODE == kLogitSample && masked) eB = ((inb >> k) & 1u) ? eB : 0.f;
+            mA = fmaxf(mA, eA);
+            mB = fmaxf(mB, eB);
+            // products rounded one by one: where r and q coincide the sum is exactly zero, as in exact arithmetic
+            const bool pos = __fadd_rn(__fmul_rn(ctA, eA), __fmul_rn(ctB, eB)) > 0.f;
+            vzA += eA;
+            vzB += eB;
+            vaA += pos ? eA : 0.f;
+            vaB += pos ? eB : 0.f;
+          }
+          if (mA > btA || mB > btB) {
+            // rare: some entry of this vector is big; the vector is done again out of line, big entries in fp64
+            const float4 r = one_sweep_big_vector<DT, MODE>(p, sh.one, base, e0, pis, masked, thr, bigacc);
+            vzA = r.x;
+            vzB = r.y;
+            vaA = r.z;
+            vaB = r.w;
+            hasbig = true;
+          }
+          zsA += vzA;
+          zsB += vzB;
+          aA += vaA;
+          aB += vaB;
+        };
+        // the channel arguments of one step from the n vectors of the lane (ensemble: the vectors themselves)
+        auto feed = [&](const uint4& r0, const uint4& r1, int s) {
+          const int e0 = (s * 32 + lane) * E;
+          if (MODE == kEnsembleSample) {
+            float xa[E], xb[E];
+            Elem<DT>::unpack(r0, xa);
+            Elem<DT>::unpack(r1, xb);
+            eat(xa, xb, 0xffffffffu, e0);
+          } else {
+            float cmb[E], vq[E];
+            unsigned inb = 0u;
+#pragma unroll
+            for (int k = 0; k < E; ++k) cmb[k] = 0.f;
+            auto take = [&](int i, const uint4& raw) {
+              float x[E];
+              Elem<DT>::unpack(raw, x);
+              const float wi = p.w[i];
+#pragma unroll
+              for (int k = 0; k < E; ++k) {
+                cmb[k] = fmaf(wi, x[k], cmb[k]);
+                if (i == pis) vq[k] = x[k];
+                if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
+              }
+            };
+            take(0, r0);
+            if (p.n >= 2) take(1, r1);
+            for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(s * 32 + lane) * 16));
+            eat(vq, cmb, inb, e0);
+          }
+        };
+        const bool pair = (MODE == kEnsembleSample) || (p.n >= 2);
+        uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+        if (s_begin < fe) {  // the first two models' vectors are fetched one step ahead
+          const char* src = row0 + static_cast<long long>(s_begin * 32 + lane) * 16;
+          nx0 = ldg_stream16(src);
+          if (pair) nx1 = ldg_stream16(src + row_step);
+        }
+        int in_group = 0, grp = 0;
+        for (int s = s_begin; s < s_end; ++s) {
+          if (s < fe) {
+            const uint4 a0 = nx0, a1 = nx1;
+            if (s + 1 < fe) {
+              const char* src = row0 + static_cast<long long>((s + 1) * 32 + lane) * 16;
+              nx0 = ldg_stream16(src);
+              if (pair) nx1 = ldg_stream16(src + row_step);
+            }
+            feed(a0, a1, s);
+          } else {
+            // ragged or unaligned step: entry by entry; entries beyond V read as -inf (no mass, outside every set)
+            const int e0 = (s * 32 + lane) * E;
+            if (MODE == kEnsembleSample) {
+              float xa[E], xb[E];
+              load_chunk<DT>(row_of(0), e0, p.V, vec_ok, xa);
+              load_chunk<DT>(row_of(1), e0, p.V, vec_ok, xb);
+              eat(xa, xb, 0xffffffffu, e0);
+            } else {
+              float cmb[E], vq[E];
+              unsigned inb = 0u;
+#pragma unroll
+              for (int k = 0; k < E; ++k) cmb[k] = 0.f;
+              for (int i = 0; i < p.n; ++i) {
+                float x[E];
+                load_chunk<DT>(row_of(i), e0, p.V, vec_ok, x);
+#pragma unroll
+                for (int k = 0; k < E; ++k) {
+                  cmb[k] = (e0 + k < p.V) ? fmaf(p.w[i], x[k], cmb[k]) : -INFINITY;
+                  if (i == pis) vq[k] = x[k];
+                  if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
+                }
+              }
+              eat(vq, cmb, inb, e0);
+            }
+          }
+          if (++in_group == gszv || s + 1 == s_end) {
+            float ra = aA, rb = aB;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+              ra += __shfl_xor_sync(0xffffffffu, ra, d);
+              rb += __shfl_xor_sync(0xffffffffu, rb, d);
+            }
+            double da = static_cast<double>(ra), db = static_cast<double>(rb);
+            if (__any_sync(0xffffffffu, hasbig)) {
+              double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
+              bigacc[2 * kThreads] = bigacc[3 * kThreads] = 0.0;
+#pragma unroll
+              for (int d = 16; d > 0; d >>= 1) {
+                ta += shfl_double(ta, lane ^ d);
+                tb += shfl_double(tb, lane ^ d);
+              }
+              da += ta;
+              db += tb;
+            }
+            if (lane == 0) {
+              sh.wtot[warp] += da;
+              sh.wincl[warp] += db;
+              if (emit) {
+                p.srung[rec_at + grp] = da;  // the group's own sums (not running totals)
+                p.srungB[rec_at + grp] = db;
+              }
+            }
+            ++grp;
+            in_group = 0;
+            aA = aB = 0.f;
+          }
+        }
+        {
+          double tA = static_cast<double>(zsA) + bigacc[0], tB = static_cast<double>(zsB) + bigacc[kThreads];
+#pragma unroll
+          for (int d = 16; d > 0; d >>= 1) {
+            tA += shfl_double(tA, lane ^ d);
+            tB += shfl_double(tB, lane ^ d);
+          }
+          if (lane == 0) {
+            sh.wsoft[warp][0].s = tA;
+            sh.wsoft[warp][0].ref = sh.fsoft[0].ref;
+            sh.wsoft[warp][1].s = tB;
+            sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
+            p.wtotg[static_cast<size_t>(uidx) * G + gwarp] = sh.wtot[warp];
+            p.wtotgB[static_cast<size_t>(uidx) * G + gwarp] = sh.wincl[warp];
+          }
+        }
+        __syncthreads();
+        if (warp < 2) {
+          float ref = (lane < kWarps) ? sh.wsoft[lane][warp].ref : -INFINITY;
+          double sum = (lane < kWarps) ? sh.wsoft[lane][warp].s : 0.0;
+          SoftPart o = warp_reduce_soft(ref, sum);
+          if (lane == 0) p.zpart[(static_cast<size_t>(uidx) * p.parts + rank) * 8 + warp] = o.s;
+        }
+        // the last block of the unit to get here completes the normalisers and locates the token
+        __syncthreads();
+        if (tid == 0) {
+          __threadfence();
+          const int prev = atomicAdd(&p.part_arrivals[uidx], 1);
+          sh.win_g = (prev == p.parts - 1) ? 1 : 0;
+          if (prev == p.parts - 1) {
+            p.part_arrivals[uidx] = 0;  // ready for the next run
+            __threadfence();
+          }
+        }
+        __syncthreads();
+        do_locate = (sh.win_g != 0);
+        __syncthreads();
+        if (do_locate) {
+          if (tid < 2) {
+            double z = 0.0;
+            for (int q = 0; q < p.parts; ++q) z += __ldcg(&p.zpart[(static_cast<size_t>(uidx) * p.parts + q) * 8 + tid]);
+            sh.fsoft[tid].s = z;
+            sh.chan_c[tid] = (tid == 0 ? kA : kB) / z;
+          }
+          __syncthreads();
+        }
+      }
+      if (STAGE == 2 || do_locate) {
       if (MODE == kEnsembleSample && tid < p.n) {
         // r - q = sum_i (w_i/Z_i - [i = proposer]/Z_i) e_i, and r = sum_i (w_i/Z_i) e_i
         const double a = p.w64[tid] / sh.fsoft[tid].s;
@@ -2131,7 +2433,6 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       };
       auto run_gsz = [&](int nst, int nrec) { return (nst + nrec - 1) / nrec > 1 ? (nst + nrec - 1) / nrec : 1; };
 
-      bool do_locate = false;
       if (STAGE == 2) {
         // ---- masses of this block's runs, to be added up and searched by the last block of the unit
         const int gszv = run_gsz(s_end - s_begin, kRecG);
@@ -2192,7 +2493,15 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       }
       if (do_locate) {
         // ---- one block per unit: add the runs up, find the run, walk it
-        for (int g = tid; g < G; g += kThreads) sh.gw[g] = __ldcg(&p.wtotg[static_cast<size_t>(uidx) * G + g]);
+        for (int g = tid; g < G; g += kThreads) {
+          const double wa = __ldcg(&p.wtotg[static_cast<size_t>(uidx) * G + g]);
+          if (STAGE == 3)  // channel sums of the run into its mass, with the completed normalisers; the products
+                           // are rounded one by one so that equal sums under opposite coefficients cancel exactly
+            sh.gw[g] = fmax(0.0, __dadd_rn(__dmul_rn(sh.chan_c[0], wa),
+                                           __dmul_rn(sh.chan_c[1], __ldcg(&p.wtotgB[static_cast<size_t>(uidx) * G + g]))));
+          else
+            sh.gw[g] = wa;
+        }
         __syncthreads();
         if (tid == 0) pick_run(sh.gw, G);
         __syncthreads();
@@ -2203,8 +2512,25 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             const int g = sh.win_g;
             const int sb = static_cast<int>(static_cast<long long>(g) * p.nsteps / G);
             const int se = static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
-            const int token = walk(sb, se, run_gsz(se - sb, kRecG), sh.base,
-                                   p.srung + (static_cast<size_t>(b) * G + g) * kRecG, sh.target, is_bonus);
+            const int gsz = run_gsz(se - sb, kRecG);
+            const double* rec = p.srung + (static_cast<size_t>(b) * G + g) * kRecG;
+            if (STAGE == 3) {
+              // masses of the run's groups from their channel sums, then running totals as the walk expects them
+              const int ngrp = (se - sb + gsz - 1) / gsz;
+              double m = 0.0;
+              if (lane < ngrp)
+                m = fmax(0.0, __dadd_rn(__dmul_rn(sh.chan_c[0], __ldcg(rec + lane)),
+                                        __dmul_rn(sh.chan_c[1], __ldcg(p.srungB + (static_cast<size_t>(b) * G + g) * kRecG + lane))));
+#pragma unroll
+              for (int d = 1; d < 32; d <<= 1) {
+                const double o = shfl_up_double(m, d);
+                if (lane >= d) m += o;
+              }
+              if (lane < kRecG) sh.srun[0][lane] = m;
+              __syncwarp();
+              rec = &sh.srun[0][0];
+            }
+            const int token = walk(sb, se, gsz, sh.base, rec, sh.target, is_bonus);
             if (lane == 0) {
               p.out_tokens[uidx] = token;  // the row's token at its first rejection, or the bonus
               // Algorithm 2's Score returns the bonus token with its probability under the law it came from
@@ -2232,6 +2558,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           }
         }
       }
+      }
       }  // stages 2 and 3
     }
     if (STAGE == 0 && rank == 0 && tid == 0) {
@@ -2246,7 +2573,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     unit = next_unit;
   }
   cluster.sync();  // no block leaves while a peer may still read its shared memory
-  if (((STAGE == 0 && p.greedy) || STAGE == 2) && tid == 0) stage_exit(p, STAGE == 0 ? 0 : 1);
+  if (((STAGE == 0 && p.greedy) || STAGE >= 2) && tid == 0) stage_exit(p, STAGE == 0 ? 0 : 1);
 }
 
 // ------------------------------------------------------------------------------------
@@ -2274,6 +2601,8 @@ struct cos_verify_ctx {
   double* d_zpart;
   double* d_wtotg;
   double* d_srung;
+  double* d_wtotgB;  // second channel of the two above, for the one-sweep drawing stage
+  double* d_srungB;
   int* d_part_arrivals;
   // optional per-stage timing (cos_verify_set_stage_timing)
   bool timing;
@@ -2307,7 +2636,7 @@ KernelFn pick_kernel(int dtype, int mode, int stage, bool dense = false) {
   }
 #define COS_CASE(DT, M, S) \
   if (dtype == DT && mode == M && stage == S) return cos_verify_kernel<DT, M, S>;
-#define COS_SAMPLING(DT, M) COS_CASE(DT, M, 0) COS_CASE(DT, M, 1) COS_CASE(DT, M, 2)
+#define COS_SAMPLING(DT, M) COS_CASE(DT, M, 0) COS_CASE(DT, M, 1) COS_CASE(DT, M, 2) COS_CASE(DT, M, 3)
   COS_SAMPLING(COS_DTYPE_F32, kEnsembleSample)
   COS_SAMPLING(COS_DTYPE_F32, kLogitSample)
   COS_CASE(COS_DTYPE_F32, kEnsembleGreedy, 0)
@@ -2425,7 +2754,7 @@ cudaError_t query_clusters(KernelFn fn, int cluster, int sm_count, int* out) {
 // attributes the kernels of one (dtype, mode) need before their first launch
 cudaError_t prepare_kernels(int dtype, int mode, int cluster_size);
 
-int stage_smem(int stage) { return stage == 2 ? kRingBytes : 0; }  // the staging ring of the token-mass sweep
+int stage_smem(int stage) { return stage >= 2 ? kRingBytes : 0; }  // the staging ring of the token-mass sweep
 
 cudaError_t launch_stage(int dtype, int mode, int stage, const KParams& p, int cluster, cudaStream_t stream,
                          bool overlap_prev = false, bool dense = false) {
@@ -2451,8 +2780,8 @@ cudaError_t launch_stage(int dtype, int mode, int stage, const KParams& p, int c
 cudaError_t prepare_kernels(int dtype, int mode, int cluster_size) {
   const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
   cudaError_t e = cudaSuccess;
-  if (draws)
-    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, 2)),
+  for (int st = 2; draws && st <= 3 && e == cudaSuccess; ++st)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, st)),
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
   if (e == cudaSuccess && cluster_size > 8)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, 0)),
@@ -2556,6 +2885,8 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   ok = ok && cudaMalloc(&ctx->d_zpart, rows * P * ctx->parts * 8 * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_wtotg, rows * P * ctx->parts * kWarps * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_srung, rows * ctx->parts * kWarps * kRecG * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_wtotgB, rows * P * ctx->parts * kWarps * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_srungB, rows * ctx->parts * kWarps * kRecG * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_part_arrivals, rows * P * sizeof(int)) == cudaSuccess;
   if (ok && config->host_staging) {
     const size_t V = static_cast<size_t>(config->vocab);
@@ -2691,6 +3022,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.wtotg = ctx->d_wtotg;
   p.srung = ctx->d_srung;
   p.part_arrivals = ctx->d_part_arrivals;
+  p.wtotgB = ctx->d_wtotgB;
+  p.srungB = ctx->d_srungB;
   p.parts = ctx->parts;
   p.max_jobs = p.num_units + a->batch;
 
@@ -2719,8 +3052,17 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     const bool all = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
     const int most = all ? p.max_jobs : a->batch;
     const int cap = 4096;  // a block walks the job list with a stride, so the grid may be smaller than the list
-    for (int st = 1; st <= 2; ++st) {
-      p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of this launch
+    p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of a drawing launch
+    // Two channel sums describe every mass when the combine is at logit level (proposer, combined logits) or
+    // mixes two models: then one sweep does the work of stages 1 and 2.  The test hooks keep the two-stage form.
+    const bool one_sweep = !all && (mode == kLogitSample || c.n == 2);
+    if (one_sweep) {
+      e = launch_stage(c.dtype, mode, 3, p, 1, stream, true);
+      if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stage)", e);
+      if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
+      ctx->ev_used = 3;
+    }
+    for (int st = 1; st <= 2 && !one_sweep; ++st) {
       e = launch_stage(c.dtype, mode, st, p, 1, stream, true);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stages)", e);
       if (ctx->timing) cudaEventRecord(ctx->ev[st + 1], stream);
@@ -2853,6 +3195,8 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_zpart);
   cudaFree(ctx->d_wtotg);
   cudaFree(ctx->d_srung);
+  cudaFree(ctx->d_wtotgB);
+  cudaFree(ctx->d_srungB);
   cudaFree(ctx->d_part_arrivals);
   for (int k = 0; k < 4; ++k)
     if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
