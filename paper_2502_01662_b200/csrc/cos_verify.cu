@@ -102,9 +102,9 @@ struct KParams {
   double* zpart;           // [B*P][parts][8]: stage 1's partial normalisers
   double* wtotg;           // [B*P][parts*16]: stage 2's mass of every warp run
   double* srung;           // [B][parts*16][kRecG]: running totals inside the runs of the row's drawing unit
+                           // (one-sweep drawing stage: [B][nsteps], first channel sum of every step)
   int* part_arrivals;      // [B*P]: blocks of the unit that finished stage 2; zero between runs
-  double* wtotgB;          // the one-sweep drawing stage: second channel of wtotg (null where that stage is not used)
-  double* srungB;          // and of srung
+  double* srungB;          // the one-sweep drawing stage: second channel of srung (null where that stage is not used)
 };
 
 // ------------------------------------------------------------------------------------
@@ -1906,14 +1906,15 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         const double drefA = static_cast<double>(sh.fsoft[0].ref), drefB = static_cast<double>(sh.fsoft[1].ref);
         const char* row0 = reinterpret_cast<const char*>(row_of(0));
         const long long row_step = p.s_model * Elem<DT>::bytes;
-        const int nst = s_end - s_begin;
-        const int gszv = (nst + kRecG - 1) / kRecG > 1 ? (nst + kRecG - 1) / kRecG : 1;
-        const size_t rec_at = (static_cast<size_t>(b) * G + gwarp) * kRecG;
-        const int nfull = vec_ok ? p.V / (32 * E) : 0;
-        const int fe = (s_end < nfull) ? s_end : nfull;  // steps [s_begin, fe) are whole aligned vectors
-        float zsA = 0.f, zsB = 0.f, aA = 0.f, aB = 0.f;  // small terms: normalisers (whole run), group sums
+        // this block's steps [blk_lo, blk_hi); its warps take them in turn, so that the block reads 8 KB of
+        // every row at a time; every step (32 lanes x E entries, in token order) leaves its two sums on record
+        const int blk_lo = static_cast<int>(static_cast<long long>(rank) * p.nsteps / lparts);
+        const int blk_hi = static_cast<int>(static_cast<long long>(rank + 1) * p.nsteps / lparts);
+        const size_t rec_at = static_cast<size_t>(b) * p.nsteps;
+        const int nfull = vec_ok ? p.V / (32 * E) : 0;  // steps below this are whole aligned vectors
+        float zsA = 0.f, zsB = 0.f, aA = 0.f, aB = 0.f;  // small terms: normalisers (all steps), sums of the step
         // the big terms of the same four sums sit in shared memory (the staging ring is idle during this sweep),
-        // one slot per thread and sum: [0] Z_A, [1] Z_B, [2] group sum A, [3] group sum B
+        // one slot per thread and sum: [0] Z_A, [1] Z_B, [2] and [3] the step's sums
         double* bigacc = reinterpret_cast<double*>(ring) + tid;
 #pragma unroll
         for (int q = 0; q < 4; ++q) bigacc[q * kThreads] = 0.0;
@@ -1931,7 +1932,6 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           c.drefA = drefA;
           c.drefB = drefB;
         }
-        if (lane == 0) sh.wtot[warp] = sh.wincl[warp] = 0.0;  // the run's sums, group by group (lane 0 only)
         __syncthreads();
         // one vector of entries: channel arguments xa (proposer's or model 0's logits) and xb (model 1's or the
         // combined logits), `inb` = inside the plausibility mask (bit per entry)
@@ -1965,7 +1965,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           aA += vaA;
           aB += vaB;
         };
-        // the channel arguments of one step from the n vectors of the lane (ensemble: the vectors themselves)
+        // the channel arguments of one step from the lane's vectors (the first two models' fetched ahead)
         auto feed = [&](const uint4& r0, const uint4& r1, int s) {
           const int e0 = (s * 32 + lane) * E;
           if (MODE == kEnsembleSample) {
@@ -1997,17 +1997,17 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         };
         const bool pair = (MODE == kEnsembleSample) || (p.n >= 2);
         uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
-        if (s_begin < fe) {  // the first two models' vectors are fetched one step ahead
-          const char* src = row0 + static_cast<long long>(s_begin * 32 + lane) * 16;
+        if (blk_lo + warp < blk_hi && blk_lo + warp < nfull) {
+          const char* src = row0 + static_cast<long long>((blk_lo + warp) * 32 + lane) * 16;
           nx0 = ldg_stream16(src);
           if (pair) nx1 = ldg_stream16(src + row_step);
         }
-        int in_group = 0, grp = 0;
-        for (int s = s_begin; s < s_end; ++s) {
-          if (s < fe) {
+        for (int s = blk_lo + warp; s < blk_hi; s += kWarps) {
+          if (s < nfull) {
             const uint4 a0 = nx0, a1 = nx1;
-            if (s + 1 < fe) {
-              const char* src = row0 + static_cast<long long>((s + 1) * 32 + lane) * 16;
+            const int sn = s + kWarps;
+            if (sn < blk_hi && sn < nfull) {
+              const char* src = row0 + static_cast<long long>(sn * 32 + lane) * 16;
               nx0 = ldg_stream16(src);
               if (pair) nx1 = ldg_stream16(src + row_step);
             }
@@ -2038,37 +2038,30 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
               eat(vq, cmb, inb, e0);
             }
           }
-          if (++in_group == gszv || s + 1 == s_end) {
-            float ra = aA, rb = aB;
+          // the step's two sums over the warp
+          float ra = aA, rb = aB;
+#pragma unroll
+          for (int d = 16; d > 0; d >>= 1) {
+            ra += __shfl_xor_sync(0xffffffffu, ra, d);
+            rb += __shfl_xor_sync(0xffffffffu, rb, d);
+          }
+          double da = static_cast<double>(ra), db = static_cast<double>(rb);
+          if (__any_sync(0xffffffffu, hasbig)) {
+            double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
+            bigacc[2 * kThreads] = bigacc[3 * kThreads] = 0.0;
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) {
-              ra += __shfl_xor_sync(0xffffffffu, ra, d);
-              rb += __shfl_xor_sync(0xffffffffu, rb, d);
+              ta += shfl_double(ta, lane ^ d);
+              tb += shfl_double(tb, lane ^ d);
             }
-            double da = static_cast<double>(ra), db = static_cast<double>(rb);
-            if (__any_sync(0xffffffffu, hasbig)) {
-              double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
-              bigacc[2 * kThreads] = bigacc[3 * kThreads] = 0.0;
-#pragma unroll
-              for (int d = 16; d > 0; d >>= 1) {
-                ta += shfl_double(ta, lane ^ d);
-                tb += shfl_double(tb, lane ^ d);
-              }
-              da += ta;
-              db += tb;
-            }
-            if (lane == 0) {
-              sh.wtot[warp] += da;
-              sh.wincl[warp] += db;
-              if (emit) {
-                p.srung[rec_at + grp] = da;  // the group's own sums (not running totals)
-                p.srungB[rec_at + grp] = db;
-              }
-            }
-            ++grp;
-            in_group = 0;
-            aA = aB = 0.f;
+            da += ta;
+            db += tb;
           }
+          if (lane == 0 && emit) {
+            p.srung[rec_at + s] = da;
+            p.srungB[rec_at + s] = db;
+          }
+          aA = aB = 0.f;
         }
         {
           double tA = static_cast<double>(zsA) + bigacc[0], tB = static_cast<double>(zsB) + bigacc[kThreads];
@@ -2082,8 +2075,6 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             sh.wsoft[warp][0].ref = sh.fsoft[0].ref;
             sh.wsoft[warp][1].s = tB;
             sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
-            p.wtotg[static_cast<size_t>(uidx) * G + gwarp] = sh.wtot[warp];
-            p.wtotgB[static_cast<size_t>(uidx) * G + gwarp] = sh.wincl[warp];
           }
         }
         __syncthreads();
@@ -2105,7 +2096,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           }
         }
         __syncthreads();
-        do_locate = (sh.win_g != 0);
+        do_locate = (sh.win_g != 0) && emit;  // (every unit listed for this stage is its row's drawing unit)
         __syncthreads();
         if (do_locate) {
           if (tid < 2) {
@@ -2493,43 +2484,95 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       }
       if (do_locate) {
         // ---- one block per unit: add the runs up, find the run, walk it
-        for (int g = tid; g < G; g += kThreads) {
-          const double wa = __ldcg(&p.wtotg[static_cast<size_t>(uidx) * G + g]);
-          if (STAGE == 3)  // channel sums of the run into its mass, with the completed normalisers; the products
-                           // are rounded one by one so that equal sums under opposite coefficients cancel exactly
-            sh.gw[g] = fmax(0.0, __dadd_rn(__dmul_rn(sh.chan_c[0], wa),
-                                           __dmul_rn(sh.chan_c[1], __ldcg(&p.wtotgB[static_cast<size_t>(uidx) * G + g]))));
-          else
-            sh.gw[g] = wa;
+        int one_step = -1;  // one-sweep stage: the step that holds the token
+        if (STAGE == 3) {
+          // Every step's channel sums turn into its mass now that the normalisers are complete (products rounded
+          // one by one, so that equal sums under opposite coefficients cancel exactly).  Threads own consecutive
+          // steps; a prefix over threads in step order gives S and the first step whose running total reaches u S.
+          const int per = (p.nsteps + kThreads - 1) / kThreads;
+          const int lo = tid * per, hi = (lo + per < p.nsteps) ? lo + per : p.nsteps;
+          const double* ra = p.srung + static_cast<size_t>(b) * p.nsteps;
+          const double* rb = p.srungB + static_cast<size_t>(b) * p.nsteps;
+          auto step_mass = [&](int st) {
+            return fmax(0.0, __dadd_rn(__dmul_rn(sh.chan_c[0], __ldcg(ra + st)), __dmul_rn(sh.chan_c[1], __ldcg(rb + st))));
+          };
+          double mine = 0.0;
+          for (int st = lo; st < hi; ++st) mine += step_mass(st);
+          double incl = mine;
+#pragma unroll
+          for (int d = 1; d < 32; d <<= 1) {
+            const double o = shfl_up_double(incl, d);
+            if (lane >= d) incl += o;
+          }
+          if (lane == 31) sh.wtot[warp] = incl;
+          if (tid == 0) {
+            sh.win_g = 0x7fffffff;
+            sh.win_rank = -1;
+          }
+          __syncthreads();
+          if (tid == 0) {
+            double run = 0.0;
+            for (int w2 = 0; w2 < kWarps; ++w2) {
+              sh.wincl[w2] = run;  // mass before the warp's steps
+              run += sh.wtot[w2];
+            }
+            sh.dec.S = run;
+            sh.target = sh.u_smp * run;
+          }
+          __syncthreads();
+          const double target = sh.target;
+          double before = sh.wincl[warp] + (incl - mine);
+          int first = 0x7fffffff, last = -1;
+          double first_base = 0.0, first_m = 0.0, last_base = 0.0, last_m = 0.0;
+          for (int st = lo; st < hi; ++st) {
+            const double m = step_mass(st);
+            if (m > 0.0) {
+              last = st;
+              last_base = before;
+              last_m = m;
+              if (first == 0x7fffffff && before + m >= target) {
+                first = st;
+                first_base = before;
+                first_m = m;
+              }
+            }
+            before += m;
+          }
+          if (first != 0x7fffffff) atomicMin(&sh.win_g, first);
+          if (last >= 0) atomicMax(&sh.win_rank, last);  // rounding corner: the last step with mass
+          __syncthreads();
+          const int wfirst = sh.win_g, wlast = sh.win_rank;
+          __syncthreads();
+          if (wfirst != 0x7fffffff) {
+            if (first == wfirst) {
+              sh.base = first_base;
+              sh.srun[0][0] = first_m;
+            }
+            one_step = wfirst;
+          } else if (wlast >= 0 && sh.dec.S > 0.0) {
+            if (last == wlast) {
+              sh.base = last_base;
+              sh.srun[0][0] = last_m;
+            }
+            one_step = wlast;
+          }
+          if (tid == 0) sh.win_g = (one_step >= 0) ? 0 : -1;
+        } else {
+          for (int g = tid; g < G; g += kThreads) sh.gw[g] = __ldcg(&p.wtotg[static_cast<size_t>(uidx) * G + g]);
+          __syncthreads();
+          if (tid == 0) pick_run(sh.gw, G);
         }
-        __syncthreads();
-        if (tid == 0) pick_run(sh.gw, G);
         __syncthreads();
         // the residual mass S (Eq. 7: 1 - alpha) is reported wherever it was computed
         if (tid == 0 && p.diag) p.diag[static_cast<long long>(uidx) * 4 + 3] = is_bonus ? __int_as_float(0x7fc00000) : static_cast<float>(sh.dec.S);
         if (sh.win_g >= 0) {
           if (emit && warp == 0) {
             const int g = sh.win_g;
-            const int sb = static_cast<int>(static_cast<long long>(g) * p.nsteps / G);
-            const int se = static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
+            // one-sweep stage: the run is the one step found above, its mass the only running total
+            const int sb = (STAGE == 3) ? one_step : static_cast<int>(static_cast<long long>(g) * p.nsteps / G);
+            const int se = (STAGE == 3) ? one_step + 1 : static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
             const int gsz = run_gsz(se - sb, kRecG);
-            const double* rec = p.srung + (static_cast<size_t>(b) * G + g) * kRecG;
-            if (STAGE == 3) {
-              // masses of the run's groups from their channel sums, then running totals as the walk expects them
-              const int ngrp = (se - sb + gsz - 1) / gsz;
-              double m = 0.0;
-              if (lane < ngrp)
-                m = fmax(0.0, __dadd_rn(__dmul_rn(sh.chan_c[0], __ldcg(rec + lane)),
-                                        __dmul_rn(sh.chan_c[1], __ldcg(p.srungB + (static_cast<size_t>(b) * G + g) * kRecG + lane))));
-#pragma unroll
-              for (int d = 1; d < 32; d <<= 1) {
-                const double o = shfl_up_double(m, d);
-                if (lane >= d) m += o;
-              }
-              if (lane < kRecG) sh.srun[0][lane] = m;
-              __syncwarp();
-              rec = &sh.srun[0][0];
-            }
+            const double* rec = (STAGE == 3) ? &sh.srun[0][0] : p.srung + (static_cast<size_t>(b) * G + g) * kRecG;
             const int token = walk(sb, se, gsz, sh.base, rec, sh.target, is_bonus);
             if (lane == 0) {
               p.out_tokens[uidx] = token;  // the row's token at its first rejection, or the bonus
@@ -2586,6 +2629,7 @@ thread_local std::string g_create_error;
 struct cos_verify_ctx {
   cos_verify_config cfg;
   int parts;            // blocks per unit in the drawing stages
+  int parts_one;        // the same in the one-sweep drawing stage
   int max_clusters[5];  // resident clusters for cluster sizes 1, 2, 4, 8, 16 (0 = not available)
   int dense_blocks;     // resident blocks of the four-per-multiprocessor build of stage 0 (0 = there is none)
   int sm_count;
@@ -2601,8 +2645,7 @@ struct cos_verify_ctx {
   double* d_zpart;
   double* d_wtotg;
   double* d_srung;
-  double* d_wtotgB;  // second channel of the two above, for the one-sweep drawing stage
-  double* d_srungB;
+  double* d_srungB;  // second channel of d_srung, for the one-sweep drawing stage
   int* d_part_arrivals;
   // optional per-stage timing (cos_verify_set_stage_timing)
   bool timing;
@@ -2724,6 +2767,22 @@ int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
   return parts;
 }
 
+// Blocks per unit in the one-sweep drawing stage.  One wave when that fills the device well (at least three
+// quarters of its block slots); otherwise several times more blocks than slots, so that the device hands them
+// out as slots come free: with one block per unit and between one and two units per multiprocessor some
+// multiprocessors would carry twice the work of others.  At least four steps per warp.
+int choose_parts_one(const cos_verify_config& c, int rows, int sm_count) {
+  const int one_wave = choose_parts(c, rows, sm_count);
+  const long long slots = 2LL * sm_count;
+  const long long blocks = static_cast<long long>(rows) * one_wave;
+  if (blocks <= slots && 4 * blocks >= 3 * slots) return one_wave;
+  const int E = entries_per_vec(c.dtype);
+  const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
+  int parts = one_wave;
+  while (parts < 8 && static_cast<long long>(rows) * parts < 3 * slots && nsteps / (2 * parts * kWarps) >= 4) parts <<= 1;
+  return parts;
+}
+
 int log2i(int c) { return c >= 16 ? 4 : (c >= 8 ? 3 : (c >= 4 ? 2 : (c >= 2 ? 1 : 0))); }
 
 // Stage 0 streams best with one block per unit (long contiguous reads, no cluster barrier);
@@ -2782,7 +2841,7 @@ cudaError_t prepare_kernels(int dtype, int mode, int cluster_size) {
   cudaError_t e = cudaSuccess;
   for (int st = 2; draws && st <= 3 && e == cudaSuccess; ++st)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, st)),
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, stage_smem(st));
   if (e == cudaSuccess && cluster_size > 8)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, 0)),
                              cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
@@ -2837,6 +2896,8 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   }
   ctx->sm_count = prop.multiProcessorCount;
   ctx->parts = choose_parts(*config, config->max_batch, ctx->sm_count);
+  ctx->parts_one = choose_parts_one(*config, config->max_batch, ctx->sm_count);
+  const size_t pmax = static_cast<size_t>(ctx->parts > ctx->parts_one ? ctx->parts : ctx->parts_one);
   KernelFn fn = pick_kernel(config->dtype, mode_of(*config), 0);
   e = prepare_kernels(config->dtype, mode_of(*config), config->cluster_size);
   if (e != cudaSuccess) {
@@ -2882,11 +2943,12 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   ok = ok && cudaMalloc(&ctx->d_job_count, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_jobs, (rows * P + rows) * sizeof(int2)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_ustats, rows * P * sizeof(UnitStats)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->d_zpart, rows * P * ctx->parts * 8 * sizeof(double)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->d_wtotg, rows * P * ctx->parts * kWarps * sizeof(double)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->d_srung, rows * ctx->parts * kWarps * kRecG * sizeof(double)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->d_wtotgB, rows * P * ctx->parts * kWarps * sizeof(double)) == cudaSuccess;
-  ok = ok && cudaMalloc(&ctx->d_srungB, rows * ctx->parts * kWarps * kRecG * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_zpart, rows * P * pmax * 8 * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_wtotg, rows * P * pmax * kWarps * sizeof(double)) == cudaSuccess;
+  const size_t steps = (static_cast<size_t>(config->vocab) + 32 * entries_per_vec(config->dtype) - 1) / (32 * entries_per_vec(config->dtype));
+  const size_t rec_per_row = steps > pmax * kWarps * kRecG ? steps : pmax * kWarps * kRecG;  // one record per step, or per group of a run
+  ok = ok && cudaMalloc(&ctx->d_srung, rows * rec_per_row * sizeof(double)) == cudaSuccess;
+  ok = ok && cudaMalloc(&ctx->d_srungB, rows * rec_per_row * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_part_arrivals, rows * P * sizeof(int)) == cudaSuccess;
   if (ok && config->host_staging) {
     const size_t V = static_cast<size_t>(config->vocab);
@@ -3022,7 +3084,6 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   p.wtotg = ctx->d_wtotg;
   p.srung = ctx->d_srung;
   p.part_arrivals = ctx->d_part_arrivals;
-  p.wtotgB = ctx->d_wtotgB;
   p.srungB = ctx->d_srungB;
   p.parts = ctx->parts;
   p.max_jobs = p.num_units + a->batch;
@@ -3057,6 +3118,8 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     // mixes two models: then one sweep does the work of stages 1 and 2.  The test hooks keep the two-stage form.
     const bool one_sweep = !all && (mode == kLogitSample || c.n == 2);
     if (one_sweep) {
+      p.parts = ctx->parts_one;
+      p.num_clusters = (most < cap ? most : cap) * p.parts;
       e = launch_stage(c.dtype, mode, 3, p, 1, stream, true);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stage)", e);
       if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
@@ -3195,7 +3258,6 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_zpart);
   cudaFree(ctx->d_wtotg);
   cudaFree(ctx->d_srung);
-  cudaFree(ctx->d_wtotgB);
   cudaFree(ctx->d_srungB);
   cudaFree(ctx->d_part_arrivals);
   for (int k = 0; k < 4; ++k)
