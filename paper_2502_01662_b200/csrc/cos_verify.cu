@@ -743,6 +743,11 @@ __device__ __noinline__ double big_token_mass(const KParams& p, const SoftPart* 
   return draw == kDrawR ? r64 : (draw == kDrawQ ? q64 : fmax(0.0, r64 - q64));
 }
 
+// 2^a and, when `in`, 2^b in fp64: the two channel terms of a big entry.  Out of line.
+__device__ __noinline__ double2 big_pair(double a, double b, bool in) {
+  return make_double2(exp2(a), in ? exp2(b) : 0.0);
+}
+
 // One-sweep drawing stage, a vector that holds a big entry (more than 2^-8 of a normaliser), done again
 // entry by entry from the stored logits: big entries in fp64 into the thread's slots `bigacc` ([0] Z_A,
 // [kThreads] Z_B, [2 kThreads] and [3 kThreads] the sums over entries with a positive mass), the others as the
@@ -1935,7 +1940,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         __syncthreads();
         // one vector of entries: channel arguments xa (proposer's or model 0's logits) and xb (model 1's or the
         // combined logits), `inb` = inside the plausibility mask (bit per entry)
-        auto eat = [&](const float (&xa)[E], const float (&xb)[E], unsigned inb, int e0) {
+        auto eat = [&](const float (&xa)[E], const float (&xb)[E], unsigned inb) -> bool {
           float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f, mA = 0.f, mB = 0.f;
 #pragma unroll
           for (int k = 0; k < E; ++k) {
@@ -1951,19 +1956,78 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             vaA += pos ? eA : 0.f;
             vaB += pos ? eB : 0.f;
           }
-          if (mA > btA || mB > btB) {
-            // rare: some entry of this vector is big; the vector is done again out of line, big entries in fp64
-            const float4 r = one_sweep_big_vector<DT, MODE>(p, sh.one, base, e0, pis, masked, thr, bigacc);
-            vzA = r.x;
-            vzB = r.y;
-            vaA = r.z;
-            vaB = r.w;
-            hasbig = true;
+          // rare: some entry of this vector is big; the caller does the vector again, big entries in fp64
+          if (mA > btA || mB > btB) return true;
+          zsA += vzA;
+          zsB += vzB;
+          aA += vaA;
+          aB += vaB;
+          return false;
+        };
+        // a vector with a big entry, entry by entry from the stored logits, out of line (ragged steps)
+        auto redo_from_memory = [&](int e0) {
+          const float4 r = one_sweep_big_vector<DT, MODE>(p, sh.one, base, e0, pis, masked, thr, bigacc);
+          zsA += r.x;
+          zsB += r.y;
+          aA += r.z;
+          aB += r.w;
+          hasbig = true;
+        };
+        // the same from the two vectors at hand (models beyond the second are read again, entry by entry)
+        auto redo = [&](const uint4& r0, const uint4& r1, int e0) {
+          float x0[E], x1[E];
+          Elem<DT>::unpack(r0, x0);
+          Elem<DT>::unpack(r1, x1);
+          float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f;
+#pragma unroll
+          for (int k = 0; k < E; ++k) {
+            float xa, xb;
+            bool in = true;
+            if (MODE == kEnsembleSample) {
+              xa = x0[k];
+              xb = x1[k];
+            } else {
+              xb = fmaf(p.w[0], x0[k], 0.f);
+              if (p.n >= 2) xb = fmaf(p.w[1], x1[k], xb);
+              for (int i = 2; i < p.n; ++i) xb = fmaf(p.w[i], Elem<DT>::load1(row_of(i), e0 + k), xb);
+              xa = (pis == 0) ? x0[k] : (pis == 1 ? x1[k] : Elem<DT>::load1(row_of(pis), e0 + k));
+              if (masked) {
+                const int mm = p.mask_model;
+                const float xm = (mm == 0) ? x0[k] : (mm == 1 ? x1[k] : Elem<DT>::load1(row_of(mm), e0 + k));
+                in = (xm >= thr);
+              }
+            }
+            const float eA = ex2_approx(fmaf(xa, p.cT, nrefA));
+            const float eB = in ? ex2_approx(fmaf(xb, p.cT, nrefB)) : 0.f;
+            if (eA > btA || eB > btB) {
+              double cb;
+              if (MODE == kEnsembleSample) {
+                cb = static_cast<double>(xb);
+              } else {
+                cb = fma(p.w64[0], static_cast<double>(x0[k]), 0.0);
+                if (p.n >= 2) cb = fma(p.w64[1], static_cast<double>(x1[k]), cb);
+                for (int i = 2; i < p.n; ++i) cb = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e0 + k)), cb);
+              }
+              const double2 d = big_pair(static_cast<double>(xa) * p.cT64 - drefA, cb * p.cT64 - drefB, in);
+              bigacc[0] += d.x;
+              bigacc[kThreads] += d.y;
+              if (ctA64 * d.x + ctB64 * d.y > 0.0) {
+                bigacc[2 * kThreads] += d.x;
+                bigacc[3 * kThreads] += d.y;
+              }
+            } else {
+              const bool pos = __fadd_rn(__fmul_rn(ctA, eA), __fmul_rn(ctB, eB)) > 0.f;
+              vzA += eA;
+              vzB += eB;
+              vaA += pos ? eA : 0.f;
+              vaB += pos ? eB : 0.f;
+            }
           }
           zsA += vzA;
           zsB += vzB;
           aA += vaA;
           aB += vaB;
+          hasbig = true;
         };
         // the channel arguments of one step from the lane's vectors (the first two models' fetched ahead)
         auto feed = [&](const uint4& r0, const uint4& r1, int s) {
@@ -1972,7 +2036,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             float xa[E], xb[E];
             Elem<DT>::unpack(r0, xa);
             Elem<DT>::unpack(r1, xb);
-            eat(xa, xb, 0xffffffffu, e0);
+            if (eat(xa, xb, 0xffffffffu)) redo(r0, r1, e0);
           } else {
             float cmb[E], vq[E];
             unsigned inb = 0u;
@@ -1992,7 +2056,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             take(0, r0);
             if (p.n >= 2) take(1, r1);
             for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(s * 32 + lane) * 16));
-            eat(vq, cmb, inb, e0);
+            if (eat(vq, cmb, inb)) redo(r0, r1, e0);
           }
         };
         const bool pair = (MODE == kEnsembleSample) || (p.n >= 2);
@@ -2019,7 +2083,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
               float xa[E], xb[E];
               load_chunk<DT>(row_of(0), e0, p.V, vec_ok, xa);
               load_chunk<DT>(row_of(1), e0, p.V, vec_ok, xb);
-              eat(xa, xb, 0xffffffffu, e0);
+              if (eat(xa, xb, 0xffffffffu)) redo_from_memory(e0);
             } else {
               float cmb[E], vq[E];
               unsigned inb = 0u;
@@ -2035,7 +2099,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
                   if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
                 }
               }
-              eat(vq, cmb, inb, e0);
+              if (eat(vq, cmb, inb)) redo_from_memory(e0);
             }
           }
           // the step's two sums over the warp
@@ -2767,19 +2831,16 @@ int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
   return parts;
 }
 
-// Blocks per unit in the one-sweep drawing stage.  One wave when that fills the device well (at least three
-// quarters of its block slots); otherwise several times more blocks than slots, so that the device hands them
-// out as slots come free: with one block per unit and between one and two units per multiprocessor some
-// multiprocessors would carry twice the work of others.  At least four steps per warp.
+// Blocks per unit in the one-sweep drawing stage.  Where a block still has enough to do (eight steps per
+// warp), several times more blocks than the device holds at once, so that it hands them out as slots come
+// free: one wave of whole units leaves some multiprocessors with twice the work of others.  Small units
+// stay at one wave: their blocks are bound by latency, not by throughput.
 int choose_parts_one(const cos_verify_config& c, int rows, int sm_count) {
-  const int one_wave = choose_parts(c, rows, sm_count);
   const long long slots = 2LL * sm_count;
-  const long long blocks = static_cast<long long>(rows) * one_wave;
-  if (blocks <= slots && 4 * blocks >= 3 * slots) return one_wave;
   const int E = entries_per_vec(c.dtype);
   const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
-  int parts = one_wave;
-  while (parts < 8 && static_cast<long long>(rows) * parts < 3 * slots && nsteps / (2 * parts * kWarps) >= 4) parts <<= 1;
+  int parts = choose_parts(c, rows, sm_count);
+  while (parts < 8 && static_cast<long long>(rows) * parts < 3 * slots && nsteps / (2 * parts * kWarps) >= 8) parts <<= 1;
   return parts;
 }
 
