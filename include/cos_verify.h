@@ -135,7 +135,8 @@ typedef struct {
   int32_t threads_per_block;
   int32_t max_clusters;      /* clusters that can be resident at once on the device                   */
   int32_t sm_count;
-  int32_t launches_per_run;  /* kernels cos_verify_run enqueues per call (3 when T > 0, else 1)        */
+  int32_t launches_per_run;  /* kernels an ordinary cos_verify_run enqueues: 1 at T = 0; at T > 0, 2 for  */
+                             /* logit-level combines and two-model ensembles, 3 otherwise             */
   int32_t reserved[3];
 } cos_verify_info;
 

@@ -13,9 +13,14 @@
 //   stage 1  listed units only: the normalisers again, terms above 2^-8 of a normaliser in fp64;
 //   stage 2  listed units only: token masses max(0, r - q) (or the law of the bonus token), every warp on
 //            a contiguous run of the vocabulary so that prefix order is token order, fp64 running totals;
-//            the last block of a unit to finish locates u * S and walks to the token.
+//            the last block of a unit to finish locates u * S and walks to the token;
+//   stage 3  stages 1 and 2 in one sweep, for logit-level combines and two-model ensembles: there a mass is
+//            k_A e_A / Z_A + k_B e_B / Z_B clipped at zero, linear in 1/Z_A and 1/Z_B over the tokens where
+//            it is positive; that set is decided with stage 0's normalisers, the sweep records the two sums
+//            of every step (256 or 128 consecutive tokens) next to the refined normalisers, and the last
+//            block of a unit turns the sums into masses, finds the step by a prefix and walks it.
 // Units are handed out from a global counter.  Between blocks there are only fences and arrival counters;
-// the three launches of a run order the stages.  Waits exist only inside a block of the barrier-free form,
+// the launches of a run (stage 0, then 3 or 1 and 2) order the stages.  Waits exist only inside a block of the barrier-free form,
 // and they are bounded: a wait that gave up marks every row with COS_ROW_FAULT and the block leaves.
 // At T = 0 stage 0 is the whole run.
 
@@ -308,6 +313,10 @@ struct OneSweep {  // constants of the one-sweep drawing stage, for its out-of-l
   double ctA64, ctB64, drefA, drefB;
 };
 
+struct Shared;
+__device__ __forceinline__ OneSweep& one_sweep_consts(Shared& sh);
+__device__ __forceinline__ double* one_sweep_coef(Shared& sh);
+
 struct Shared {
   Xchg x[2];
   FreeRun fr;
@@ -316,7 +325,8 @@ struct Shared {
   double wtot[kWarps];        // this block's per-warp totals of sweep 2
   double wincl[kWarps];       // their running sum
   double srun[kWarps][kRec];  // a warp's running total after each group of steps
-  double gw[kMaxParts * kWarps];  // locating the token: mass of every warp run of the unit
+  double gw[kMaxParts * kWarps];  // locating the token: mass of every warp run of the unit (the one-sweep stage,
+                                  // which has no runs, keeps its constants here: see one_sweep_consts)
   int win_g;
   SoftPart fsoft[kMaxSlots];  // merged over the cluster
   ArgPart farg[kMaxSlots];
@@ -332,10 +342,14 @@ struct Shared {
   int next_local, next;
   float thr32;  // plausibility threshold rounded up to fp32
   float big_thr[kMaxSlots];  // sweep 2: terms above this share of a normaliser are redone in fp64
-  double chan_c[2];          // one-sweep drawing stage: exact coefficients of the two channel sums in a mass
-  OneSweep one;
   float ldraft[COS_MAX_MODELS];  // the n logits at the draft token, fetched before sweep 1
 };
+
+// The one-sweep drawing stage never fills gw[]; its constants and the two exact coefficients of the channel
+// sums live there, so that the layout of Shared is the same for every stage.
+static_assert(sizeof(OneSweep) <= 16 * sizeof(double), "OneSweep must fit in front of the coefficients");
+__device__ __forceinline__ OneSweep& one_sweep_consts(Shared& sh) { return *reinterpret_cast<OneSweep*>(&sh.gw[0]); }
+__device__ __forceinline__ double* one_sweep_coef(Shared& sh) { return &sh.gw[16]; }
 
 // lane accumulator of a softmax normaliser in the base-2 domain: s = sum 2^(v*c - ref)
 struct LaneSoft {
@@ -1925,7 +1939,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         for (int q = 0; q < 4; ++q) bigacc[q * kThreads] = 0.0;
         bool hasbig = false;
         if (tid == 0) {
-          OneSweep& c = sh.one;
+          OneSweep& c = one_sweep_consts(sh);
           c.ctA = ctA;
           c.ctB = ctB;
           c.nrefA = nrefA;
@@ -1966,7 +1980,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         };
         // a vector with a big entry, entry by entry from the stored logits, out of line (ragged steps)
         auto redo_from_memory = [&](int e0) {
-          const float4 r = one_sweep_big_vector<DT, MODE>(p, sh.one, base, e0, pis, masked, thr, bigacc);
+          const float4 r = one_sweep_big_vector<DT, MODE>(p, one_sweep_consts(sh), base, e0, pis, masked, thr, bigacc);
           zsA += r.x;
           zsB += r.y;
           aA += r.z;
@@ -2167,12 +2181,12 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             double z = 0.0;
             for (int q = 0; q < p.parts; ++q) z += __ldcg(&p.zpart[(static_cast<size_t>(uidx) * p.parts + q) * 8 + tid]);
             sh.fsoft[tid].s = z;
-            sh.chan_c[tid] = (tid == 0 ? kA : kB) / z;
+            one_sweep_coef(sh)[tid] = (tid == 0 ? kA : kB) / z;
           }
           __syncthreads();
         }
       }
-      if (STAGE == 2 || do_locate) {
+      if (STAGE != 3 || do_locate) {
       if (MODE == kEnsembleSample && tid < p.n) {
         // r - q = sum_i (w_i/Z_i - [i = proposer]/Z_i) e_i, and r = sum_i (w_i/Z_i) e_i
         const double a = p.w64[tid] / sh.fsoft[tid].s;
@@ -2558,7 +2572,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           const double* ra = p.srung + static_cast<size_t>(b) * p.nsteps;
           const double* rb = p.srungB + static_cast<size_t>(b) * p.nsteps;
           auto step_mass = [&](int st) {
-            return fmax(0.0, __dadd_rn(__dmul_rn(sh.chan_c[0], __ldcg(ra + st)), __dmul_rn(sh.chan_c[1], __ldcg(rb + st))));
+            return fmax(0.0, __dadd_rn(__dmul_rn(one_sweep_coef(sh)[0], __ldcg(ra + st)), __dmul_rn(one_sweep_coef(sh)[1], __ldcg(rb + st))));
           };
           double mine = 0.0;
           for (int st = lo; st < hi; ++st) mine += step_mass(st);
@@ -3301,8 +3315,15 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
   info->threads_per_block = kThreads;
   info->max_clusters = ctx->max_clusters[log2i(info->cluster_size)];
   info->sm_count = ctx->sm_count;
-  info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? 3 : 1;
+  {
+    // ordinary runs (no test hook): one launch at T = 0; else stage 0 and the one-sweep drawing stage where two
+    // channel sums describe a mass, stages 0, 1 and 2 otherwise
+    const int mode = mode_of(ctx->cfg);
+    const bool one_sweep = (mode == kLogitSample) || (mode == kEnsembleSample && ctx->cfg.n == 2);
+    info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? (one_sweep ? 2 : 3) : 1;
+  }
   info->reserved[0] = ctx->parts;
+  info->reserved[1] = ctx->parts_one;
   return COS_OK;
 }
 
