@@ -30,7 +30,7 @@ from paper_2502_01662_b200.binding import COS_RUN_EARLY_EXIT  # noqa: E402
 
 HEADLINE = "cfg3"
 # dram read + write bytes of one stage-0 launch from the ncu capture summarised under profiles/
-TRAFFIC_BYTES = {"cfg3": 355656448}
+TRAFFIC_BYTES = {"cfg3": 355332096}
 FALLBACK_HBM_GBS = 6650.0
 L2_BYTES = 126 * 1024 * 1024
 

@@ -53,6 +53,39 @@ def test_small_cases_match_oracle(w):
         assert np.array_equal(plain[k], gpu[k]), k
 
 
+# The one-sweep drawing stage with more than two models at logit level: the first two models' vectors come from
+# registers, the others are read in the sweep (and again, entry by entry, for a vector that holds a big term);
+# with the plausibility mask on the third model; unaligned rows (scalar loads throughout); sharp distributions
+# (low temperature) so that big terms are common.
+LOGIT_N = [
+    synth.Workload("logit3", 3, synth.COMBINE_LOGIT_LINEAR, (1.2, -0.4, 0.2), 0.9, 6, 3, 20011, "bf16", "gauss",
+                   sigma=3.0, rho=0.7, proposer_rule="cycle"),
+    synth.Workload("logit3_masked", 3, synth.COMBINE_LOGIT_LINEAR, (1.0, -0.3, 0.3), 0.6, 6, 3, 20480, "bf16", "gauss",
+                   sigma=3.0, rho=0.7, proposer_rule="cycle", mask_model=2, mask_alpha=0.05),
+    synth.Workload("logit4_f32_unaligned", 4, synth.COMBINE_LOGIT_LINEAR, (0.9, 0.3, -0.1, -0.1), 0.5, 4, 2, 4099, "f32",
+                   "gauss", sigma=2.5, rho=0.8, proposer_rule="cycle"),
+    synth.Workload("logit3_zipf_f16", 3, synth.COMBINE_LOGIT_LINEAR, (1.5, -0.25, -0.25), 0.7, 5, 4, 50000, "f16",
+                   "gumbel_zipf", rho=0.85, proposer_rule="cycle"),
+]
+
+
+@pytest.mark.parametrize("w", LOGIT_N, ids=[w.name for w in LOGIT_N])
+def test_one_sweep_drawing_stage_with_more_than_two_models(w):
+    inputs = synth.make_inputs(w, "cuda")
+    ref = helpers.run_oracle(w, inputs)
+    plain = helpers.run_gpu(w, inputs, diag=True)                       # stage 0, then the one-sweep stage
+    stats = helpers.check_parity(w, plain, ref)
+    assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
+    hooked = helpers.run_gpu(w, inputs, flags=COS_RUN_ALL_RESIDUALS)    # stages 0, 1 and 2
+    for k in ("accept_count", "out_tokens", "row_status"):
+        assert np.array_equal(plain[k], hooked[k]), k
+    for m in range(w.n):                                                # bonus token from a named model
+        refm = helpers.run_oracle(w, inputs, bonus_model=m)
+        gpum = helpers.run_gpu(w, inputs, diag=True, bonus_model=m)
+        statm = helpers.check_parity(w, gpum, refm)
+        assert statm["excused_accept"] + statm["excused_sample"] <= 1, statm
+
+
 # Both forms of the streaming stage at small sizes: cluster_size 1 runs it without block barriers (one block
 # per position, unless a plausibility mask is set), larger sizes split a position across a cluster.
 FORMS = [SMALL[i] for i in (1, 3, 4, 6, 7, 8)]
