@@ -1953,25 +1953,26 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         }
         __syncthreads();
         // one vector of entries: channel arguments xa (proposer's or model 0's logits) and xb (model 1's or the
-        // combined logits), `inb` = inside the plausibility mask (bit per entry)
-        auto eat = [&](const float (&xa)[E], const float (&xb)[E], unsigned inb) -> bool {
-          float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f, mA = 0.f, mB = 0.f;
+        // combined logits)
+        // (entries outside the mask arrive with xb = -inf: their e_B is zero)
+        const float nctA = -ctA;
+        auto eat = [&](const float (&xa)[E], const float (&xb)[E]) -> bool {
+          float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f;
 #pragma unroll
           for (int k = 0; k < E; ++k) {
             const float eA = ex2_approx(fmaf(xa[k], p.cT, nrefA));
-            float eB = ex2_approx(fmaf(xb[k], p.cT, nrefB));
-            if (MODE == kLogitSample && masked) eB = ((inb >> k) & 1u) ? eB : 0.f;
-            mA = fmaxf(mA, eA);
-            mB = fmaxf(mB, eB);
-            // products rounded one by one: where r and q coincide the sum is exactly zero, as in exact arithmetic
-            const bool pos = __fadd_rn(__fmul_rn(ctA, eA), __fmul_rn(ctB, eB)) > 0.f;
+            const float eB = ex2_approx(fmaf(xb[k], p.cT, nrefB));
+            // k_A e_A / Z_A + k_B e_B / Z_B > 0 with the products rounded one by one: where r and q coincide
+            // neither side exceeds the other, as in exact arithmetic
+            const float in_p = (__fmul_rn(ctB, eB) > __fmul_rn(nctA, eA)) ? 1.f : 0.f;
             vzA += eA;
             vzB += eB;
-            vaA += pos ? eA : 0.f;
-            vaB += pos ? eB : 0.f;
+            vaA = fmaf(in_p, eA, vaA);
+            vaB = fmaf(in_p, eB, vaB);
           }
-          // rare: some entry of this vector is big; the caller does the vector again, big entries in fp64
-          if (mA > btA || mB > btB) return true;
+          // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum
+          // big); the caller does the vector again, big entries in fp64
+          if (vzA > btA || vzB > btB) return true;
           zsA += vzA;
           zsB += vzB;
           aA += vaA;
@@ -2050,7 +2051,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             float xa[E], xb[E];
             Elem<DT>::unpack(r0, xa);
             Elem<DT>::unpack(r1, xb);
-            if (eat(xa, xb, 0xffffffffu)) redo(r0, r1, e0);
+            if (eat(xa, xb)) redo(r0, r1, e0);
           } else {
             float cmb[E], vq[E];
             unsigned inb = 0u;
@@ -2070,7 +2071,11 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             take(0, r0);
             if (p.n >= 2) take(1, r1);
             for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(s * 32 + lane) * 16));
-            if (eat(vq, cmb, inb)) redo(r0, r1, e0);
+            if (masked) {
+#pragma unroll
+              for (int k = 0; k < E; ++k) cmb[k] = ((inb >> k) & 1u) ? cmb[k] : -INFINITY;
+            }
+            if (eat(vq, cmb)) redo(r0, r1, e0);
           }
         };
         const bool pair = (MODE == kEnsembleSample) || (p.n >= 2);
@@ -2097,7 +2102,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
               float xa[E], xb[E];
               load_chunk<DT>(row_of(0), e0, p.V, vec_ok, xa);
               load_chunk<DT>(row_of(1), e0, p.V, vec_ok, xb);
-              if (eat(xa, xb, 0xffffffffu)) redo_from_memory(e0);
+              if (eat(xa, xb)) redo_from_memory(e0);
             } else {
               float cmb[E], vq[E];
               unsigned inb = 0u;
@@ -2113,7 +2118,11 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
                   if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
                 }
               }
-              if (eat(vq, cmb, inb)) redo_from_memory(e0);
+              if (masked) {
+#pragma unroll
+                for (int k = 0; k < E; ++k) cmb[k] = ((inb >> k) & 1u) ? cmb[k] : -INFINITY;
+              }
+              if (eat(vq, cmb)) redo_from_memory(e0);
             }
           }
           // the step's two sums over the warp
