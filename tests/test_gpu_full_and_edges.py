@@ -39,6 +39,28 @@ def _small(cfg, **kw):
     return C[cfg].scaled(**kw)
 
 
+@pytest.mark.parametrize("name,kw", [("cfg3", dict(batch=100, gamma=1)), ("cfg5", dict(batch=80, gamma=1)),
+                                     ("cfg3", dict(batch=300, vocab=40000, gamma=1))])
+def test_batches_that_do_not_fill_whole_waves(name, kw):
+    """Between one and two drawing positions per multiprocessor (and more than two): the one-sweep drawing
+    stage then splits a position over more blocks than the device holds at once; every row against the oracle
+    on a sample, the residual mass it reports against the oracle's."""
+    w = C[name].scaled(name=f"{name}_b{kw['batch']}", **kw)
+    inputs = synth.make_inputs(w, "cuda")
+    rows = sorted(np.random.default_rng(11).choice(w.batch, size=24, replace=False).tolist())
+    gpu = helpers.run_gpu(w, inputs, diag=True)
+    ref = helpers.run_oracle(w, inputs, rows=rows)
+    stats = helpers.check_parity(w, gpu, ref, rows=rows)
+    assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
+    acc = gpu["accept_count"]
+    assert np.all(gpu["out_tokens"][np.arange(w.batch), acc] >= 0)
+    again = helpers.run_gpu(w, inputs, diag=True)
+    for k in ("accept_count", "out_tokens", "row_status"):
+        assert np.array_equal(gpu[k], again[k]), k
+    del inputs
+    torch.cuda.empty_cache()
+
+
 def test_statistics_of_acceptance_match_eq7():
     """Mean accept flag against mean alpha_j = 1 - sum max(0, r - q) (Eq. 7) from the kernel's own S."""
     w = _small("cfg4", batch=32, vocab=12808, gamma=6, name="stat")
