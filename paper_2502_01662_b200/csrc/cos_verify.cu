@@ -1906,8 +1906,9 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         // (logit level), and (k_A, k_B) says what is drawn: max(0, r - q), r, or q.  The set of tokens with a
         // positive mass is decided with the normalisers stage 0 left (they are good to 1e-7, and a token whose sign
         // that could change carries no mass to speak of); over that set the mass is LINEAR in 1/Z_A and 1/Z_B,
-        // so this sweep only adds up e_A and e_B per group of steps, and with them the refined normalisers of
-        // stage 1.  Whoever locates the token turns the sums into masses once the normalisers are complete.
+        // so this sweep only adds up e_A and e_B over that set, step by step, and over everything for the refined
+        // normalisers of stage 1.  Whoever locates the token turns the sums into masses once the normalisers are
+        // complete.
         // Terms above 2^-8 of a normaliser go through fp64, as in stage 1.
         double kA, kB;
         if (MODE == kEnsembleSample) {
