@@ -604,7 +604,7 @@ __device__ void publish_unit(const KParams& p, int b, int j, int accept, int sta
     if (status) mine |= 1 << (6 + kPackedP + j);
   }
   const int prev = atomicAdd(&p.row_arrivals[b], mine);
-  if ((prev & 63) != p.P - 1) return;
+  if ((packed ? (prev & 63) : prev) != p.P - 1) return;  // longer rows keep a plain count in the word
   // last unit of the row: every other unit's result is visible after the fence below
   __threadfence();
   int a = p.gamma;

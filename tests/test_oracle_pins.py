@@ -583,3 +583,149 @@ def test_proposer_per_position_changes_q_position_by_position():
     b = orc.verify(logits, "f32", drafts, np.array([1]), cfg, 3, 1)
     for k in ("accept_count", "out_tokens", "row_status"):
         assert np.array_equal(a[k], b[k])
+
+
+# --------------------------------------------------------------------------------------
+# the disclosed boundary cases, and the conventions for q(x) = 0, an empty residual and
+# non-finite logits at T = 0
+# --------------------------------------------------------------------------------------
+def test_accept_boundary_flag_is_the_1e5_band_around_the_threshold():
+    """A position is a disclosed boundary case of the accept test iff |u - min(1, r(x)/q(x))| < 1e-5
+    (the band in which an fp32 evaluation of Eq. 6 may decide differently from an fp64 one)."""
+    V = 12
+    l = rng_logits(41, 2, V)
+    cfg = cfg_we(2, V, [0.5, 0.5])
+    p0, p1 = sp_softmax(l[0]), sp_softmax(l[1])
+    ratios = (0.5 * p0 + 0.5 * p1) / p0
+    d = int(np.argmin(np.abs(ratios - 0.8)))          # a draft whose threshold lies strictly inside (0, 1)
+    thr = float(ratios[d])
+    assert 0.55 < thr < 0.999
+    for delta, want in ((0.9e-5, True), (-0.9e-5, True), (1.1e-5, False), (-1.1e-5, False), (0.0, True)):
+        res = orc.verify_position(l, cfg, 0, d, thr + delta, 0.5)
+        assert res.boundary_accept is want, (delta, res.boundary_accept)
+        assert res.accept is (delta <= 0.0)
+    # a threshold clipped at 1: the band is measured from 1, not from the ratio
+    d1 = int(np.argmax(ratios))
+    assert ratios[d1] > 1.0 + 1e-3
+    assert orc.verify_position(l, cfg, 0, d1, 1.0 - 0.9e-5, 0.5).boundary_accept
+    assert not orc.verify_position(l, cfg, 0, d1, 1.0 - 1.1e-5, 0.5).boundary_accept
+
+
+def test_sample_boundary_flag_is_the_1e6_band_around_the_normalised_cdf_edges():
+    """A drawn token is a disclosed boundary case iff one of its two CDF edges, divided by the total
+    mass, lies within 1e-6 of the uniform."""
+    V = 9
+    l = rng_logits(43, 2, V)
+    cfg = cfg_we(2, V, [0.5, 0.5], gamma=0)
+    r = 0.5 * sp_softmax(l[0]) + 0.5 * sp_softmax(l[1])
+    cdf = np.cumsum(r) / np.sum(r)
+    k = 4
+    lo, hi = float(cdf[k - 1]), float(cdf[k])
+    assert hi - lo > 1e-4                             # the token is wide enough to sit strictly inside
+    for u, want_tok, want_flag in ((lo + 0.9e-6, k, True), (lo + 1.1e-6, k, False), (hi - 0.9e-6, k, True),
+                                   (hi - 1.1e-6, k, False), (lo - 0.9e-6, k - 1, True), (hi + 0.9e-6, k + 1, True),
+                                   (0.5 * (lo + hi), k, False)):
+        res = orc.verify_position(l, cfg, 0, None, 0.5, u)
+        assert res.cand == want_tok and res.boundary_sample is want_flag, (u, res.cand, res.boundary_sample)
+    # the residual's edges are normalised by the residual mass S, not by 1
+    cfg1 = cfg_we(2, V, [0.5, 0.5])
+    q = sp_softmax(l[0])
+    resid = np.maximum(0.0, r - q)
+    S = resid.sum()
+    assert 0.01 < S < 0.9
+    c = np.cumsum(resid) / S
+    kk = int(np.argmax(resid))
+    lo_r = float(c[kk - 1]) if kk > 0 else 0.0
+    assert orc.verify_position(l, cfg1, 0, 0, 0.99999, lo_r + 0.9e-6).boundary_sample
+    assert not orc.verify_position(l, cfg1, 0, 0, 0.99999, lo_r + 1.1e-6 + 1e-9).boundary_sample
+    assert orc.verify_position(l, cfg1, 0, 0, 0.99999, lo_r + 1.1e-6 + 1e-9).cand == kk
+
+
+def test_q_zero_convention_ratio_is_infinite_iff_r_is_positive():
+    """A convention of this build, not of the paper (which never meets q(x) = 0 because the draft is
+    drawn from q): the ratio is +inf when r(x) > 0 (accepted for every u) and 0 otherwise (rejected
+    for every u); the position reports Q_ZERO either way.  Reached at T = 0 with a draft that is
+    not the proposer's argmax."""
+    V = 6
+    l = np.zeros((2, V))
+    l[0, 1] = 3.0          # proposer's argmax: token 1
+    l[1, 4] = 3.0          # the other model's argmax: token 4
+    cfg = cfg_we(2, V, [0.5, 0.5], T=0.0)
+    for u in (lattice_u(0), lattice_u(LATTICE - 1)):
+        res = orc.verify_position(l, cfg, 0, 4, u, 0.5)              # r(4) = 0.5 > 0 = q(4)
+        assert res.status == orc.STATUS_Q_ZERO and res.ratio == math.inf and res.accept
+        res = orc.verify_position(l, cfg, 0, 2, u, 0.5)              # r(2) = 0 = q(2)
+        assert res.status & orc.STATUS_Q_ZERO and res.ratio == 0.0 and not res.accept
+        res = orc.verify_position(l, cfg, 0, 1, u, 0.5)              # q(1) = 1: the ordinary branch
+        assert res.status == 0 and res.ratio == 0.5
+    # whole row: the flag is reported, the accepted draft is kept
+    logits = np.broadcast_to(l[:, None, None, :], (2, 1, 2, V)).copy()
+    out = orc.verify(logits, "f64", [[4]], [0], cfg, 3, 0)
+    assert out["accept_count"][0] == 1 and out["row_status"][0] == orc.STATUS_Q_ZERO
+
+
+def test_empty_residual_convention_draws_from_r_and_reports_only_on_rejection():
+    """A convention of this build: when r and q coincide the residual max(0, r - q) has no mass; in exact
+    arithmetic no rejection can then happen, so the case only arises from a bad draft.  The token is
+    drawn from r with the same uniform and RESIDUAL_EMPTY is reported only if the position rejected."""
+    V = 7
+    l = rng_logits(47, 2, V)
+    l[1] = l[0]                                                       # both models identical: r == q exactly
+    cfg = cfg_we(2, V, [0.5, 0.5])
+    p = sp_softmax(l[0])
+    cdf = np.cumsum(p)
+    for u in (0.1, 0.5, 0.93):
+        k_want = int(np.searchsorted(cdf, u * cdf[-1]))
+        res = orc.verify_position(l, cfg, 0, V + 3, 0.5, u)           # a bad draft forces the rejection
+        assert res.status == (orc.STATUS_BAD_DRAFT | orc.STATUS_RESIDUAL_EMPTY)
+        assert res.S == 0.0 and res.cand == k_want
+        res = orc.verify_position(l, cfg, 0, 2, 0.5, u)               # accepted (ratio 1): candidate unused, no flag
+        assert res.accept and res.status == 0 and res.cand == k_want
+
+
+def test_greedy_with_non_finite_logits_reports_the_position():
+    """T = 0 reading: a NaN or +inf anywhere among the position's logits, or a model (or the masked
+    combination) without a finite maximum, makes the one-hot distributions undefined; the position
+    then counts as rejected with no candidate.  Logits of -inf are legal as long as a finite maximum remains."""
+    V = 8
+    base = rng_logits(53, 2, V)
+    we, ll = cfg_we(2, V, [0.5, 0.5], T=0.0), cfg_ll(2, V, [1.5, -0.5], T=0.0)
+    llm = cfg_ll(2, V, [1.0, -0.5], T=0.0, mask_model=0, alpha=0.1)
+    for cfg in (we, ll, llm):
+        for bad in (np.nan, np.inf):
+            for model in (0, 1):
+                l = base.copy()
+                l[model, 3] = bad
+                r, q, ok = orc.position_distributions(l, cfg, 0)
+                assert not ok and np.all(np.isnan(r))
+                res = orc.verify_position(l, cfg, 0, 2, 0.5, 0.5)
+                assert res.status == orc.STATUS_NONFINITE and not res.accept and res.cand == -1
+        l = base.copy()
+        k = int(np.argmin(base[0]))                                   # never an argmax, inside no mask
+        l[0, k] = -np.inf                                             # ruled-out token: still well defined
+        r, q, ok = orc.position_distributions(l, cfg, 0)
+        assert ok and q[int(np.argmax(l[0]))] == 1.0 and abs(r.sum() - 1.0) < 1e-15 and r[k] == 0.0
+        if cfg is not we:
+            l = base.copy()
+            l[1, 3] = -np.inf                                         # times a negative weight: a combined logit of +inf
+            assert not orc.position_distributions(l, cfg if cfg is ll else ll, 0)[2]
+        l = base.copy()
+        l[1, :] = -np.inf                                             # a model with no finite maximum
+        _, _, ok = orc.position_distributions(l, cfg, 0)
+        assert not ok
+    # logit level: +inf * negative weight would give -inf - harmless in a max - but the input itself is rejected
+    l = base.copy()
+    l[1, 5] = np.inf
+    assert not orc.position_distributions(l, ll, 0)[2]
+    # whole row at T = 0: the non-finite position stops the row and emits -1
+    logits = np.broadcast_to(base[:, None, None, :], (2, 1, 3, V)).copy()
+    logits[0, 0, 1, 0] = np.nan
+    d = int(np.argmax(base[0]))
+    out = orc.verify(logits, "f64", [[d, d]], [0], cfg_we(2, V, [0.5, 0.5], T=0.0, gamma=2), 5, 0)
+    # position 0: the draft is the proposer's argmax, so r(d) >= 0.5 = ratio and some uniforms accept
+    a = int(out["accept_count"][0])
+    assert a <= 1
+    if a == 1:
+        assert out["out_tokens"][0, 1] == -1 and out["row_status"][0] & orc.STATUS_NONFINITE
+    else:
+        assert out["row_status"][0] == 0
