@@ -1,16 +1,19 @@
 """Builds libcos_verify.so in-tree with nvcc for sm_100a (cross-compiles without a GPU)."""
 from __future__ import annotations
 
+import glob
 import os
 import shutil
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
-SRC = os.path.join(PKG_DIR, "csrc", "cos_verify.cu")
+CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG_DIR, "libcos_verify.so")
+OBJ_DIR = os.path.join(PKG_DIR, "_build")
 
 
 def nvcc_path() -> str:
@@ -20,28 +23,50 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found; set NVCC or put it on PATH")
 
 
+def sources():
+    return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
+
+
+def dependencies():
+    return sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + [os.path.join(INCLUDE, "cos_verify.h")]
+
+
 def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [SRC, os.path.join(INCLUDE, "cos_verify.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+    return any(os.path.getmtime(d) > t for d in dependencies())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the CUDA library if it is missing or older than its sources; return its path."""
-    if not force and not needs_build():
-        return LIB
+def _compile(src: str, verbose: bool):
+    obj = os.path.join(OBJ_DIR, os.path.splitext(os.path.basename(src))[0] + ".o")
     cmd = [
         nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-        "-Xptxas", "-v" if verbose else "-O3", "-shared", "-Xcompiler", "-fPIC",
-        "-I", INCLUDE, "-o", LIB, SRC, "-lcudart",
+        "-Xptxas", "-v" if verbose else "-O3", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC, "-c", "-o", obj, src,
     ]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + " ".join(cmd) + "\n" + res.stdout + res.stderr)
+    return obj, res.stdout + res.stderr
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the CUDA library if it is missing or older than its sources; return its path.
+    Every csrc/*.cu is one translation unit; they are compiled side by side and linked into one library."""
+    if not force and not needs_build():
+        return LIB
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    srcs = sources()
+    with ThreadPoolExecutor(max_workers=len(srcs)) as pool:
+        done = list(pool.map(lambda s: _compile(s, verbose), srcs))
+    cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC", "-o", LIB]
+    cmd += [obj for obj, _ in done] + ["-lcudart"]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("link failed:\n" + " ".join(cmd) + "\n" + res.stdout + res.stderr)
     if verbose:
-        sys.stderr.write(res.stdout + res.stderr)
+        for _, log in done:
+            sys.stderr.write(log)
     return LIB
 
 
