@@ -26,12 +26,15 @@ import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 from paper_2502_01662_b200 import synth  # noqa: E402
-from paper_2502_01662_b200.binding import COS_RUN_EARLY_EXIT  # noqa: E402
+from paper_2502_01662_b200.binding import COS_RUN_EARLY_EXIT  # noqa: E402,F401
 
 HEADLINE = "cfg3"
-# dram read + write bytes of one stage-0 launch from the ncu capture summarised under profiles/
-TRAFFIC_BYTES = {"cfg3": 355332096}
+# dram read + write bytes of one launch of the dominant kernel, as RECORDED in the ncu capture summarised under
+# profiles/ (kernel name -> bytes); reported only while the kernel that runs carries the same name
+TRAFFIC_BYTES = {}
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+REPORTED = ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg5_greedy")
 L2_BYTES = 126 * 1024 * 1024
 
 
@@ -240,29 +243,139 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def kernel_names(w, info):
+    """What the launches of one call are (for the roofline's stage list)."""
+    if info["one_launch"]:
+        return ["cos_fused_kernel (every position: sweep, accept tests, row scan, token draw)"]
+    names = ["cos_verify_kernel stage 0 (every position: sweep, accept tests, row scan)"]
+    if info["launches_per_run"] == 2:
+        names.append("cos_verify_kernel stage 3 (token draw, one sweep)")
+    elif info["launches_per_run"] == 3:
+        names += ["cos_verify_kernel stage 1 (normalisers of the drawing positions)",
+                  "cos_verify_kernel stage 2 (token masses and draw)"]
+    return names
+
+
+def measure_workload(w, dev, local, steps, warmup, row_base=0, sampler=None, cluster=0, stage_runs=30):
+    """One workload on one GPU: K back-to-back calls between two events, then the launches of a call one by one."""
+    peak, _ = measured_peak()
+    sets = rotating_inputs(w, dev, 0)
+    verifier = make_verifier(w, device=local, cluster_size=cluster)
+    info = verifier.info()
+    elapsed, outs = time_device(w, verifier, sets, steps, warmup, row_base, sampler)
+    verifier.set_stage_timing(True)
+    acc = None
+    touts = verifier._alloc_outs(w.batch, w.gamma + 1, w.vocab, dev, False, False)
+    for k in range(stage_runs + 5):
+        s_ = sets[k % len(sets)]
+        verifier.run(s_["logits"], s_["drafts"], s_["proposer"], s_["seed"], s_["offset"] + k, row_base=row_base, outs=touts)
+        ms = verifier.stage_ms()
+        if k >= 5:
+            acc = ms if acc is None else [a_ + b_ for a_, b_ in zip(acc, ms)]
+    stage_us = [1e3 * a_ / stage_runs for a_ in acc]
+    verifier.set_stage_timing(False)
+    verifier.close()
+    nbytes = w.positions * w.bytes_per_position
+    per_call = elapsed / steps
+    stages = []
+    for name, us in zip(kernel_names(w, info), stage_us):
+        # every launch is charged the whole call's algorithmic bytes only if it reads them: the first one does
+        gbps = nbytes / (us * 1e-6) / 1e9 if not stages else None
+        stages.append({"kernel": name, "us": us, "GBps": gbps, "frac": (gbps / peak) if gbps else None})
+    res = {"us_per_call": 1e6 * per_call, "positions_per_s": w.positions / per_call, "GBps": nbytes / per_call / 1e9,
+           "frac": nbytes / per_call / 1e9 / peak, "frac_of_nominal_8TBps": nbytes / per_call / 1e9 / NOMINAL_HBM_GBS,
+           "bytes_per_call": nbytes, "launches_per_call": info["launches_per_run"], "stages": stages,
+           "buffers": len(sets), "one_launch": info["one_launch"]}
+    return res, elapsed, outs, info, sets
+
+
+def sustained_small_calls(w, dev, local, calls=256, contexts=8):
+    """Many independent calls of a small workload on distinct buffers, spread over several contexts and streams,
+    so that calls overlap on the device: the time per call once launch latency is hidden."""
+    sets = rotating_inputs(w, dev, 0)
+    vs = [make_verifier(w, device=local) for _ in range(contexts)]
+    streams = [torch.cuda.Stream(device=dev) for _ in range(contexts)]
+    outs = [v._alloc_outs(w.batch, w.gamma + 1, w.vocab, dev, False, False) for v in vs]
+    def go(n, base):
+        for k in range(n):
+            c = k % contexts
+            s_ = sets[(base + k) % len(sets)]
+            vs[c].run(s_["logits"], s_["drafts"], s_["proposer"], s_["seed"], s_["offset"] + base + k, outs=outs[c],
+                      stream=streams[c])
+    torch.cuda.synchronize(dev)
+    go(2 * contexts, 0)
+    torch.cuda.synchronize(dev)
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(torch.cuda.current_stream(dev))
+    for st in streams:
+        st.wait_stream(torch.cuda.current_stream(dev))
+    go(calls, 1000)
+    for st in streams:
+        torch.cuda.current_stream(dev).wait_stream(st)
+    t1.record(torch.cuda.current_stream(dev))
+    torch.cuda.synchronize(dev)
+    for v in vs:
+        v.close()
+    sec = t0.elapsed_time(t1) / 1e3 / calls
+    nbytes = w.positions * w.bytes_per_position
+    return {"us_per_call_sustained": 1e6 * sec, "positions_per_s_sustained": w.positions / sec,
+            "GBps_sustained": nbytes / sec / 1e9, "contexts": contexts, "calls": calls, "buffers": len(sets)}
+
+
+def ceilings(dev):
+    """Read-only and read-plus-exponential streaming ceilings of this device (library micro-kernels)."""
+    from paper_2502_01662_b200.binding import measure_ceiling
+    buf = (torch.randn(512 * 1024 * 1024, device=dev, dtype=torch.float32) * 3.0).to(torch.bfloat16)   # 1 GiB
+    out = {"read_ceiling_GBps": measure_ceiling(0, buf), "ex2_ceiling_GBps": measure_ceiling(1, buf),
+           "bytes": buf.numel() * 2, "what": "128-bit streaming loads over 1 GiB of bf16; ex2: one ex2.approx per entry"}
+    del buf
+    return out
+
+
+def self_launch(args):
+    """`--gpus N` without a launcher around us: start the N ranks here (one process per GPU)."""
+    import socket
+    with socket.socket() as s_:
+        s_.bind(("127.0.0.1", 0))
+        port = s_.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", default=HEADLINE, choices=sorted(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cluster", type=int, default=0, help="thread blocks per position (0 = library default)")
-    ap.add_argument("--all-configs", action="store_true", help="also time the other workloads (short loops)")
+    ap.add_argument("--headline-only", action="store_true", help="skip the per-workload table and the ceilings")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="gloo: launcher self-test on CPU (no verification is timed; see tests/test_bench_launcher.py)")
     args = ap.parse_args()
     w = synth.CONFIGS[args.config]
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        self_launch(args)
     if args.impl == "reference":
         run_reference(args, w)
         return
     if args.warmup < 3:
         args.warmup = 3
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.backend == "gloo":
+        launcher_self_test(args, world, rank)
+        return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
@@ -273,36 +386,20 @@ def main():
     # each rank verifies its own shard of rows (the whole workload per rank: weak scaling);
     # rows are independent, so there is no collective on the data path
     row_base = rank * w.batch
-    sets = rotating_inputs(w, dev, rank)
-    verifier = make_verifier(w, device=local, cluster_size=args.cluster)
-    info = verifier.info()
     sampler = ClockSampler(local) if rank == 0 else None
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize(dev)
-    elapsed, outs = time_device(w, verifier, sets, args.steps, args.warmup, row_base, sampler)
+    head, elapsed, outs, info, sets = measure_workload(w, dev, local, args.steps, args.warmup, row_base, sampler,
+                                                       cluster=args.cluster)
     if dist is not None:
         t = torch.tensor([elapsed], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         elapsed = float(t.item())
         dist.barrier()
-    # the dominant kernel (stage 0: every position once) timed by itself: CUDA events recorded by the
-    # library on the launching stream around each of its launches
-    stage_ms = None
-    verifier.set_stage_timing(True)
-    acc = None
-    B, P, V = w.batch, w.gamma + 1, w.vocab
-    touts = verifier._alloc_outs(B, P, V, dev, False, False)
-    for k in range(60):
-        s_ = sets[k % len(sets)]
-        verifier.run(s_["logits"], s_["drafts"], s_["proposer"], s_["seed"], s_["offset"] + k, row_base=row_base, outs=touts)
-        ms = verifier.stage_ms()
-        if k >= 10:
-            acc = ms if acc is None else [a_ + b_ for a_, b_ in zip(acc, ms)]
-    stage_ms = [a_ / 50.0 for a_ in acc]
-    verifier.set_stage_timing(False)
-    verifier.close()
     mean_accept = float(outs["accept_count"].float().mean().item())
+    n_sets = len(sets)
+    del sets
 
     e2e = None
     if not args.skip_e2e:
@@ -315,43 +412,25 @@ def main():
         e2e = {"value": world * w.positions * e_steps / et, "unit": "positions/s", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": e_steps}
 
-    extra = None
-    if args.all_configs and world == 1:
-        extra = {}
-        for name, ww in synth.CONFIGS.items():
+    table, ceil = None, None
+    extra_launches = 0
+    if not args.headline_only and world == 1:
+        table = {}
+        for name in REPORTED:
+            ww = synth.CONFIGS[name]
             torch.cuda.empty_cache()
-            s2 = rotating_inputs(ww, dev, 0)
-            v2 = make_verifier(ww, device=local)
-            k2 = max(20, args.steps // 4)
-            t2, _ = time_device(ww, v2, s2, k2, 5, 0)
-            # a variant, not the metric: with the early-exit hint positions behind a reported rejection go unread
-            t3, _ = time_device(ww, v2, s2, k2, 5, 0, flags=COS_RUN_EARLY_EXIT)
-            # the same calls captured once in a CUDA graph and replayed (one call per input copy, 64 at most)
-            outs2 = v2._alloc_outs(ww.batch, ww.gamma + 1, ww.vocab, dev, False, False)
-            ncap = min(len(s2), 64)
-            graph = torch.cuda.CUDAGraph()
-            torch.cuda.synchronize(dev)
-            with torch.cuda.graph(graph):
-                for q in range(ncap):
-                    v2.run(s2[q]["logits"], s2[q]["drafts"], s2[q]["proposer"], s2[q]["seed"], s2[q]["offset"], outs=outs2)
-            reps = max(3, k2 // ncap)
-            for _ in range(2):
-                graph.replay()
-            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            ev0.record()
-            for _ in range(reps):
-                graph.replay()
-            ev1.record()
-            torch.cuda.synchronize(dev)
-            t4 = ev0.elapsed_time(ev1) / 1e3
-            del graph
-            extra[name] = {"us_per_call": 1e6 * t2 / k2, "positions_per_s": ww.positions * k2 / t2,
-                           "us_per_call_graph": 1e6 * t4 / (reps * ncap),
-                           "GBps": ww.positions * ww.bytes_per_position * k2 / t2 / 1e9,
-                           "cluster": v2.info()["cluster_size"], "buffers": len(s2),
-                           "us_per_call_early_exit": 1e6 * t3 / k2}
-            v2.close()
+            if name == w.name:
+                table[name] = {k: v for k, v in head.items()}
+                continue
+            k2 = 400 if ww.positions * ww.bytes_per_position < (1 << 30) else 100
+            res, _, _, inf2, s2 = measure_workload(ww, dev, local, k2, 5, stage_runs=20)
             del s2
+            extra_launches += (k2 + 5 + 25) * inf2["launches_per_run"]
+            if name == "cfg2":
+                res.update(sustained_small_calls(ww, dev, local))
+            table[name] = res
+        torch.cuda.empty_cache()
+        ceil = ceilings(dev)
 
     if rank != 0:
         if dist is not None:
@@ -359,40 +438,64 @@ def main():
         return
     peak, peak_kind = measured_peak()
     per_call = elapsed / args.steps
-    bytes_per_launch = w.positions * w.bytes_per_position
-    stage0 = stage_ms[0] / 1e3                      # seconds per launch of the dominant kernel
-    achieved = bytes_per_launch / stage0 / 1e9
-    per_launch = per_call
+    bytes_per_call = w.positions * w.bytes_per_position
+    achieved = bytes_per_call / per_call / 1e9
+    dominant = head["stages"][0]["kernel"].split(" ")[0]
     line = {
         "metric": "verified draft positions/sec", "value": world * w.positions * args.steps / elapsed,
         "unit": "positions/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1e3 * per_launch, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "ms_per_step": 1e3 * per_call, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "input_dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "n": w.n, "combine": "prob_ensemble" if w.combine == 0 else "logit_linear",
                    "T": w.temperature, "B": w.batch, "gamma": w.gamma, "V": w.vocab, "logits": w.dtype,
-                   "l2": "inputs larger than L2" if len(sets) == 1 else f"rotating over {len(sets)} input copies",
+                   "l2": "inputs larger than L2" if n_sets == 1 else f"rotating over {n_sets} input copies",
                    "cluster_size": info["cluster_size"], "resident_clusters": info["max_clusters"],
+                   "one_launch": info["one_launch"], "items_per_position": info["items_per_position"],
                    "mean_accept_count": mean_accept},
+        # the WHOLE call: algorithmic bytes of the batch over the time of all launches of a call
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": TRAFFIC_BYTES.get(w.name), "peak_kind": peak_kind, "bytes_per_launch": bytes_per_launch,
-                     "kernel": "cos_verify_kernel, stage 0 (every position: sweep, accept tests, row scan)",
-                     "launch_us": [1e3 * m for m in stage_ms],
-                     "whole_call": {"achieved": bytes_per_launch / per_call / 1e9,
-                                    "frac": bytes_per_launch / per_call / 1e9 / peak}},
+                     "traffic": TRAFFIC_BYTES.get(dominant), "peak_kind": peak_kind, "bytes_per_launch": bytes_per_call,
+                     "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS, "kernel": head["stages"][0]["kernel"],
+                     "launches_per_call": head["launches_per_call"], "stages": head["stages"]},
         "gpu_launches": args.steps * info["launches_per_run"],
         "clocks": sampler.summary() if sampler else None,
     }
     if e2e:
         line["e2e"] = e2e
-    if extra:
-        line["all_configs"] = extra
+    if table:
+        line["configs"] = table
+    if ceil:
+        line["ceilings"] = ceil
     if not args.skip_cpu:
-        v, rows, dt, passes = oracle_sample(w)
-        line["cpu_baseline"] = {"value": v, "unit": "positions/s", "cores": 1, "kind": "oracle",
-                                "sample": f"first {rows} rows x {w.gamma + 1} positions of {w.name}, {passes} pass(es), {dt:.1f} s"}
+        line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def cpu_baseline(w):
+    """The oracle, as it stands, on this machine's host cores: on one core, on a bounded sample of the workload."""
+    v, rows, dt, passes = oracle_sample(w)
+    return {"value": v, "unit": "positions/s", "cores": 1, "box_cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"first {rows} rows x {w.gamma + 1} positions of {w.name}, {passes} pass(es), {dt:.1f} s"}
+
+
+def launcher_self_test(args, world, rank):
+    """CPU check of the multi-rank plumbing (no GPU, no verification): ranks meet, each times a stand-in step,
+    the maximum over ranks is taken, rank 0 prints the line with n_gpus = world size."""
+    import torch.distributed as dist
+    dist.init_process_group("gloo")
+    dist.barrier()
+    t0 = time.perf_counter()
+    time.sleep(0.01 * (rank + 1))            # rank r "works" for (r + 1) * 10 ms
+    elapsed = time.perf_counter() - t0
+    t = torch.tensor([elapsed], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": "launcher self-test", "n_gpus": world, "max_elapsed_s": float(t.item()),
+                          "own_elapsed_s": elapsed, "backend": "gloo", "gpu_launches": 0}))
+    dist.destroy_process_group()
 
 
 if __name__ == "__main__":

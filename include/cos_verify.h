@@ -135,9 +135,11 @@ typedef struct {
   int32_t threads_per_block;
   int32_t max_clusters;      /* clusters that can be resident at once on the device                   */
   int32_t sm_count;
-  int32_t launches_per_run;  /* kernels an ordinary cos_verify_run enqueues: 1 at T = 0; at T > 0, 2 for  */
-                             /* logit-level combines and two-model ensembles, 3 otherwise             */
-  int32_t reserved[3];
+  int32_t launches_per_run;  /* kernels an ordinary cos_verify_run enqueues: 1 at T = 0 and wherever the  */
+                             /* one-launch form covers the configuration (reserved[2] == 1); else 2   */
+                             /* for logit-level combines and two-model ensembles, 3 otherwise         */
+  int32_t reserved[3];       /* [0], [1]: work items per position when streaming / drawing; [2]: 1    */
+                             /* when an ordinary run is one launch                                    */
 } cos_verify_info;
 
 /*
@@ -217,6 +219,29 @@ cos_status cos_verify_run_static(const cos_verify_config* config, const cos_veri
  */
 cos_status cos_verify_set_stage_timing(cos_verify_ctx* ctx, int enable);
 cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, int32_t* count);
+
+/*
+ * Failure detection of the one-launch form of a run (sampling modes without mask or test hook): every wait
+ * inside the kernel is a bounded poll.  A block that sees no progress for `polls` polls (about 0.2 us each; the
+ * default of 2^20 is about a fifth of a second) sets COS_ROW_FAULT on every row and leaves; the kernel always
+ * terminates and the device stays usable.  `polls` must be at least 16.  `test_drop_report` != 0 is a test
+ * hook: one streaming warp of block 0 then never reports its first work item, so the waits of that block run
+ * out and the run ends with COS_ROW_FAULT; the context clears its scratch before its next run.
+ * The paper has no counterpart; this follows from running the whole step (Sec. 3.1-3.2) as one launch.
+ */
+cos_status cos_verify_set_wait_limit(cos_verify_ctx* ctx, uint32_t polls, int32_t test_drop_report);
+
+/*
+ * Measurement aid (the paper has no counterpart): the two ceilings the streaming pass is compared with, measured
+ * on the current device.  kind 0 reads `bytes` of `device_buf` once with 128-bit streaming loads; kind 1 does the
+ * same and evaluates one fast base-2 exponential per 16-bit entry, which is what a softmax normaliser (Sec. 3.1)
+ * costs per bf16 logit.  Same launch shape as the verification kernels.  `device_out` is scratch of at least
+ * 1024 floats per multiprocessor (`out_floats` says how many it holds).  Runs two untimed and `reps` timed
+ * launches on `cuda_stream`, waits for them, and returns the fastest in *best_ms.  `device_buf` must be 16-byte
+ * aligned; its contents only matter as numbers (any bf16 data will do).
+ */
+cos_status cos_verify_measure_ceiling(int32_t kind, const void* device_buf, uint64_t bytes, float* device_out,
+                                      uint64_t out_floats, int32_t reps, float* best_ms, void* cuda_stream);
 
 /* Launch geometry chosen at creation. */
 cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info);

@@ -32,7 +32,7 @@ _STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR
 
 EXPORTS = ("cos_verify_create", "cos_verify_run", "cos_verify_run_host", "cos_verify_get_info",
            "cos_verify_destroy", "cos_verify_last_error", "cos_verify_set_stage_timing", "cos_verify_get_stage_ms",
-           "cos_verify_run_static")
+           "cos_verify_run_static", "cos_verify_set_wait_limit", "cos_verify_measure_ceiling")
 
 
 class CosVerifyError(RuntimeError):
@@ -92,6 +92,12 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.cos_verify_set_stage_timing.restype = ctypes.c_int
     lib.cos_verify_get_stage_ms.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.cos_verify_get_stage_ms.restype = ctypes.c_int
+    lib.cos_verify_set_wait_limit.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_int32]
+    lib.cos_verify_set_wait_limit.restype = ctypes.c_int
+    lib.cos_verify_measure_ceiling.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p,
+                                               ctypes.c_uint64, ctypes.c_int32, ctypes.POINTER(ctypes.c_float),
+                                               ctypes.c_void_p]
+    lib.cos_verify_measure_ceiling.restype = ctypes.c_int
     lib.cos_verify_destroy.argtypes = [ctypes.c_void_p]
     lib.cos_verify_destroy.restype = ctypes.c_int
     lib.cos_verify_last_error.argtypes = [ctypes.c_void_p]
@@ -146,8 +152,11 @@ class CosVerifier:
     def info(self) -> dict:
         inf = cos_verify_info()
         self._check(self._lib.cos_verify_get_info(self._ctx, ctypes.byref(inf)))
-        return {k: getattr(inf, k) for k in ("cluster_size", "threads_per_block", "max_clusters", "sm_count",
-                                             "launches_per_run")}
+        out = {k: getattr(inf, k) for k in ("cluster_size", "threads_per_block", "max_clusters", "sm_count",
+                                            "launches_per_run")}
+        out["items_per_position"], out["draw_items_per_position"] = inf.reserved[0], inf.reserved[1]
+        out["one_launch"] = bool(inf.reserved[2])
+        return out
 
     def _fill_args(self, logits, drafts, proposer, seed, offset, row_base, flags, outs,
                    bonus_model=None, offset_device=None) -> cos_verify_args:
@@ -183,6 +192,10 @@ class CosVerifier:
         a.bonus_model = bonus_model if (bonus_model is not None and bonus_model >= 0) else 0
         a.offset_device = offset_device.data_ptr() if offset_device is not None else None
         return a
+
+    def set_wait_limit(self, polls: int, test_drop_report: bool = False):
+        """cos_verify_set_wait_limit: bound of the kernel's internal polls (and the test hook that makes one run out)."""
+        self._check(self._lib.cos_verify_set_wait_limit(self._ctx, int(polls), int(bool(test_drop_report))))
 
     def set_stage_timing(self, enable: bool):
         """cos_verify_set_stage_timing: record events around every launch of later runs."""
@@ -274,6 +287,24 @@ class CosVerifier:
 
     def __exit__(self, *exc):
         self.close()
+
+
+def measure_ceiling(kind: int, buf, reps: int = 10, stream=None) -> float:
+    """cos_verify_measure_ceiling: GB/s of a read-only streaming pass over the device tensor `buf` (kind 0), or of
+    the same pass with one fast exponential per 16-bit entry (kind 1)."""
+    import torch
+    lib = load_library()
+    out = torch.empty(1024 * torch.cuda.get_device_properties(buf.device).multi_processor_count, dtype=torch.float32,
+                      device=buf.device)
+    ms = ctypes.c_float(0.0)
+    nbytes = buf.numel() * buf.element_size()
+    s = torch.cuda.current_stream(buf.device) if stream is None else stream
+    with torch.cuda.device(buf.device):
+        st = lib.cos_verify_measure_ceiling(kind, buf.data_ptr(), nbytes, out.data_ptr(), out.numel(), reps,
+                                            ctypes.byref(ms), ctypes.c_void_p(s.cuda_stream))
+    if st != COS_OK:
+        raise CosVerifyError(st, "cos_verify_measure_ceiling")
+    return nbytes / (ms.value * 1e-3) / 1e9
 
 
 def run_static(n: int, combine: int, weights: Sequence[float], temperature: float, gamma: int, vocab: int,

@@ -1,0 +1,1160 @@
+// CoS verification in ONE persistent launch (sampling modes, T > 0): combine (Eq. 3-5), accept test (Eq. 6),
+// first-rejection scan and the residual / bonus draw (Sec. 3.1-3.2) without a second pass over the batch.
+//
+// The run is cut into work items that any block can take:
+//   streaming item  one chunk (a contiguous range of steps, ~128 KB) of the n logit rows of one (row, position):
+//                   per-model softmax statistics of the chunk.  The block that completes the last chunk of a
+//                   position merges the chunks in order, takes the accept test and publishes the position.
+//   drawing item    one chunk of the one position of a row that must emit a token (its first rejection, or the
+//                   bonus position): per step (32 lanes x one 16-byte vector) the channel sums over the tokens
+//                   with a positive mass, plus the refined normalisers.  The block that completes the last chunk
+//                   turns the sums into masses, finds the step by a prefix and walks it to the token.
+// Streaming items come from a counter in row-major order; a row is settled as soon as every position up to its
+// first rejection has been published (rows resolve from the front), and its drawing items then go to a queue
+// that blocks look at before they take the next streaming item, while the position's logits are still in L2.
+//
+// A block is fifteen streaming warps and one service warp.  Streaming warps run from item to item without
+// block barriers and leave their partial sums in a ring of four slots in shared memory; the service warp fetches
+// items one ahead, merges the partials, talks to the other blocks (fences, arrival counters, the queue) and does
+// all serial work (decision, row scan, locating a token), so none of it sits on the streaming warps' path.
+// No block depends on a particular other block: any item can be taken by any block, and a block with nothing to
+// do polls the queue until every position is published and every row has its token.  All polls are bounded.
+
+#include "cos_fused.h"
+
+using namespace cosv;
+
+namespace {
+
+constexpr int kFT = 512;          // threads per block
+constexpr int kSW = 15;           // streaming warps
+constexpr int kST = kSW * 32;     // streaming threads
+constexpr int kRing = 4;          // items a block may have open
+constexpr int kCh = 4;            // channels of a drawing sweep (ensembles of up to four models; logit level: two)
+constexpr int kItemStream = 0, kItemDraw = 1, kItemExit = 3;
+constexpr int kCtrNext = 0, kCtrEvents = 1, kCtrHead = 2, kCtrTail = 3, kCtrGone = 4, kCtrFault = 5;
+
+struct FParams {
+  KParams k;
+  FusedPlan plan;
+  FusedScratch s;
+  int num_items;          // streaming items of this run
+  int nvec;               // 16-byte vectors per logit row
+  unsigned total_events;  // positions to publish + rows to settle
+  unsigned poll_limit;
+  int debug_drop;
+};
+
+struct ItemCtx {
+  int kind, b, j, chunk;
+  int pis;          // model whose distribution is q (valid index)
+  int lo, hi;       // streaming: vectors [lo, hi) of every row; drawing: steps [lo, hi)
+  int dkind;        // drawing: what the token is drawn from
+  float ct[kCh], nref[kCh], bt[kCh];
+  double ct64[kCh], dref[kCh];
+};
+
+struct FShared {
+  int tag[kRing];       // seq + 1 once ctx[seq & 3] is valid
+  int arrive[kRing];    // streaming warps that have finished the item of that slot
+  int started;          // number of items some warp has begun
+  int fault;
+  ItemCtx ctx[kRing];
+  SoftPart part[kRing][kSW][kCh];
+};
+
+__device__ __forceinline__ int vol_load(const int* p) { return *reinterpret_cast<const volatile int*>(p); }
+__device__ __forceinline__ unsigned vol_load(const unsigned* p) { return *reinterpret_cast<const volatile unsigned*>(p); }
+
+template <int DT>
+__device__ __forceinline__ uint4 ninf_vec() {
+  const unsigned w = (DT == COS_DTYPE_F32) ? 0xff800000u : (DT == COS_DTYPE_BF16 ? 0xff80ff80u : 0xfc00fc00u);
+  return make_uint4(w, w, w, w);
+}
+
+__device__ __forceinline__ const char* unit_base(const KParams& p, int b, int j, int eb) {
+  return reinterpret_cast<const char*>(p.logits) + (static_cast<long long>(b) * p.s_row + static_cast<long long>(j) * p.s_pos) * eb;
+}
+
+// coefficient of channel i in the mass that is drawn from: max(0, r - q), r, or q
+template <int MODE>
+__device__ __forceinline__ double channel_k(const KParams& p, int i, int pis, int dkind) {
+  if (MODE == kEnsembleSample) {
+    const double sel = (i == pis) ? 1.0 : 0.0;
+    return dkind == kDrawResidual ? p.w64[i] - sel : (dkind == kDrawQ ? sel : p.w64[i]);
+  }
+  if (i == 0) return dkind == kDrawResidual ? -1.0 : (dkind == kDrawQ ? 1.0 : 0.0);
+  return dkind == kDrawQ ? 0.0 : 1.0;
+}
+
+// ------------------------------------------------------------------------------------
+// streaming warps
+// ------------------------------------------------------------------------------------
+template <int DT, int MODE>
+__device__ __forceinline__ void stream_item(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
+  const KParams& p = fp.k;
+  const int lane = stid & 31;
+  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
+  Slice sl;
+  sl.v_lo = it.lo;
+  sl.v_hi = it.hi;
+  sl.e_lo = sl.e_hi = 0;
+  if (MODE == kEnsembleSample) {
+    for (int i = 0; i < p.n; ++i) {
+      LaneSoft acc = soft_slice<DT, kST>(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, sl, stid, p.cT);
+      warp_merge_soft(acc, &part[i], lane);
+    }
+  } else {
+    LaneSoft accq, accc;
+    logit_soft_slice<DT, kST>(p, base, sl, stid, it.pis, false, -INFINITY, accq, accc);
+    warp_merge_soft(accq, &part[0], lane);
+    warp_merge_soft(accc, &part[1], lane);
+  }
+}
+
+// A vector of a drawing sweep that holds a big entry (more than 2^-8 of a normaliser), done again entry by entry from
+// the stored logits: big entries in fp64 into the thread's slots (`bigacc[q * kST]`: q < NCH the normalisers,
+// NCH <= q < 2 NCH the step sums), the others as the sweep does them, returned in zs / as.  Rare; out of line.
+template <int DT, int MODE, int NCH>
+__device__ __noinline__ void draw_big_vector(const KParams& p, const ItemCtx& c, const char* base, int e0, double* bigacc,
+                                             float* zs, float* as) {
+  constexpr int E = Elem<DT>::E;
+  for (int k = 0; k < E; ++k) {
+    const int e = e0 + k;
+    if (e >= p.V) break;
+    float x[NCH];
+    double x64[NCH];
+    if (MODE == kEnsembleSample) {
+      for (int i = 0; i < NCH; ++i) {
+        x[i] = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
+        x64[i] = static_cast<double>(x[i]);
+      }
+    } else {
+      float xb = 0.f, xa = 0.f;
+      double cb = 0.0;
+      for (int i = 0; i < p.n; ++i) {
+        const float v = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
+        xb = fmaf(p.w[i], v, xb);
+        cb = fma(p.w64[i], static_cast<double>(v), cb);
+        if (i == c.pis) xa = v;
+      }
+      x[0] = xa;
+      x[1] = xb;
+      x64[0] = static_cast<double>(xa);
+      x64[1] = cb;
+    }
+    float ee[NCH];
+    bool big = false;
+    for (int i = 0; i < NCH; ++i) {
+      ee[i] = ex2_approx(fmaf(x[i], p.cT, c.nref[i]));
+      big |= ee[i] > c.bt[i];
+    }
+    if (big) {
+      double d[NCH], tot = 0.0;
+      for (int i = 0; i < NCH; ++i) {
+        d[i] = exp2(x64[i] * p.cT64 - c.dref[i]);
+        tot += c.ct64[i] * d[i];
+      }
+      for (int i = 0; i < NCH; ++i) {
+        bigacc[i * kST] += d[i];
+        if (tot > 0.0) bigacc[(NCH + i) * kST] += d[i];
+      }
+    } else {
+      float acc = 0.f;
+      for (int i = 0; i < NCH; ++i) acc = __fadd_rn(acc, __fmul_rn(c.ct[i], ee[i]));
+      const bool pos = acc > 0.f;
+      for (int i = 0; i < NCH; ++i) {
+        zs[i] += ee[i];
+        as[i] += pos ? ee[i] : 0.f;
+      }
+    }
+  }
+}
+
+// One chunk of a drawing sweep.  A token's mass is sum_i k_i e_i / Z_i clipped at zero, with the channels i the
+// models (ensemble) or the proposer's and the combined logits (logit level), e_i = 2^(arg_i - ref_i).  Which tokens
+// have a positive mass is decided with the normalisers of the streaming pass (products rounded one by one, so that
+// r == q gives exactly zero); over those tokens the mass is linear in the 1/Z_i, so the sweep records, per step,
+// the sums of e_i over them, and adds up the refined normalisers (terms above 2^-8 of one in fp64).
+template <int DT, int MODE, int NCH>
+__device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid, double* bigacc) {
+  constexpr int E = Elem<DT>::E;
+  const KParams& p = fp.k;
+  const int lane = stid & 31, warp = stid >> 5;
+  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
+  const long long row_step = p.s_model * Elem<DT>::bytes;
+  float ct[NCH], nref[NCH], bt[NCH];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    ct[i] = it.ct[i];
+    nref[i] = it.nref[i];
+    bt[i] = it.bt[i];
+  }
+  float zs[NCH], as[NCH];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) zs[i] = as[i] = 0.f;
+#pragma unroll
+  for (int q = 0; q < 2 * NCH; ++q) bigacc[q * kST] = 0.0;
+  bool zbig = false;
+  constexpr int NL = (MODE == kEnsembleSample) ? NCH : 2;  // rows fetched one step ahead
+  const int nl = (MODE == kEnsembleSample) ? NCH : (p.n < 2 ? p.n : 2);
+  uint4 nx[NL];
+  auto fetch = [&](int s) {
+    const int v = s * 32 + lane;
+#pragma unroll
+    for (int i = 0; i < NL; ++i)
+      nx[i] = (v < fp.nvec && i < nl) ? ldg_stream16(base + i * row_step + static_cast<long long>(v) * 16) : ninf_vec<DT>();
+  };
+  double* rec = fp.s.srec + static_cast<size_t>(it.b) * p.nsteps * NCH;
+  if (it.lo + warp < it.hi) fetch(it.lo + warp);
+  for (int s = it.lo + warp; s < it.hi; s += kSW) {
+    uint4 cur[NL];
+#pragma unroll
+    for (int i = 0; i < NL; ++i) cur[i] = nx[i];
+    if (s + kSW < it.hi) fetch(s + kSW);
+    const int v = s * 32 + lane;
+    float xc[NCH][E];  // channel arguments
+    if (MODE == kEnsembleSample) {
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) Elem<DT>::unpack(cur[i], xc[i]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < E; ++k) xc[1][k] = 0.f;
+      auto take = [&](int i, const uint4& raw) {
+        float x[E];
+        Elem<DT>::unpack(raw, x);
+        const float wi = p.w[i];
+#pragma unroll
+        for (int k = 0; k < E; ++k) {
+          xc[1][k] = fmaf(wi, x[k], xc[1][k]);
+          if (i == it.pis) xc[0][k] = x[k];
+        }
+      };
+      take(0, cur[0]);
+      if (p.n >= 2) take(1, cur[1]);
+      for (int i = 2; i < p.n; ++i)
+        take(i, v < fp.nvec ? ldg_stream16(base + i * row_step + static_cast<long long>(v) * 16) : ninf_vec<DT>());
+      if (v >= fp.nvec) {
+#pragma unroll
+        for (int k = 0; k < E; ++k) xc[0][k] = xc[1][k] = -INFINITY;
+      }
+    }
+    float vz[NCH], va[NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) vz[i] = va[i] = 0.f;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+      float e[NCH];
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) {
+        e[i] = ex2_approx(fmaf(xc[i][k], p.cT, nref[i]));
+        vz[i] += e[i];
+        acc = __fadd_rn(acc, __fmul_rn(ct[i], e[i]));
+      }
+      const float in_p = (acc > 0.f) ? 1.f : 0.f;
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) va[i] = fmaf(in_p, e[i], va[i]);
+    }
+    bool big = false;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) big |= vz[i] > bt[i];
+    // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum big)
+    if (big) {
+      float rz[NCH], ra[NCH];
+      for (int i = 0; i < NCH; ++i) rz[i] = ra[i] = 0.f;
+      draw_big_vector<DT, MODE, NCH>(p, it, base, v * E, bigacc, rz, ra);
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) {
+        zs[i] += rz[i];
+        as[i] = ra[i];
+      }
+      zbig = true;
+    } else {
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) {
+        zs[i] += vz[i];
+        as[i] = va[i];
+      }
+    }
+    // the step's sums over the warp
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) as[i] += __shfl_xor_sync(0xffffffffu, as[i], d);
+    }
+    double da[NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) da[i] = static_cast<double>(as[i]);
+    if (__any_sync(0xffffffffu, big)) {
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) {
+        double t = bigacc[(NCH + i) * kST];
+        bigacc[(NCH + i) * kST] = 0.0;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+        da[i] += t;
+      }
+    }
+    if (lane < NCH) {
+      double mine = da[0];
+#pragma unroll
+      for (int i = 1; i < NCH; ++i) mine = (lane == i) ? da[i] : mine;
+      __stcg(rec + static_cast<size_t>(s) * NCH + lane, mine);
+      __threadfence();
+    }
+  }
+  // this warp's share of the refined normalisers
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    double t = static_cast<double>(zs[i]) + (__any_sync(0xffffffffu, zbig) ? bigacc[i * kST] : 0.0);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+    if (lane == 0) {
+      part[i].s = t;
+      part[i].ref = 0.f;
+    }
+  }
+}
+
+template <int DT, int MODE, int NCH>
+__device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, double* bigacc_all) {
+  const int stid = threadIdx.x, lane = stid & 31, warp = stid >> 5;
+  double* bigacc = bigacc_all + stid;
+  for (int seq = 0;; ++seq) {
+    const int slot = seq & (kRing - 1);
+    // the service warp posts the item; it is normally there already (fetched one ahead)
+    int ok = 0;
+    if (lane == 0) {
+      // (bounded, but longer than the service warp's own patience: when nothing moves it is the one that gives up)
+      for (unsigned long long it = 0; it < 8ull * fp.poll_limit; ++it) {
+        if (vol_load(&sh.tag[slot]) == seq + 1) {
+          ok = 1;
+          break;
+        }
+        if (vol_load(&sh.fault)) break;
+        __nanosleep(100);
+      }
+      __threadfence_block();
+      if (ok) atomicMax(&sh.started, seq + 1);
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) return;
+    __syncwarp();
+    const ItemCtx& it = sh.ctx[slot];
+    if (it.kind == kItemExit) return;
+    if (it.kind == kItemStream)
+      stream_item<DT, MODE>(fp, it, &sh.part[slot][warp][0], stid);
+    else
+      draw_item<DT, MODE, NCH>(fp, it, &sh.part[slot][warp][0], stid, bigacc);
+    __syncwarp();
+    if (lane == 0) {
+      const bool drop = fp.debug_drop && blockIdx.x == 0 && warp == 0 && seq == 0;  // test hook: a report that never comes
+      __threadfence();  // a drawing item's step records are read by another block
+      if (!drop) atomicAdd(&sh.arrive[slot], 1);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------
+// service warp
+// ------------------------------------------------------------------------------------
+struct Unif {
+  double u_acc, u_smp;
+};
+__device__ __forceinline__ Unif position_uniforms(const KParams& p, int b, int j) {
+  unsigned rnd[4];
+  const unsigned long long grow = static_cast<unsigned long long>(p.row_base + b);
+  philox4x32_10(static_cast<unsigned>(grow), static_cast<unsigned>(j), offset_lo(p), offset_hi(p), p.seed_lo, p.seed_hi, rnd);
+  Unif u;
+  u.u_acc = word_to_uniform(rnd[0]);
+  u.u_smp = word_to_uniform(rnd[1]);
+  return u;
+}
+
+__device__ __forceinline__ SoftPart ldcg_part(const SoftPart* q) {
+  const int4 raw = __ldcg(reinterpret_cast<const int4*>(q));
+  SoftPart o;
+  o.s = __hiloint2double(raw.y, raw.x);
+  o.ref = __int_as_float(raw.z);
+  o.pad = 0;
+  return o;
+}
+__device__ __forceinline__ void stcg_part(SoftPart* q, const SoftPart& v) {
+  __stcg(reinterpret_cast<int4*>(q), make_int4(__double2loint(v.s), __double2hiint(v.s), __float_as_int(v.ref), 0));
+}
+
+__device__ __forceinline__ void add_events(const FParams& fp, unsigned n) {
+  __threadfence();
+  atomicAdd(&fp.s.ctr[kCtrEvents], n);
+}
+
+// one thread: the drawing items of row b go to the queue
+__device__ __forceinline__ void push_draw(const FParams& fp, int b) {
+  __threadfence();
+  const unsigned at = atomicAdd(&fp.s.ctr[kCtrTail], static_cast<unsigned>(fp.plan.dchunks));
+  for (int c = 0; c < fp.plan.dchunks; ++c) {
+    const int desc = (kItemDraw << 30) | (b << 8) | c;
+    if (at + c < static_cast<unsigned>(fp.plan.dq_cap)) atomicExch(&fp.s.dq[at + c], desc + 1);
+  }
+}
+
+// Publish a position (Sec. 3.1).  The row's 64-bit word holds four bits per position: published, "the row stops
+// here" (rejected, or the bonus position), "reported status bits", "a token can be drawn here".  Every position
+// adds its own bits once, so the value the atomic returns tells the publisher whether it was the one that settled
+// the row: every position up to the first stop is in.  That publisher writes the row's outputs and queues the
+// row's drawing items; positions behind the first stop are still verified but decide nothing.
+__device__ __forceinline__ void publish_position(const FParams& fp, int b, int j, int accept, int status, int drawable) {
+  const KParams& p = fp.k;
+  const bool stop = (!accept) || (j == p.gamma);
+  const unsigned long long nib = 1ull | (stop ? 2ull : 0ull) | (status ? 4ull : 0ull) | (drawable ? 8ull : 0ull);
+  const unsigned long long mine = nib << (4 * j);
+  __threadfence();
+  const unsigned long long prev = atomicAdd(&fp.s.row_word[b], mine);
+  const unsigned long long total = prev + mine;
+  const unsigned long long ones = 0x1111111111111111ull;
+  const unsigned long long rowmask = (p.P >= 16) ? ~0ull : ((1ull << (4 * p.P)) - 1ull);
+  auto settled = [&](unsigned long long w, int* first_stop) -> bool {
+    const unsigned long long stops = (w >> 1) & ones;
+    if (stops == 0ull) return false;
+    const int fs = (__ffsll(static_cast<long long>(stops)) - 1) >> 2;
+    const unsigned long long missing = ~w & ones & rowmask;
+    const int fm = missing ? ((__ffsll(static_cast<long long>(missing)) - 1) >> 2) : p.P;
+    *first_stop = fs;
+    return fs < fm;
+  };
+  int a = 0, a_prev = 0;
+  const bool now = settled(total, &a), before = settled(prev, &a_prev);
+  if ((total & ones & rowmask) == (ones & rowmask)) fp.s.row_word[b] = 0ull;  // the row's last position: clean for the next run
+  unsigned events = 1;
+  if (now && !before) {
+    __threadfence();
+    unsigned st = 0;
+    for (int k = 0; k <= a; ++k)
+      if ((total >> (4 * k + 2)) & 1ull) st |= static_cast<unsigned>(__ldcg(&p.unit_res[b * p.P + k]).y);
+    const bool can_draw = ((total >> (4 * a + 3)) & 1ull) != 0ull;
+    p.accept_count[b] = a;
+    int* o = p.out_tokens + static_cast<long long>(b) * p.P;
+    for (int k = 0; k < p.P; ++k) o[k] = (k < a) ? p.drafts[b * p.gamma + k] : -1;
+    p.row_status[b] = st;
+    if (p.bonus_prob != nullptr) p.bonus_prob[b] = __int_as_float(0x7fc00000);
+    if (can_draw) {
+      const int dkind = (a < p.gamma) ? kDrawResidual : (p.bonus_model >= 0 ? kDrawQ : kDrawR);
+      __stcg(&fp.s.row_draw[b], a | (dkind << 8));
+      push_draw(fp, b);
+    } else {
+      events += 1;  // nothing can be drawn (a non-finite position): the row is settled
+    }
+  }
+  add_events(fp, events);
+}
+
+// The last chunk of a position has arrived: merge the chunks in order, take the accept test in fp64 (Eq. 6) and
+// publish.  Whole warp; `own` (chunks == 1) are the block's merged statistics.
+template <int DT, int MODE>
+__device__ __forceinline__ void finish_position(const FParams& fp, int b, int j, int pi_raw, const SoftPart* own) {
+  const KParams& p = fp.k;
+  const int lane = threadIdx.x & 31;
+  const int ns = fp.plan.nslots, C = fp.plan.chunks;
+  const int uidx = b * p.P + j;
+  SoftPart fs[kCh > 2 ? kCh : 2];
+  for (int k = 0; k < ns; ++k) {
+    if (C == 1) {
+      fs[k] = own[k];
+    } else {
+      SoftPart in;
+      in.s = 0.0;
+      in.ref = -INFINITY;
+      if (lane < C) in = ldcg_part(&fp.s.chunk_part[(static_cast<size_t>(uidx) * C + lane) * ns + k]);
+      fs[k] = warp_reduce_soft(in.ref, in.s);
+    }
+  }
+  const bool is_bonus = (j == p.gamma);
+  const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
+  const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
+  const bool pi_ok = (pi_raw >= 0 && pi_raw < p.n);
+  const int pi = pi_raw;
+  const char* base = unit_base(p, b, j, Elem<DT>::bytes);
+  float ld = 0.f;
+  if (lane < p.n && !is_bonus && draft_ok) ld = Elem<DT>::load1(base + static_cast<long long>(lane) * p.s_model * Elem<DT>::bytes, draft);
+  const Unif un = position_uniforms(p, b, j);
+  const double kNaN = __longlong_as_double(0x7ff8000000000000LL);
+  const double kInf = __longlong_as_double(0x7ff0000000000000LL);
+  bool finite = pi_ok;
+  for (int k = 0; k < ns; ++k) finite = finite && isfinite(fs[k].ref) && isfinite(fs[k].s) && (fs[k].s > 0.0);
+  int accept = 0, status = 0;
+  double ratio = kNaN, r_d = kNaN, q_d = kNaN;
+  if (!finite) {
+    status |= COS_ROW_NONFINITE;
+  } else if (!is_bonus) {
+    if (draft_ok) {
+      double rr = 0.0, qq = 0.0;
+      if (MODE == kEnsembleSample) {
+        for (int i = 0; i < p.n; ++i) {
+          const double li = static_cast<double>(__shfl_sync(0xffffffffu, ld, i));
+          const double pd = exp2(li * p.cT64 - static_cast<double>(fs[i].ref)) / fs[i].s;
+          rr += p.w64[i] * pd;
+          if (i == pi) qq = pd;
+        }
+      } else {
+        double cd = 0.0, lq = 0.0;
+        for (int i = 0; i < p.n; ++i) {
+          const double li = static_cast<double>(__shfl_sync(0xffffffffu, ld, i));
+          cd = fma(p.w64[i], li, cd);
+          if (i == pi) lq = li;
+        }
+        rr = exp2(cd * p.cT64 - static_cast<double>(fs[1].ref)) / fs[1].s;
+        qq = exp2(lq * p.cT64 - static_cast<double>(fs[0].ref)) / fs[0].s;
+      }
+      r_d = rr;
+      q_d = qq;
+      if (qq > 0.0) {
+        ratio = rr / qq;
+      } else {
+        status |= COS_ROW_Q_ZERO;
+        ratio = (rr > 0.0) ? kInf : 0.0;
+      }
+      accept = (un.u_acc <= fmin(1.0, ratio)) ? 1 : 0;
+    } else {
+      status |= COS_ROW_BAD_DRAFT;
+    }
+  }
+  const int drawable = finite ? 1 : 0;
+  if (lane < ns) {
+    double sv = fs[0].s;
+    float rv = fs[0].ref;
+    for (int k = 1; k < ns; ++k) {
+      sv = (lane == k) ? fs[k].s : sv;
+      rv = (lane == k) ? fs[k].ref : rv;
+    }
+    __stcg(&p.ustats[uidx].s[lane], sv);
+    __stcg(&p.ustats[uidx].ref[lane], rv);
+    __threadfence();
+  }
+  __syncwarp();
+  if (lane == 0) {
+    if (p.diag) {
+      float* d = p.diag + static_cast<long long>(uidx) * 4;
+      d[0] = static_cast<float>(ratio);
+      d[1] = static_cast<float>(r_d);
+      d[2] = static_cast<float>(q_d);
+      d[3] = static_cast<float>(kNaN);
+    }
+    __stcg(&p.unit_res[uidx], make_int4(accept, status, -1, drawable));
+    publish_position(fp, b, j, accept, status, drawable);
+  }
+  __syncwarp();
+}
+
+// ---- locating the token of a row once its drawing sweep is complete -------------------------------------------
+struct WalkConst {
+  double zs[kCh];    // refined normalisers (ensemble: per model; logit level: proposer, combined)
+  float ref[kCh];    // reference exponents
+  float big_thr[kCh];
+  float a_resid[kCh], a_draw[kCh];  // ensemble: coefficient of e_i in r - q, and in the law a bonus token follows
+  float inv_zq, inv_zc;             // logit level
+  int pis;
+  bool draw_q;
+};
+
+// Mass of one big token in fp64 from the stored logits: r - q clipped at zero, r, or q.  Rare; out of line.
+template <int DT, int MODE>
+__device__ __noinline__ double big_token(const KParams& p, const WalkConst& w, const char* base, int e, int draw) {
+  if (e >= p.V) return 0.0;
+  double r64 = 0.0, q64 = 0.0;
+  float lv[COS_MAX_MODELS];
+  for (int i = 0; i < p.n; ++i) lv[i] = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
+  if (MODE == kEnsembleSample) {
+    for (int i = 0; i < p.n; ++i) {
+      const double pr = exp2(static_cast<double>(lv[i]) * p.cT64 - static_cast<double>(w.ref[i])) / w.zs[i];
+      r64 += p.w64[i] * pr;
+      if (i == w.pis) q64 = pr;
+    }
+  } else {
+    double cd = 0.0;
+    for (int i = 0; i < p.n; ++i) cd = fma(p.w64[i], static_cast<double>(lv[i]), cd);
+    r64 = exp2(cd * p.cT64 - static_cast<double>(w.ref[1])) / w.zs[1];
+    q64 = exp2(static_cast<double>(lv[w.pis]) * p.cT64 - static_cast<double>(w.ref[0])) / w.zs[0];
+  }
+  return draw == kDrawR ? r64 : (draw == kDrawQ ? q64 : fmax(0.0, r64 - q64));
+}
+
+// fp32 masses of the E tokens of one lane of a step (products rounded one by one, so that r == q cancels exactly);
+// tokens holding more than 2^-8 of a normaliser are flagged in `bigbits` and get mass 0 here.
+template <int DT, int MODE>
+__device__ __forceinline__ void token_masses(const KParams& p, const WalkConst& w, const char* base, int e0, bool use_r,
+                                             float (&mass32)[Elem<DT>::E], unsigned& bigbits) {
+  constexpr int E = Elem<DT>::E;
+  float acc[E];
+  bool anybig = false;
+  bigbits = 0u;
+#pragma unroll
+  for (int k = 0; k < E; ++k) acc[k] = 0.f;
+  if (MODE == kEnsembleSample) {
+    for (int i = 0; i < p.n; ++i) {
+      float v[E];
+      load_chunk<DT>(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e0, p.V, true, v);
+      const float co = use_r ? w.a_draw[i] : w.a_resid[i], rf = -w.ref[i];
+      float emax = 0.f;
+#pragma unroll
+      for (int k = 0; k < E; ++k) {
+        const float e = ex2_approx(fmaf(v[k], p.cT, rf));
+        emax = fmaxf(emax, e);
+        acc[k] = __fadd_rn(acc[k], __fmul_rn(co, e));
+        bigbits |= (e > w.big_thr[i]) ? (1u << k) : 0u;
+      }
+      anybig |= emax > w.big_thr[i];
+    }
+  } else {
+    float cmb[E], eq[E];
+#pragma unroll
+    for (int k = 0; k < E; ++k) cmb[k] = eq[k] = 0.f;
+    for (int i = 0; i < p.n; ++i) {
+      float v[E];
+      load_chunk<DT>(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e0, p.V, true, v);
+      const float wi = p.w[i];
+#pragma unroll
+      for (int k = 0; k < E; ++k) {
+        cmb[k] = fmaf(wi, v[k], cmb[k]);
+        if (i == w.pis) eq[k] = ex2_approx(fmaf(v[k], p.cT, -w.ref[0]));
+      }
+    }
+    const bool from_q = use_r && w.draw_q;
+    const float qco = use_r ? 0.f : w.inv_zq;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+      const bool in = (e0 + k < p.V);
+      const float ec = in ? ex2_approx(fmaf(cmb[k], p.cT, -w.ref[1])) : 0.f;
+      const float eqk = in ? eq[k] : 0.f;
+      const float rr = ec * w.inv_zc;
+      acc[k] = from_q ? __fmul_rn(eqk, w.inv_zq) : __fsub_rn(rr, __fmul_rn(eqk, qco));
+      const bool big = (ec > w.big_thr[1]) || (eqk > w.big_thr[0]);
+      bigbits |= big ? (1u << k) : 0u;
+      anybig |= big;
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < E; ++k) mass32[k] = ((bigbits >> k) & 1u) ? 0.f : fmaxf(0.f, acc[k]);
+  if (!anybig) bigbits = 0u;
+}
+
+// The token inside one step: `before` is the mass in front of the step.  An fp64 prefix over the lanes, then the
+// lane's tokens one by one.  Whole warp; returns the token (or the step's last token with mass).
+template <int DT, int MODE>
+__device__ __forceinline__ int walk_step(const KParams& p, const WalkConst& w, const char* base, int step, double before,
+                                         double target, bool use_r) {
+  constexpr int E = Elem<DT>::E;
+  const int lane = threadIdx.x & 31;
+  const int e0 = (step * 32 + lane) * E;
+  const int draw = use_r ? (w.draw_q ? kDrawQ : kDrawR) : kDrawResidual;
+  float mass32[E];
+  unsigned bigbits;
+  token_masses<DT, MODE>(p, w, base, e0, use_r, mass32, bigbits);
+  double m64[E];
+#pragma unroll
+  for (int k = 0; k < E; ++k) m64[k] = static_cast<double>(mass32[k]);
+  float ls = 0.f;
+#pragma unroll
+  for (int k = 0; k < E; ++k) ls += mass32[k];
+  double own = static_cast<double>(ls);
+  if (bigbits) {
+    for (int k = 0; k < E; ++k)
+      if (bigbits & (1u << k)) {
+        m64[k] = big_token<DT, MODE>(p, w, base, e0 + k, draw);
+        own += m64[k];
+      }
+  }
+  double inc = own;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const double o = shfl_up_double(inc, d);
+    if (lane >= d) inc += o;
+  }
+  double excl = shfl_up_double(inc, 1);
+  if (lane == 0) excl = 0.0;
+  const double incl = excl + own;
+  const bool hit = (own > 0.0) && (before + incl >= target);
+  const unsigned hits = __ballot_sync(0xffffffffu, hit);
+  const unsigned pos_lanes = __ballot_sync(0xffffffffu, own > 0.0);
+  if (hits == 0u && pos_lanes == 0u) return -1;
+  const int src = hits ? (__ffs(hits) - 1) : (31 - __clz(pos_lanes));
+  int found = -1;
+  if (lane == src) {
+    double part = 0.0;
+    int lastk = -1;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+      part += m64[k];
+      if (m64[k] > 0.0) {
+        lastk = k;
+        if (found < 0 && before + (excl + part) >= target) found = e0 + k;
+      }
+    }
+    if (found < 0) found = e0 + lastk;
+  }
+  return __shfl_sync(0xffffffffu, found, src);
+}
+
+// The drawing sweep of row b is complete.  Whole warp.
+template <int DT, int MODE, int NCH>
+__device__ __forceinline__ void locate_token(const FParams& fp, int b) {
+  const KParams& p = fp.k;
+  const int lane = threadIdx.x & 31;
+  const int rd = __ldcg(&fp.s.row_draw[b]);
+  const int j = rd & 0xff, dkind = rd >> 8;
+  const int uidx = b * p.P + j;
+  const bool is_bonus = (j == p.gamma);
+  const int pis = proposer_of(p, b, j);
+  const char* base = unit_base(p, b, j, Elem<DT>::bytes);
+  WalkConst w;
+  w.pis = pis;
+  w.draw_q = (dkind == kDrawQ);
+  double coef[NCH];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    double z = 0.0;
+    for (int c = 0; c < fp.plan.dchunks; ++c) z += __ldcg(&fp.s.dzpart[(static_cast<size_t>(b) * fp.plan.dchunks + c) * NCH + i]);
+    w.zs[i] = z;
+    w.ref[i] = __ldcg(&p.ustats[uidx].ref[i]);
+    w.big_thr[i] = static_cast<float>(__ldcg(&p.ustats[uidx].s[i]) * kBigShare);  // from the first estimate, as in the sweep
+    coef[i] = channel_k<MODE>(p, i, pis, dkind) / z;
+  }
+  if (MODE == kEnsembleSample) {
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+      const double a = p.w64[i] / w.zs[i];
+      const double sel = (i == pis) ? 1.0 / w.zs[i] : 0.0;
+      w.a_resid[i] = static_cast<float>(a - sel);
+      w.a_draw[i] = w.draw_q ? static_cast<float>(sel) : static_cast<float>(a);
+    }
+  } else {
+    w.inv_zq = static_cast<float>(1.0 / w.zs[0]);
+    w.inv_zc = static_cast<float>(1.0 / w.zs[1]);
+  }
+  // every step's channel sums turn into its mass (products rounded one by one: equal sums under opposite
+  // coefficients cancel exactly); lanes own consecutive steps, a prefix over the lanes gives S
+  const double* rec = fp.s.srec + static_cast<size_t>(b) * p.nsteps * NCH;
+  auto step_mass = [&](int st) {
+    double acc = __dmul_rn(coef[0], __ldcg(rec + static_cast<size_t>(st) * NCH));
+#pragma unroll
+    for (int i = 1; i < NCH; ++i) acc = __dadd_rn(acc, __dmul_rn(coef[i], __ldcg(rec + static_cast<size_t>(st) * NCH + i)));
+    return fmax(0.0, acc);
+  };
+  const int per = (p.nsteps + 31) / 32;
+  const int lo = lane * per, hi = (lo + per < p.nsteps) ? lo + per : p.nsteps;
+  double mine = 0.0;
+  for (int st = lo; st < hi; ++st) mine += step_mass(st);
+  double incl = mine;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const double o = shfl_up_double(incl, d);
+    if (lane >= d) incl += o;
+  }
+  const double S = shfl_double(incl, 31);
+  const Unif un = position_uniforms(p, b, j);
+  const double target = un.u_smp * S;
+  double before = incl - mine;
+  int first = 0x7fffffff, last = -1;
+  double first_base = 0.0, last_base = 0.0;
+  for (int st = lo; st < hi; ++st) {
+    const double m = step_mass(st);
+    if (m > 0.0) {
+      last = st;
+      last_base = before;
+      if (first == 0x7fffffff && before + m >= target) {
+        first = st;
+        first_base = before;
+      }
+    }
+    before += m;
+  }
+  int step = -1;
+  double step_base = 0.0;
+  const unsigned found = __ballot_sync(0xffffffffu, first != 0x7fffffff);
+  const unsigned have = __ballot_sync(0xffffffffu, last >= 0);
+  if (found) {
+    const int src = __ffs(found) - 1;
+    step = __shfl_sync(0xffffffffu, first, src);
+    step_base = shfl_double(first_base, src);
+  } else if (have && S > 0.0) {  // rounding corner: the last step with mass
+    const int src = 31 - __clz(have);
+    step = __shfl_sync(0xffffffffu, last, src);
+    step_base = shfl_double(last_base, src);
+  }
+  if (lane == 0 && p.diag && dkind == kDrawResidual)
+    p.diag[static_cast<long long>(uidx) * 4 + 3] = static_cast<float>(S);
+  if (step >= 0) {
+    const bool use_r = (dkind != kDrawResidual);
+    const int token = walk_step<DT, MODE>(p, w, base, step, step_base, target, use_r);
+    if (lane == 0) {
+      p.out_tokens[uidx] = token;
+      // Algorithm 2's Score returns the bonus token with its probability under the law it came from
+      if (is_bonus && p.bonus_prob != nullptr && token >= 0)
+        p.bonus_prob[b] = static_cast<float>(big_token<DT, MODE>(p, w, base, token, w.draw_q ? kDrawQ : kDrawR));
+      add_events(fp, 1);
+    }
+  } else if (dkind == kDrawResidual) {
+    // a token is needed although max(0, r - q) has no mass: the row draws from r instead, with the same uniform
+    if (lane == 0) {
+      atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_RESIDUAL_EMPTY));
+      __stcg(&fp.s.row_draw[b], j | (kDrawR << 8));
+      push_draw(fp, b);
+    }
+  } else {
+    if (lane == 0) add_events(fp, 1);  // nothing to draw from: the row keeps -1
+  }
+  __syncwarp();
+}
+
+// one thread: the next item of this block, or -1.  Drawing items first (their logits are still in L2).
+__device__ __forceinline__ int take_item(const FParams& fp, bool& static_left) {
+  unsigned h = vol_load(&fp.s.ctr[kCtrHead]);
+  for (int tries = 0; tries < 8; ++tries) {
+    if (h >= static_cast<unsigned>(fp.plan.dq_cap)) break;
+    const int v = vol_load(&fp.s.dq[h]);
+    if (v == 0) break;
+    const unsigned old = atomicCAS(&fp.s.ctr[kCtrHead], h, h + 1);
+    if (old == h) {
+      fp.s.dq[h] = 0;  // clean for the next run
+      __threadfence();
+      return v - 1;
+    }
+    h = old;
+  }
+  if (static_left) {
+    const unsigned t = atomicAdd(&fp.s.ctr[kCtrNext], 1u);
+    if (t < static_cast<unsigned>(fp.num_items)) {
+      const int unit = static_cast<int>(t) / fp.plan.chunks, c = static_cast<int>(t) % fp.plan.chunks;
+      return (kItemStream << 30) | (unit << 8) | c;
+    }
+    static_left = false;
+  }
+  return -1;
+}
+
+template <int MODE>
+__device__ __forceinline__ void fill_ctx(const FParams& fp, ItemCtx& cx, int desc) {
+  const KParams& p = fp.k;
+  const int lane = threadIdx.x & 31;
+  const int kind = (desc >> 30) & 3, id = (desc >> 8) & 0x3fffff, c = desc & 0xff;
+  if (kind == kItemStream) {
+    const int b = id / p.P, j = id % p.P;  // row-major: a row's positions come one after the other
+    if (lane == 0) {
+      cx.kind = kItemStream;
+      cx.b = b;
+      cx.j = j;
+      cx.chunk = c;
+      const int pi = proposer_of(p, b, j);
+      cx.dkind = pi;  // as given; checked when the position is decided
+      cx.pis = (pi >= 0 && pi < p.n) ? pi : 0;
+      const int lo = c * fp.plan.chunk_steps * 32, hi = lo + fp.plan.chunk_steps * 32;
+      cx.lo = lo;
+      cx.hi = hi < fp.nvec ? hi : fp.nvec;
+    }
+  } else {
+    const int b = id;
+    const int rd = __ldcg(&fp.s.row_draw[b]);
+    const int j = rd & 0xff, dkind = rd >> 8;
+    const int pis = proposer_of(p, b, j);
+    const int uidx = b * p.P + j;
+    if (lane == 0) {
+      cx.kind = kItemDraw;
+      cx.b = b;
+      cx.j = j;
+      cx.chunk = c;
+      cx.pis = pis;
+      cx.dkind = dkind;
+      const int lo = c * fp.plan.dchunk_steps, hi = lo + fp.plan.dchunk_steps;
+      cx.lo = lo;
+      cx.hi = hi < p.nsteps ? hi : p.nsteps;
+    }
+    if (lane < fp.plan.nch) {
+      const double z0 = __ldcg(&p.ustats[uidx].s[lane]);
+      const float ref = __ldcg(&p.ustats[uidx].ref[lane]);
+      const double c64 = channel_k<MODE>(p, lane, pis, dkind) / z0;  // with the first estimates: signs only
+      cx.ct64[lane] = c64;
+      cx.ct[lane] = static_cast<float>(c64);
+      cx.nref[lane] = -ref;
+      cx.dref[lane] = static_cast<double>(ref);
+      cx.bt[lane] = static_cast<float>(z0 * kBigShare);
+    }
+  }
+  __syncwarp();
+}
+
+template <int DT, int MODE, int NCH>
+__device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
+  const KParams& p = fp.k;
+  const int lane = threadIdx.x & 31;
+  int fetched = 0, processed = 0;
+  bool static_left = true;
+  unsigned idle = 0;
+  bool failed = false;
+  while (true) {
+    bool did = false;
+    // ---- fetch one item ahead of the fastest streaming warp
+    if (fetched < processed + kRing && fetched <= vol_load(&sh.started)) {
+      int desc = -1;
+      if (lane == 0) desc = take_item(fp, static_left);
+      desc = __shfl_sync(0xffffffffu, desc, 0);
+      static_left = __shfl_sync(0xffffffffu, static_left ? 1 : 0, 0) != 0;
+      if (desc >= 0) {
+        fill_ctx<MODE>(fp, sh.ctx[fetched & (kRing - 1)], desc);
+        if (lane == 0) {
+          __threadfence_block();
+          *reinterpret_cast<volatile int*>(&sh.tag[fetched & (kRing - 1)]) = fetched + 1;
+        }
+        ++fetched;
+        did = true;
+      } else if (processed == fetched) {
+        // nothing open here and nothing to take: done once every position is published and every row settled
+        unsigned ev = 0;
+        if (lane == 0) ev = vol_load(&fp.s.ctr[kCtrEvents]);
+        ev = __shfl_sync(0xffffffffu, ev, 0);
+        if (ev >= fp.total_events) break;
+      }
+    }
+    // ---- the oldest open item, once every streaming warp has reported it
+    if (processed < fetched) {
+      const int slot = processed & (kRing - 1);
+      int in = 0;
+      if (lane == 0) in = vol_load(&sh.arrive[slot]);
+      in = __shfl_sync(0xffffffffu, in, 0);
+      if (in == kSW) {
+        __threadfence_block();
+        const ItemCtx& cx = sh.ctx[slot];
+        const int b = cx.b, j = cx.j, c = cx.chunk;
+        if (cx.kind == kItemStream) {
+          const int ns = fp.plan.nslots, C = fp.plan.chunks;
+          const int uidx = b * p.P + j;
+          SoftPart merged[kCh > 2 ? kCh : 2];
+          for (int k = 0; k < ns; ++k) {
+            const float ref = (lane < kSW) ? sh.part[slot][lane][k].ref : -INFINITY;
+            const double s = (lane < kSW) ? sh.part[slot][lane][k].s : 0.0;
+            merged[k] = warp_reduce_soft(ref, s);
+          }
+          bool last = true;
+          if (C > 1) {
+            if (lane < ns) {
+              SoftPart mine = merged[0];
+              for (int k = 1; k < ns; ++k) mine = (lane == k) ? merged[k] : mine;
+              stcg_part(&fp.s.chunk_part[(static_cast<size_t>(uidx) * C + c) * ns + lane], mine);
+              __threadfence();
+            }
+            __syncwarp();
+            int prev = 0;
+            if (lane == 0) {
+              __threadfence();
+              prev = atomicAdd(&fp.s.unit_arrivals[uidx], 1);
+              if (prev == C - 1) {
+                fp.s.unit_arrivals[uidx] = 0;  // clean for the next run
+                __threadfence();
+              }
+            }
+            prev = __shfl_sync(0xffffffffu, prev, 0);
+            last = (prev == C - 1);
+          }
+          if (last) finish_position<DT, MODE>(fp, b, j, cx.dkind, merged);
+        } else {
+          // this block's share of the refined normalisers; the last chunk of the row locates the token
+          for (int i = 0; i < NCH; ++i) {
+            double t = (lane < kSW) ? sh.part[slot][lane][i].s : 0.0;
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+            if (lane == 0) __stcg(&fp.s.dzpart[(static_cast<size_t>(b) * fp.plan.dchunks + c) * NCH + i], t);
+          }
+          int prev = 0;
+          if (lane == 0) {
+            __threadfence();
+            prev = atomicAdd(&fp.s.draw_arrivals[b], 1);
+            if (prev == fp.plan.dchunks - 1) {
+              fp.s.draw_arrivals[b] = 0;
+              __threadfence();
+            }
+          }
+          prev = __shfl_sync(0xffffffffu, prev, 0);
+          if (prev == fp.plan.dchunks - 1) locate_token<DT, MODE, NCH>(fp, b);
+        }
+        if (lane == 0) {
+          *reinterpret_cast<volatile int*>(&sh.arrive[slot]) = 0;
+          __threadfence_block();
+        }
+        ++processed;
+        did = true;
+      }
+    }
+    if (did) {
+      idle = 0;
+    } else {
+      if (++idle > fp.poll_limit) {
+        failed = true;
+        break;
+      }
+      __nanosleep(processed < fetched ? 100 : 200);
+    }
+  }
+  if (failed) {
+    // no progress anywhere for the whole limit (a defect, never the data): mark every row, let everybody leave
+    if (lane == 0) {
+      *reinterpret_cast<volatile int*>(&sh.fault) = 1;
+      atomicExch(&fp.s.ctr[kCtrFault], 1u);
+    }
+    for (int b = lane; b < p.B; b += 32) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_FAULT));
+  }
+  // tell the streaming warps to leave
+  if (lane == 0) {
+    ItemCtx& cx = sh.ctx[fetched & (kRing - 1)];
+    cx.kind = kItemExit;
+    __threadfence_block();
+    *reinterpret_cast<volatile int*>(&sh.tag[fetched & (kRing - 1)]) = fetched + 1;
+    // the last block to leave puts the counters back: every run starts from the same state
+    __threadfence();
+    const unsigned gone = atomicAdd(&fp.s.ctr[kCtrGone], 1u);
+    if (gone == gridDim.x - 1) {
+      const bool faulted = vol_load(&fp.s.ctr[kCtrFault]) != 0u;
+      fp.s.ctr[kCtrNext] = 0u;
+      fp.s.ctr[kCtrEvents] = 0u;
+      fp.s.ctr[kCtrHead] = 0u;
+      fp.s.ctr[kCtrTail] = 0u;
+      fp.s.ctr[kCtrGone] = 0u;
+      fp.s.ctr[kCtrFault] = faulted ? 2u : 0u;  // 2: the scratch may be dirty; the host clears it before the next run
+      __threadfence();
+    }
+  }
+}
+
+template <int DT, int MODE, int NCH>
+__global__ void __launch_bounds__(kFT, 2) cos_fused_kernel(const __grid_constant__ FParams fp) {
+  __shared__ FShared sh;
+  extern __shared__ double bigacc[];  // [2 * NCH][kST]: fp64 sums of the big terms of a drawing sweep, one slot per thread
+  const int tid = threadIdx.x;
+  if (tid < kRing) {
+    sh.tag[tid] = 0;
+    sh.arrive[tid] = 0;
+  }
+  if (tid == 0) {
+    sh.started = 0;
+    sh.fault = 0;
+  }
+  __syncthreads();
+  if (tid < kST)
+    stream_role<DT, MODE, NCH>(fp, sh, bigacc);
+  else
+    service_role<DT, MODE, NCH>(fp, sh);
+}
+
+using FusedFn = void (*)(const FParams);
+
+template <int DT>
+FusedFn pick_dt(int mode, int n) {
+  if (mode == kLogitSample) return cos_fused_kernel<DT, kLogitSample, 2>;
+  if (mode == kEnsembleSample) {
+    if (n == 1) return cos_fused_kernel<DT, kEnsembleSample, 1>;
+    if (n == 2) return cos_fused_kernel<DT, kEnsembleSample, 2>;
+    if (n == 3) return cos_fused_kernel<DT, kEnsembleSample, 3>;
+    if (n == 4) return cos_fused_kernel<DT, kEnsembleSample, 4>;
+  }
+  return nullptr;
+}
+
+FusedFn pick_fused(int dtype, int mode, int n) {
+  if (dtype == COS_DTYPE_F32) return pick_dt<COS_DTYPE_F32>(mode, n);
+  if (dtype == COS_DTYPE_BF16) return pick_dt<COS_DTYPE_BF16>(mode, n);
+  if (dtype == COS_DTYPE_F16) return pick_dt<COS_DTYPE_F16>(mode, n);
+  return nullptr;
+}
+
+int channels_of(int mode, int n) { return mode == kEnsembleSample ? n : 2; }
+size_t fused_smem(int mode, int n) { return static_cast<size_t>(2 * channels_of(mode, n)) * kST * sizeof(double); }
+
+}  // namespace
+
+namespace cosv {
+
+bool fused_covers(int dtype, int mode, int n, int vocab, int gamma, int mask_model, long long max_units) {
+  if (mode != kEnsembleSample && mode != kLogitSample) return false;
+  if (mode == kEnsembleSample && n > kCh) return false;
+  if (mask_model >= 0) return false;
+  if (gamma + 1 > 16) return false;            // four bits per position in the row's word
+  if (max_units > 0x3fffffLL) return false;    // item descriptors keep 22 bits for the position
+  const int E = (dtype == COS_DTYPE_F32) ? 4 : 8;
+  if (vocab % E != 0) return false;            // whole 16-byte vectors only
+  return pick_fused(dtype, mode, n) != nullptr;
+}
+
+FusedPlan fused_plan(int dtype, int mode, int n, int vocab, int gamma, int max_batch, int sm_count, int blocks_per_sm) {
+  FusedPlan pl;
+  const int E = (dtype == COS_DTYPE_F32) ? 4 : 8;
+  const int nvec = vocab / E;
+  const int nsteps = (nvec + 31) / 32;
+  // streaming chunks of about 128 KB over all models, at least two steps per streaming warp, 32 chunks at most
+  const long long step_bytes = 512LL * n;
+  int cs = static_cast<int>((128 * 1024 + step_bytes - 1) / step_bytes);
+  if (cs < 2 * kSW) cs = 2 * kSW;
+  int chunks = (nsteps + cs - 1) / cs;
+  if (chunks > 32) chunks = 32;
+  if (chunks < 1) chunks = 1;
+  pl.chunks = chunks;
+  pl.chunk_steps = (nsteps + chunks - 1) / chunks;
+  pl.chunks = (nsteps + pl.chunk_steps - 1) / pl.chunk_steps;
+  // drawing chunks: half that size (the sweep costs about twice as much per byte), 64 at most
+  int ds = cs / 2;
+  if (ds < kSW) ds = kSW;
+  int dchunks = (nsteps + ds - 1) / ds;
+  if (dchunks > 64) dchunks = 64;
+  if (dchunks < 1) dchunks = 1;
+  pl.dchunk_steps = (nsteps + dchunks - 1) / dchunks;
+  pl.dchunks = (nsteps + pl.dchunk_steps - 1) / pl.dchunk_steps;
+  pl.nslots = (mode == kEnsembleSample) ? n : 2;
+  pl.nch = channels_of(mode, n);
+  pl.blocks = sm_count * (blocks_per_sm > 0 ? blocks_per_sm : 1);
+  pl.dq_cap = 2 * max_batch * pl.dchunks;  // a row queues its items once, twice when the residual turns out empty
+  (void)gamma;
+  return pl;
+}
+
+void fused_scratch_bytes(const FusedPlan& pl, int vocab, int dtype, int gamma, int max_batch, size_t out[9]) {
+  const size_t B = static_cast<size_t>(max_batch), P = static_cast<size_t>(gamma) + 1;
+  const int E = (dtype == COS_DTYPE_F32) ? 4 : 8;
+  const size_t nsteps = (static_cast<size_t>(vocab / E) + 31) / 32;
+  out[0] = 8 * sizeof(unsigned);
+  out[1] = B * sizeof(unsigned long long);
+  out[2] = B * P * sizeof(int);
+  out[3] = B * P * pl.chunks * pl.nslots * sizeof(SoftPart);
+  out[4] = static_cast<size_t>(pl.dq_cap) * sizeof(int);
+  out[5] = B * sizeof(int);
+  out[6] = B * sizeof(int);
+  out[7] = B * pl.dchunks * pl.nch * sizeof(double);
+  out[8] = B * nsteps * pl.nch * sizeof(double);
+}
+
+cudaError_t fused_occupancy(int dtype, int mode, int n, int* blocks_per_sm) {
+  FusedFn fn = pick_fused(dtype, mode, n);
+  if (fn == nullptr) return cudaErrorInvalidDeviceFunction;
+  cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(fused_smem(mode, n)));
+  if (e != cudaSuccess) return e;
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void*>(fn), kFT, fused_smem(mode, n));
+}
+
+cudaError_t fused_launch(int dtype, int mode, const KParams& p, const FusedPlan& plan, const FusedScratch& scratch,
+                         unsigned poll_limit, int debug_drop, cudaStream_t stream) {
+  FusedFn fn = pick_fused(dtype, mode, p.n);
+  if (fn == nullptr) return cudaErrorInvalidDeviceFunction;
+  FParams fp;
+  fp.k = p;
+  fp.plan = plan;
+  fp.s = scratch;
+  fp.num_items = p.num_units * plan.chunks;
+  const int E = (dtype == COS_DTYPE_F32) ? 4 : 8;
+  fp.nvec = p.V / E;
+  fp.total_events = static_cast<unsigned>(p.num_units + p.B);
+  fp.poll_limit = poll_limit;
+  fp.debug_drop = debug_drop;
+  int blocks = plan.blocks;
+  if (blocks > fp.num_items) blocks = fp.num_items;
+  fn<<<blocks, kFT, fused_smem(mode, p.n), stream>>>(fp);
+  return cudaGetLastError();
+}
+
+}  // namespace cosv

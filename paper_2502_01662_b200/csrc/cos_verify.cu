@@ -25,6 +25,7 @@
 // At T = 0 stage 0 is the whole run.
 
 #include "cos_common.cuh"
+#include "cos_fused.h"
 
 using namespace cosv;
 
@@ -2119,6 +2120,14 @@ struct cos_verify_ctx {
   cudaEvent_t ev[4];
   int ev_used;  // events recorded by the last run
   // optional staging for host-pointer runs
+  // the one-launch form of a run (sampling modes the fused kernel covers, no cluster size requested)
+  bool fused;
+  FusedPlan fplan;
+  FusedScratch fscr;
+  void* fused_mem[9];
+  size_t fused_bytes[9];
+  unsigned wait_limit;  // idle polls after which a block of the one-launch kernel gives up
+  int test_drop;        // test hook: one streaming warp never reports its first item
   void* d_logits;
   int* d_drafts;
   int* d_proposer;
@@ -2330,6 +2339,12 @@ cos_status init_scratch(cos_verify_ctx* ctx, cudaStream_t stream) {
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_job_count, 0, 2 * sizeof(int), stream);
   if (e == cudaSuccess)
     e = cudaMemsetAsync(ctx->d_part_arrivals, 0, rows * (static_cast<size_t>(ctx->cfg.gamma) + 1) * sizeof(int), stream);
+  if (ctx->fused) {
+    // counters, row words, arrival counters and the queue start at zero; the rest is written before it is read
+    static const int kClear[] = {0, 1, 2, 4, 5, 6};
+    for (int k : kClear)
+      if (e == cudaSuccess) e = cudaMemsetAsync(ctx->fused_mem[k], 0, ctx->fused_bytes[k], stream);
+  }
   if (e != cudaSuccess) return cuda_fail(ctx, "scratch reset", e);
   ctx->scratch_dirty = false;
   return COS_OK;
@@ -2414,6 +2429,36 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   ok = ok && cudaMalloc(&ctx->d_srung, rows * rec_per_row * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_srungB, rows * rec_per_row * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_part_arrivals, rows * P * sizeof(int)) == cudaSuccess;
+  ctx->wait_limit = 1u << 20;
+  ctx->test_drop = 0;
+  ctx->fused = false;
+  if (ok && config->cluster_size == 0 &&
+      fused_covers(config->dtype, mode_of(*config), config->n, config->vocab, config->gamma,
+                   config->combine == COS_COMBINE_LOGIT_LINEAR ? config->mask_model : -1,
+                   static_cast<long long>(rows) * static_cast<long long>(P))) {
+    int per_sm = 0;
+    e = fused_occupancy(config->dtype, mode_of(*config), config->n, &per_sm);
+    if (e != cudaSuccess || per_sm < 1) {
+      (void)cudaGetLastError();
+    } else {
+      ctx->fplan = fused_plan(config->dtype, mode_of(*config), config->n, config->vocab, config->gamma, config->max_batch,
+                              ctx->sm_count, per_sm);
+      fused_scratch_bytes(ctx->fplan, config->vocab, config->dtype, config->gamma, config->max_batch, ctx->fused_bytes);
+      for (int k = 0; k < 9; ++k) ok = ok && cudaMalloc(&ctx->fused_mem[k], ctx->fused_bytes[k]) == cudaSuccess;
+      if (ok) {
+        ctx->fscr.ctr = static_cast<unsigned*>(ctx->fused_mem[0]);
+        ctx->fscr.row_word = static_cast<unsigned long long*>(ctx->fused_mem[1]);
+        ctx->fscr.unit_arrivals = static_cast<int*>(ctx->fused_mem[2]);
+        ctx->fscr.chunk_part = static_cast<SoftPart*>(ctx->fused_mem[3]);
+        ctx->fscr.dq = static_cast<int*>(ctx->fused_mem[4]);
+        ctx->fscr.row_draw = static_cast<int*>(ctx->fused_mem[5]);
+        ctx->fscr.draw_arrivals = static_cast<int*>(ctx->fused_mem[6]);
+        ctx->fscr.dzpart = static_cast<double*>(ctx->fused_mem[7]);
+        ctx->fscr.srec = static_cast<double*>(ctx->fused_mem[8]);
+        ctx->fused = true;
+      }
+    }
+  }
   if (ok && config->host_staging) {
     const size_t V = static_cast<size_t>(config->vocab);
     ok = ok && cudaMalloc(&ctx->d_logits, static_cast<size_t>(config->n) * rows * P * V * elem_bytes(config->dtype)) == cudaSuccess;
@@ -2554,6 +2599,19 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
 
   const int mode = mode_of(c);
   const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
+  // One launch does the whole run where the fused kernel covers it: aligned rows, no test hook.  (The hint to
+  // leave positions unread is not taken there: every position is read once.)
+  if (ctx->fused && p.vec_ok && a->dump_r == nullptr && !(a->flags & COS_RUN_ALL_RESIDUALS)) {
+    p.early_exit = 0;
+    ctx->scratch_dirty = true;
+    if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
+    e = fused_launch(c.dtype, mode, p, ctx->fplan, ctx->fscr, ctx->wait_limit, ctx->test_drop, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (one-launch form)", e);
+    if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
+    ctx->ev_used = 2;
+    ctx->scratch_dirty = (ctx->test_drop != 0);  // a run that was made to give up leaves its counters behind
+    return COS_OK;
+  }
   // stage 0: every unit once (statistics, accept tests, row scans)
   const int c0 = choose_stream_cluster(c, p.num_units, ctx->sm_count);
   const int mc0 = ctx->max_clusters[log2i(c0)];
@@ -2697,6 +2755,17 @@ extern "C" cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, in
   return COS_OK;
 }
 
+extern "C" cos_status cos_verify_set_wait_limit(cos_verify_ctx* ctx, uint32_t polls, int32_t test_drop_report) {
+  if (!ctx) return COS_ERR_INVALID_ARG;
+  if (polls < 16) {
+    ctx->err = "wait limit below 16 polls";
+    return COS_ERR_INVALID_ARG;
+  }
+  ctx->wait_limit = polls;
+  ctx->test_drop = test_drop_report ? 1 : 0;
+  return COS_OK;
+}
+
 extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_info* info) {
   if (!ctx || !info) return COS_ERR_INVALID_ARG;
   memset(info, 0, sizeof(*info));
@@ -2709,10 +2778,11 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
     // channel sums describe a mass, stages 0, 1 and 2 otherwise
     const int mode = mode_of(ctx->cfg);
     const bool one_sweep = (mode == kLogitSample) || (mode == kEnsembleSample && ctx->cfg.n == 2);
-    info->launches_per_run = (ctx->cfg.temperature > 0.0f) ? (one_sweep ? 2 : 3) : 1;
+    info->launches_per_run = (ctx->cfg.temperature > 0.0f && !ctx->fused) ? (one_sweep ? 2 : 3) : 1;
   }
-  info->reserved[0] = ctx->parts;
-  info->reserved[1] = ctx->parts_one;
+  info->reserved[0] = ctx->fused ? ctx->fplan.chunks : ctx->parts;
+  info->reserved[1] = ctx->fused ? ctx->fplan.dchunks : ctx->parts_one;
+  info->reserved[2] = ctx->fused ? 1 : 0;
   return COS_OK;
 }
 
@@ -2734,6 +2804,7 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   for (int k = 0; k < 4; ++k)
     if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
   cudaFree(ctx->d_unit_res);
+  for (int k = 0; k < 9; ++k) cudaFree(ctx->fused_mem[k]);
   cudaFree(ctx->d_logits);
   cudaFree(ctx->d_drafts);
   cudaFree(ctx->d_proposer);
