@@ -22,8 +22,17 @@ def oracle_config(w: synth.Workload, bonus_model: int = -1) -> orc.OracleConfig:
                             bonus_model=bonus_model)
 
 
-def run_oracle(w: synth.Workload, inputs: dict, rows=None, return_r=False, row_base=0, bonus_model: int = -1) -> dict:
+def run_oracle(w: synth.Workload, inputs: dict, rows=None, return_r=False, row_base=0, bonus_model: int = -1,
+               native: bool = False, threads: int = 0) -> dict:
+    """The oracle on the inputs of a GPU run.  `native` runs its C++ twin (same rows, spread over host threads),
+    which is how full-size workloads are checked on every row."""
     logits = inputs["logits"]
+    if native:
+        from oracle import cos_oracle_native as nat
+        assert not return_r
+        return nat.verify(synth.logits_as_numpy(logits), w.dtype, inputs["drafts"].cpu().numpy(),
+                          inputs["proposer"].cpu().numpy(), oracle_config(w, bonus_model), inputs["seed"], inputs["offset"],
+                          row_base=row_base, rows=rows, threads=threads)
     if rows is not None:
         # copy only the sampled rows to the host (full-size cases hold gigabytes)
         sel = logits[:, list(rows)]

@@ -12,18 +12,19 @@ pytestmark = pytest.mark.gpu
 C = synth.CONFIGS
 
 
-@pytest.mark.parametrize("name,nrows", [("cfg1", 1), ("cfg2", 8), ("cfg3", 10), ("cfg4", 8), ("cfg5", 8), ("cfg5_greedy", 8)])
-def test_full_size_workloads_on_sampled_rows(name, nrows):
+@pytest.mark.parametrize("name,nrows", [("cfg1", 1), ("cfg2", 8), ("cfg3", 64), ("cfg4", 32), ("cfg5", 48), ("cfg5_greedy", 48)])
+def test_full_size_workloads(name, nrows):
     """The launch configuration bench.py times (default cluster choice, full batch), compared with the
-    oracle on a seeded sample of rows; a row's result does not depend on the other rows."""
+    oracle's C++ twin on every row (workloads 1 to 4) or on a seeded sample of rows (the 2.4 GB workload 5);
+    a row's result does not depend on the other rows."""
     w = C[name]
     inputs = synth.make_inputs(w, "cuda")
     rows = sorted(np.random.default_rng(7).choice(w.batch, size=min(nrows, w.batch), replace=False).tolist())
     gpu = helpers.run_gpu(w, inputs, diag=True)
-    ref = helpers.run_oracle(w, inputs, rows=rows)
+    ref = helpers.run_oracle(w, inputs, rows=rows, native=True)
     stats = helpers.check_parity(w, gpu, ref, rows=rows)
-    assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
-    # the sampled rows are not degenerate: some rows reject, and sampling modes do not reject everything at 0
+    assert stats["excused_accept"] + stats["excused_sample"] <= 2, stats
+    # the rows are not degenerate: some rows reject, and sampling modes do not reject everything at 0
     acc = gpu["accept_count"]
     assert acc.min() >= 0 and acc.max() <= w.gamma
     assert np.all(gpu["out_tokens"][np.arange(w.batch), acc] >= 0)
