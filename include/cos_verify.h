@@ -221,6 +221,18 @@ cos_status cos_verify_set_stage_timing(cos_verify_ctx* ctx, int enable);
 cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, int32_t* count);
 
 /*
+ * The one-launch form of a run (Sec. 3.1-3.2 as ONE persistent kernel): streaming work items of about 128 KB,
+ * rows settled as soon as every position up to their first rejection is published, the token draw queued inside
+ * the same launch.  It covers sampling runs (T > 0) of ensembles of up to four models and of logit-level combines
+ * without mask, with 16-byte aligned rows, at most 16 positions per row and no test hook; `enable` != 0 makes
+ * later runs of this context take it (COS_ERR_UNSUPPORTED when the configuration is not covered), 0 returns to
+ * the staged launches, which are the default because they are the faster form on the measured workloads.
+ * Results are those of the staged form (same arithmetic per position; sums are merged in another order, so
+ * probabilities may differ in the last bits).  COS_RUN_EARLY_EXIT is ignored there: every position is read.
+ */
+cos_status cos_verify_set_one_launch(cos_verify_ctx* ctx, int32_t enable);
+
+/*
  * Failure detection of the one-launch form of a run (sampling modes without mask or test hook): every wait
  * inside the kernel is a bounded poll.  A block that sees no progress for `polls` polls (about 0.2 us each; the
  * default of 2^20 is about a fifth of a second) sets COS_ROW_FAULT on every row and leaves; the kernel always

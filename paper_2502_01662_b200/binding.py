@@ -32,7 +32,7 @@ _STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR
 
 EXPORTS = ("cos_verify_create", "cos_verify_run", "cos_verify_run_host", "cos_verify_get_info",
            "cos_verify_destroy", "cos_verify_last_error", "cos_verify_set_stage_timing", "cos_verify_get_stage_ms",
-           "cos_verify_run_static", "cos_verify_set_wait_limit", "cos_verify_measure_ceiling")
+           "cos_verify_run_static", "cos_verify_set_wait_limit", "cos_verify_measure_ceiling", "cos_verify_set_one_launch")
 
 
 class CosVerifyError(RuntimeError):
@@ -92,6 +92,8 @@ def load_library(rebuild: bool = False) -> ctypes.CDLL:
     lib.cos_verify_set_stage_timing.restype = ctypes.c_int
     lib.cos_verify_get_stage_ms.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.cos_verify_get_stage_ms.restype = ctypes.c_int
+    lib.cos_verify_set_one_launch.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+    lib.cos_verify_set_one_launch.restype = ctypes.c_int
     lib.cos_verify_set_wait_limit.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_int32]
     lib.cos_verify_set_wait_limit.restype = ctypes.c_int
     lib.cos_verify_measure_ceiling.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p,
@@ -192,6 +194,10 @@ class CosVerifier:
         a.bonus_model = bonus_model if (bonus_model is not None and bonus_model >= 0) else 0
         a.offset_device = offset_device.data_ptr() if offset_device is not None else None
         return a
+
+    def set_one_launch(self, enable: bool = True):
+        """cos_verify_set_one_launch: later runs take the one-launch kernel (raises if the configuration is not covered)."""
+        self._check(self._lib.cos_verify_set_one_launch(self._ctx, int(bool(enable))))
 
     def set_wait_limit(self, polls: int, test_drop_report: bool = False):
         """cos_verify_set_wait_limit: bound of the kernel's internal polls (and the test hook that makes one run out)."""

@@ -14,7 +14,7 @@
 // that blocks look at before they take the next streaming item, while the position's logits are still in L2.
 //
 // A block is fifteen streaming warps and one service warp.  Streaming warps run from item to item without
-// block barriers and leave their partial sums in a ring of four slots in shared memory; the service warp fetches
+// block barriers and leave their partial sums in a ring of eight slots in shared memory; the service warp fetches
 // items one ahead, merges the partials, talks to the other blocks (fences, arrival counters, the queue) and does
 // all serial work (decision, row scan, locating a token), so none of it sits on the streaming warps' path.
 // No block depends on a particular other block: any item can be taken by any block, and a block with nothing to
@@ -29,10 +29,29 @@ namespace {
 constexpr int kFT = 512;          // threads per block
 constexpr int kSW = 15;           // streaming warps
 constexpr int kST = kSW * 32;     // streaming threads
-constexpr int kRing = 4;          // items a block may have open
+constexpr int kRing = 8;          // items a block may have open
 constexpr int kCh = 4;            // channels of a drawing sweep (ensembles of up to four models; logit level: two)
 constexpr int kItemStream = 0, kItemDraw = 1, kItemExit = 3;
-constexpr int kCtrNext = 0, kCtrEvents = 1, kCtrHead = 2, kCtrTail = 3, kCtrGone = 4, kCtrFault = 5;
+// counters, each on a 128-byte line of its own (the queue's head and tail share one: they are read together)
+constexpr int kCtrNext = 0, kCtrEvents = 32, kCtrHead = 64, kCtrTail = 65, kCtrGone = 96, kCtrFault = 128;
+constexpr int kCtrWords = 160;
+
+// Optional timeline accounting (build with -DCOS_FUSED_PROFILE): cycles the service warp and streaming warp 0 of
+// every block spend in each activity, summed over blocks into g_prof.  Compiled out of ordinary builds.
+#ifdef COS_FUSED_PROFILE
+__device__ unsigned long long g_prof[32];
+#define PROF_DECL unsigned long long prof_acc[16] = {0}; long long prof_t0 = 0; (void)prof_t0
+#define PROF_T0 prof_t0 = clock64()
+#define PROF_ADD(k) do { const long long t1_ = clock64(); prof_acc[k] += static_cast<unsigned long long>(t1_ - prof_t0); prof_t0 = t1_; } while (0)
+#define PROF_COUNT(k) prof_acc[k] += 1
+#define PROF_FLUSH(base) do { if ((threadIdx.x & 31) == 0) for (int q_ = 0; q_ < 16; ++q_) if (prof_acc[q_]) atomicAdd(&g_prof[(base) + q_], prof_acc[q_]); } while (0)
+#else
+#define PROF_DECL
+#define PROF_T0
+#define PROF_ADD(k)
+#define PROF_COUNT(k)
+#define PROF_FLUSH(base)
+#endif
 
 struct FParams {
   KParams k;
@@ -55,7 +74,7 @@ struct ItemCtx {
 };
 
 struct FShared {
-  int tag[kRing];       // seq + 1 once ctx[seq & 3] is valid
+  int tag[kRing];       // seq + 1 once ctx[seq % kRing] is valid
   int arrive[kRing];    // streaming warps that have finished the item of that slot
   int started;          // number of items some warp has begun
   int fault;
@@ -90,21 +109,135 @@ __device__ __forceinline__ double channel_k(const KParams& p, int i, int pis, in
 // ------------------------------------------------------------------------------------
 // streaming warps
 // ------------------------------------------------------------------------------------
+constexpr int kU = 8;  // 16-byte loads a streaming thread issues back to back
+
+// A streaming load that stays where it is written (a batch of loads is issued first, then consumed).
+__device__ __forceinline__ uint4 ldg_ahead16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// One row's share of one thread again in the running-maximum form (after an overflow or a non-finite input).
+template <int DT>
+__device__ __noinline__ LaneSoft online_redo(const char* row, int v_first, int v_hi, float c) {
+  constexpr int E = Elem<DT>::E;
+  LaneSoft acc;
+  acc.init();
+  for (int v = v_first; v < v_hi; v += kST) {
+    float x[E];
+    Elem<DT>::unpack(ldg_stream16(row + static_cast<long long>(v) * 16), x);
+    acc.add_online(x, c);
+  }
+  return acc;
+}
+
+// Ensemble: the softmax statistics of the chunk [lo, hi) of every model's row, row after row.  Threads are
+// interleaved over the 16-byte vectors; a thread issues kU loads back to back and then consumes them (no warp
+// waits for another, so the other warps' loads cover the gap).  Fixed reference exponent per row and thread, seeded
+// from the thread's first vector (a whole number, so that sums rescale exactly); overflow or a non-finite input
+// redoes the thread's share of that row in the running-maximum form.
+template <int DT>
+__device__ __forceinline__ void stream_ensemble(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
+  constexpr int E = Elem<DT>::E;
+  const KParams& p = fp.k;
+  const int lane = stid & 31;
+  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
+  const long long row_step = p.s_model * Elem<DT>::bytes;
+  const int v0 = it.lo + stid;
+  for (int i = 0; i < p.n; ++i) {
+    const char* row = base + i * row_step;
+    LaneSoft acc;
+    acc.init();
+    bool first = true;
+    for (int v = v0; v < it.hi; v += kU * kST) {
+      uint4 raw[kU];
+#pragma unroll
+      for (int u = 0; u < kU; ++u)
+        if (v + u * kST < it.hi) raw[u] = ldg_ahead16(row + static_cast<long long>(v + u * kST) * 16);
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+        if (v + u * kST < it.hi) {
+          float x[E];
+          Elem<DT>::unpack(raw[u], x);
+          if (u == 0 && first) {
+            acc.seed(x, p.cT);
+            first = false;
+          }
+          acc.add_fixed(x, p.cT);
+        }
+      }
+    }
+    if (!(acc.s < INFINITY)) acc = online_redo<DT>(row, v0, it.hi, p.cT);
+    warp_merge_soft(acc, &part[i], lane);
+  }
+}
+
+// Logit level with two models: proposer's softmax and the softmax of the combined logits, one vector of each model
+// per trip, kU / 2 trips per batch.  Same reference-exponent scheme as above.  False when some lane of the warp
+// met an overflow or a non-finite input (the caller then takes the general form).
+template <int DT>
+__device__ __forceinline__ bool stream_logit2(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
+  constexpr int E = Elem<DT>::E;
+  constexpr int T = kU / 2;
+  const KParams& p = fp.k;
+  const int lane = stid & 31;
+  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
+  const long long row_step = p.s_model * Elem<DT>::bytes;
+  const int v0 = it.lo + stid;
+  const float w0 = p.w[0], w1 = p.w[1];
+  const bool q_is_0 = (it.pis == 0);
+  LaneSoft accq, accc;
+  accq.init();
+  accc.init();
+  bool first = true;
+  for (int v = v0; v < it.hi; v += T * kST) {
+    uint4 r0[T], r1[T];
+#pragma unroll
+    for (int u = 0; u < T; ++u)
+      if (v + u * kST < it.hi) {
+        r0[u] = ldg_ahead16(base + static_cast<long long>(v + u * kST) * 16);
+        r1[u] = ldg_ahead16(base + row_step + static_cast<long long>(v + u * kST) * 16);
+      }
+#pragma unroll
+    for (int u = 0; u < T; ++u) {
+      if (v + u * kST < it.hi) {
+        float x0[E], x1[E], cmb[E];
+        Elem<DT>::unpack(r0[u], x0);
+        Elem<DT>::unpack(r1[u], x1);
+#pragma unroll
+        for (int k = 0; k < E; ++k) cmb[k] = fmaf(w1, x1[k], fmaf(w0, x0[k], 0.f));
+        if (u == 0 && first) {
+          if (q_is_0) accq.seed(x0, p.cT); else accq.seed(x1, p.cT);
+          accc.seed(cmb, p.cT);
+          first = false;
+        }
+        if (q_is_0) accq.add_fixed(x0, p.cT); else accq.add_fixed(x1, p.cT);
+        accc.add_fixed(cmb, p.cT);
+      }
+    }
+  }
+  const bool settled = (accq.s < INFINITY) && (accc.s < INFINITY);
+  if (!__all_sync(0xffffffffu, settled)) return false;
+  warp_merge_soft(accq, &part[0], lane);
+  warp_merge_soft(accc, &part[1], lane);
+  return true;
+}
+
 template <int DT, int MODE>
 __device__ __forceinline__ void stream_item(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
   const KParams& p = fp.k;
   const int lane = stid & 31;
-  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
-  Slice sl;
-  sl.v_lo = it.lo;
-  sl.v_hi = it.hi;
-  sl.e_lo = sl.e_hi = 0;
   if (MODE == kEnsembleSample) {
-    for (int i = 0; i < p.n; ++i) {
-      LaneSoft acc = soft_slice<DT, kST>(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, sl, stid, p.cT);
-      warp_merge_soft(acc, &part[i], lane);
-    }
+    stream_ensemble<DT>(fp, it, part, stid);
   } else {
+    if (p.n == 2 && stream_logit2<DT>(fp, it, part, stid)) return;
+    // any other number of models, and the warps that met an overflow or a non-finite input
+    const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
+    Slice sl;
+    sl.v_lo = it.lo;
+    sl.v_hi = it.hi;
+    sl.e_lo = sl.e_hi = 0;
     LaneSoft accq, accc;
     logit_soft_slice<DT, kST>(p, base, sl, stid, it.pis, false, -INFINITY, accq, accc);
     warp_merge_soft(accq, &part[0], lane);
@@ -203,7 +336,7 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
     const int v = s * 32 + lane;
 #pragma unroll
     for (int i = 0; i < NL; ++i)
-      nx[i] = (v < fp.nvec && i < nl) ? ldg_stream16(base + i * row_step + static_cast<long long>(v) * 16) : ninf_vec<DT>();
+      nx[i] = (v < fp.nvec && i < nl) ? ldg_ahead16(base + i * row_step + static_cast<long long>(v) * 16) : ninf_vec<DT>();
   };
   double* rec = fp.s.srec + static_cast<size_t>(it.b) * p.nsteps * NCH;
   if (it.lo + warp < it.hi) fetch(it.lo + warp);
@@ -301,7 +434,6 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
 #pragma unroll
       for (int i = 1; i < NCH; ++i) mine = (lane == i) ? da[i] : mine;
       __stcg(rec + static_cast<size_t>(s) * NCH + lane, mine);
-      __threadfence();
     }
   }
   // this warp's share of the refined normalisers
@@ -321,6 +453,8 @@ template <int DT, int MODE, int NCH>
 __device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, double* bigacc_all) {
   const int stid = threadIdx.x, lane = stid & 31, warp = stid >> 5;
   double* bigacc = bigacc_all + stid;
+  PROF_DECL;
+  PROF_T0;
   for (int seq = 0;; ++seq) {
     const int slot = seq & (kRing - 1);
     // the service warp posts the item; it is normally there already (fetched one ahead)
@@ -339,21 +473,30 @@ __device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, doub
       if (ok) atomicMax(&sh.started, seq + 1);
     }
     ok = __shfl_sync(0xffffffffu, ok, 0);
-    if (!ok) return;
+    PROF_ADD(0);  // waiting for an item
+    if (!ok) break;
     __syncwarp();
     const ItemCtx& it = sh.ctx[slot];
-    if (it.kind == kItemExit) return;
-    if (it.kind == kItemStream)
+    if (it.kind == kItemExit) break;
+    if (it.kind == kItemStream) {
       stream_item<DT, MODE>(fp, it, &sh.part[slot][warp][0], stid);
-    else
+      PROF_ADD(1);
+      PROF_COUNT(4);
+    } else {
       draw_item<DT, MODE, NCH>(fp, it, &sh.part[slot][warp][0], stid, bigacc);
+      PROF_ADD(2);
+      PROF_COUNT(5);
+    }
+    if (it.kind == kItemDraw) __threadfence();  // the step records of a drawing item are read by another block
     __syncwarp();
     if (lane == 0) {
       const bool drop = fp.debug_drop && blockIdx.x == 0 && warp == 0 && seq == 0;  // test hook: a report that never comes
-      __threadfence();  // a drawing item's step records are read by another block
+      __threadfence_block();
       if (!drop) atomicAdd(&sh.arrive[slot], 1);
     }
+    PROF_ADD(3);  // reporting
   }
+  if (warp == 0) PROF_FLUSH(0);
 }
 
 // ------------------------------------------------------------------------------------
@@ -452,7 +595,7 @@ __device__ __forceinline__ void publish_position(const FParams& fp, int b, int j
 // The last chunk of a position has arrived: merge the chunks in order, take the accept test in fp64 (Eq. 6) and
 // publish.  Whole warp; `own` (chunks == 1) are the block's merged statistics.
 template <int DT, int MODE>
-__device__ __forceinline__ void finish_position(const FParams& fp, int b, int j, int pi_raw, const SoftPart* own) {
+__device__ __forceinline__ void finish_position(const FParams& fp, int b, int j, const SoftPart* own) {
   const KParams& p = fp.k;
   const int lane = threadIdx.x & 31;
   const int ns = fp.plan.nslots, C = fp.plan.chunks;
@@ -472,8 +615,8 @@ __device__ __forceinline__ void finish_position(const FParams& fp, int b, int j,
   const bool is_bonus = (j == p.gamma);
   const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
   const bool draft_ok = is_bonus || (draft >= 0 && draft < p.V);
-  const bool pi_ok = (pi_raw >= 0 && pi_raw < p.n);
-  const int pi = pi_raw;
+  const int pi = proposer_of(p, b, j);
+  const bool pi_ok = (pi >= 0 && pi < p.n);
   const char* base = unit_base(p, b, j, Elem<DT>::bytes);
   float ld = 0.f;
   if (lane < p.n && !is_bonus && draft_ok) ld = Elem<DT>::load1(base + static_cast<long long>(lane) * p.s_model * Elem<DT>::bytes, draft);
@@ -743,6 +886,7 @@ __device__ __forceinline__ void locate_token(const FParams& fp, int b) {
   const int per = (p.nsteps + 31) / 32;
   const int lo = lane * per, hi = (lo + per < p.nsteps) ? lo + per : p.nsteps;
   double mine = 0.0;
+#pragma unroll 8
   for (int st = lo; st < hi; ++st) mine += step_mass(st);
   double incl = mine;
 #pragma unroll
@@ -756,6 +900,7 @@ __device__ __forceinline__ void locate_token(const FParams& fp, int b) {
   double before = incl - mine;
   int first = 0x7fffffff, last = -1;
   double first_base = 0.0, last_base = 0.0;
+#pragma unroll 4
   for (int st = lo; st < hi; ++st) {
     const double m = step_mass(st);
     if (m > 0.0) {
@@ -806,20 +951,30 @@ __device__ __forceinline__ void locate_token(const FParams& fp, int b) {
   __syncwarp();
 }
 
-// one thread: the next item of this block, or -1.  Drawing items first (their logits are still in L2).
-__device__ __forceinline__ int take_item(const FParams& fp, bool& static_left) {
-  unsigned h = vol_load(&fp.s.ctr[kCtrHead]);
-  for (int tries = 0; tries < 8; ++tries) {
-    if (h >= static_cast<unsigned>(fp.plan.dq_cap)) break;
-    const int v = vol_load(&fp.s.dq[h]);
-    if (v == 0) break;
-    const unsigned old = atomicCAS(&fp.s.ctr[kCtrHead], h, h + 1);
-    if (old == h) {
-      fp.s.dq[h] = 0;  // clean for the next run
+__device__ __forceinline__ uint2 vol_load2(const unsigned* p) {
+  uint2 v;
+  asm volatile("ld.volatile.global.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+
+// One thread: the next item of this block, or -1.  Drawing items first (their logits are still in L2).
+// The queue hands out tickets: a block that sees entries beyond the head takes the next ticket with one atomic
+// add.  Under a race the ticket may lie beyond the tail; it then names the entry this block takes as soon as
+// somebody writes it (`ticket` is kept across calls; a block holds one ticket at most).  Nobody spins on the
+// queue, and every entry has exactly one taker, who cannot leave before the run is complete.
+__device__ __forceinline__ int take_item(const FParams& fp, bool& static_left, int& ticket) {
+  if (ticket < 0) {
+    const uint2 ht = vol_load2(&fp.s.ctr[kCtrHead]);  // head, tail
+    if (ht.y > ht.x) ticket = static_cast<int>(atomicAdd(&fp.s.ctr[kCtrHead], 1u));
+  }
+  if (ticket >= 0 && ticket < fp.plan.dq_cap) {
+    const int v = vol_load(&fp.s.dq[ticket]);
+    if (v != 0) {
+      fp.s.dq[ticket] = 0;  // clean for the next run
+      ticket = -1;
       __threadfence();
       return v - 1;
     }
-    h = old;
   }
   if (static_left) {
     const unsigned t = atomicAdd(&fp.s.ctr[kCtrNext], 1u);
@@ -844,8 +999,8 @@ __device__ __forceinline__ void fill_ctx(const FParams& fp, ItemCtx& cx, int des
       cx.b = b;
       cx.j = j;
       cx.chunk = c;
-      const int pi = proposer_of(p, b, j);
-      cx.dkind = pi;  // as given; checked when the position is decided
+      // (only the logit-level sweep needs to know whose distribution q is; the decision looks it up itself)
+      const int pi = (MODE == kLogitSample) ? proposer_of(p, b, j) : 0;
       cx.pis = (pi >= 0 && pi < p.n) ? pi : 0;
       const int lo = c * fp.plan.chunk_steps * 32, hi = lo + fp.plan.chunk_steps * 32;
       cx.lo = lo;
@@ -888,18 +1043,23 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
   const int lane = threadIdx.x & 31;
   int fetched = 0, processed = 0;
   bool static_left = true;
+  int ticket = -1;
   unsigned idle = 0;
   bool failed = false;
+  PROF_DECL;
+  PROF_T0;
   while (true) {
     bool did = false;
-    // ---- fetch one item ahead of the fastest streaming warp
-    if (fetched < processed + kRing && fetched <= vol_load(&sh.started)) {
+    // ---- fetch up to two items ahead of the fastest streaming warp
+    if (fetched < processed + kRing && fetched <= vol_load(&sh.started) + 1) {
       int desc = -1;
-      if (lane == 0) desc = take_item(fp, static_left);
+      if (lane == 0) desc = take_item(fp, static_left, ticket);
       desc = __shfl_sync(0xffffffffu, desc, 0);
       static_left = __shfl_sync(0xffffffffu, static_left ? 1 : 0, 0) != 0;
       if (desc >= 0) {
+        PROF_ADD(0);  // taking an item
         fill_ctx<MODE>(fp, sh.ctx[fetched & (kRing - 1)], desc);
+        PROF_ADD(1);
         if (lane == 0) {
           __threadfence_block();
           *reinterpret_cast<volatile int*>(&sh.tag[fetched & (kRing - 1)]) = fetched + 1;
@@ -935,15 +1095,9 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
           }
           bool last = true;
           if (C > 1) {
-            if (lane < ns) {
-              SoftPart mine = merged[0];
-              for (int k = 1; k < ns; ++k) mine = (lane == k) ? merged[k] : mine;
-              stcg_part(&fp.s.chunk_part[(static_cast<size_t>(uidx) * C + c) * ns + lane], mine);
-              __threadfence();
-            }
-            __syncwarp();
             int prev = 0;
             if (lane == 0) {
+              for (int k = 0; k < ns; ++k) stcg_part(&fp.s.chunk_part[(static_cast<size_t>(uidx) * C + c) * ns + k], merged[k]);
               __threadfence();
               prev = atomicAdd(&fp.s.unit_arrivals[uidx], 1);
               if (prev == C - 1) {
@@ -954,7 +1108,12 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
             prev = __shfl_sync(0xffffffffu, prev, 0);
             last = (prev == C - 1);
           }
-          if (last) finish_position<DT, MODE>(fp, b, j, cx.dkind, merged);
+          PROF_ADD(2);  // a streaming chunk reported
+          if (last) {
+            finish_position<DT, MODE>(fp, b, j, merged);
+            PROF_ADD(3);
+            PROF_COUNT(8);
+          }
         } else {
           // this block's share of the refined normalisers; the last chunk of the row locates the token
           for (int i = 0; i < NCH; ++i) {
@@ -973,7 +1132,12 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
             }
           }
           prev = __shfl_sync(0xffffffffu, prev, 0);
-          if (prev == fp.plan.dchunks - 1) locate_token<DT, MODE, NCH>(fp, b);
+          PROF_ADD(4);  // a drawing chunk reported
+          if (prev == fp.plan.dchunks - 1) {
+            locate_token<DT, MODE, NCH>(fp, b);
+            PROF_ADD(5);
+            PROF_COUNT(9);
+          }
         }
         if (lane == 0) {
           *reinterpret_cast<volatile int*>(&sh.arrive[slot]) = 0;
@@ -986,6 +1150,7 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
     if (did) {
       idle = 0;
     } else {
+      PROF_ADD(processed < fetched ? 6 : 7);  // waiting for the streaming warps / for work
       if (++idle > fp.poll_limit) {
         failed = true;
         break;
@@ -1001,6 +1166,7 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
     }
     for (int b = lane; b < p.B; b += 32) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_FAULT));
   }
+  PROF_FLUSH(16);
   // tell the streaming warps to leave
   if (lane == 0) {
     ItemCtx& cx = sh.ctx[fetched & (kRing - 1)];
@@ -1069,6 +1235,17 @@ size_t fused_smem(int mode, int n) { return static_cast<size_t>(2 * channels_of(
 
 }  // namespace
 
+#ifdef COS_FUSED_PROFILE
+extern "C" int cos_fused_profile_read(unsigned long long* out32, int reset) {
+  if (cudaMemcpyFromSymbol(out32, g_prof, sizeof(g_prof)) != cudaSuccess) return -1;
+  if (reset) {
+    unsigned long long z[32] = {0};
+    if (cudaMemcpyToSymbol(g_prof, z, sizeof(z)) != cudaSuccess) return -1;
+  }
+  return 0;
+}
+#endif
+
 namespace cosv {
 
 bool fused_covers(int dtype, int mode, int n, int vocab, int gamma, int mask_model, long long max_units) {
@@ -1089,16 +1266,21 @@ FusedPlan fused_plan(int dtype, int mode, int n, int vocab, int gamma, int max_b
   const int nsteps = (nvec + 31) / 32;
   // streaming chunks of about 128 KB over all models, at least two steps per streaming warp, 32 chunks at most
   const long long step_bytes = 512LL * n;
-  int cs = static_cast<int>((128 * 1024 + step_bytes - 1) / step_bytes);
+  const long long chunk_kb = 256, dchunk_kb = 64;  // the fastest of the measured sizes (64 to 640 KB, 32 to 128 KB)
+  int cs = static_cast<int>((chunk_kb * 1024 + step_bytes - 1) / step_bytes);
   if (cs < 2 * kSW) cs = 2 * kSW;
   int chunks = (nsteps + cs - 1) / cs;
   if (chunks > 32) chunks = 32;
   if (chunks < 1) chunks = 1;
   pl.chunks = chunks;
   pl.chunk_steps = (nsteps + chunks - 1) / chunks;
+  // whole batches: kSW steps give every streaming thread one vector, a batch is kU of them (kU / 2 per row with the
+  // two rows of a logit-level pair in one trip)
+  const int batch = kSW * (mode == kEnsembleSample ? kU : kU / 2);
+  if (pl.chunk_steps > batch && chunks > 1) pl.chunk_steps = (pl.chunk_steps + batch - 1) / batch * batch;
   pl.chunks = (nsteps + pl.chunk_steps - 1) / pl.chunk_steps;
   // drawing chunks: half that size (the sweep costs about twice as much per byte), 64 at most
-  int ds = cs / 2;
+  int ds = static_cast<int>((dchunk_kb * 1024 + step_bytes - 1) / step_bytes);
   if (ds < kSW) ds = kSW;
   int dchunks = (nsteps + ds - 1) / ds;
   if (dchunks > 64) dchunks = 64;
@@ -1117,7 +1299,7 @@ void fused_scratch_bytes(const FusedPlan& pl, int vocab, int dtype, int gamma, i
   const size_t B = static_cast<size_t>(max_batch), P = static_cast<size_t>(gamma) + 1;
   const int E = (dtype == COS_DTYPE_F32) ? 4 : 8;
   const size_t nsteps = (static_cast<size_t>(vocab / E) + 31) / 32;
-  out[0] = 8 * sizeof(unsigned);
+  out[0] = kCtrWords * sizeof(unsigned);
   out[1] = B * sizeof(unsigned long long);
   out[2] = B * P * sizeof(int);
   out[3] = B * P * pl.chunks * pl.nslots * sizeof(SoftPart);

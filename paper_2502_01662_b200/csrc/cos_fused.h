@@ -21,7 +21,7 @@ struct FusedPlan {
 
 // Device scratch of the one-launch kernel (all of it zero between runs).
 struct FusedScratch {
-  unsigned* ctr;                 // [8]: next streaming item, events done, queue head, queue tail, blocks gone, fault
+  unsigned* ctr;                 // next streaming item, events done, queue head and tail, blocks gone, fault (a line each)
   unsigned long long* row_word;  // [B]
   int* unit_arrivals;            // [B * P]
   SoftPart* chunk_part;          // [B * P][chunks][nslots]

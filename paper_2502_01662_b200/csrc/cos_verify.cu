@@ -2121,7 +2121,8 @@ struct cos_verify_ctx {
   int ev_used;  // events recorded by the last run
   // optional staging for host-pointer runs
   // the one-launch form of a run (sampling modes the fused kernel covers, no cluster size requested)
-  bool fused;
+  bool fused;      // the one-launch kernel covers this configuration (its scratch is allocated)
+  bool use_fused;  // and runs take it (cos_verify_set_one_launch)
   FusedPlan fplan;
   FusedScratch fscr;
   void* fused_mem[9];
@@ -2601,7 +2602,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
   // One launch does the whole run where the fused kernel covers it: aligned rows, no test hook.  (The hint to
   // leave positions unread is not taken there: every position is read once.)
-  if (ctx->fused && p.vec_ok && a->dump_r == nullptr && !(a->flags & COS_RUN_ALL_RESIDUALS)) {
+  if (ctx->fused && ctx->use_fused && p.vec_ok && a->dump_r == nullptr && !(a->flags & COS_RUN_ALL_RESIDUALS)) {
     p.early_exit = 0;
     ctx->scratch_dirty = true;
     if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
@@ -2755,6 +2756,16 @@ extern "C" cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, in
   return COS_OK;
 }
 
+extern "C" cos_status cos_verify_set_one_launch(cos_verify_ctx* ctx, int32_t enable) {
+  if (!ctx) return COS_ERR_INVALID_ARG;
+  if (enable && !ctx->fused) {
+    ctx->err = "the one-launch form does not cover this configuration";
+    return COS_ERR_UNSUPPORTED;
+  }
+  ctx->use_fused = enable != 0;
+  return COS_OK;
+}
+
 extern "C" cos_status cos_verify_set_wait_limit(cos_verify_ctx* ctx, uint32_t polls, int32_t test_drop_report) {
   if (!ctx) return COS_ERR_INVALID_ARG;
   if (polls < 16) {
@@ -2778,11 +2789,11 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
     // channel sums describe a mass, stages 0, 1 and 2 otherwise
     const int mode = mode_of(ctx->cfg);
     const bool one_sweep = (mode == kLogitSample) || (mode == kEnsembleSample && ctx->cfg.n == 2);
-    info->launches_per_run = (ctx->cfg.temperature > 0.0f && !ctx->fused) ? (one_sweep ? 2 : 3) : 1;
+    info->launches_per_run = (ctx->cfg.temperature > 0.0f && !(ctx->fused && ctx->use_fused)) ? (one_sweep ? 2 : 3) : 1;
   }
   info->reserved[0] = ctx->fused ? ctx->fplan.chunks : ctx->parts;
   info->reserved[1] = ctx->fused ? ctx->fplan.dchunks : ctx->parts_one;
-  info->reserved[2] = ctx->fused ? 1 : 0;
+  info->reserved[2] = (ctx->fused && ctx->use_fused) ? 1 : 0;
   return COS_OK;
 }
 
