@@ -106,7 +106,9 @@ typedef struct {
   int64_t stride_model, stride_row, stride_pos;
   const int32_t* draft_tokens; /* [B][gamma]; may be NULL when gamma == 0                               */
   const int32_t* proposer;     /* [B], index in [0, n) of the model that proposed the row's drafts      */
-                               /* ([B][gamma+1] with COS_RUN_PROPOSER_PER_POSITION)                     */
+                               /* ([B][gamma+1] with COS_RUN_PROPOSER_PER_POSITION).  An index outside  */
+                               /* [0, n) names no distribution q: the positions it governs report       */
+                               /* COS_ROW_NONFINITE (rejected, token -1); nothing is read out of bounds */
   int32_t batch;               /* B, 1..max_batch                                                       */
   int32_t flags;               /* COS_RUN_* bits                                                        */
   int64_t row_base;            /* global index of row 0 (for row-sharded batches); enters the RNG only  */

@@ -316,7 +316,7 @@ def measure_ceiling(kind: int, buf, reps: int = 10, stream=None) -> float:
 def run_static(n: int, combine: int, weights: Sequence[float], temperature: float, gamma: int, vocab: int,
                logits, drafts, proposer, seed: int, offset: int, mask_model: int = -1, mask_alpha: float = 1.0,
                device: int = 0, cluster_size: int = 0, row_base: int = 0, flags: int = 0, outs: dict = None,
-               stream=None) -> dict:
+               stream=None, bonus_model: Optional[int] = None) -> dict:
     """cos_verify_run_static: one verification pass with no context and no device allocation.
 
     For hosts that cannot call cudaMalloc where they verify (a device fully owned by an engine's
@@ -346,6 +346,10 @@ def run_static(n: int, combine: int, weights: Sequence[float], temperature: floa
     a.stride_model, a.stride_row, a.stride_pos = logits.stride(0), logits.stride(1), logits.stride(2)
     a.draft_tokens = drafts.data_ptr() if (drafts is not None and drafts.numel() > 0) else None
     a.proposer = proposer.data_ptr()
+    if proposer.dim() == 2:
+        flags |= COS_RUN_PROPOSER_PER_POSITION
+    if bonus_model is not None and bonus_model >= 0:
+        flags |= COS_RUN_BONUS_FROM_MODEL
     a.batch, a.flags, a.row_base = logits.shape[1], flags, row_base
     a.seed, a.offset = seed & 0xFFFFFFFFFFFFFFFF, offset & 0xFFFFFFFFFFFFFFFF
     a.accept_count = outs["accept_count"].data_ptr()
@@ -354,7 +358,7 @@ def run_static(n: int, combine: int, weights: Sequence[float], temperature: floa
     a.diag = outs["diag"].data_ptr() if "diag" in outs else None
     a.dump_r = None
     a.bonus_prob = outs["bonus_prob"].data_ptr() if "bonus_prob" in outs else None
-    a.bonus_model = 0
+    a.bonus_model = bonus_model if (bonus_model is not None and bonus_model >= 0) else 0
     s = torch.cuda.current_stream(logits.device) if stream is None else stream
     st = lib.cos_verify_run_static(ctypes.byref(cfg), ctypes.byref(a), ctypes.c_void_p(s.cuda_stream))
     if st != COS_OK:

@@ -24,6 +24,8 @@
 // and they are bounded: a wait that gave up marks every row with COS_ROW_FAULT and the block leaves.
 // At T = 0 stage 0 is the whole run.
 
+#include <mutex>
+
 #include "cos_common.cuh"
 #include "cos_fused.h"
 
@@ -2332,6 +2334,54 @@ cos_status cuda_fail(cos_verify_ctx* ctx, const char* what, cudaError_t e) {
   return COS_ERR_CUDA;
 }
 
+// What a launch needs from the configuration and the arguments of a run (everything but the scratch pointers).
+void fill_params(const cos_verify_config& c, const cos_verify_args* a, KParams& p) {
+  memset(&p, 0, sizeof(p));
+  p.logits = a->logits;
+  p.s_model = a->stride_model;
+  p.s_row = a->stride_row;
+  p.s_pos = a->stride_pos;
+  p.drafts = a->draft_tokens;
+  p.proposer = a->proposer;
+  p.n = c.n;
+  p.V = c.vocab;
+  p.gamma = c.gamma;
+  p.P = c.gamma + 1;
+  p.B = a->batch;
+  p.mask_model = (c.combine == COS_COMBINE_LOGIT_LINEAR) ? c.mask_model : -1;
+  const int E = entries_per_vec(c.dtype);
+  const int eb = elem_bytes(c.dtype);
+  p.vec_ok = (reinterpret_cast<uintptr_t>(a->logits) % 16 == 0) && ((a->stride_model * eb) % 16 == 0) &&
+             ((a->stride_row * eb) % 16 == 0) && ((a->stride_pos * eb) % 16 == 0);
+  p.nsteps = (c.vocab + 32 * E - 1) / (32 * E);
+  p.flags = a->flags;
+  p.num_units = a->batch * (c.gamma + 1);
+  for (int i = 0; i < COS_MAX_MODELS; ++i) {
+    p.w[i] = (i < c.n) ? c.weights[i] : 0.f;
+    p.w64[i] = static_cast<double>(p.w[i]);
+  }
+  if (c.temperature > 0.0f) {
+    p.cT = static_cast<float>(1.4426950408889634 / static_cast<double>(c.temperature));
+    p.cT64 = static_cast<double>(p.cT);
+  }
+  p.ln_alpha = (p.mask_model >= 0) ? log(static_cast<double>(c.mask_alpha)) : 0.0;
+  p.seed_lo = static_cast<unsigned>(a->seed);
+  p.seed_hi = static_cast<unsigned>(a->seed >> 32);
+  p.off_lo = static_cast<unsigned>(a->offset);
+  p.off_hi = static_cast<unsigned>(a->offset >> 32);
+  p.off_dev = reinterpret_cast<const unsigned long long*>(a->offset_device);
+  p.row_base = a->row_base;
+  p.accept_count = a->accept_count;
+  p.out_tokens = a->out_tokens;
+  p.row_status = a->row_status;
+  p.diag = a->diag;
+  p.dump_r = a->dump_r;
+  p.bonus_prob = a->bonus_prob;
+  p.per_pos = (a->flags & COS_RUN_PROPOSER_PER_POSITION) ? 1 : 0;
+  p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
+  p.greedy = (c.temperature == 0.0f) ? 1 : 0;
+}
+
 cos_status init_scratch(cos_verify_ctx* ctx, cudaStream_t stream) {
   const size_t rows = static_cast<size_t>(ctx->cfg.max_batch);
   cudaError_t e = cudaMemsetAsync(ctx->d_work_counter, 0, 4 * sizeof(unsigned), stream);  // counter and the two exit counts
@@ -2538,49 +2588,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   }
 
   KParams p;
-  memset(&p, 0, sizeof(p));
-  p.logits = a->logits;
-  p.s_model = a->stride_model;
-  p.s_row = a->stride_row;
-  p.s_pos = a->stride_pos;
-  p.drafts = a->draft_tokens;
-  p.proposer = a->proposer;
-  p.n = c.n;
-  p.V = c.vocab;
-  p.gamma = c.gamma;
-  p.P = c.gamma + 1;
-  p.B = a->batch;
-  p.mask_model = (c.combine == COS_COMBINE_LOGIT_LINEAR) ? c.mask_model : -1;
-  const int E = entries_per_vec(c.dtype);
-  p.vec_ok = (reinterpret_cast<uintptr_t>(a->logits) % 16 == 0) && ((a->stride_model * eb) % 16 == 0) &&
-             ((a->stride_row * eb) % 16 == 0) && ((a->stride_pos * eb) % 16 == 0);
-  p.nsteps = (c.vocab + 32 * E - 1) / (32 * E);
-  p.flags = a->flags;
-  p.num_units = a->batch * (c.gamma + 1);
-  for (int i = 0; i < COS_MAX_MODELS; ++i) {
-    p.w[i] = (i < c.n) ? c.weights[i] : 0.f;
-    p.w64[i] = static_cast<double>(p.w[i]);
-  }
-  if (c.temperature > 0.0f) {
-    p.cT = static_cast<float>(1.4426950408889634 / static_cast<double>(c.temperature));
-    p.cT64 = static_cast<double>(p.cT);
-  }
-  p.ln_alpha = (p.mask_model >= 0) ? log(static_cast<double>(c.mask_alpha)) : 0.0;
-  p.seed_lo = static_cast<unsigned>(a->seed);
-  p.seed_hi = static_cast<unsigned>(a->seed >> 32);
-  p.off_lo = static_cast<unsigned>(a->offset);
-  p.off_hi = static_cast<unsigned>(a->offset >> 32);
-  p.off_dev = reinterpret_cast<const unsigned long long*>(a->offset_device);
-  p.row_base = a->row_base;
-  p.accept_count = a->accept_count;
-  p.out_tokens = a->out_tokens;
-  p.row_status = a->row_status;
-  p.diag = a->diag;
-  p.dump_r = a->dump_r;
-  p.bonus_prob = a->bonus_prob;
-  p.per_pos = (a->flags & COS_RUN_PROPOSER_PER_POSITION) ? 1 : 0;
-  p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
-  p.greedy = (c.temperature == 0.0f) ? 1 : 0;
+  fill_params(c, a, p);
   p.work_counter = ctx->d_work_counter;
   p.exit_count = ctx->d_work_counter + 1;
   p.row_arrivals = ctx->d_row_arrivals;
@@ -2849,6 +2857,7 @@ constexpr int kStaticMaxDevices = 64;
 // stand-in, never an address a kernel may use, so the address is asked for once per device.
 unsigned char* g_static_addr[kStaticMaxDevices];
 bool g_static_ready[kStaticMaxDevices];
+std::mutex g_static_mutex;  // first calls from several host threads look the address up once
 
 cos_status static_fail(cos_status st, const char* msg) {
   g_create_error = msg;
@@ -2879,6 +2888,8 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     return static_fail(COS_ERR_INVALID_ARG, "bonus_model outside [0, n)");
   if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4)
     return static_fail(COS_ERR_ALIGNMENT, "bonus_prob is not 4-byte aligned");
+  if (a->offset_device && reinterpret_cast<uintptr_t>(a->offset_device) % 8)
+    return static_fail(COS_ERR_ALIGNMENT, "offset_device is not 8-byte aligned");
   const int eb = elem_bytes(c.dtype);
   if (reinterpret_cast<uintptr_t>(a->logits) % eb) return static_fail(COS_ERR_ALIGNMENT, "logits pointer not aligned to its element type");
   if (reinterpret_cast<uintptr_t>(a->proposer) % 4 || reinterpret_cast<uintptr_t>(a->accept_count) % 4 ||
@@ -2891,13 +2902,16 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   cudaError_t e = cudaSetDevice(c.device);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaSetDevice", e);
   KernelFn fn = pick_kernel(c.dtype, mode_of(c), 0);
-  if (!g_static_ready[c.device]) {
-    // once per device, with that device current: the device address of the built-in array
-    void* addr = nullptr;
-    e = cudaGetSymbolAddress(&addr, g_static_scratch);
-    if (e != cudaSuccess || addr == nullptr) return cuda_fail(nullptr, "cudaGetSymbolAddress(built-in scratch)", e);
-    g_static_addr[c.device] = static_cast<unsigned char*>(addr);
-    g_static_ready[c.device] = true;
+  {
+    std::lock_guard<std::mutex> guard(g_static_mutex);
+    if (!g_static_ready[c.device]) {
+      // once per device, with that device current: the device address of the built-in array
+      void* addr = nullptr;
+      e = cudaGetSymbolAddress(&addr, g_static_scratch);
+      if (e != cudaSuccess || addr == nullptr) return cuda_fail(nullptr, "cudaGetSymbolAddress(built-in scratch)", e);
+      g_static_addr[c.device] = static_cast<unsigned char*>(addr);
+      g_static_ready[c.device] = true;
+    }
   }
   e = prepare_kernels(c.dtype, mode_of(c), c.cluster_size);
   if (e != cudaSuccess) return cuda_fail(nullptr, "cudaFuncSetAttribute", e);
@@ -2932,49 +2946,8 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
   if (e != cudaSuccess) return cuda_fail(nullptr, "clearing the built-in scratch", e);
 
   KParams p;
-  memset(&p, 0, sizeof(p));
-  p.logits = a->logits;
-  p.s_model = a->stride_model;
-  p.s_row = a->stride_row;
-  p.s_pos = a->stride_pos;
-  p.drafts = a->draft_tokens;
-  p.proposer = a->proposer;
-  p.n = c.n;
-  p.V = c.vocab;
-  p.gamma = c.gamma;
-  p.P = c.gamma + 1;
-  p.B = a->batch;
-  p.mask_model = (c.combine == COS_COMBINE_LOGIT_LINEAR) ? c.mask_model : -1;
-  const int E = entries_per_vec(c.dtype);
-  p.vec_ok = (reinterpret_cast<uintptr_t>(a->logits) % 16 == 0) && ((a->stride_model * eb) % 16 == 0) &&
-             ((a->stride_row * eb) % 16 == 0) && ((a->stride_pos * eb) % 16 == 0);
-  p.nsteps = (c.vocab + 32 * E - 1) / (32 * E);
-  p.flags = a->flags;
+  fill_params(c, a, p);
   p.num_units = static_cast<int>(units);
-  for (int i = 0; i < COS_MAX_MODELS; ++i) {
-    p.w[i] = (i < c.n) ? c.weights[i] : 0.f;
-    p.w64[i] = static_cast<double>(p.w[i]);
-  }
-  if (c.temperature > 0.0f) {
-    p.cT = static_cast<float>(1.4426950408889634 / static_cast<double>(c.temperature));
-    p.cT64 = static_cast<double>(p.cT);
-  }
-  p.ln_alpha = (p.mask_model >= 0) ? log(static_cast<double>(c.mask_alpha)) : 0.0;
-  p.seed_lo = static_cast<unsigned>(a->seed);
-  p.seed_hi = static_cast<unsigned>(a->seed >> 32);
-  p.off_lo = static_cast<unsigned>(a->offset);
-  p.off_hi = static_cast<unsigned>(a->offset >> 32);
-  p.off_dev = reinterpret_cast<const unsigned long long*>(a->offset_device);
-  p.row_base = a->row_base;
-  p.accept_count = a->accept_count;
-  p.out_tokens = a->out_tokens;
-  p.row_status = a->row_status;
-  p.diag = a->diag;
-  p.dump_r = a->dump_r;
-  p.bonus_prob = a->bonus_prob;
-  p.per_pos = (a->flags & COS_RUN_PROPOSER_PER_POSITION) ? 1 : 0;
-  p.bonus_model = (a->flags & COS_RUN_BONUS_FROM_MODEL) ? a->bonus_model : -1;
-  p.greedy = (c.temperature == 0.0f) ? 1 : 0;
   p.work_counter = d_counter;
   p.exit_count = d_counter + 1;
   p.row_arrivals = d_arrivals;

@@ -165,6 +165,56 @@ def test_greedy_ensemble_atoms_and_q_zero():
     assert gpu["row_status"][0] & COS_ROW_Q_ZERO
 
 
+@pytest.mark.parametrize("name", ["cfg5_greedy", "cfg2_greedy", "we_greedy"])
+def test_greedy_with_non_finite_logits(name):
+    """T = 0 (Sec. 4.1: one-hot distributions): a NaN or +inf among a position's logits, or a model without a
+    finite maximum, leaves the argmax undefined: the position counts as rejected, no token, NONFINITE; -inf
+    entries are legal while a finite maximum remains.  Rows against the oracle."""
+    if name == "cfg5_greedy":
+        w = C["cfg5_greedy"].scaled(batch=8, vocab=16000, gamma=3, name="greedy_nonfinite")
+    elif name == "cfg2_greedy":
+        w = synth.Workload("cd_greedy", 2, 1, (1.0, -0.5), 0.0, 8, 3, 9001, "bf16", "gauss", sigma=3.0, rho=0.7,
+                           proposer_rule="cycle", mask_model=0, mask_alpha=0.1)
+    else:
+        w = synth.Workload("we_greedy_nf", 3, 0, (0.5, 0.3, 0.2), 0.0, 8, 3, 5000, "f32", "gauss", sigma=2.0, rho=0.5,
+                           proposer_rule="cycle")
+    inputs = synth.make_inputs(w, "cuda")
+    logits = inputs["logits"].clone()
+    logits[0, 0, 0, 17] = float("nan")            # row 0 stops at position 0
+    logits[1, 1, 1, 3] = float("inf")             # row 1 at position 1 at the latest
+    logits[w.n - 1, 2, 2, :] = float("-inf")      # a model with no finite maximum
+    worst = int(torch.argmin(logits[0, 3, 0].float()))
+    logits[0, 3, :, worst] = float("-inf")        # a ruled-out token that is nobody's argmax: harmless
+    mod = dict(inputs, logits=logits)
+    gpu = helpers.run_gpu(w, mod, diag=True)
+    ref = helpers.run_oracle(w, mod)
+    helpers.check_parity(w, gpu, ref, check_diag=False)
+    assert gpu["accept_count"][0] == 0 and gpu["out_tokens"][0, 0] == -1 and gpu["row_status"][0] & COS_ROW_NONFINITE
+    assert gpu["accept_count"][1] <= 1 and gpu["accept_count"][2] <= 2
+    for b in (1, 2):
+        if gpu["row_status"][b] & COS_ROW_NONFINITE:
+            assert gpu["out_tokens"][b, gpu["accept_count"][b]] == -1
+    assert not (gpu["row_status"][3] & COS_ROW_NONFINITE)
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg5", "cfg5_greedy"])
+def test_proposer_index_outside_the_models_is_reported_per_row(name):
+    """A proposer index outside [0, n) names no distribution q: every position of that row reports NONFINITE
+    (so the row stops at position 0 without a token); the other rows are those of the oracle."""
+    w = C[name].scaled(batch=6, vocab=8192, gamma=3, name=f"{name}_bad_proposer")
+    inputs = synth.make_inputs(w, "cuda")
+    prop = inputs["proposer"].clone()
+    prop[1] = w.n
+    prop[4] = -1
+    gpu = helpers.run_gpu(w, dict(inputs, proposer=prop), diag=True)
+    ref = helpers.run_oracle(w, inputs)
+    good = [0, 2, 3, 5]
+    helpers.check_parity(w, gpu, ref, rows=good)
+    for b in (1, 4):
+        assert gpu["accept_count"][b] == 0 and gpu["row_status"][b] & COS_ROW_NONFINITE
+        assert np.all(gpu["out_tokens"][b] == -1)
+
+
 def test_invalid_arguments_return_errors():
     w = _small("cfg3", batch=2, vocab=1024, gamma=2, name="args")
     inputs = synth.make_inputs(w, "cuda")
@@ -213,6 +263,10 @@ def test_early_exit_hint_gives_the_rows_of_the_full_run(name):
         assert np.array_equal(hint[k], full[k]), k
         assert np.array_equal(again[k], full[k]), k
     assert np.array_equal(np.isnan(hint["bonus_prob"]), np.isnan(full["bonus_prob"]))
+    # and a sample of the hinted run's rows against the oracle itself
+    rows = sorted(np.random.default_rng(13).choice(w.batch, size=24, replace=False).tolist())
+    ref = helpers.run_oracle(w, inputs, rows=rows, native=True)
+    helpers.check_parity(w, hint, ref, rows=rows, check_diag=False)
     a = full["accept_count"]
     g = w.gamma
     unread = 0

@@ -51,8 +51,63 @@ def test_static_entry_matches_context_entry_twice(w):
             # ratio, r(x), q(x): same arithmetic, compared within the tolerance of the parity tests
             got, ref = outs["diag"][..., :3].cpu().numpy(), want["diag"][..., :3].cpu().numpy()
             np.testing.assert_allclose(got, ref, rtol=helpers.TOL_R[w.dtype], atol=1e-30, equal_nan=True)
+            # and against the oracle itself, with the bar of the parity tests
+            oracle = helpers.run_oracle(w, dict(inputs, offset=offset))
+            helpers.check_parity(w, {k: t.cpu().numpy() for k, t in outs.items()}, oracle)
     finally:
         verifier.close()
+
+
+def _static_outs(B, P, extra=()):
+    outs = {
+        "accept_count": torch.full((B,), -7, dtype=torch.int32, device="cuda"),
+        "out_tokens": torch.full((B, P), -7, dtype=torch.int32, device="cuda"),
+        "row_status": torch.full((B,), -7, dtype=torch.int32, device="cuda"),
+        "diag": torch.zeros((B, P, 4), dtype=torch.float32, device="cuda"),
+    }
+    if "bonus_prob" in extra:
+        outs["bonus_prob"] = torch.zeros(B, dtype=torch.float32, device="cuda")
+    return outs
+
+
+def _call_static(w, inputs, outs, offset, **kw):
+    binding.run_static(w.n, w.combine, w.weights, w.temperature, w.gamma, w.vocab, inputs["logits"], inputs["drafts"],
+                       inputs["proposer"], inputs["seed"], offset, mask_model=w.mask_model, mask_alpha=w.mask_alpha,
+                       outs=outs, **kw)
+    torch.cuda.synchronize()
+    return {k: t.cpu().numpy() for k, t in outs.items()}
+
+
+def test_static_entry_at_its_limits_and_a_small_call_after_a_large_one():
+    """8192 positions in 1024 rows (both limits at once), then a few rows on the array the large call used."""
+    big = C["cfg1"].scaled(batch=1024, vocab=64, gamma=7, name="static_limits")
+    small = C["cfg3"].scaled(batch=3, vocab=20008, gamma=4, name="static_after_large")
+    for w in (big, small, big):
+        inputs = synth.make_inputs(w, "cuda")
+        got = _call_static(w, inputs, _static_outs(w.batch, w.gamma + 1), inputs["offset"])
+        ref = helpers.run_oracle(w, inputs, native=True)
+        helpers.check_parity(w, got, ref)
+
+
+def test_static_entry_with_the_optional_arguments():
+    """Residual mass everywhere (the job list grows to positions + rows), a named bonus model with its
+    probability, a proposer per position, and a forced cluster size: each twice in a row, against the oracle."""
+    from paper_2502_01662_b200 import COS_RUN_ALL_RESIDUALS
+    w = C["cfg4"].scaled(batch=6, vocab=12808, gamma=3, name="static_opts")
+    inputs = synth.make_inputs(w, "cuda")
+    g = np.random.default_rng(2)
+    table = torch.as_tensor(g.integers(0, w.n, size=(w.batch, w.gamma + 1)).astype(np.int32), device="cuda")
+    for call in range(2):
+        off = inputs["offset"] + call
+        got = _call_static(w, inputs, _static_outs(w.batch, w.gamma + 1), off, flags=COS_RUN_ALL_RESIDUALS)
+        ref = helpers.run_oracle(w, dict(inputs, offset=off), native=True)
+        helpers.check_parity(w, got, ref)
+        np.testing.assert_allclose(got["diag"][:, : w.gamma, 3], ref["S"][:, : w.gamma], rtol=1e-5, atol=1e-7)
+        mod = dict(inputs, proposer=table, offset=off)
+        got = _call_static(w, mod, _static_outs(w.batch, w.gamma + 1, ("bonus_prob",)), off, bonus_model=1)
+        helpers.check_parity(w, got, helpers.run_oracle(w, mod, bonus_model=1, native=True))
+        got = _call_static(w, inputs, _static_outs(w.batch, w.gamma + 1), off, cluster_size=2)
+        helpers.check_parity(w, got, ref)
 
 
 def test_static_entry_rejects_sizes_beyond_the_built_in_scratch():
