@@ -31,7 +31,7 @@ from paper_2502_01662_b200.binding import COS_RUN_EARLY_EXIT  # noqa: E402,F401
 HEADLINE = "cfg3"
 # dram read + write bytes of one launch of the dominant kernel, as RECORDED in the ncu capture summarised under
 # profiles/ (kernel name -> bytes); reported only while the kernel that runs carries the same name
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {"cos_verify_kernel": 355740928}   # profiles/cos_verify_kernel_cfg3.md, stage 0 on workload 3
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 REPORTED = ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "cfg5_greedy")
@@ -196,47 +196,42 @@ def oracle_sample(w, target_seconds=15.0, max_rows=None):
 
 
 def run_reference(args, w):
-    """The oracle, as it stands, on host cores: each step verifies a bounded sample of the workload
-    (whole rows, or the first positions of one row when the step budget is small), sized so that
-    the run ends within a few minutes whatever --steps says."""
+    """The oracle, as it stands, on host cores (its C++ twin, OpenMP over rows, all threads): each step verifies a
+    bounded sample of the workload (whole rows), sized so that the run ends within a few minutes whatever --steps
+    says.  Rank 0 alone runs it."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     import helpers
+    from oracle import cos_oracle_native as nat
     P = w.gamma + 1
-    max_rows = min(4, w.batch)
-    base = synth.make_inputs(w.scaled(batch=max_rows, name=w.name), "cpu")
-    def run_units(units):
-        if units >= P:
-            rows = min(max_rows, units // P)
-            small = w.scaled(batch=max_rows, name=w.name)
-            t0 = time.perf_counter()
-            helpers.run_oracle(small, base, rows=range(rows))
-            return rows * P, time.perf_counter() - t0
-        small = w.scaled(batch=1, gamma=units - 1, name=w.name)
-        part = dict(base, logits=base["logits"][:, :1, :units].contiguous(), drafts=base["drafts"][:1, :units - 1].contiguous(),
-                    proposer=base["proposer"][:1])
+    threads = nat.max_threads()
+    max_rows = min(w.batch, max(1, threads))
+    small = w.scaled(batch=max_rows, name=w.name)
+    base = synth.make_inputs(small, "cpu")
+    def run_rows(rows):
         t0 = time.perf_counter()
-        helpers.run_oracle(small, part)
-        return units, time.perf_counter() - t0
-    _, t_unit = run_units(1)
+        helpers.run_oracle(small, base, rows=range(rows), native=True)
+        return time.perf_counter() - t0
+    t_all = run_rows(max_rows)
     budget = 150.0 / max(1, args.steps + args.warmup)
-    units = int(max(1, min(max_rows * P, budget / max(t_unit, 1e-6))))
+    rows = max_rows if t_all <= budget else max(1, int(max_rows * budget / t_all))
     total_pos, total_t = 0, 0.0
     for k in range(args.warmup + args.steps):
-        done, dt = run_units(units)
+        dt = run_rows(rows)
         if k >= args.warmup:
-            total_pos += done
+            total_pos += rows * P
             total_t += dt
     value = total_pos / total_t
-    sample = (f"{units // P} rows x {P} positions" if units >= P else f"first {units} positions of one row") + f" of {w.name} per step"
+    sample = f"{rows} rows x {P} positions of {w.name} per step (C++ twin of the oracle, {threads} threads)"
     line = {
         "impl": "reference", "metric": "verified draft positions/sec", "value": value, "unit": "positions/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "n": w.n, "B": w.batch, "gamma": w.gamma, "V": w.vocab, "logits": w.dtype},
-        "cpu_baseline": {"value": value, "unit": "positions/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "positions/s", "cores": min(threads, rows), "box_cores": os.cpu_count(),
+                         "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "positions/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -248,7 +243,9 @@ def kernel_names(w, info):
     if info["one_launch"]:
         return ["cos_fused_kernel (every position: sweep, accept tests, row scan, token draw)"]
     names = ["cos_verify_kernel stage 0 (every position: sweep, accept tests, row scan)"]
-    if info["launches_per_run"] == 2:
+    if info["launches_per_run"] == 2 and info.get("draw_items"):
+        names.append("cos_fused_kernel, drawing items only (token draw, one sweep)")
+    elif info["launches_per_run"] == 2:
         names.append("cos_verify_kernel stage 3 (token draw, one sweep)")
     elif info["launches_per_run"] == 3:
         names += ["cos_verify_kernel stage 1 (normalisers of the drawing positions)",
@@ -256,11 +253,14 @@ def kernel_names(w, info):
     return names
 
 
-def measure_workload(w, dev, local, steps, warmup, row_base=0, sampler=None, cluster=0, stage_runs=30):
+def measure_workload(w, dev, local, steps, warmup, row_base=0, sampler=None, cluster=0, stage_runs=30,
+                     try_one_launch=False, one_launch=False):
     """One workload on one GPU: K back-to-back calls between two events, then the launches of a call one by one."""
     peak, _ = measured_peak()
     sets = rotating_inputs(w, dev, 0)
     verifier = make_verifier(w, device=local, cluster_size=cluster)
+    if one_launch:
+        verifier.set_one_launch(True)
     info = verifier.info()
     elapsed, outs = time_device(w, verifier, sets, steps, warmup, row_base, sampler)
     verifier.set_stage_timing(True)
@@ -282,10 +282,27 @@ def measure_workload(w, dev, local, steps, warmup, row_base=0, sampler=None, clu
         # every launch is charged the whole call's algorithmic bytes only if it reads them: the first one does
         gbps = nbytes / (us * 1e-6) / 1e9 if not stages else None
         stages.append({"kernel": name, "us": us, "GBps": gbps, "frac": (gbps / peak) if gbps else None})
+    one_launch_us = drawing_launch_us = None
+    if try_one_launch:
+        v2 = make_verifier(w, device=local)
+        try:
+            v2.set_one_launch(1)
+            t2, _ = time_device(w, v2, sets, max(20, steps // 4), 5, row_base)
+            one_launch_us = 1e6 * t2 / max(20, steps // 4)
+            v2.set_one_launch(2)
+            t3, _ = time_device(w, v2, sets, max(20, steps // 4), 5, row_base)
+            drawing_launch_us = 1e6 * t3 / max(20, steps // 4)
+        except Exception:
+            one_launch_us = None          # the one-launch form does not cover this configuration
+        finally:
+            v2.close()
     res = {"us_per_call": 1e6 * per_call, "positions_per_s": w.positions / per_call, "GBps": nbytes / per_call / 1e9,
            "frac": nbytes / per_call / 1e9 / peak, "frac_of_nominal_8TBps": nbytes / per_call / 1e9 / NOMINAL_HBM_GBS,
            "bytes_per_call": nbytes, "launches_per_call": info["launches_per_run"], "stages": stages,
            "buffers": len(sets), "one_launch": info["one_launch"]}
+    if one_launch_us is not None:
+        res["us_per_call_one_launch_form"] = one_launch_us   # the opt-in single-kernel form of the same run
+        res["us_per_call_persistent_drawing_launch"] = drawing_launch_us   # staged streaming + the persistent kernel's drawing items
     return res, elapsed, outs, info, sets
 
 
@@ -352,6 +369,7 @@ def main():
     ap.add_argument("--config", default=HEADLINE, choices=sorted(synth.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cluster", type=int, default=0, help="thread blocks per position (0 = library default)")
+    ap.add_argument("--one-launch", action="store_true", help="time the opt-in single-kernel form of a run instead")
     ap.add_argument("--headline-only", action="store_true", help="skip the per-workload table and the ceilings")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
@@ -391,7 +409,7 @@ def main():
         dist.barrier()
     torch.cuda.synchronize(dev)
     head, elapsed, outs, info, sets = measure_workload(w, dev, local, args.steps, args.warmup, row_base, sampler,
-                                                       cluster=args.cluster)
+                                                       cluster=args.cluster, one_launch=args.one_launch)
     if dist is not None:
         t = torch.tensor([elapsed], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -423,7 +441,7 @@ def main():
                 table[name] = {k: v for k, v in head.items()}
                 continue
             k2 = 400 if ww.positions * ww.bytes_per_position < (1 << 30) else 100
-            res, _, _, inf2, s2 = measure_workload(ww, dev, local, k2, 5, stage_runs=20)
+            res, _, _, inf2, s2 = measure_workload(ww, dev, local, k2, 5, stage_runs=20, try_one_launch=True)
             del s2
             extra_launches += (k2 + 5 + 25) * inf2["launches_per_run"]
             if name == "cfg2":
@@ -473,11 +491,35 @@ def main():
         dist.destroy_process_group()
 
 
+def native_sample(w, threads, target_seconds=6.0):
+    """The oracle's C++ twin on the first rows of the workload with `threads` host threads (0 = all)."""
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import helpers
+    from oracle import cos_oracle_native as nat
+    used = threads if threads > 0 else nat.max_threads()
+    rows = min(w.batch, max(1, used))
+    small = w.scaled(batch=rows, name=w.name)
+    inputs = synth.make_inputs(small, "cpu")
+    t0 = time.perf_counter()
+    helpers.run_oracle(small, inputs, native=True, threads=threads)
+    t1 = time.perf_counter() - t0
+    reps = int(max(0, min(2000, target_seconds / max(t1, 1e-3) - 1)))
+    for _ in range(reps):
+        helpers.run_oracle(small, inputs, native=True, threads=threads)
+    total = time.perf_counter() - t0
+    return (reps + 1) * rows * (w.gamma + 1) / total, rows, total, used
+
+
 def cpu_baseline(w):
-    """The oracle, as it stands, on this machine's host cores: on one core, on a bounded sample of the workload."""
-    v, rows, dt, passes = oracle_sample(w)
-    return {"value": v, "unit": "positions/s", "cores": 1, "box_cores": os.cpu_count(), "kind": "oracle",
-            "sample": f"first {rows} rows x {w.gamma + 1} positions of {w.name}, {passes} pass(es), {dt:.1f} s"}
+    """The oracle, as it stands, on this machine's host cores, on a bounded sample of the workload: its C++ twin on all
+    cores (the headline value) and on one, and the Python oracle on one core."""
+    v_all, rows_all, dt_all, used = native_sample(w, 0)
+    v_one, rows_one, dt_one, _ = native_sample(w, 1, target_seconds=4.0)
+    v_py, rows_py, dt_py, passes = oracle_sample(w, target_seconds=6.0)
+    return {"value": v_all, "unit": "positions/s", "cores": used, "box_cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"first {rows_all} rows x {w.gamma + 1} positions of {w.name}, {dt_all:.1f} s (C++ twin of the oracle, OpenMP over rows)",
+            "one_thread": {"value": v_one, "sample": f"{rows_one} row(s), {dt_one:.1f} s"},
+            "python_oracle_one_thread": {"value": v_py, "sample": f"{rows_py} row(s), {passes} pass(es), {dt_py:.1f} s"}}
 
 
 def launcher_self_test(args, world, rank):

@@ -140,8 +140,9 @@ typedef struct {
   int32_t launches_per_run;  /* kernels an ordinary cos_verify_run enqueues: 1 at T = 0 and wherever the  */
                              /* one-launch form covers the configuration (reserved[2] == 1); else 2   */
                              /* for logit-level combines and two-model ensembles, 3 otherwise         */
-  int32_t reserved[3];       /* [0], [1]: work items per position when streaming / drawing; [2]: 1    */
-                             /* when an ordinary run is one launch                                    */
+  int32_t reserved[3];       /* [0], [1]: work items per position when streaming / drawing; [2]: bit  */
+                             /* 0: an ordinary run is one launch; bit 1: the tokens of a staged run   */
+                             /* are drawn by the persistent kernel's drawing items                    */
 } cos_verify_info;
 
 /*
@@ -226,11 +227,14 @@ cos_status cos_verify_get_stage_ms(cos_verify_ctx* ctx, float* ms, int32_t* coun
  * The one-launch form of a run (Sec. 3.1-3.2 as ONE persistent kernel): streaming work items of about 128 KB,
  * rows settled as soon as every position up to their first rejection is published, the token draw queued inside
  * the same launch.  It covers sampling runs (T > 0) of ensembles of up to four models and of logit-level combines
- * without mask, with 16-byte aligned rows, at most 16 positions per row and no test hook; `enable` != 0 makes
- * later runs of this context take it (COS_ERR_UNSUPPORTED when the configuration is not covered), 0 returns to
- * the staged launches, which are the default because they are the faster form on the measured workloads.
- * Results are those of the staged form (same arithmetic per position; sums are merged in another order, so
- * probabilities may differ in the last bits).  COS_RUN_EARLY_EXIT is ignored there: every position is read.
+ * without mask, with 16-byte aligned rows, at most 16 positions per row and no test hook.  `enable` = 1 makes
+ * later runs of this context take it (COS_ERR_UNSUPPORTED when the configuration is not covered); `enable` = 2
+ * keeps the staged streaming launch and lets the same persistent kernel draw the tokens in a second launch that
+ * runs only its drawing items (one sweep with a channel sum per model, also for ensembles of three and four
+ * models); 0 returns to the staged launches, which are the default because they are the faster form on the
+ * measured workloads.  Results are those of the staged form (same arithmetic per position; sums are merged in
+ * another order, so probabilities may differ in the last bits).  COS_RUN_EARLY_EXIT is ignored by form 1: every
+ * position is read.
  */
 cos_status cos_verify_set_one_launch(cos_verify_ctx* ctx, int32_t enable);
 

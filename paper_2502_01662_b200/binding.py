@@ -157,7 +157,8 @@ class CosVerifier:
         out = {k: getattr(inf, k) for k in ("cluster_size", "threads_per_block", "max_clusters", "sm_count",
                                             "launches_per_run")}
         out["items_per_position"], out["draw_items_per_position"] = inf.reserved[0], inf.reserved[1]
-        out["one_launch"] = bool(inf.reserved[2])
+        out["one_launch"] = bool(inf.reserved[2] & 1)
+        out["draw_items"] = bool(inf.reserved[2] & 2)   # tokens are drawn by the persistent kernel's drawing items
         return out
 
     def _fill_args(self, logits, drafts, proposer, seed, offset, row_base, flags, outs,
@@ -195,9 +196,10 @@ class CosVerifier:
         a.offset_device = offset_device.data_ptr() if offset_device is not None else None
         return a
 
-    def set_one_launch(self, enable: bool = True):
-        """cos_verify_set_one_launch: later runs take the one-launch kernel (raises if the configuration is not covered)."""
-        self._check(self._lib.cos_verify_set_one_launch(self._ctx, int(bool(enable))))
+    def set_one_launch(self, enable=True):
+        """cos_verify_set_one_launch: 1 / True: later runs take the one-launch kernel; 2: staged streaming launch, tokens
+        drawn by that kernel's drawing items; 0: the staged launches (raises if the configuration is not covered)."""
+        self._check(self._lib.cos_verify_set_one_launch(self._ctx, int(enable)))
 
     def set_wait_limit(self, polls: int, test_drop_report: bool = False):
         """cos_verify_set_wait_limit: bound of the kernel's internal polls (and the test hook that makes one run out)."""

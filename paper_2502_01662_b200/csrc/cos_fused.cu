@@ -31,7 +31,7 @@ constexpr int kSW = 15;           // streaming warps
 constexpr int kST = kSW * 32;     // streaming threads
 constexpr int kRing = 8;          // items a block may have open
 constexpr int kCh = 4;            // channels of a drawing sweep (ensembles of up to four models; logit level: two)
-constexpr int kItemStream = 0, kItemDraw = 1, kItemExit = 3;
+constexpr int kItemStream = 0, kItemDraw = 1, kItemJob = 2, kItemExit = 3;  // kItemJob: a drawing item named by its place in the job list
 // counters, each on a 128-byte line of its own (the queue's head and tail share one: they are read together)
 constexpr int kCtrNext = 0, kCtrEvents = 32, kCtrHead = 64, kCtrTail = 65, kCtrGone = 96, kCtrFault = 128;
 constexpr int kCtrWords = 160;
@@ -44,6 +44,7 @@ __device__ unsigned long long g_prof[32];
 #define PROF_T0 prof_t0 = clock64()
 #define PROF_ADD(k) do { const long long t1_ = clock64(); prof_acc[k] += static_cast<unsigned long long>(t1_ - prof_t0); prof_t0 = t1_; } while (0)
 #define PROF_COUNT(k) prof_acc[k] += 1
+__device__ __forceinline__ unsigned long long prof_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define PROF_FLUSH(base) do { if ((threadIdx.x & 31) == 0) for (int q_ = 0; q_ < 16; ++q_) if (prof_acc[q_]) atomicAdd(&g_prof[(base) + q_], prof_acc[q_]); } while (0)
 #else
 #define PROF_DECL
@@ -62,6 +63,7 @@ struct FParams {
   unsigned total_events;  // positions to publish + rows to settle
   unsigned poll_limit;
   int debug_drop;
+  int draw_only;          // the positions were published by an earlier launch; this one draws the tokens of its job list
 };
 
 struct ItemCtx {
@@ -78,6 +80,11 @@ struct FShared {
   int arrive[kRing];    // streaming warps that have finished the item of that slot
   int started;          // number of items some warp has begun
   int fault;
+  int num_items;        // items handed out by the counter
+  unsigned total_events;
+  // drawing-only launch: rows whose drawing sweep is complete, handed from the service warp to the locating warp
+  int loc_ring[8];
+  int loc_tail, loc_head, loc_exit;
   ItemCtx ctx[kRing];
   SoftPart part[kRing][kSW][kCh];
 };
@@ -245,13 +252,22 @@ __device__ __forceinline__ void stream_item(const FParams& fp, const ItemCtx& it
   }
 }
 
+template <int N>
+struct RawSet {
+  uint4 r[N];
+};
+
 // A vector of a drawing sweep that holds a big entry (more than 2^-8 of a normaliser), done again entry by entry from
-// the stored logits: big entries in fp64 into the thread's slots (`bigacc[q * kST]`: q < NCH the normalisers,
-// NCH <= q < 2 NCH the step sums), the others as the sweep does them, returned in zs / as.  Rare; out of line.
-template <int DT, int MODE, int NCH>
-__device__ __noinline__ void draw_big_vector(const KParams& p, const ItemCtx& c, const char* base, int e0, double* bigacc,
-                                             float* zs, float* as) {
+// the vectors at hand (models beyond those are read again): big entries in fp64 into the thread's slots
+// (`bigacc[q * kST]`: q < NCH the normalisers, NCH <= q < 2 NCH the step sums), the others as the sweep does
+// them, returned in zs / as.  Rare; out of line.
+template <int DT, int MODE, int NCH, int NL>
+__device__ __noinline__ void draw_big_vector(const KParams& p, const ItemCtx& c, RawSet<NL> raw, const char* base, int e0,
+                                             double* bigacc, float* zs, float* as) {
   constexpr int E = Elem<DT>::E;
+  float xs[NL][E];
+#pragma unroll
+  for (int i = 0; i < NL; ++i) Elem<DT>::unpack(raw.r[i], xs[i]);
   for (int k = 0; k < E; ++k) {
     const int e = e0 + k;
     if (e >= p.V) break;
@@ -259,14 +275,14 @@ __device__ __noinline__ void draw_big_vector(const KParams& p, const ItemCtx& c,
     double x64[NCH];
     if (MODE == kEnsembleSample) {
       for (int i = 0; i < NCH; ++i) {
-        x[i] = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
+        x[i] = xs[i < NL ? i : 0][k];
         x64[i] = static_cast<double>(x[i]);
       }
     } else {
       float xb = 0.f, xa = 0.f;
       double cb = 0.0;
       for (int i = 0; i < p.n; ++i) {
-        const float v = Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
+        const float v = (i < NL) ? xs[i][k] : Elem<DT>::load1(base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes, e);
         xb = fmaf(p.w[i], v, xb);
         cb = fma(p.w64[i], static_cast<double>(v), cb);
         if (i == c.pis) xa = v;
@@ -339,6 +355,10 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
       nx[i] = (v < fp.nvec && i < nl) ? ldg_ahead16(base + i * row_step + static_cast<long long>(v) * 16) : ninf_vec<DT>();
   };
   double* rec = fp.s.srec + static_cast<size_t>(it.b) * p.nsteps * NCH;
+#ifdef COS_FUSED_PROFILE
+  long long dt0 = clock64(), dt_first = 0;
+  unsigned long long dsteps = 0;
+#endif
   if (it.lo + warp < it.hi) fetch(it.lo + warp);
   for (int s = it.lo + warp; s < it.hi; s += kSW) {
     uint4 cur[NL];
@@ -396,7 +416,10 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
     if (big) {
       float rz[NCH], ra[NCH];
       for (int i = 0; i < NCH; ++i) rz[i] = ra[i] = 0.f;
-      draw_big_vector<DT, MODE, NCH>(p, it, base, v * E, bigacc, rz, ra);
+      RawSet<NL> rs;
+#pragma unroll
+      for (int i = 0; i < NL; ++i) rs.r[i] = cur[i];
+      draw_big_vector<DT, MODE, NCH, NL>(p, it, rs, base, v * E, bigacc, rz, ra);
 #pragma unroll
       for (int i = 0; i < NCH; ++i) {
         zs[i] += rz[i];
@@ -435,7 +458,14 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
       for (int i = 1; i < NCH; ++i) mine = (lane == i) ? da[i] : mine;
       __stcg(rec + static_cast<size_t>(s) * NCH + lane, mine);
     }
+#ifdef COS_FUSED_PROFILE
+    if (dsteps == 0) dt_first = clock64();
+    ++dsteps;
+#endif
   }
+#ifdef COS_FUSED_PROFILE
+  const long long dt_loop = clock64();
+#endif
   // this warp's share of the refined normalisers
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
@@ -447,9 +477,18 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
       part[i].ref = 0.f;
     }
   }
+#ifdef COS_FUSED_PROFILE
+  if (warp == 0 && lane == 0 && dsteps > 0) {
+    atomicAdd(&g_prof[8], static_cast<unsigned long long>(dt_first - dt0));   // up to the end of the first step
+    atomicAdd(&g_prof[9], static_cast<unsigned long long>(dt_loop - dt_first)); // the other steps
+    atomicAdd(&g_prof[10], static_cast<unsigned long long>(clock64() - dt_loop)); // normaliser shares
+    atomicAdd(&g_prof[11], dsteps - 1);
+    atomicAdd(&g_prof[12], 1ull);
+  }
+#endif
 }
 
-template <int DT, int MODE, int NCH>
+template <int DT, int MODE, int NCH, bool DRAW_ONLY>
 __device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, double* bigacc_all) {
   const int stid = threadIdx.x, lane = stid & 31, warp = stid >> 5;
   double* bigacc = bigacc_all + stid;
@@ -478,7 +517,7 @@ __device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, doub
     __syncwarp();
     const ItemCtx& it = sh.ctx[slot];
     if (it.kind == kItemExit) break;
-    if (it.kind == kItemStream) {
+    if (!DRAW_ONLY && it.kind == kItemStream) {
       stream_item<DT, MODE>(fp, it, &sh.part[slot][warp][0], stid);
       PROF_ADD(1);
       PROF_COUNT(4);
@@ -962,7 +1001,7 @@ __device__ __forceinline__ uint2 vol_load2(const unsigned* p) {
 // add.  Under a race the ticket may lie beyond the tail; it then names the entry this block takes as soon as
 // somebody writes it (`ticket` is kept across calls; a block holds one ticket at most).  Nobody spins on the
 // queue, and every entry has exactly one taker, who cannot leave before the run is complete.
-__device__ __forceinline__ int take_item(const FParams& fp, bool& static_left, int& ticket) {
+__device__ __forceinline__ int take_item(const FParams& fp, int num_items, bool& static_left, int& ticket) {
   if (ticket < 0) {
     const uint2 ht = vol_load2(&fp.s.ctr[kCtrHead]);  // head, tail
     if (ht.y > ht.x) ticket = static_cast<int>(atomicAdd(&fp.s.ctr[kCtrHead], 1u));
@@ -978,7 +1017,11 @@ __device__ __forceinline__ int take_item(const FParams& fp, bool& static_left, i
   }
   if (static_left) {
     const unsigned t = atomicAdd(&fp.s.ctr[kCtrNext], 1u);
-    if (t < static_cast<unsigned>(fp.num_items)) {
+    if (t < static_cast<unsigned>(num_items)) {
+      if (fp.draw_only) {
+        const int job = static_cast<int>(t) / fp.plan.dchunks, c = static_cast<int>(t) % fp.plan.dchunks;
+        return (kItemJob << 30) | (job << 8) | c;
+      }
       const int unit = static_cast<int>(t) / fp.plan.chunks, c = static_cast<int>(t) % fp.plan.chunks;
       return (kItemStream << 30) | (unit << 8) | c;
     }
@@ -1007,9 +1050,19 @@ __device__ __forceinline__ void fill_ctx(const FParams& fp, ItemCtx& cx, int des
       cx.hi = hi < fp.nvec ? hi : fp.nvec;
     }
   } else {
-    const int b = id;
-    const int rd = __ldcg(&fp.s.row_draw[b]);
-    const int j = rd & 0xff, dkind = rd >> 8;
+    int b = id, j, dkind;
+    if (kind == kItemJob) {
+      // the id-th entry of the job list an earlier launch left: the one position of its row that draws a token
+      const int idx = __ldcg(&p.jobs[id]).x;
+      b = idx / p.P;
+      j = idx % p.P;
+      dkind = (j < p.gamma) ? kDrawResidual : (p.bonus_model >= 0 ? kDrawQ : kDrawR);
+      if (lane == 0) __stcg(&fp.s.row_draw[b], j | (dkind << 8));  // every chunk of the row writes the same word
+    } else {
+      const int rd = __ldcg(&fp.s.row_draw[b]);
+      j = rd & 0xff;
+      dkind = rd >> 8;
+    }
     const int pis = proposer_of(p, b, j);
     const int uidx = b * p.P + j;
     if (lane == 0) {
@@ -1037,7 +1090,24 @@ __device__ __forceinline__ void fill_ctx(const FParams& fp, ItemCtx& cx, int des
   __syncwarp();
 }
 
-template <int DT, int MODE, int NCH>
+constexpr int kLocateChunk = 0xff;  // a queue entry with this chunk number asks for a row's token to be located
+
+// Service warp: hand row b to this block's locating warp if that warp has nothing else to do.  Whole warp.
+__device__ __forceinline__ bool hand_to_locator(FShared& sh, int b, int lane) {
+  int ok = 0;
+  if (lane == 0) {
+    const int tail = vol_load(&sh.loc_tail), head = vol_load(&sh.loc_head);
+    if (tail == head) {
+      *reinterpret_cast<volatile int*>(&sh.loc_ring[tail & 7]) = b;
+      __threadfence_block();
+      *reinterpret_cast<volatile int*>(&sh.loc_tail) = tail + 1;
+      ok = 1;
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+template <int DT, int MODE, int NCH, bool DRAW_ONLY>
 __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
   const KParams& p = fp.k;
   const int lane = threadIdx.x & 31;
@@ -1046,17 +1116,34 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
   int ticket = -1;
   unsigned idle = 0;
   bool failed = false;
+  // Looking for work reads two lines of L2 that every block shares.  A block that found nothing looks again only
+  // after a pause that grows with every empty look (to a few loop turns): hundreds of blocks asking every 100 ns keep one
+  // L2 slice so busy that every load of the device that maps to it waits behind them.
+  unsigned empty_looks = 0, skip = 0;
+#ifdef COS_FUSED_PROFILE
+  const unsigned long long t_begin = prof_now();
+  bool stamped = false;
+#endif
   PROF_DECL;
   PROF_T0;
   while (true) {
     bool did = false;
     // ---- fetch up to two items ahead of the fastest streaming warp
-    if (fetched < processed + kRing && fetched <= vol_load(&sh.started) + 1) {
+    if (skip > 0) --skip;
+    // (a drawing-only launch has few, short items per block: one item ahead, so that no block sits on work another
+    // block is idle for)
+    if (skip == 0 && fetched < processed + kRing && fetched <= vol_load(&sh.started) + (DRAW_ONLY ? 0 : 1)) {
       int desc = -1;
-      if (lane == 0) desc = take_item(fp, static_left, ticket);
+      if (lane == 0) desc = take_item(fp, sh.num_items, static_left, ticket);
       desc = __shfl_sync(0xffffffffu, desc, 0);
       static_left = __shfl_sync(0xffffffffu, static_left ? 1 : 0, 0) != 0;
-      if (desc >= 0) {
+      if (DRAW_ONLY && desc != -1 && (desc & 0xff) == kLocateChunk) {
+        // a row whose sweep is complete, passed on by a block whose locating warp was busy
+        const int b = (desc >> 8) & 0x3fffff;
+        if (!hand_to_locator(sh, b, lane)) locate_token<DT, MODE, NCH>(fp, b);
+        did = true;
+        empty_looks = 0;
+      } else if (desc != -1) {
         PROF_ADD(0);  // taking an item
         fill_ctx<MODE>(fp, sh.ctx[fetched & (kRing - 1)], desc);
         PROF_ADD(1);
@@ -1066,12 +1153,21 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
         }
         ++fetched;
         did = true;
-      } else if (processed == fetched) {
+        empty_looks = 0;
+      } else {
+#ifdef COS_FUSED_PROFILE
+        if (!stamped && !static_left && lane == 0) atomicMax(&g_prof[13], prof_now() - t_begin);
+        if (!static_left) stamped = true;
+#endif
+        empty_looks = empty_looks < 4 ? empty_looks + 1 : 4;
+        skip = empty_looks;  // loop turns (each sleeps 100 to 200 ns, in practice rather more)
+      }
+      if (desc == -1 && processed == fetched) {
         // nothing open here and nothing to take: done once every position is published and every row settled
         unsigned ev = 0;
         if (lane == 0) ev = vol_load(&fp.s.ctr[kCtrEvents]);
         ev = __shfl_sync(0xffffffffu, ev, 0);
-        if (ev >= fp.total_events) break;
+        if (ev >= sh.total_events) break;
       }
     }
     // ---- the oldest open item, once every streaming warp has reported it
@@ -1084,7 +1180,7 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
         __threadfence_block();
         const ItemCtx& cx = sh.ctx[slot];
         const int b = cx.b, j = cx.j, c = cx.chunk;
-        if (cx.kind == kItemStream) {
+        if (!DRAW_ONLY && cx.kind == kItemStream) {
           const int ns = fp.plan.nslots, C = fp.plan.chunks;
           const int uidx = b * p.P + j;
           SoftPart merged[kCh > 2 ? kCh : 2];
@@ -1134,7 +1230,22 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
           prev = __shfl_sync(0xffffffffu, prev, 0);
           PROF_ADD(4);  // a drawing chunk reported
           if (prev == fp.plan.dchunks - 1) {
-            locate_token<DT, MODE, NCH>(fp, b);
+            // the row's sweep is complete.  A drawing-only launch has a warp that does nothing but locate tokens,
+            // so that this warp stays free to report the other rows' chunks; it takes the row unless its ring is full
+            // ... so that this warp stays free; if that warp is busy the row goes to the queue, for any block to take
+            bool handed = false;
+            if (DRAW_ONLY) {
+              handed = hand_to_locator(sh, b, lane);
+              if (!handed) {
+                if (lane == 0) {
+                  __threadfence();
+                  const unsigned at = atomicAdd(&fp.s.ctr[kCtrTail], 1u);
+                  if (at < static_cast<unsigned>(fp.plan.dq_cap)) atomicExch(&fp.s.dq[at], ((kItemDraw << 30) | (b << 8) | kLocateChunk) + 1);
+                }
+                handed = true;
+              }
+            }
+            if (!handed) locate_token<DT, MODE, NCH>(fp, b);
             PROF_ADD(5);
             PROF_COUNT(9);
           }
@@ -1167,8 +1278,12 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
     for (int b = lane; b < p.B; b += 32) atomicOr(&p.row_status[b], static_cast<unsigned>(COS_ROW_FAULT));
   }
   PROF_FLUSH(16);
-  // tell the streaming warps to leave
+#ifdef COS_FUSED_PROFILE
+  if (lane == 0) atomicMax(&g_prof[14], prof_now() - t_begin);
+#endif
+  // tell the streaming warps (and the locating warp) to leave
   if (lane == 0) {
+    *reinterpret_cast<volatile int*>(&sh.loc_exit) = 1;
     ItemCtx& cx = sh.ctx[fetched & (kRing - 1)];
     cx.kind = kItemExit;
     __threadfence_block();
@@ -1184,13 +1299,20 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
       fp.s.ctr[kCtrTail] = 0u;
       fp.s.ctr[kCtrGone] = 0u;
       fp.s.ctr[kCtrFault] = faulted ? 2u : 0u;  // 2: the scratch may be dirty; the host clears it before the next run
+      if (fp.draw_only) {  // what the staged launches leave clean for the next run
+        *fp.k.job_count = 0;
+        *fp.k.work_counter = 0u;
+      }
       __threadfence();
     }
   }
 }
 
-template <int DT, int MODE, int NCH>
-__global__ void __launch_bounds__(kFT, 2) cos_fused_kernel(const __grid_constant__ FParams fp) {
+// DRAW_ONLY: the launch that only draws tokens (after a staged launch published the positions).  It is compiled
+// without the streaming code and for one block per multiprocessor, so that the drawing sweep keeps its working set in
+// registers; the one-launch form needs two blocks per multiprocessor to stream at full rate.
+template <int DT, int MODE, int NCH, bool DRAW_ONLY>
+__global__ void __launch_bounds__(DRAW_ONLY ? kFT + 32 : kFT, 1) cos_fused_kernel(const __grid_constant__ FParams fp) {
   __shared__ FShared sh;
   extern __shared__ double bigacc[];  // [2 * NCH][kST]: fp64 sums of the big terms of a drawing sweep, one slot per thread
   const int tid = threadIdx.x;
@@ -1198,35 +1320,91 @@ __global__ void __launch_bounds__(kFT, 2) cos_fused_kernel(const __grid_constant
     sh.tag[tid] = 0;
     sh.arrive[tid] = 0;
   }
+  // (after a launch that published the positions: started while it drained; nothing it wrote is read before this)
+  if (fp.draw_only) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid == 0) {
     sh.started = 0;
     sh.fault = 0;
+    sh.loc_tail = sh.loc_head = sh.loc_exit = 0;
+    if (fp.draw_only) {
+      int njobs = __ldcg(fp.k.job_count);
+      njobs = njobs < fp.k.max_jobs ? njobs : fp.k.max_jobs;
+      sh.num_items = njobs * fp.plan.dchunks;
+      sh.total_events = static_cast<unsigned>(njobs);
+    } else {
+      sh.num_items = fp.num_items;
+      sh.total_events = fp.total_events;
+    }
   }
   __syncthreads();
-  if (tid < kST)
-    stream_role<DT, MODE, NCH>(fp, sh, bigacc);
-  else
-    service_role<DT, MODE, NCH>(fp, sh);
+  if (tid < kST) {
+    stream_role<DT, MODE, NCH, DRAW_ONLY>(fp, sh, bigacc);
+  } else if (tid < kFT) {
+    service_role<DT, MODE, NCH, DRAW_ONLY>(fp, sh);
+  } else {
+    // the locating warp of a drawing-only launch: rows in the order the service warp hands them over
+    const int lane = tid & 31;
+    int head = 0;
+    for (unsigned long long it = 0; it < 16ull * fp.poll_limit; ++it) {
+      int tail = 0, leave = 0;
+      if (lane == 0) {
+        tail = vol_load(&sh.loc_tail);
+        leave = vol_load(&sh.loc_exit) | vol_load(&sh.fault);
+      }
+      tail = __shfl_sync(0xffffffffu, tail, 0);
+      leave = __shfl_sync(0xffffffffu, leave, 0);
+      if (head < tail) {
+        __syncwarp();
+        const int b = vol_load(&sh.loc_ring[head & 7]);
+#ifdef COS_FUSED_PROFILE
+        const unsigned long long tl0 = prof_now();
+#endif
+        locate_token<DT, MODE, NCH>(fp, b);
+#ifdef COS_FUSED_PROFILE
+        if (lane == 0) {
+          atomicAdd(&g_prof[7], prof_now() - tl0);
+          atomicAdd(&g_prof[15], 1ull);
+        }
+#endif
+        ++head;
+        if (lane == 0) {
+          __threadfence_block();
+          *reinterpret_cast<volatile int*>(&sh.loc_head) = head;
+        }
+        it = 0;
+      } else if (leave) {
+        break;
+      } else {
+        __nanosleep(100);
+      }
+    }
+  }
 }
 
 using FusedFn = void (*)(const FParams);
 
-template <int DT>
+template <int DT, bool DRAW_ONLY>
 FusedFn pick_dt(int mode, int n) {
-  if (mode == kLogitSample) return cos_fused_kernel<DT, kLogitSample, 2>;
+  if (mode == kLogitSample) return cos_fused_kernel<DT, kLogitSample, 2, DRAW_ONLY>;
   if (mode == kEnsembleSample) {
-    if (n == 1) return cos_fused_kernel<DT, kEnsembleSample, 1>;
-    if (n == 2) return cos_fused_kernel<DT, kEnsembleSample, 2>;
-    if (n == 3) return cos_fused_kernel<DT, kEnsembleSample, 3>;
-    if (n == 4) return cos_fused_kernel<DT, kEnsembleSample, 4>;
+    if (n == 1) return cos_fused_kernel<DT, kEnsembleSample, 1, DRAW_ONLY>;
+    if (n == 2) return cos_fused_kernel<DT, kEnsembleSample, 2, DRAW_ONLY>;
+    if (n == 3) return cos_fused_kernel<DT, kEnsembleSample, 3, DRAW_ONLY>;
+    if (n == 4) return cos_fused_kernel<DT, kEnsembleSample, 4, DRAW_ONLY>;
   }
   return nullptr;
 }
 
-FusedFn pick_fused(int dtype, int mode, int n) {
-  if (dtype == COS_DTYPE_F32) return pick_dt<COS_DTYPE_F32>(mode, n);
-  if (dtype == COS_DTYPE_BF16) return pick_dt<COS_DTYPE_BF16>(mode, n);
-  if (dtype == COS_DTYPE_F16) return pick_dt<COS_DTYPE_F16>(mode, n);
+FusedFn pick_fused(int dtype, int mode, int n, bool draw_only = false) {
+  if (draw_only) {
+    if (dtype == COS_DTYPE_F32) return pick_dt<COS_DTYPE_F32, true>(mode, n);
+    if (dtype == COS_DTYPE_BF16) return pick_dt<COS_DTYPE_BF16, true>(mode, n);
+    if (dtype == COS_DTYPE_F16) return pick_dt<COS_DTYPE_F16, true>(mode, n);
+    return nullptr;
+  }
+  if (dtype == COS_DTYPE_F32) return pick_dt<COS_DTYPE_F32, false>(mode, n);
+  if (dtype == COS_DTYPE_BF16) return pick_dt<COS_DTYPE_BF16, false>(mode, n);
+  if (dtype == COS_DTYPE_F16) return pick_dt<COS_DTYPE_F16, false>(mode, n);
   return nullptr;
 }
 
@@ -1290,7 +1468,8 @@ FusedPlan fused_plan(int dtype, int mode, int n, int vocab, int gamma, int max_b
   pl.nslots = (mode == kEnsembleSample) ? n : 2;
   pl.nch = channels_of(mode, n);
   pl.blocks = sm_count * (blocks_per_sm > 0 ? blocks_per_sm : 1);
-  pl.dq_cap = 2 * max_batch * pl.dchunks;  // a row queues its items once, twice when the residual turns out empty
+  pl.draw_blocks = sm_count;
+  pl.dq_cap = 2 * max_batch * (pl.dchunks + 1);  // a row queues its items once (twice when the residual turns out empty), and may be queued for locating
   (void)gamma;
   return pl;
 }
@@ -1315,13 +1494,16 @@ cudaError_t fused_occupancy(int dtype, int mode, int n, int* blocks_per_sm) {
   if (fn == nullptr) return cudaErrorInvalidDeviceFunction;
   cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(fused_smem(mode, n)));
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_fused(dtype, mode, n, true)),
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem(mode, n)));
   if (e != cudaSuccess) return e;
   return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void*>(fn), kFT, fused_smem(mode, n));
 }
 
 cudaError_t fused_launch(int dtype, int mode, const KParams& p, const FusedPlan& plan, const FusedScratch& scratch,
-                         unsigned poll_limit, int debug_drop, cudaStream_t stream) {
-  FusedFn fn = pick_fused(dtype, mode, p.n);
+                         unsigned poll_limit, int debug_drop, bool draw_only, cudaStream_t stream) {
+  FusedFn fn = pick_fused(dtype, mode, p.n, draw_only);
   if (fn == nullptr) return cudaErrorInvalidDeviceFunction;
   FParams fp;
   fp.k = p;
@@ -1333,10 +1515,21 @@ cudaError_t fused_launch(int dtype, int mode, const KParams& p, const FusedPlan&
   fp.total_events = static_cast<unsigned>(p.num_units + p.B);
   fp.poll_limit = poll_limit;
   fp.debug_drop = debug_drop;
-  int blocks = plan.blocks;
-  if (blocks > fp.num_items) blocks = fp.num_items;
-  fn<<<blocks, kFT, fused_smem(mode, p.n), stream>>>(fp);
-  return cudaGetLastError();
+  fp.draw_only = draw_only ? 1 : 0;
+  int blocks = draw_only ? plan.draw_blocks : plan.blocks;
+  const int most = draw_only ? p.B * plan.dchunks : fp.num_items;
+  if (blocks > most) blocks = most;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  lc.blockDim = dim3(draw_only ? kFT + 32 : kFT, 1, 1);
+  lc.dynamicSmemBytes = fused_smem(mode, p.n);
+  lc.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at;
+  lc.numAttrs = draw_only ? 1 : 0;  // a drawing launch starts while the launch before it drains
+  return cudaLaunchKernelEx(&lc, fn, fp);
 }
 
 }  // namespace cosv

@@ -15,7 +15,8 @@ struct FusedPlan {
   int dchunks, dchunk_steps;  // drawing: the same for the one (row, position) of a row that draws a token
   int nslots;                 // softmax statistics per (row, position): n (ensemble) or 2 (logit level)
   int nch;                    // channel sums per step of a drawing sweep: n (ensemble) or 2
-  int blocks;                 // persistent blocks of the launch
+  int blocks;                 // persistent blocks of the one-launch form (two per multiprocessor)
+  int draw_blocks;            // persistent blocks of a launch that only draws tokens (one per multiprocessor)
   int dq_cap;                 // entries of the queue of drawing items
 };
 
@@ -46,8 +47,10 @@ cudaError_t fused_occupancy(int dtype, int mode, int n, int* blocks_per_sm);
 // Enqueue the launch.  `p` is filled as for the staged kernels; plan/scratch come from the context.
 // `poll_limit`: idle polls after which a block that sees no progress gives up (COS_ROW_FAULT on every row).
 // `debug_drop`: test hook; when non-zero, one streaming warp of block 0 never reports its first item.
+// `draw_only`: the positions were published by the staged launch before this one (its job list names, per row, the
+// position that draws a token); this launch then only draws those tokens.
 cudaError_t fused_launch(int dtype, int mode, const KParams& p, const FusedPlan& plan, const FusedScratch& scratch,
-                         unsigned poll_limit, int debug_drop, cudaStream_t stream);
+                         unsigned poll_limit, int debug_drop, bool draw_only, cudaStream_t stream);
 
 }  // namespace cosv
 

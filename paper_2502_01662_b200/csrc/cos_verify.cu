@@ -2125,6 +2125,7 @@ struct cos_verify_ctx {
   // the one-launch form of a run (sampling modes the fused kernel covers, no cluster size requested)
   bool fused;      // the one-launch kernel covers this configuration (its scratch is allocated)
   bool use_fused;  // and runs take it (cos_verify_set_one_launch)
+  bool draw_fused; // staged runs draw their tokens with that kernel's drawing items
   FusedPlan fplan;
   FusedScratch fscr;
   void* fused_mem[9];
@@ -2483,6 +2484,7 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   ctx->wait_limit = 1u << 20;
   ctx->test_drop = 0;
   ctx->fused = false;
+  ctx->draw_fused = false;
   if (ok && config->cluster_size == 0 &&
       fused_covers(config->dtype, mode_of(*config), config->n, config->vocab, config->gamma,
                    config->combine == COS_COMBINE_LOGIT_LINEAR ? config->mask_model : -1,
@@ -2614,7 +2616,7 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     p.early_exit = 0;
     ctx->scratch_dirty = true;
     if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
-    e = fused_launch(c.dtype, mode, p, ctx->fplan, ctx->fscr, ctx->wait_limit, ctx->test_drop, stream);
+    e = fused_launch(c.dtype, mode, p, ctx->fplan, ctx->fscr, ctx->wait_limit, ctx->test_drop, false, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (one-launch form)", e);
     if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
     ctx->ev_used = 2;
@@ -2648,6 +2650,16 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
     // Two channel sums describe every mass when the combine is at logit level (proposer, combined logits) or
     // mixes two models: then one sweep does the work of stages 1 and 2.  The test hooks keep the two-stage form.
     const bool one_sweep = !all && (mode == kLogitSample || c.n == 2);
+    if (!all && ctx->fused && ctx->draw_fused && p.vec_ok) {
+      // the tokens are drawn by the persistent kernel's drawing items (one sweep with a channel sum per model, any
+      // block takes any chunk of any row) instead of the drawing stages
+      e = fused_launch(c.dtype, mode, p, ctx->fplan, ctx->fscr, ctx->wait_limit, 0, true, stream);
+      if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing items)", e);
+      if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
+      ctx->ev_used = 3;
+      ctx->scratch_dirty = false;
+      return COS_OK;
+    }
     if (one_sweep) {
       p.parts = ctx->parts_one;
       p.num_clusters = (most < cap ? most : cap) * p.parts;
@@ -2770,7 +2782,8 @@ extern "C" cos_status cos_verify_set_one_launch(cos_verify_ctx* ctx, int32_t ena
     ctx->err = "the one-launch form does not cover this configuration";
     return COS_ERR_UNSUPPORTED;
   }
-  ctx->use_fused = enable != 0;
+  ctx->use_fused = (enable == 1);
+  ctx->draw_fused = (enable == 2);
   return COS_OK;
 }
 
@@ -2796,12 +2809,13 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
     // ordinary runs (no test hook): one launch at T = 0; else stage 0 and the one-sweep drawing stage where two
     // channel sums describe a mass, stages 0, 1 and 2 otherwise
     const int mode = mode_of(ctx->cfg);
-    const bool one_sweep = (mode == kLogitSample) || (mode == kEnsembleSample && ctx->cfg.n == 2);
+    const bool one_sweep = (mode == kLogitSample) || (mode == kEnsembleSample && ctx->cfg.n == 2) ||
+                           (ctx->fused && ctx->draw_fused);
     info->launches_per_run = (ctx->cfg.temperature > 0.0f && !(ctx->fused && ctx->use_fused)) ? (one_sweep ? 2 : 3) : 1;
   }
   info->reserved[0] = ctx->fused ? ctx->fplan.chunks : ctx->parts;
   info->reserved[1] = ctx->fused ? ctx->fplan.dchunks : ctx->parts_one;
-  info->reserved[2] = (ctx->fused && ctx->use_fused) ? 1 : 0;
+  info->reserved[2] = ((ctx->fused && ctx->use_fused) ? 1 : 0) | ((ctx->fused && ctx->draw_fused) ? 2 : 0);
   return COS_OK;
 }
 

@@ -11,10 +11,12 @@ pytestmark = pytest.mark.gpu
 C = synth.CONFIGS
 
 
-def one_launch_verifier(w, **kw):
+def one_launch_verifier(w, form=1, **kw):
+    """form 1: the whole run in one launch; form 2: staged streaming launch, tokens drawn by the persistent kernel."""
     v = helpers.make_verifier(w, **kw)
-    v.set_one_launch(True)
-    assert v.info()["one_launch"] and v.info()["launches_per_run"] == 1
+    v.set_one_launch(form)
+    info = v.info()
+    assert (info["one_launch"] and info["launches_per_run"] == 1) if form == 1 else (info["draw_items"] and info["launches_per_run"] == 2)
     return v
 
 
@@ -37,10 +39,11 @@ SMALL = [
 ]
 
 
+@pytest.mark.parametrize("form", [1, 2])
 @pytest.mark.parametrize("w", SMALL, ids=[w.name for w in SMALL])
-def test_one_launch_matches_the_oracle(w):
+def test_one_launch_matches_the_oracle(w, form):
     inputs = synth.make_inputs(w, "cuda")
-    v = one_launch_verifier(w)
+    v = one_launch_verifier(w, form)
     try:
         gpu = helpers.run_gpu(w, inputs, verifier=v, diag=True)
         again = helpers.run_gpu(w, inputs, verifier=v, diag=True)      # the scratch was left clean; results do not depend on scheduling
@@ -60,12 +63,13 @@ def test_one_launch_matches_the_oracle(w):
             np.testing.assert_allclose(gpu["diag"][b, a[b], 3], ref["S"][b, a[b]], rtol=1e-5, atol=1e-7)
 
 
+@pytest.mark.parametrize("form", [1, 2])
 @pytest.mark.parametrize("name,nrows", [("cfg3", 64), ("cfg4", 32), ("cfg5", 32)])
-def test_one_launch_full_size(name, nrows):
+def test_one_launch_full_size(name, nrows, form):
     w = C[name]
     inputs = synth.make_inputs(w, "cuda")
     rows = sorted(np.random.default_rng(5).choice(w.batch, size=min(nrows, w.batch), replace=False).tolist())
-    v = one_launch_verifier(w)
+    v = one_launch_verifier(w, form)
     try:
         gpu = helpers.run_gpu(w, inputs, verifier=v, diag=True)
         again = helpers.run_gpu(w, inputs, verifier=v)
@@ -95,13 +99,14 @@ def test_one_launch_alternate_proposals_and_bonus_model():
     drafts[:4] = torch.argmax(inputs["logits"][0, :4, : w.gamma].float(), dim=-1).to(torch.int32)
     mod = dict(inputs, proposer=table, drafts=drafts)
     for bonus in (-1, 2):
-        v = one_launch_verifier(w)
-        try:
-            gpu = helpers.run_gpu(w, mod, verifier=v, diag=True, bonus_model=bonus if bonus >= 0 else None)
-        finally:
-            v.close()
         ref = helpers.run_oracle(w, mod, bonus_model=bonus, native=True)
-        helpers.check_parity(w, gpu, ref)
+        for form in (1, 2):
+            v = one_launch_verifier(w, form)
+            try:
+                gpu = helpers.run_gpu(w, mod, verifier=v, diag=True, bonus_model=bonus if bonus >= 0 else None)
+            finally:
+                v.close()
+            helpers.check_parity(w, gpu, ref)
 
 
 def test_one_launch_bad_drafts_non_finite_logits_and_empty_residual():
@@ -116,13 +121,14 @@ def test_one_launch_bad_drafts_non_finite_logits_and_empty_residual():
     logits[1, 5] = logits[0, 5]                  # identical models: r == q, the residual is empty
     drafts[5, 0] = w.vocab                       # ... and a bad draft forces a token all the same
     mod = dict(inputs, logits=logits, drafts=drafts)
-    v = one_launch_verifier(w)
-    try:
-        gpu = helpers.run_gpu(w, mod, verifier=v, diag=True)
-    finally:
-        v.close()
     ref = helpers.run_oracle(w, mod, native=True)
-    helpers.check_parity(w, gpu, ref)
+    for form in (2, 1):
+        v = one_launch_verifier(w, form)
+        try:
+            gpu = helpers.run_gpu(w, mod, verifier=v, diag=True)
+        finally:
+            v.close()
+        helpers.check_parity(w, gpu, ref)
     assert gpu["row_status"][0] & COS_ROW_BAD_DRAFT
     assert gpu["row_status"][2] & COS_ROW_NONFINITE and gpu["out_tokens"][2, 0] == -1
     assert gpu["row_status"][5] == (COS_ROW_BAD_DRAFT | COS_ROW_RESIDUAL_EMPTY)
