@@ -135,6 +135,26 @@ def test_one_launch_bad_drafts_non_finite_logits_and_empty_residual():
     assert 0 <= gpu["out_tokens"][5, 0] < w.vocab
 
 
+@pytest.mark.parametrize("form", [1, 2])
+def test_one_launch_partial_batches_strides_and_row_base(form):
+    """A context sized for more rows than a run passes, logits that are a strided view, and a row offset."""
+    w = C["cfg3"].scaled(batch=5, vocab=20008, gamma=3, name="layout_one_launch")
+    inputs = synth.make_inputs(w, "cuda")
+    n, B, P, V = inputs["logits"].shape
+    padded = torch.zeros((n, B, P + 1, V + 64), dtype=inputs["logits"].dtype, device="cuda")
+    padded[:, :, :P, :V] = inputs["logits"]
+    view = padded[:, :, :P, :V]                       # same values, other strides (rows still 16-byte aligned)
+    v = one_launch_verifier(w, form, max_batch=16)
+    try:
+        outs = v.run(view, inputs["drafts"], inputs["proposer"], inputs["seed"], inputs["offset"], row_base=1000, diag=True)
+        torch.cuda.synchronize()
+        gpu = {k: t.cpu().numpy() for k, t in outs.items()}
+    finally:
+        v.close()
+    ref = helpers.run_oracle(w, inputs, row_base=1000, native=True)
+    helpers.check_parity(w, gpu, ref)
+
+
 def test_one_launch_is_refused_where_it_does_not_apply():
     for w in (C["cfg2"].scaled(batch=2, vocab=4096, gamma=2), C["cfg5_greedy"].scaled(batch=2, vocab=4096, gamma=2),
               C["cfg3"].scaled(batch=2, vocab=4100, gamma=2)):
