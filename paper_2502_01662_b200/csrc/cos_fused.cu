@@ -13,12 +13,16 @@
 // first rejection has been published (rows resolve from the front), and its drawing items then go to a queue
 // that blocks look at before they take the next streaming item, while the position's logits are still in L2.
 //
-// A block is fifteen streaming warps and one service warp.  Streaming warps run from item to item without
-// block barriers and leave their partial sums in a ring of eight slots in shared memory; the service warp fetches
-// items one ahead, merges the partials, talks to the other blocks (fences, arrival counters, the queue) and does
-// all serial work (decision, row scan, locating a token), so none of it sits on the streaming warps' path.
+// A block (one per multiprocessor) is fifteen streaming warps, a service warp, a producer warp and a locating warp.
+// The producer (one thread) follows the block's items and fills a ring of five 30 KB stages in shared memory with
+// 1-D bulk copies that complete on mbarriers, running ahead across item boundaries; the streaming warps consume the
+// stages without block barriers and leave their partial sums in a ring of eight item slots.  Drawing items are read by
+// the streaming warps themselves.  The service warp fetches items one ahead, merges the partials, talks to the other
+// blocks (fences, arrival counters, the queue) and decides positions; the locating warp turns a row's recorded step
+// sums into its token, so none of the serial work sits on the streaming warps' path.
 // No block depends on a particular other block: any item can be taken by any block, and a block with nothing to
-// do polls the queue until every position is published and every row has its token.  All polls are bounded.
+// do looks at the queue (with a growing pause) until every position is published and every row has its token.
+// All waits are bounded.
 
 #include "cos_fused.h"
 
@@ -26,10 +30,15 @@ using namespace cosv;
 
 namespace {
 
-constexpr int kFT = 512;          // threads per block
+constexpr int kFT = 576;          // threads per block: fifteen streaming warps, then the service, producer and locating warps
 constexpr int kSW = 15;           // streaming warps
 constexpr int kST = kSW * 32;     // streaming threads
 constexpr int kRing = 8;          // items a block may have open
+constexpr int kSvcWarp = kSW, kProdWarp = kSW + 1;  // the last warp locates tokens
+constexpr int kNST = 5;                    // stages of the shared-memory ring the producer fills with bulk copies
+constexpr int kVPT = 4;                    // 16-byte vectors per streaming thread and stage
+constexpr int kStageVecs = kST * kVPT;     // 1920 vectors
+constexpr int kStageBytes = kStageVecs * 16;  // 30 KB
 constexpr int kCh = 4;            // channels of a drawing sweep (ensembles of up to four models; logit level: two)
 constexpr int kItemStream = 0, kItemDraw = 1, kItemJob = 2, kItemExit = 3;  // kItemJob: a drawing item named by its place in the job list
 // counters, each on a 128-byte line of its own (the queue's head and tail share one: they are read together)
@@ -39,7 +48,8 @@ constexpr int kCtrWords = 160;
 // Optional timeline accounting (build with -DCOS_FUSED_PROFILE): cycles the service warp and streaming warp 0 of
 // every block spend in each activity, summed over blocks into g_prof.  Compiled out of ordinary builds.
 #ifdef COS_FUSED_PROFILE
-__device__ unsigned long long g_prof[32];
+__device__ unsigned long long g_prof[48];
+__device__ unsigned long long g_prof_t0;  // globaltimer at the start of the launch (block 0)
 #define PROF_DECL unsigned long long prof_acc[16] = {0}; long long prof_t0 = 0; (void)prof_t0
 #define PROF_T0 prof_t0 = clock64()
 #define PROF_ADD(k) do { const long long t1_ = clock64(); prof_acc[k] += static_cast<unsigned long long>(t1_ - prof_t0); prof_t0 = t1_; } while (0)
@@ -85,12 +95,51 @@ struct FShared {
   // drawing-only launch: rows whose drawing sweep is complete, handed from the service warp to the locating warp
   int loc_ring[8];
   int loc_tail, loc_head, loc_exit;
+  // the ring of stages: `full` completes when a stage's bulk copies have landed, `empty` when the fifteen
+  // streaming warps have read it
+  unsigned long long full[kNST], empty[kNST];
   ItemCtx ctx[kRing];
   SoftPart part[kRing][kSW][kCh];
 };
 
 __device__ __forceinline__ int vol_load(const int* p) { return *reinterpret_cast<const volatile int*>(p); }
 __device__ __forceinline__ unsigned vol_load(const unsigned* p) { return *reinterpret_cast<const volatile unsigned*>(p); }
+
+// ---- mbarriers and 1-D bulk copies (global -> shared, completing on an mbarrier) --------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(void* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(void* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok)
+               : "r"(smem_u32(bar)), "r"(parity)
+               : "memory");
+  return ok != 0;
+}
+// Bounded wait for the phase of `parity` to complete.  False when it gave up (it then raises the block's fault
+// flag) or when another warp already has.
+__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, int* fault, unsigned limit) {
+  for (unsigned long long it = 0; it < 64ull * limit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (vol_load(fault)) return false;
+  }
+  *reinterpret_cast<volatile int*>(fault) = 1;
+  return false;
+}
+// both addresses 16-byte aligned, `bytes` a multiple of 16
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, void* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
 
 template <int DT>
 __device__ __forceinline__ uint4 ninf_vec() {
@@ -116,8 +165,6 @@ __device__ __forceinline__ double channel_k(const KParams& p, int i, int pis, in
 // ------------------------------------------------------------------------------------
 // streaming warps
 // ------------------------------------------------------------------------------------
-constexpr int kU = 8;  // 16-byte loads a streaming thread issues back to back
-
 // A streaming load that stays where it is written (a batch of loads is issued first, then consumed).
 __device__ __forceinline__ uint4 ldg_ahead16(const void* p) {
   uint4 v;
@@ -139,82 +186,95 @@ __device__ __noinline__ LaneSoft online_redo(const char* row, int v_first, int v
   return acc;
 }
 
-// Ensemble: the softmax statistics of the chunk [lo, hi) of every model's row, row after row.  Threads are
-// interleaved over the 16-byte vectors; a thread issues kU loads back to back and then consumes them (no warp
-// waits for another, so the other warps' loads cover the gap).  Fixed reference exponent per row and thread, seeded
-// from the thread's first vector (a whole number, so that sums rescale exactly); overflow or a non-finite input
-// redoes the thread's share of that row in the running-maximum form.
+// How a streaming item maps to stages of the ring.  The producer warp and the streaming warps walk the same sequence:
+// ensemble: row after row, 1920 vectors of one row per stage; logit level with two models: 960 vectors of each of the
+// two rows per stage (the second row in the stage's upper half).  `k` counts stages since the launch began.
+
+// Ensemble: the softmax statistics of the chunk [lo, hi) of every model's row.  A thread's vectors are those at
+// lo + stid + 480 m, four per stage, read from shared memory once the stage's bulk copy has landed.  Fixed reference
+// exponent per row and thread, seeded from the thread's first vector (a whole number, so that sums rescale exactly);
+// overflow or a non-finite input redoes the thread's share of that row from global memory in the running-maximum
+// form.  False when a wait gave up.
 template <int DT>
-__device__ __forceinline__ void stream_ensemble(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
+__device__ __forceinline__ bool stream_ensemble(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid, FShared& sh,
+                                                const unsigned char* ring, unsigned& k) {
   constexpr int E = Elem<DT>::E;
   const KParams& p = fp.k;
   const int lane = stid & 31;
   const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
   const long long row_step = p.s_model * Elem<DT>::bytes;
-  const int v0 = it.lo + stid;
   for (int i = 0; i < p.n; ++i) {
-    const char* row = base + i * row_step;
     LaneSoft acc;
     acc.init();
     bool first = true;
-    for (int v = v0; v < it.hi; v += kU * kST) {
-      uint4 raw[kU];
+    for (int v = it.lo; v < it.hi; v += kStageVecs, ++k) {
+      const unsigned slot = k % kNST;
+      if (!mbar_wait(&sh.full[slot], (k / kNST) & 1u, &sh.fault, fp.poll_limit)) return false;
+      const int nv = (it.hi - v < kStageVecs) ? it.hi - v : kStageVecs;
+      const uint4* st = reinterpret_cast<const uint4*>(ring + static_cast<size_t>(slot) * kStageBytes);
+      uint4 raw[kVPT];
 #pragma unroll
-      for (int u = 0; u < kU; ++u)
-        if (v + u * kST < it.hi) raw[u] = ldg_ahead16(row + static_cast<long long>(v + u * kST) * 16);
+      for (int j = 0; j < kVPT; ++j)
+        if (stid + j * kST < nv) raw[j] = st[stid + j * kST];
 #pragma unroll
-      for (int u = 0; u < kU; ++u) {
-        if (v + u * kST < it.hi) {
+      for (int j = 0; j < kVPT; ++j) {
+        if (stid + j * kST < nv) {
           float x[E];
-          Elem<DT>::unpack(raw[u], x);
-          if (u == 0 && first) {
+          Elem<DT>::unpack(raw[j], x);
+          if (j == 0 && first) {
             acc.seed(x, p.cT);
             first = false;
           }
           acc.add_fixed(x, p.cT);
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.empty[slot]);
     }
-    if (!(acc.s < INFINITY)) acc = online_redo<DT>(row, v0, it.hi, p.cT);
+    if (!(acc.s < INFINITY)) acc = online_redo<DT>(base + i * row_step, it.lo + stid, it.hi, p.cT);
     warp_merge_soft(acc, &part[i], lane);
   }
+  return true;
 }
 
-// Logit level with two models: proposer's softmax and the softmax of the combined logits, one vector of each model
-// per trip, kU / 2 trips per batch.  Same reference-exponent scheme as above.  False when some lane of the warp
-// met an overflow or a non-finite input (the caller then takes the general form).
+// Logit level with two models: proposer's softmax and the softmax of the combined logits.  `settled` comes back
+// false when some lane of the warp met an overflow or a non-finite input (the caller then takes the general form
+// from global memory).  False when a wait gave up.
 template <int DT>
-__device__ __forceinline__ bool stream_logit2(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
+__device__ __forceinline__ bool stream_logit2(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid, FShared& sh,
+                                              const unsigned char* ring, unsigned& k, bool& settled_all) {
   constexpr int E = Elem<DT>::E;
-  constexpr int T = kU / 2;
+  constexpr int HV = kStageVecs / 2, HT = kVPT / 2;  // vectors of each row per stage, per thread
   const KParams& p = fp.k;
   const int lane = stid & 31;
-  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
-  const long long row_step = p.s_model * Elem<DT>::bytes;
-  const int v0 = it.lo + stid;
   const float w0 = p.w[0], w1 = p.w[1];
   const bool q_is_0 = (it.pis == 0);
   LaneSoft accq, accc;
   accq.init();
   accc.init();
   bool first = true;
-  for (int v = v0; v < it.hi; v += T * kST) {
-    uint4 r0[T], r1[T];
+  for (int v = it.lo; v < it.hi; v += HV, ++k) {
+    const unsigned slot = k % kNST;
+    if (!mbar_wait(&sh.full[slot], (k / kNST) & 1u, &sh.fault, fp.poll_limit)) return false;
+    const int nv = (it.hi - v < HV) ? it.hi - v : HV;
+    const uint4* st0 = reinterpret_cast<const uint4*>(ring + static_cast<size_t>(slot) * kStageBytes);
+    const uint4* st1 = st0 + HV;
+    uint4 r0[HT], r1[HT];
 #pragma unroll
-    for (int u = 0; u < T; ++u)
-      if (v + u * kST < it.hi) {
-        r0[u] = ldg_ahead16(base + static_cast<long long>(v + u * kST) * 16);
-        r1[u] = ldg_ahead16(base + row_step + static_cast<long long>(v + u * kST) * 16);
+    for (int j = 0; j < HT; ++j)
+      if (stid + j * kST < nv) {
+        r0[j] = st0[stid + j * kST];
+        r1[j] = st1[stid + j * kST];
       }
 #pragma unroll
-    for (int u = 0; u < T; ++u) {
-      if (v + u * kST < it.hi) {
+    for (int j = 0; j < HT; ++j) {
+      if (stid + j * kST < nv) {
         float x0[E], x1[E], cmb[E];
-        Elem<DT>::unpack(r0[u], x0);
-        Elem<DT>::unpack(r1[u], x1);
+        Elem<DT>::unpack(r0[j], x0);
+        Elem<DT>::unpack(r1[j], x1);
 #pragma unroll
-        for (int k = 0; k < E; ++k) cmb[k] = fmaf(w1, x1[k], fmaf(w0, x0[k], 0.f));
-        if (u == 0 && first) {
+        for (int q = 0; q < E; ++q) cmb[q] = fmaf(w1, x1[q], fmaf(w0, x0[q], 0.f));
+        if (j == 0 && first) {
           if (q_is_0) accq.seed(x0, p.cT); else accq.seed(x1, p.cT);
           accc.seed(cmb, p.cT);
           first = false;
@@ -223,33 +283,82 @@ __device__ __forceinline__ bool stream_logit2(const FParams& fp, const ItemCtx& 
         accc.add_fixed(cmb, p.cT);
       }
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.empty[slot]);
   }
   const bool settled = (accq.s < INFINITY) && (accc.s < INFINITY);
-  if (!__all_sync(0xffffffffu, settled)) return false;
-  warp_merge_soft(accq, &part[0], lane);
-  warp_merge_soft(accc, &part[1], lane);
-  return true;
-}
-
-template <int DT, int MODE>
-__device__ __forceinline__ void stream_item(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid) {
-  const KParams& p = fp.k;
-  const int lane = stid & 31;
-  if (MODE == kEnsembleSample) {
-    stream_ensemble<DT>(fp, it, part, stid);
-  } else {
-    if (p.n == 2 && stream_logit2<DT>(fp, it, part, stid)) return;
-    // any other number of models, and the warps that met an overflow or a non-finite input
-    const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
-    Slice sl;
-    sl.v_lo = it.lo;
-    sl.v_hi = it.hi;
-    sl.e_lo = sl.e_hi = 0;
-    LaneSoft accq, accc;
-    logit_soft_slice<DT, kST>(p, base, sl, stid, it.pis, false, -INFINITY, accq, accc);
+  settled_all = __all_sync(0xffffffffu, settled);
+  if (settled_all) {
     warp_merge_soft(accq, &part[0], lane);
     warp_merge_soft(accc, &part[1], lane);
   }
+  return true;
+}
+
+// The producer warp's side of a streaming item (one thread): the stages in the order the streaming warps read them.
+// A stage is refilled once the fifteen warps have released its previous contents.  False when a wait gave up.
+template <int MODE>
+__device__ __forceinline__ bool produce_item(const FParams& fp, const ItemCtx& it, FShared& sh, unsigned char* ring, unsigned& k,
+                                             int eb) {
+  const KParams& p = fp.k;
+  const char* base = unit_base(p, it.b, it.j, eb);
+  const long long row_step = p.s_model * eb;
+  auto acquire = [&](unsigned slot) -> bool {
+    return k < static_cast<unsigned>(kNST) || mbar_wait(&sh.empty[slot], ((k / kNST) - 1u) & 1u, &sh.fault, fp.poll_limit);
+  };
+  if (MODE == kEnsembleSample) {
+    for (int i = 0; i < p.n; ++i)
+      for (int v = it.lo; v < it.hi; v += kStageVecs, ++k) {
+        const unsigned slot = k % kNST;
+        if (!acquire(slot)) return false;
+        const unsigned bytes = static_cast<unsigned>((it.hi - v < kStageVecs ? it.hi - v : kStageVecs)) * 16u;
+        mbar_expect_tx(&sh.full[slot], bytes);
+        bulk_load(ring + static_cast<size_t>(slot) * kStageBytes, base + i * row_step + static_cast<long long>(v) * 16, bytes,
+                  &sh.full[slot]);
+      }
+  } else {
+    constexpr int HV = kStageVecs / 2;
+    for (int v = it.lo; v < it.hi; v += HV, ++k) {
+      const unsigned slot = k % kNST;
+      if (!acquire(slot)) return false;
+      const unsigned bytes = static_cast<unsigned>((it.hi - v < HV ? it.hi - v : HV)) * 16u;
+      unsigned char* dst = ring + static_cast<size_t>(slot) * kStageBytes;
+      mbar_expect_tx(&sh.full[slot], 2u * bytes);
+      bulk_load(dst, base + static_cast<long long>(v) * 16, bytes, &sh.full[slot]);
+      bulk_load(dst + HV * 16, base + row_step + static_cast<long long>(v) * 16, bytes, &sh.full[slot]);
+    }
+  }
+  return true;
+}
+
+// Whether a streaming item goes through the ring (the producer and the streaming warps must agree).
+template <int MODE>
+__device__ __forceinline__ bool item_uses_ring(const KParams& p) {
+  return MODE == kEnsembleSample || p.n == 2;
+}
+
+template <int DT, int MODE>
+__device__ __forceinline__ bool stream_item(const FParams& fp, const ItemCtx& it, SoftPart* part, int stid, FShared& sh,
+                                            const unsigned char* ring, unsigned& k) {
+  const KParams& p = fp.k;
+  const int lane = stid & 31;
+  if (MODE == kEnsembleSample) return stream_ensemble<DT>(fp, it, part, stid, sh, ring, k);
+  if (item_uses_ring<MODE>(p)) {
+    bool settled = false;
+    if (!stream_logit2<DT>(fp, it, part, stid, sh, ring, k, settled)) return false;
+    if (settled) return true;
+  }
+  // any other number of models, and the warps that met an overflow or a non-finite input: from global memory
+  const char* base = unit_base(p, it.b, it.j, Elem<DT>::bytes);
+  Slice sl;
+  sl.v_lo = it.lo;
+  sl.v_hi = it.hi;
+  sl.e_lo = sl.e_hi = 0;
+  LaneSoft accq, accc;
+  logit_soft_slice<DT, kST>(p, base, sl, stid, it.pis, false, -INFINITY, accq, accc);
+  warp_merge_soft(accq, &part[0], lane);
+  warp_merge_soft(accc, &part[1], lane);
+  return true;
 }
 
 template <int N>
@@ -489,9 +598,10 @@ __device__ __forceinline__ void draw_item(const FParams& fp, const ItemCtx& it, 
 }
 
 template <int DT, int MODE, int NCH, bool DRAW_ONLY>
-__device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, double* bigacc_all) {
+__device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, double* bigacc_all, const unsigned char* ring) {
   const int stid = threadIdx.x, lane = stid & 31, warp = stid >> 5;
   double* bigacc = bigacc_all + stid;
+  unsigned k = 0;  // stages of the ring consumed so far
   PROF_DECL;
   PROF_T0;
   for (int seq = 0;; ++seq) {
@@ -518,7 +628,10 @@ __device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, doub
     const ItemCtx& it = sh.ctx[slot];
     if (it.kind == kItemExit) break;
     if (!DRAW_ONLY && it.kind == kItemStream) {
-      stream_item<DT, MODE>(fp, it, &sh.part[slot][warp][0], stid);
+      if (!stream_item<DT, MODE>(fp, it, &sh.part[slot][warp][0], stid, sh, ring, k)) break;
+#ifdef COS_FUSED_PROFILE
+      if (warp == 0 && lane == 0) atomicMax(&g_prof[32], prof_now() - g_prof_t0);
+#endif
       PROF_ADD(1);
       PROF_COUNT(4);
     } else {
@@ -536,6 +649,43 @@ __device__ __forceinline__ void stream_role(const FParams& fp, FShared& sh, doub
     PROF_ADD(3);  // reporting
   }
   if (warp == 0) PROF_FLUSH(0);
+}
+
+// The producer warp: one thread follows the block's items in order and fills the ring with the stages of the
+// streaming items, as far ahead of the streaming warps as the ring and the posted items allow (across the change
+// from one item to the next, so that the stream never drains).  Drawing items are read by the streaming warps
+// themselves.  Before it leaves it makes sure that every copy it issued has landed.
+template <int DT, int MODE>
+__device__ __forceinline__ void producer_role(const FParams& fp, FShared& sh, unsigned char* ring) {
+  if ((threadIdx.x & 31) != 0) return;
+  unsigned k = 0;
+  for (int seq = 0;; ++seq) {
+    const int slot = seq & (kRing - 1);
+    bool ok = false;
+    for (unsigned long long it = 0; it < 8ull * fp.poll_limit; ++it) {
+      if (vol_load(&sh.tag[slot]) == seq + 1) {
+        ok = true;
+        break;
+      }
+      if (vol_load(&sh.fault)) break;
+      __nanosleep(100);
+    }
+    if (!ok) break;
+    __threadfence_block();
+    atomicMax(&sh.started, seq + 1);
+    const ItemCtx& it = sh.ctx[slot];
+    const int kind = *reinterpret_cast<const volatile int*>(&it.kind);
+    if (kind == kItemExit) break;
+    if (kind != kItemStream || !item_uses_ring<MODE>(fp.k)) continue;
+    if (!produce_item<MODE>(fp, it, sh, ring, k, Elem<DT>::bytes)) break;
+  }
+  // every stage issued completes its `full` phase when its bytes are in, whoever reads them: wait for the last
+  // use of every slot (bounded), so that no copy is in flight when the block's shared memory is given back
+  for (unsigned back = 0; back < static_cast<unsigned>(kNST) && back < k; ++back) {
+    const unsigned use = k - 1u - back;
+    for (unsigned it = 0; it < (1u << 20); ++it)
+      if (mbar_try_wait(&sh.full[use % kNST], (use / kNST) & 1u)) break;
+  }
 }
 
 // ------------------------------------------------------------------------------------
@@ -878,8 +1028,10 @@ __device__ __forceinline__ int walk_step(const KParams& p, const WalkConst& w, c
 }
 
 // The drawing sweep of row b is complete.  Whole warp.
+constexpr int kLocBufSteps = 2048;  // steps whose masses fit the locating warp's buffer in shared memory (16 KB)
+
 template <int DT, int MODE, int NCH>
-__device__ __forceinline__ void locate_token(const FParams& fp, int b) {
+__device__ __forceinline__ void locate_token(const FParams& fp, int b, double* mbuf = nullptr) {
   const KParams& p = fp.k;
   const int lane = threadIdx.x & 31;
   const int rd = __ldcg(&fp.s.row_draw[b]);
@@ -888,6 +1040,12 @@ __device__ __forceinline__ void locate_token(const FParams& fp, int b) {
   const bool is_bonus = (j == p.gamma);
   const int pis = proposer_of(p, b, j);
   const char* base = unit_base(p, b, j, Elem<DT>::bytes);
+#ifdef COS_FUSED_PROFILE
+  unsigned long long lt0 = prof_now();
+#define LOC_STAMP(k) do { const unsigned long long t_ = prof_now(); if (lane == 0) atomicAdd(&g_prof[k], t_ - lt0); lt0 = t_; } while (0)
+#else
+#define LOC_STAMP(k)
+#endif
   WalkConst w;
   w.pis = pis;
   w.draw_q = (dkind == kDrawQ);
@@ -913,63 +1071,82 @@ __device__ __forceinline__ void locate_token(const FParams& fp, int b) {
     w.inv_zq = static_cast<float>(1.0 / w.zs[0]);
     w.inv_zc = static_cast<float>(1.0 / w.zs[1]);
   }
-  // every step's channel sums turn into its mass (products rounded one by one: equal sums under opposite
-  // coefficients cancel exactly); lanes own consecutive steps, a prefix over the lanes gives S
+  // Every step's channel sums turn into its mass (products rounded one by one: equal sums under opposite
+  // coefficients cancel exactly).  Steps are taken 32 at a time (lane l has step 32 t + l, so the records are read
+  // coalesced); an inclusive scan over the lanes and a running total over the tiles give the mass in front of every
+  // step.  First pass: the total S.  Second pass, same arithmetic: the first step whose running total reaches u S.
   const double* rec = fp.s.srec + static_cast<size_t>(b) * p.nsteps * NCH;
   auto step_mass = [&](int st) {
+    if (st >= p.nsteps) return 0.0;
     double acc = __dmul_rn(coef[0], __ldcg(rec + static_cast<size_t>(st) * NCH));
 #pragma unroll
     for (int i = 1; i < NCH; ++i) acc = __dadd_rn(acc, __dmul_rn(coef[i], __ldcg(rec + static_cast<size_t>(st) * NCH + i)));
     return fmax(0.0, acc);
   };
-  const int per = (p.nsteps + 31) / 32;
-  const int lo = lane * per, hi = (lo + per < p.nsteps) ? lo + per : p.nsteps;
-  double mine = 0.0;
-#pragma unroll 8
-  for (int st = lo; st < hi; ++st) mine += step_mass(st);
-  double incl = mine;
+  auto scan32 = [&](double m) {
+    double incl = m;
 #pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const double o = shfl_up_double(incl, d);
-    if (lane >= d) incl += o;
+    for (int d = 1; d < 32; d <<= 1) {
+      const double o = shfl_up_double(incl, d);
+      if (lane >= d) incl += o;
+    }
+    return incl;
+  };
+  LOC_STAMP(26);
+  const int ntiles = (p.nsteps + 31) / 32;
+  // With a buffer in shared memory (the locating warp has one) the masses are computed once, with nothing between
+  // the loads of a lane, and the search runs on shared memory; without one the second pass reads the records again.
+  const bool buffered = (mbuf != nullptr) && (p.nsteps <= kLocBufSteps);
+  double mine = 0.0;
+  if (buffered) {
+#pragma unroll 8
+    for (int t = 0; t < ntiles; ++t) {
+      const double m = step_mass(t * 32 + lane);
+      mbuf[t * 32 + lane] = m;
+      mine += m;
+    }
+    __syncwarp();
+  } else {
+#pragma unroll 8
+    for (int t = 0; t < ntiles; ++t) mine += step_mass(t * 32 + lane);
   }
-  const double S = shfl_double(incl, 31);
+  double S = mine;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) S += shfl_double(S, lane ^ d);
+  LOC_STAMP(27);
   const Unif un = position_uniforms(p, b, j);
   const double target = un.u_smp * S;
-  double before = incl - mine;
-  int first = 0x7fffffff, last = -1;
-  double first_base = 0.0, last_base = 0.0;
-#pragma unroll 4
-  for (int st = lo; st < hi; ++st) {
-    const double m = step_mass(st);
-    if (m > 0.0) {
-      last = st;
-      last_base = before;
-      if (first == 0x7fffffff && before + m >= target) {
-        first = st;
-        first_base = before;
-      }
+  int step = -1, last = -1;
+  double step_base = 0.0, last_base = 0.0, run = 0.0;
+  for (int t = 0; t < ntiles && step < 0; ++t) {
+    const int st = t * 32 + lane;
+    const double m = buffered ? mbuf[st] : step_mass(st);
+    const double incl = scan32(m);
+    const double before = run + (incl - m);
+    const unsigned hit = __ballot_sync(0xffffffffu, m > 0.0 && before + m >= target);
+    const unsigned mass = __ballot_sync(0xffffffffu, m > 0.0);
+    if (hit) {
+      const int src = __ffs(hit) - 1;
+      step = t * 32 + src;
+      step_base = shfl_double(before, src);
+    } else if (mass) {
+      const int src = 31 - __clz(mass);
+      last = t * 32 + src;
+      last_base = shfl_double(before, src);
     }
-    before += m;
+    run += shfl_double(incl, 31);
   }
-  int step = -1;
-  double step_base = 0.0;
-  const unsigned found = __ballot_sync(0xffffffffu, first != 0x7fffffff);
-  const unsigned have = __ballot_sync(0xffffffffu, last >= 0);
-  if (found) {
-    const int src = __ffs(found) - 1;
-    step = __shfl_sync(0xffffffffu, first, src);
-    step_base = shfl_double(first_base, src);
-  } else if (have && S > 0.0) {  // rounding corner: the last step with mass
-    const int src = 31 - __clz(have);
-    step = __shfl_sync(0xffffffffu, last, src);
-    step_base = shfl_double(last_base, src);
+  if (step < 0 && last >= 0 && S > 0.0) {  // rounding corner: the last step with mass
+    step = last;
+    step_base = last_base;
   }
+  LOC_STAMP(28);
   if (lane == 0 && p.diag && dkind == kDrawResidual)
     p.diag[static_cast<long long>(uidx) * 4 + 3] = static_cast<float>(S);
   if (step >= 0) {
     const bool use_r = (dkind != kDrawResidual);
     const int token = walk_step<DT, MODE>(p, w, base, step, step_base, target, use_r);
+    LOC_STAMP(29);
     if (lane == 0) {
       p.out_tokens[uidx] = token;
       // Algorithm 2's Score returns the bonus token with its probability under the law it came from
@@ -988,6 +1165,8 @@ __device__ __forceinline__ void locate_token(const FParams& fp, int b) {
     if (lane == 0) add_events(fp, 1);  // nothing to draw from: the row keeps -1
   }
   __syncwarp();
+  LOC_STAMP(30);
+#undef LOC_STAMP
 }
 
 __device__ __forceinline__ uint2 vol_load2(const unsigned* p) {
@@ -1036,7 +1215,10 @@ __device__ __forceinline__ void fill_ctx(const FParams& fp, ItemCtx& cx, int des
   const int lane = threadIdx.x & 31;
   const int kind = (desc >> 30) & 3, id = (desc >> 8) & 0x3fffff, c = desc & 0xff;
   if (kind == kItemStream) {
-    const int b = id / p.P, j = id % p.P;  // row-major: a row's positions come one after the other
+    // Row-major order: a row's positions one after the other.  A row settles as soon as the position of its first
+    // rejection is decided (the earlier ones came before it), while its later positions are still being streamed.
+    // (Position-major over the batch, and over groups of 32 rows, measured 10 % slower on workloads 3 and 4.)
+    const int b = id / p.P, j = id % p.P;
     if (lane == 0) {
       cx.kind = kItemStream;
       cx.b = b;
@@ -1128,16 +1310,15 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
   PROF_T0;
   while (true) {
     bool did = false;
-    // ---- fetch up to two items ahead of the fastest streaming warp
+    // ---- fetch up to two items ahead of the fastest of the streaming and producer warps
     if (skip > 0) --skip;
-    // (a drawing-only launch has few, short items per block: one item ahead, so that no block sits on work another
-    // block is idle for)
+    // (and where items are few and short, no block should sit on work another block is idle for)
     if (skip == 0 && fetched < processed + kRing && fetched <= vol_load(&sh.started) + (DRAW_ONLY ? 0 : 1)) {
       int desc = -1;
       if (lane == 0) desc = take_item(fp, sh.num_items, static_left, ticket);
       desc = __shfl_sync(0xffffffffu, desc, 0);
       static_left = __shfl_sync(0xffffffffu, static_left ? 1 : 0, 0) != 0;
-      if (DRAW_ONLY && desc != -1 && (desc & 0xff) == kLocateChunk) {
+      if (desc != -1 && ((desc >> 30) & 3) == kItemDraw && (desc & 0xff) == kLocateChunk) {
         // a row whose sweep is complete, passed on by a block whose locating warp was busy
         const int b = (desc >> 8) & 0x3fffff;
         if (!hand_to_locator(sh, b, lane)) locate_token<DT, MODE, NCH>(fp, b);
@@ -1207,6 +1388,9 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
           PROF_ADD(2);  // a streaming chunk reported
           if (last) {
             finish_position<DT, MODE>(fp, b, j, merged);
+#ifdef COS_FUSED_PROFILE
+            if (lane == 0) atomicMax(&g_prof[33], prof_now() - g_prof_t0);
+#endif
             PROF_ADD(3);
             PROF_COUNT(8);
           }
@@ -1228,13 +1412,16 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
             }
           }
           prev = __shfl_sync(0xffffffffu, prev, 0);
+#ifdef COS_FUSED_PROFILE
+          if (lane == 0) atomicMax(&g_prof[34], prof_now() - g_prof_t0);
+#endif
           PROF_ADD(4);  // a drawing chunk reported
           if (prev == fp.plan.dchunks - 1) {
             // the row's sweep is complete.  A drawing-only launch has a warp that does nothing but locate tokens,
             // so that this warp stays free to report the other rows' chunks; it takes the row unless its ring is full
             // ... so that this warp stays free; if that warp is busy the row goes to the queue, for any block to take
             bool handed = false;
-            if (DRAW_ONLY) {
+            {
               handed = hand_to_locator(sh, b, lane);
               if (!handed) {
                 if (lane == 0) {
@@ -1312,16 +1499,31 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
 // without the streaming code and for one block per multiprocessor, so that the drawing sweep keeps its working set in
 // registers; the one-launch form needs two blocks per multiprocessor to stream at full rate.
 template <int DT, int MODE, int NCH, bool DRAW_ONLY>
-__global__ void __launch_bounds__(DRAW_ONLY ? kFT + 32 : kFT, 1) cos_fused_kernel(const __grid_constant__ FParams fp) {
+__global__ void __launch_bounds__(kFT, 1) cos_fused_kernel(const __grid_constant__ FParams fp) {
   __shared__ FShared sh;
-  extern __shared__ double bigacc[];  // [2 * NCH][kST]: fp64 sums of the big terms of a drawing sweep, one slot per thread
+  // dynamic shared memory: [2 * NCH][kST] fp64 sums of the big terms of a drawing sweep (one slot per thread), the
+  // locating warp's buffer of step masses, then (one-launch form) the ring of kNST stages the producer fills
+  extern __shared__ __align__(128) unsigned char dyn_smem[];
+  double* bigacc = reinterpret_cast<double*>(dyn_smem);
+  double* locbuf = reinterpret_cast<double*>(dyn_smem + ((2 * NCH * kST * sizeof(double) + 127) / 128) * 128);
+  unsigned char* ring = reinterpret_cast<unsigned char*>(locbuf + kLocBufSteps);
   const int tid = threadIdx.x;
   if (tid < kRing) {
     sh.tag[tid] = 0;
     sh.arrive[tid] = 0;
   }
+  if (tid == 0) {
+    for (int q = 0; q < kNST; ++q) {
+      mbar_init(&sh.full[q], 1);       // the producer's arrival, with the bytes it announces
+      mbar_init(&sh.empty[q], kSW);    // one arrival per streaming warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   // (after a launch that published the positions: started while it drained; nothing it wrote is read before this)
   if (fp.draw_only) asm volatile("griddepcontrol.wait;" ::: "memory");
+#ifdef COS_FUSED_PROFILE
+  if (tid == 0 && blockIdx.x == 0) g_prof_t0 = prof_now();
+#endif
   if (tid == 0) {
     sh.started = 0;
     sh.fault = 0;
@@ -1337,12 +1539,15 @@ __global__ void __launch_bounds__(DRAW_ONLY ? kFT + 32 : kFT, 1) cos_fused_kerne
     }
   }
   __syncthreads();
-  if (tid < kST) {
-    stream_role<DT, MODE, NCH, DRAW_ONLY>(fp, sh, bigacc);
-  } else if (tid < kFT) {
+  const int role = tid >> 5;
+  if (role < kSW) {
+    stream_role<DT, MODE, NCH, DRAW_ONLY>(fp, sh, bigacc, ring);
+  } else if (role == kSvcWarp) {
     service_role<DT, MODE, NCH, DRAW_ONLY>(fp, sh);
+  } else if (role == kProdWarp) {
+    if (!DRAW_ONLY) producer_role<DT, MODE>(fp, sh, ring);
   } else {
-    // the locating warp of a drawing-only launch: rows in the order the service warp hands them over
+    // the locating warp: rows in the order the service warp hands them over
     const int lane = tid & 31;
     int head = 0;
     for (unsigned long long it = 0; it < 16ull * fp.poll_limit; ++it) {
@@ -1359,9 +1564,10 @@ __global__ void __launch_bounds__(DRAW_ONLY ? kFT + 32 : kFT, 1) cos_fused_kerne
 #ifdef COS_FUSED_PROFILE
         const unsigned long long tl0 = prof_now();
 #endif
-        locate_token<DT, MODE, NCH>(fp, b);
+        locate_token<DT, MODE, NCH>(fp, b, locbuf);
 #ifdef COS_FUSED_PROFILE
         if (lane == 0) {
+          atomicMax(&g_prof[35], prof_now() - g_prof_t0);
           atomicAdd(&g_prof[7], prof_now() - tl0);
           atomicAdd(&g_prof[15], 1ull);
         }
@@ -1409,15 +1615,18 @@ FusedFn pick_fused(int dtype, int mode, int n, bool draw_only = false) {
 }
 
 int channels_of(int mode, int n) { return mode == kEnsembleSample ? n : 2; }
-size_t fused_smem(int mode, int n) { return static_cast<size_t>(2 * channels_of(mode, n)) * kST * sizeof(double); }
+size_t fused_smem(int mode, int n, bool draw_only) {
+  const size_t big = ((static_cast<size_t>(2 * channels_of(mode, n)) * kST * sizeof(double) + 127) / 128) * 128;
+  return big + kLocBufSteps * sizeof(double) + (draw_only ? 0 : static_cast<size_t>(kNST) * kStageBytes);
+}
 
 }  // namespace
 
 #ifdef COS_FUSED_PROFILE
-extern "C" int cos_fused_profile_read(unsigned long long* out32, int reset) {
+extern "C" int cos_fused_profile_read(unsigned long long* out32, int reset) {  // 48 words
   if (cudaMemcpyFromSymbol(out32, g_prof, sizeof(g_prof)) != cudaSuccess) return -1;
   if (reset) {
-    unsigned long long z[32] = {0};
+    unsigned long long z[48] = {0};
     if (cudaMemcpyToSymbol(g_prof, z, sizeof(z)) != cudaSuccess) return -1;
   }
   return 0;
@@ -1442,22 +1651,29 @@ FusedPlan fused_plan(int dtype, int mode, int n, int vocab, int gamma, int max_b
   const int E = (dtype == COS_DTYPE_F32) ? 4 : 8;
   const int nvec = vocab / E;
   const int nsteps = (nvec + 31) / 32;
-  // streaming chunks of about 128 KB over all models, at least two steps per streaming warp, 32 chunks at most
+  // Streaming chunks.  A whole position per item where that still gives every block several items (one report to the
+  // other blocks less per item); else just enough chunks of at least 256 KB (over all models) to give the persistent
+  // blocks about four items each; 32 chunks at most, whole stages of the ring.
   const long long step_bytes = 512LL * n;
-  const long long chunk_kb = 256, dchunk_kb = 64;  // the fastest of the measured sizes (64 to 640 KB, 32 to 128 KB)
-  int cs = static_cast<int>((chunk_kb * 1024 + step_bytes - 1) / step_bytes);
-  if (cs < 2 * kSW) cs = 2 * kSW;
-  int chunks = (nsteps + cs - 1) / cs;
-  if (chunks > 32) chunks = 32;
-  if (chunks < 1) chunks = 1;
+  const long long dchunk_kb = 64;
+  const long long units = static_cast<long long>(max_batch) * (gamma + 1);
+  const long long blocks_ll = sm_count;
+  int chunks = 1;
+  if (units * 2 < 7 * blocks_ll) {
+    chunks = static_cast<int>((7 * blocks_ll + 2 * units - 1) / (2 * units));
+    const long long most = (nsteps * step_bytes) / (256 * 1024);
+    if (chunks > most) chunks = static_cast<int>(most);
+    if (chunks > 32) chunks = 32;
+    if (chunks < 1) chunks = 1;
+  }
+  int cs = (nsteps + chunks - 1) / chunks;
   pl.chunks = chunks;
-  pl.chunk_steps = (nsteps + chunks - 1) / chunks;
-  // whole batches: kSW steps give every streaming thread one vector, a batch is kU of them (kU / 2 per row with the
-  // two rows of a logit-level pair in one trip)
-  const int batch = kSW * (mode == kEnsembleSample ? kU : kU / 2);
-  if (pl.chunk_steps > batch && chunks > 1) pl.chunk_steps = (pl.chunk_steps + batch - 1) / batch * batch;
+  pl.chunk_steps = cs;
+  // (a stage of the ring is 60 steps of one row, or 30 of each row of a logit-level pair)
+  const int batch = (mode == kEnsembleSample) ? kStageVecs / 32 : kStageVecs / 64;
+  if (chunks > 1) pl.chunk_steps = (pl.chunk_steps + batch - 1) / batch * batch;
   pl.chunks = (nsteps + pl.chunk_steps - 1) / pl.chunk_steps;
-  // drawing chunks: half that size (the sweep costs about twice as much per byte), 64 at most
+  // drawing chunks of about 64 KB, 64 at most
   int ds = static_cast<int>((dchunk_kb * 1024 + step_bytes - 1) / step_bytes);
   if (ds < kSW) ds = kSW;
   int dchunks = (nsteps + ds - 1) / ds;
@@ -1470,7 +1686,6 @@ FusedPlan fused_plan(int dtype, int mode, int n, int vocab, int gamma, int max_b
   pl.blocks = sm_count * (blocks_per_sm > 0 ? blocks_per_sm : 1);
   pl.draw_blocks = sm_count;
   pl.dq_cap = 2 * max_batch * (pl.dchunks + 1);  // a row queues its items once (twice when the residual turns out empty), and may be queued for locating
-  (void)gamma;
   return pl;
 }
 
@@ -1493,12 +1708,13 @@ cudaError_t fused_occupancy(int dtype, int mode, int n, int* blocks_per_sm) {
   FusedFn fn = pick_fused(dtype, mode, n);
   if (fn == nullptr) return cudaErrorInvalidDeviceFunction;
   cudaError_t e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(fused_smem(mode, n)));
+                                       static_cast<int>(fused_smem(mode, n, false)));
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_fused(dtype, mode, n, true)),
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem(mode, n)));
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fused_smem(mode, n, true)));
   if (e != cudaSuccess) return e;
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void*>(fn), kFT, fused_smem(mode, n));
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, reinterpret_cast<const void*>(fn), kFT,
+                                                       fused_smem(mode, n, false));
 }
 
 cudaError_t fused_launch(int dtype, int mode, const KParams& p, const FusedPlan& plan, const FusedScratch& scratch,
@@ -1521,8 +1737,8 @@ cudaError_t fused_launch(int dtype, int mode, const KParams& p, const FusedPlan&
   if (blocks > most) blocks = most;
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
-  lc.blockDim = dim3(draw_only ? kFT + 32 : kFT, 1, 1);
-  lc.dynamicSmemBytes = fused_smem(mode, p.n);
+  lc.blockDim = dim3(kFT, 1, 1);
+  lc.dynamicSmemBytes = fused_smem(mode, p.n, draw_only);
   lc.stream = stream;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
