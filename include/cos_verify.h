@@ -130,6 +130,11 @@ typedef struct {
   const uint64_t* offset_device; /* optional: device address of the counter offset, read by the kernels */
                                /* in place of `offset` (8-byte aligned); lets a captured run be         */
                                /* replayed with fresh uniforms; may be NULL                             */
+  float* lse;                  /* optional out [B][gamma+1][S]: the log-sum-exp ln sum_x exp(l(x) / T)  */
+                               /* behind every softmax of a position (Sec. 3.1).  Ensemble: S = n, one  */
+                               /* per model; logit level: S = 2, the proposer's logits and the combined */
+                               /* (masked) logits.  NaN at T = 0 and where the position is not finite.  */
+                               /* One more small launch per run; may be NULL                            */
 } cos_verify_args;
 
 typedef struct {
@@ -172,7 +177,7 @@ cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* args, void
  * context, runs, copies accept_count / out_tokens / row_status (and diag if given)
  * back and waits for the stream.  Requires config.host_staging != 0 and contiguous
  * logits (stride_pos = V, stride_row = (gamma+1) V, stride_model = B (gamma+1) V).
- * dump_r is not supported here.
+ * dump_r and lse are not supported here.
  */
 cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* args, void* cuda_stream);
 

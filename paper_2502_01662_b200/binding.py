@@ -59,7 +59,7 @@ class cos_verify_args(ctypes.Structure):
         ("seed", ctypes.c_uint64), ("offset", ctypes.c_uint64), ("accept_count", ctypes.c_void_p),
         ("out_tokens", ctypes.c_void_p), ("row_status", ctypes.c_void_p), ("diag", ctypes.c_void_p),
         ("dump_r", ctypes.c_void_p), ("bonus_prob", ctypes.c_void_p), ("bonus_model", ctypes.c_int32),
-        ("offset_device", ctypes.c_void_p),
+        ("offset_device", ctypes.c_void_p), ("lse", ctypes.c_void_p),
     ]
 
 
@@ -194,6 +194,7 @@ class CosVerifier:
         a.bonus_prob = outs["bonus_prob"].data_ptr() if "bonus_prob" in outs else None
         a.bonus_model = bonus_model if (bonus_model is not None and bonus_model >= 0) else 0
         a.offset_device = offset_device.data_ptr() if offset_device is not None else None
+        a.lse = outs["lse"].data_ptr() if "lse" in outs else None
         return a
 
     def set_one_launch(self, enable=True):
@@ -237,7 +238,7 @@ class CosVerifier:
     # -- the calls -------------------------------------------------------------------
     def run(self, logits, drafts, proposer, seed: int, offset: int, row_base: int = 0, flags: int = 0,
             diag: bool = False, dump_r: bool = False, outs: Optional[dict] = None, stream=None,
-            bonus_model: Optional[int] = None, offset_device=None) -> dict:
+            bonus_model: Optional[int] = None, offset_device=None, lse: bool = False) -> dict:
         """cos_verify_run on device tensors; asynchronous on `stream` (default: torch's current stream).
 
         `proposer` is [B], or [B, gamma+1] to name the proposer of every draft (Algorithm 2); `bonus_model`
@@ -254,6 +255,9 @@ class CosVerifier:
         n, B, P, V = logits.shape
         if outs is None:
             outs = self._alloc_outs(B, P, V, logits.device, diag, dump_r)
+            if lse:     # log-sum-exp behind every softmax of a position: [B, gamma+1, n] (ensemble) or [B, gamma+1, 2]
+                slots = self.cfg.n if self.cfg.combine == COS_COMBINE_PROB_ENSEMBLE else 2
+                outs["lse"] = torch.empty((B, P, slots), dtype=torch.float32, device=logits.device)
         if offset_device is not None and (offset_device.dtype != torch.int64 or not offset_device.is_cuda):
             raise ValueError("offset_device must be an int64 device tensor")
         a = self._fill_args(logits, drafts, proposer, seed, offset, row_base, flags, outs, bonus_model, offset_device)

@@ -2089,6 +2089,20 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   if (((STAGE == 0 && p.greedy) || STAGE >= 2) && tid == 0) stage_exit(p, STAGE == 0 ? 0 : 1);
 }
 
+// The log-sum-exp behind every softmax of a position, from the merged statistics a run leaves per position:
+// ln sum_x exp(l(x) / T) = (ref + log2 s) ln 2.  One thread per (position, slot).
+__global__ void export_lse_kernel(const UnitStats* ustats, const int4* unit_res, float* lse, int units, int slots, int sampling) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= units * slots) return;
+  const int u = t / slots, k = t % slots;
+  float v = __int_as_float(0x7fc00000);
+  if (sampling && !(__ldcg(&unit_res[u]).y & COS_ROW_NONFINITE)) {
+    const double sum = ustats[u].s[k];
+    v = static_cast<float>((static_cast<double>(ustats[u].ref[k]) + log2(sum)) * 0.6931471805599453);
+  }
+  lse[t] = v;
+}
+
 // ------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------
@@ -2543,7 +2557,9 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   return COS_OK;
 }
 
-extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* a, void* cuda_stream) {
+namespace {
+// the launches of one run (everything but the optional export of the log-sum-exps)
+cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cuda_stream) {
   if (!ctx) return COS_ERR_INVALID_ARG;
   if (!a) {
     ctx->err = "null args";
@@ -2681,6 +2697,26 @@ extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args*
   return COS_OK;
 }
 
+}  // namespace
+
+extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* a, void* cuda_stream) {
+  if (ctx && a && a->lse && reinterpret_cast<uintptr_t>(a->lse) % 4) {
+    ctx->err = "lse is not 4-byte aligned";
+    return COS_ERR_ALIGNMENT;
+  }
+  const cos_status st = run_launches(ctx, a, cuda_stream);
+  if (st != COS_OK || a->lse == nullptr) return st;
+  const cos_verify_config& c = ctx->cfg;
+  const int units = a->batch * (c.gamma + 1);
+  const int slots = (c.combine == COS_COMBINE_PROB_ENSEMBLE) ? c.n : 2;
+  const int total = units * slots;
+  export_lse_kernel<<<(total + 255) / 256, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      ctx->d_ustats, ctx->d_unit_res, a->lse, units, slots, c.temperature > 0.0f ? 1 : 0);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (log-sum-exp export)", e);
+  return COS_OK;
+}
+
 extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_args* a, void* cuda_stream) {
   if (!ctx) return COS_ERR_INVALID_ARG;
   if (!a) {
@@ -2696,8 +2732,8 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
     ctx->err = "batch outside 1..max_batch";
     return COS_ERR_INVALID_ARG;
   }
-  if (a->dump_r) {
-    ctx->err = "dump_r is not available for host-pointer runs";
+  if (a->dump_r || a->lse) {
+    ctx->err = "dump_r and lse are not available for host-pointer runs";
     return COS_ERR_UNSUPPORTED;
   }
   if (!a->logits || !a->proposer || !a->accept_count || !a->out_tokens || !a->row_status || (c.gamma > 0 && !a->draft_tokens)) {
@@ -2904,6 +2940,7 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     return static_fail(COS_ERR_ALIGNMENT, "bonus_prob is not 4-byte aligned");
   if (a->offset_device && reinterpret_cast<uintptr_t>(a->offset_device) % 8)
     return static_fail(COS_ERR_ALIGNMENT, "offset_device is not 8-byte aligned");
+  if (a->lse) return static_fail(COS_ERR_UNSUPPORTED, "lse is not available from the allocation-free entry point");
   const int eb = elem_bytes(c.dtype);
   if (reinterpret_cast<uintptr_t>(a->logits) % eb) return static_fail(COS_ERR_ALIGNMENT, "logits pointer not aligned to its element type");
   if (reinterpret_cast<uintptr_t>(a->proposer) % 4 || reinterpret_cast<uintptr_t>(a->accept_count) % 4 ||

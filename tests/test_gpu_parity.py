@@ -144,3 +144,46 @@ def test_proposer_per_position_and_named_bonus_model(w, cs):
     other = helpers.run_oracle(w, dict(inputs, proposer=torch.as_tensor((table + 1) % w.n)), bonus_model=-1)
     assert w.n == 1 or not np.array_equal(other["accept_count"], ref["accept_count"]) or \
         not np.array_equal(other["out_tokens"], ref["out_tokens"])
+
+
+@pytest.mark.parametrize("name,kw", [("cfg3", dict(batch=5, vocab=20008, gamma=3)), ("cfg4", dict(batch=4, vocab=12808, gamma=2)),
+                                     ("cfg2", dict(batch=4, vocab=9001, gamma=3)), ("cfg5", dict(batch=3, vocab=50000, gamma=2)),
+                                     ("cfg1", dict(batch=2, vocab=32000, gamma=4)), ("cfg5_greedy", dict(batch=2, vocab=8000, gamma=2))])
+@pytest.mark.parametrize("form", [0, 1])
+def test_log_sum_exp_of_every_softmax(name, kw, form):
+    """The optional `lse` output against scipy's logsumexp of the stored logits over T (Sec. 3.1): one value per model
+    (ensemble), or the proposer's and the combined, masked logits' (logit level); NaN at T = 0."""
+    from scipy.special import logsumexp
+    from oracle import cos_oracle as orc
+    w = synth.CONFIGS[name].scaled(**kw)
+    inputs = synth.make_inputs(w, "cuda")
+    v = helpers.make_verifier(w)
+    try:
+        if form == 1:
+            try:
+                v.set_one_launch(1)
+            except Exception:
+                pytest.skip("the one-launch form does not cover this configuration")
+        outs = v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], inputs["seed"], inputs["offset"], lse=True)
+        torch.cuda.synchronize()
+        got = outs["lse"].cpu().numpy()
+    finally:
+        v.close()
+    if w.temperature == 0.0:
+        assert np.all(np.isnan(got))
+        return
+    host = synth.logits_as_numpy(inputs["logits"])
+    prop = inputs["proposer"].cpu().numpy()
+    T = float(np.float32(w.temperature))
+    wts = np.asarray(w.weights, dtype=np.float32).astype(np.float64)
+    for b in range(w.batch):
+        for j in range(w.gamma + 1):
+            l = orc.to_float64(host[:, b, j, :], w.dtype)
+            if w.combine == 0:
+                want = [logsumexp(l[i] / T) for i in range(w.n)]
+            else:
+                c = sum(wts[i] * l[i] for i in range(w.n))
+                if w.mask_model >= 0:
+                    c = np.where(orc.plausibility_mask(l[w.mask_model], float(np.float32(w.mask_alpha))), c, -np.inf)
+                want = [logsumexp(l[int(prop[b])] / T), logsumexp(c / T)]
+            np.testing.assert_allclose(got[b, j], want, rtol=0, atol=2e-5)
