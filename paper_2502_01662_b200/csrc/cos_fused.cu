@@ -2,7 +2,7 @@
 // first-rejection scan and the residual / bonus draw (Sec. 3.1-3.2) without a second pass over the batch.
 //
 // The run is cut into work items that any block can take:
-//   streaming item  one chunk (a contiguous range of steps, ~128 KB) of the n logit rows of one (row, position):
+//   streaming item  one (row, position), or one chunk of it (a contiguous range of steps of its n logit rows):
 //                   per-model softmax statistics of the chunk.  The block that completes the last chunk of a
 //                   position merges the chunks in order, takes the accept test and publishes the position.
 //   drawing item    one chunk of the one position of a row that must emit a token (its first rejection, or the
@@ -11,13 +11,13 @@
 //                   turns the sums into masses, finds the step by a prefix and walks it to the token.
 // Streaming items come from a counter in row-major order; a row is settled as soon as every position up to its
 // first rejection has been published (rows resolve from the front), and its drawing items then go to a queue
-// that blocks look at before they take the next streaming item, while the position's logits are still in L2.
+// that blocks look at before they take the next streaming item.
 //
 // A block (one per multiprocessor) is fifteen streaming warps, a service warp, a producer warp and a locating warp.
 // The producer (one thread) follows the block's items and fills a ring of five 30 KB stages in shared memory with
 // 1-D bulk copies that complete on mbarriers, running ahead across item boundaries; the streaming warps consume the
 // stages without block barriers and leave their partial sums in a ring of eight item slots.  Drawing items are read by
-// the streaming warps themselves.  The service warp fetches items one ahead, merges the partials, talks to the other
+// the streaming warps themselves.  The service warp fetches items ahead, merges the partials, talks to the other
 // blocks (fences, arrival counters, the queue) and decides positions; the locating warp turns a row's recorded step
 // sums into its token, so none of the serial work sits on the streaming warps' path.
 // No block depends on a particular other block: any item can be taken by any block, and a block with nothing to
@@ -1417,9 +1417,8 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
 #endif
           PROF_ADD(4);  // a drawing chunk reported
           if (prev == fp.plan.dchunks - 1) {
-            // the row's sweep is complete.  A drawing-only launch has a warp that does nothing but locate tokens,
-            // so that this warp stays free to report the other rows' chunks; it takes the row unless its ring is full
-            // ... so that this warp stays free; if that warp is busy the row goes to the queue, for any block to take
+            // the row's sweep is complete: its token is located by the block's locating warp, so that this warp
+            // stays free to report other chunks; if that warp is busy the row goes to the queue, for any block to take
             bool handed = false;
             {
               handed = hand_to_locator(sh, b, lane);
@@ -1495,9 +1494,9 @@ __device__ __forceinline__ void service_role(const FParams& fp, FShared& sh) {
   }
 }
 
-// DRAW_ONLY: the launch that only draws tokens (after a staged launch published the positions).  It is compiled
-// without the streaming code and for one block per multiprocessor, so that the drawing sweep keeps its working set in
-// registers; the one-launch form needs two blocks per multiprocessor to stream at full rate.
+// DRAW_ONLY: the launch that only draws tokens (after a staged launch published the positions); it is compiled
+// without the streaming code.  One block per multiprocessor in both forms: the drawing sweep then keeps its working
+// set in registers, and the ring of stages, not the number of resident warps, keeps the stream going.
 template <int DT, int MODE, int NCH, bool DRAW_ONLY>
 __global__ void __launch_bounds__(kFT, 1) cos_fused_kernel(const __grid_constant__ FParams fp) {
   __shared__ FShared sh;
