@@ -88,6 +88,8 @@ struct KParams {
                            // (one-sweep drawing stage: [B][nsteps], first channel sum of every step)
   int* part_arrivals;      // [B*P]: blocks of the unit that finished stage 2; zero between runs
   double* srungB;          // the one-sweep drawing stage: second channel of srung (null where that stage is not used)
+  double* srungC;          // ... third and fourth channel (ensembles of three or four models; null otherwise)
+  double* srungD;
 };
 
 // ------------------------------------------------------------------------------------

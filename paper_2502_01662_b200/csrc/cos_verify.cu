@@ -71,6 +71,15 @@ struct OneSweep {  // constants of the one-sweep drawing stage, for its out-of-l
   double ctA64, ctB64, drefA, drefB;
 };
 
+struct OneSweepN {  // the same for the one-sweep stage that keeps a channel per model (ensembles of three or four)
+  float ct[4], nref[4], bt[4];
+  double ct64[4], dref[4];
+};
+
+struct Raw4 {  // one lane's vector of each of up to four models
+  uint4 r[4];
+};
+
 struct Shared;
 __device__ __forceinline__ OneSweep& one_sweep_consts(Shared& sh);
 __device__ __forceinline__ double* one_sweep_coef(Shared& sh);
@@ -106,6 +115,8 @@ struct Shared {
 // The one-sweep drawing stage never fills gw[]; its constants and the two exact coefficients of the channel
 // sums live there, so that the layout of Shared is the same for every stage.
 static_assert(sizeof(OneSweep) <= 16 * sizeof(double), "OneSweep must fit in front of the coefficients");
+static_assert(sizeof(OneSweepN) <= 16 * sizeof(double), "OneSweepN must fit in front of the coefficients");
+__device__ __forceinline__ OneSweepN& one_sweep_consts_n(Shared& sh) { return *reinterpret_cast<OneSweepN*>(&sh.gw[0]); }
 __device__ __forceinline__ OneSweep& one_sweep_consts(Shared& sh) { return *reinterpret_cast<OneSweep*>(&sh.gw[0]); }
 __device__ __forceinline__ double* one_sweep_coef(Shared& sh) { return &sh.gw[16]; }
 
@@ -358,6 +369,184 @@ __device__ __noinline__ float4 one_sweep_big_vector(const KParams& p, const OneS
     }
   }
   return out;
+}
+
+// The one-sweep drawing stage with a channel per model (ensembles of three or four; Eq. 4): r - q, r and q are all
+// sums over the models of k_i e_i / Z_i with e_i = 2^(l_i c - ref_i), so a token's mass is that sum clipped at zero.
+// One big entry (more than 2^-8 of a normaliser) of that sweep, in fp64 from its logits: into the thread's slots
+// `bigacc` ([i kThreads] Z_i, [(4 + i) kThreads] the sum of e_i where the mass is positive).  Rare; out of line.
+__device__ __noinline__ void one_sweep_big_token_n(const KParams& p, const OneSweepN& c, float x0, float x1, float x2, float x3,
+                                                   double* bigacc) {
+  const float x[4] = {x0, x1, x2, x3};
+  double d[4], tot = 0.0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    d[i] = exp2(static_cast<double>(x[i]) * p.cT64 - c.dref[i]);  // (a model the ensemble does not have: -inf, no term)
+    tot += c.ct64[i] * d[i];
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    bigacc[i * kThreads] += d[i];
+    if (tot > 0.0) bigacc[(4 + i) * kThreads] += d[i];
+  }
+}
+
+// The sweep itself: this block's steps [rank, rank + 1) / lparts of the unit's steps, its warps taking them in
+// turn; every step (32 lanes x E entries, in token order) leaves, per model, the sum of e_i over its tokens with a
+// positive mass (the set is decided with the normalisers of stage 0, products rounded one by one so that equal
+// terms cancel exactly; over that set the mass is linear in the 1/Z_i), and the warp's share of the refined
+// normalisers goes to sh.wsoft.  `kc` returns the coefficients k_i of what is drawn: max(0, r - q), r, or q.
+template <int DT>
+__device__ __forceinline__ void one_sweep_channels(const KParams& p, Shared& sh, uint4* ring, const char* base, int b, int rank,
+                                                   int lparts, int pis, bool is_bonus, bool draw_q, int emit, bool vec_ok,
+                                                   double (&kc)[4]) {
+  constexpr int E = Elem<DT>::E;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float ct[4], nref[4], bt[4];
+  double ct64[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const bool live = i < p.n;
+    const double sel = (i == pis) ? 1.0 : 0.0;
+    kc[i] = !live ? 0.0 : (!is_bonus ? p.w64[i] - sel : (draw_q ? sel : p.w64[i]));
+    ct64[i] = live ? kc[i] / sh.fsoft[i].s : 0.0;  // with the first estimates: signs only
+    ct[i] = static_cast<float>(ct64[i]);
+    nref[i] = live ? -sh.fsoft[i].ref : 0.f;
+    bt[i] = live ? sh.big_thr[i] : INFINITY;
+  }
+  if (tid == 0) {
+    OneSweepN& c = one_sweep_consts_n(sh);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      c.ct[i] = ct[i];
+      c.nref[i] = nref[i];
+      c.bt[i] = bt[i];
+      c.ct64[i] = ct64[i];
+      c.dref[i] = (i < p.n) ? static_cast<double>(sh.fsoft[i].ref) : 0.0;
+    }
+  }
+  // the big terms sit in shared memory (the staging ring is idle during this sweep), one slot per thread and sum
+  double* bigacc = reinterpret_cast<double*>(ring) + tid;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) bigacc[q * kThreads] = 0.0;
+  __syncthreads();
+  const long long row_step = p.s_model * Elem<DT>::bytes;
+  const int blk_lo = static_cast<int>(static_cast<long long>(rank) * p.nsteps / lparts);
+  const int blk_hi = static_cast<int>(static_cast<long long>(rank + 1) * p.nsteps / lparts);
+  const size_t rec_at = static_cast<size_t>(b) * p.nsteps;
+  const int nfull = vec_ok ? p.V / (32 * E) : 0;  // steps below this are whole aligned vectors
+  float zs[4] = {0.f, 0.f, 0.f, 0.f};
+  bool hasbig = false;
+  Raw4 nx;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) nx.r[i] = make_uint4(0u, 0u, 0u, 0u);
+  auto fetch = [&](int s) {
+    const char* src = base + static_cast<long long>(s * 32 + lane) * 16;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (i < p.n) nx.r[i] = ldg_stream16(src + i * row_step);
+  };
+  if (blk_lo + warp < blk_hi && blk_lo + warp < nfull) fetch(blk_lo + warp);
+  for (int s = blk_lo + warp; s < blk_hi; s += kWarps) {
+    const int e0 = (s * 32 + lane) * E;
+    const bool have_raw = s < nfull;
+    const Raw4 cur = nx;
+    float x[4][E];
+    if (have_raw) {
+      const int sn = s + kWarps;
+      if (sn < blk_hi && sn < nfull) fetch(sn);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) Elem<DT>::unpack(cur.r[i], x[i]);
+    } else {
+      // ragged or unaligned step: entry by entry; entries beyond V read as -inf (no mass, outside every set)
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (i < p.n) load_chunk<DT>(base + i * row_step, e0, p.V, vec_ok, x[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (i >= p.n) {
+#pragma unroll
+        for (int k = 0; k < E; ++k) x[i][k] = -INFINITY;
+      }
+    }
+    float vz[4] = {0.f, 0.f, 0.f, 0.f}, va[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+      float e[4], acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        e[i] = ex2_approx(fmaf(x[i][k], p.cT, nref[i]));
+        vz[i] += e[i];
+        acc = __fadd_rn(acc, __fmul_rn(ct[i], e[i]));
+      }
+      const float in_p = (acc > 0.f) ? 1.f : 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) va[i] = fmaf(in_p, e[i], va[i]);
+    }
+    // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum big)
+    const bool big = (vz[0] > bt[0]) || (vz[1] > bt[1]) || (vz[2] > bt[2]) || (vz[3] > bt[3]);
+    if (big) {
+      // the vector again, its big entries in fp64 (entries beyond V and models the ensemble does not have are -inf)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) vz[i] = va[i] = 0.f;
+#pragma unroll
+      for (int k = 0; k < E; ++k) {
+        float e[4], acc = 0.f;
+        bool bigtok = false;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          e[i] = ex2_approx(fmaf(x[i][k], p.cT, nref[i]));
+          bigtok |= e[i] > bt[i];
+          acc = __fadd_rn(acc, __fmul_rn(ct[i], e[i]));
+        }
+        if (bigtok) {
+          one_sweep_big_token_n(p, one_sweep_consts_n(sh), x[0][k], x[1][k], x[2][k], x[3][k], bigacc);
+        } else {
+          const float in_p = (acc > 0.f) ? 1.f : 0.f;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            vz[i] += e[i];
+            va[i] = fmaf(in_p, e[i], va[i]);
+          }
+        }
+      }
+      hasbig = true;
+    }
+    // the step's sums over the warp
+    double mine = 0.0;
+    const bool anybig = __any_sync(0xffffffffu, hasbig);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      zs[i] += vz[i];
+      float r = va[i];
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) r += __shfl_xor_sync(0xffffffffu, r, d);
+      double dr = static_cast<double>(r);
+      if (anybig) {
+        double t = bigacc[(4 + i) * kThreads];
+        bigacc[(4 + i) * kThreads] = 0.0;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+        dr += t;
+      }
+      if (lane == i) mine = dr;
+    }
+    if (emit && lane < 4) {
+      double* dst = (lane == 0) ? p.srung : (lane == 1 ? p.srungB : (lane == 2 ? p.srungC : p.srungD));
+      dst[rec_at + s] = mine;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    double t = static_cast<double>(zs[i]) + bigacc[i * kThreads];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) t += shfl_double(t, lane ^ d);
+    if (lane == 0) {
+      sh.wsoft[warp][i].s = t;
+      sh.wsoft[warp][i].ref = (i < p.n) ? sh.fsoft[i].ref : 0.f;
+    }
+  }
 }
 
 // Combined logit of one token in fp64, from the stored logits: the chain of fused multiply-adds that
@@ -899,6 +1088,10 @@ template <int DT, int MODE, int STAGE, int MINB = 2>
 __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid_constant__ KParams p) {
   constexpr int E = Elem<DT>::E;
   constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
+  // the drawing stages in one sweep: stage 3 with two channel sums per step, stage 4 with one per model of an
+  // ensemble of three or four
+  constexpr bool kOneSweep = (STAGE == 3 || STAGE == 4);
+  constexpr int NCH = (STAGE == 4) ? 4 : 2;
   cg::cluster_group cluster = cg::this_cluster();
   // stage 0 shares a unit among the blocks of a cluster; stages 1 and 2 among `parts` independent
   // blocks (they meet only through global memory: partial sums between the launches, an arrival counter within stage 2)
@@ -925,7 +1118,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   // later stages are launched while the previous one drains (programmatic dependent launch);
   // nothing it wrote is read before this point
   if (STAGE >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if ((STAGE == 1 || STAGE == 3) && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
+  if ((STAGE == 1 || kOneSweep) && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
   const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
   if (STAGE == 0) {
@@ -1282,7 +1475,11 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       }
       } else {
       bool do_locate = false;
-      if (STAGE == 3) {
+      if (kOneSweep) {
+        double kc[4] = {0.0, 0.0, 0.0, 0.0};  // coefficient of every channel in what is drawn
+        if (STAGE == 4) {
+          one_sweep_channels<DT>(p, sh, ring, base, b, rank, lparts, pis, is_bonus, draw_q, emit, vec_ok, kc);
+        } else {
         // ---- the drawing stages in one sweep.  A token's mass is k_A e_A / Z_A + k_B e_B / Z_B clipped at zero,
         // where the two channels are the two models (ensemble, n = 2) or the proposer's and the combined logits
         // (logit level), and (k_A, k_B) says what is drawn: max(0, r - q), r, or q.  The set of tokens with a
@@ -1547,8 +1744,11 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
           }
         }
+        kc[0] = kA;
+        kc[1] = kB;
+        }
         __syncthreads();
-        if (warp < 2) {
+        if (warp < NCH) {
           float ref = (lane < kWarps) ? sh.wsoft[lane][warp].ref : -INFINITY;
           double sum = (lane < kWarps) ? sh.wsoft[lane][warp].s : 0.0;
           SoftPart o = warp_reduce_soft(ref, sum);
@@ -1569,16 +1769,20 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         do_locate = (sh.win_g != 0) && emit;  // (every unit listed for this stage is its row's drawing unit)
         __syncthreads();
         if (do_locate) {
-          if (tid < 2) {
+          if (tid < NCH) {
             double z = 0.0;
             for (int q = 0; q < p.parts; ++q) z += __ldcg(&p.zpart[(static_cast<size_t>(uidx) * p.parts + q) * 8 + tid]);
-            sh.fsoft[tid].s = z;
-            one_sweep_coef(sh)[tid] = (tid == 0 ? kA : kB) / z;
+            double kmine = kc[0];
+#pragma unroll
+            for (int i = 1; i < NCH; ++i) kmine = (tid == i) ? kc[i] : kmine;
+            const bool live = (STAGE != 4) || tid < p.n;  // an ensemble of three leaves the fourth channel empty
+            if (live) sh.fsoft[tid].s = z;
+            one_sweep_coef(sh)[tid] = live ? kmine / z : 0.0;
           }
           __syncthreads();
         }
       }
-      if (STAGE != 3 || do_locate) {
+      if (!kOneSweep || do_locate) {
       if (MODE == kEnsembleSample && tid < p.n) {
         // r - q = sum_i (w_i/Z_i - [i = proposer]/Z_i) e_i, and r = sum_i (w_i/Z_i) e_i
         const double a = p.w64[tid] / sh.fsoft[tid].s;
@@ -1955,7 +2159,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       if (do_locate) {
         // ---- one block per unit: add the runs up, find the run, walk it
         int one_step = -1;  // one-sweep stage: the step that holds the token
-        if (STAGE == 3) {
+        if (kOneSweep) {
           // Every step's channel sums turn into its mass now that the normalisers are complete (products rounded
           // one by one, so that equal sums under opposite coefficients cancel exactly).  Threads own consecutive
           // steps; a prefix over threads in step order gives S and the first step whose running total reaches u S.
@@ -1963,8 +2167,15 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           const int lo = tid * per, hi = (lo + per < p.nsteps) ? lo + per : p.nsteps;
           const double* ra = p.srung + static_cast<size_t>(b) * p.nsteps;
           const double* rb = p.srungB + static_cast<size_t>(b) * p.nsteps;
+          const double* rc = (STAGE == 4) ? p.srungC + static_cast<size_t>(b) * p.nsteps : nullptr;
+          const double* rd = (STAGE == 4) ? p.srungD + static_cast<size_t>(b) * p.nsteps : nullptr;
           auto step_mass = [&](int st) {
-            return fmax(0.0, __dadd_rn(__dmul_rn(one_sweep_coef(sh)[0], __ldcg(ra + st)), __dmul_rn(one_sweep_coef(sh)[1], __ldcg(rb + st))));
+            double acc = __dadd_rn(__dmul_rn(one_sweep_coef(sh)[0], __ldcg(ra + st)), __dmul_rn(one_sweep_coef(sh)[1], __ldcg(rb + st)));
+            if (STAGE == 4) {
+              acc = __dadd_rn(acc, __dmul_rn(one_sweep_coef(sh)[2], __ldcg(rc + st)));
+              acc = __dadd_rn(acc, __dmul_rn(one_sweep_coef(sh)[3], __ldcg(rd + st)));
+            }
+            return fmax(0.0, acc);
           };
           double mine = 0.0;
           for (int st = lo; st < hi; ++st) mine += step_mass(st);
@@ -2039,10 +2250,10 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           if (emit && warp == 0) {
             const int g = sh.win_g;
             // one-sweep stage: the run is the one step found above, its mass the only running total
-            const int sb = (STAGE == 3) ? one_step : static_cast<int>(static_cast<long long>(g) * p.nsteps / G);
-            const int se = (STAGE == 3) ? one_step + 1 : static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
+            const int sb = kOneSweep ? one_step : static_cast<int>(static_cast<long long>(g) * p.nsteps / G);
+            const int se = kOneSweep ? one_step + 1 : static_cast<int>(static_cast<long long>(g + 1) * p.nsteps / G);
             const int gsz = run_gsz(se - sb, kRecG);
-            const double* rec = (STAGE == 3) ? &sh.srun[0][0] : p.srung + (static_cast<size_t>(b) * G + g) * kRecG;
+            const double* rec = kOneSweep ? &sh.srun[0][0] : p.srung + (static_cast<size_t>(b) * G + g) * kRecG;
             const int token = walk(sb, se, gsz, sh.base, rec, sh.target, is_bonus);
             if (lane == 0) {
               p.out_tokens[uidx] = token;  // the row's token at its first rejection, or the bonus
@@ -2129,6 +2340,8 @@ struct cos_verify_ctx {
   double* d_zpart;
   double* d_wtotg;
   double* d_srung;
+  double* d_srungC;  // third and fourth channel of the one-sweep stage (ensembles of three or four models)
+  double* d_srungD;
   double* d_srungB;  // second channel of d_srung, for the one-sweep drawing stage
   int* d_part_arrivals;
   // optional per-stage timing (cos_verify_set_stage_timing)
@@ -2174,6 +2387,14 @@ KernelFn pick_kernel(int dtype, int mode, int stage, bool dense = false) {
 #define COS_CASE(DT, M, S) \
   if (dtype == DT && mode == M && stage == S) return cos_verify_kernel<DT, M, S>;
 #define COS_SAMPLING(DT, M) COS_CASE(DT, M, 0) COS_CASE(DT, M, 1) COS_CASE(DT, M, 2) COS_CASE(DT, M, 3)
+  // (stage 4, the one-sweep drawing stage with a channel per model, exists for ensembles only)
+  // its sweep holds four vectors per lane and the next four: built for one block per multiprocessor (the
+  // 64-register build spills a kilobyte per thread and is slower than the two-stage form)
+  if (mode == kEnsembleSample && stage == 4) {
+    if (dtype == COS_DTYPE_F32) return cos_verify_kernel<COS_DTYPE_F32, kEnsembleSample, 4, 1>;
+    if (dtype == COS_DTYPE_BF16) return cos_verify_kernel<COS_DTYPE_BF16, kEnsembleSample, 4, 1>;
+    if (dtype == COS_DTYPE_F16) return cos_verify_kernel<COS_DTYPE_F16, kEnsembleSample, 4, 1>;
+  }
   COS_SAMPLING(COS_DTYPE_F32, kEnsembleSample)
   COS_SAMPLING(COS_DTYPE_F32, kLogitSample)
   COS_CASE(COS_DTYPE_F32, kEnsembleGreedy, 0)
@@ -2252,6 +2473,15 @@ int choose_cluster(const cos_verify_config& c) {
 
 // Blocks per unit in the drawing stages: as many as fit on the device in one wave (two blocks per
 // multiprocessor), at least two steps per warp.
+// The stage that draws the tokens in one sweep: 3 where two channel sums describe every mass (the combine is at
+// logit level: proposer and combined logits; or it mixes two models), 4 for ensembles of three or four models (a
+// channel per model); 0: the two-stage form (more models, one model, greedy decoding).
+int one_sweep_stage(const cos_verify_config& c) {
+  if (c.temperature == 0.0f) return 0;
+  if (c.combine != COS_COMBINE_PROB_ENSEMBLE) return 3;
+  return c.n == 2 ? 3 : ((c.n == 3 || c.n == 4) ? 4 : 0);
+}
+
 int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
   int parts = 1;
   while (parts < kMaxParts && rows * parts * 2 <= 2 * sm_count) parts <<= 1;
@@ -2266,7 +2496,7 @@ int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
 // free: one wave of whole units leaves some multiprocessors with twice the work of others.  Small units
 // stay at one wave: their blocks are bound by latency, not by throughput.
 int choose_parts_one(const cos_verify_config& c, int rows, int sm_count) {
-  const long long slots = 2LL * sm_count;
+  const long long slots = (one_sweep_stage(c) == 4 ? 1LL : 2LL) * sm_count;  // blocks the device holds at once
   const int E = entries_per_vec(c.dtype);
   const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
   int parts = choose_parts(c, rows, sm_count);
@@ -2330,9 +2560,11 @@ cudaError_t launch_stage(int dtype, int mode, int stage, const KParams& p, int c
 cudaError_t prepare_kernels(int dtype, int mode, int cluster_size) {
   const bool draws = (mode == kEnsembleSample || mode == kLogitSample);
   cudaError_t e = cudaSuccess;
-  for (int st = 2; draws && st <= 3 && e == cudaSuccess; ++st)
-    e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, st)),
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, stage_smem(st));
+  for (int st = 2; draws && st <= 4 && e == cudaSuccess; ++st) {
+    KernelFn fn = pick_kernel(dtype, mode, st);
+    if (fn != nullptr)
+      e = cudaFuncSetAttribute(reinterpret_cast<const void*>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, stage_smem(st));
+  }
   if (e == cudaSuccess && cluster_size > 8)
     e = cudaFuncSetAttribute(reinterpret_cast<const void*>(pick_kernel(dtype, mode, 0)),
                              cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
@@ -2494,6 +2726,10 @@ extern "C" cos_status cos_verify_create(const cos_verify_config* config, cos_ver
   const size_t rec_per_row = steps > pmax * kWarps * kRecG ? steps : pmax * kWarps * kRecG;  // one record per step, or per group of a run
   ok = ok && cudaMalloc(&ctx->d_srung, rows * rec_per_row * sizeof(double)) == cudaSuccess;
   ok = ok && cudaMalloc(&ctx->d_srungB, rows * rec_per_row * sizeof(double)) == cudaSuccess;
+  if (one_sweep_stage(*config) == 4) {
+    ok = ok && cudaMalloc(&ctx->d_srungC, rows * rec_per_row * sizeof(double)) == cudaSuccess;
+    ok = ok && cudaMalloc(&ctx->d_srungD, rows * rec_per_row * sizeof(double)) == cudaSuccess;
+  }
   ok = ok && cudaMalloc(&ctx->d_part_arrivals, rows * P * sizeof(int)) == cudaSuccess;
   ctx->wait_limit = 1u << 20;
   ctx->test_drop = 0;
@@ -2621,6 +2857,8 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
   p.srung = ctx->d_srung;
   p.part_arrivals = ctx->d_part_arrivals;
   p.srungB = ctx->d_srungB;
+  p.srungC = ctx->d_srungC;
+  p.srungD = ctx->d_srungD;
   p.parts = ctx->parts;
   p.max_jobs = p.num_units + a->batch;
 
@@ -2665,7 +2903,8 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
     p.num_clusters = (most < cap ? most : cap) * p.parts;  // blocks of a drawing launch
     // Two channel sums describe every mass when the combine is at logit level (proposer, combined logits) or
     // mixes two models: then one sweep does the work of stages 1 and 2.  The test hooks keep the two-stage form.
-    const bool one_sweep = !all && (mode == kLogitSample || c.n == 2);
+    const int sweep_stage = one_sweep_stage(c);
+    const bool one_sweep = !all && sweep_stage != 0;
     if (!all && ctx->fused && ctx->draw_fused && p.vec_ok) {
       // the tokens are drawn by the persistent kernel's drawing items (one sweep with a channel sum per model, any
       // block takes any chunk of any row) instead of the drawing stages
@@ -2679,7 +2918,7 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
     if (one_sweep) {
       p.parts = ctx->parts_one;
       p.num_clusters = (most < cap ? most : cap) * p.parts;
-      e = launch_stage(c.dtype, mode, 3, p, 1, stream, true);
+      e = launch_stage(c.dtype, mode, sweep_stage, p, 1, stream, true);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stage)", e);
       if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
       ctx->ev_used = 3;
@@ -2842,11 +3081,10 @@ extern "C" cos_status cos_verify_get_info(const cos_verify_ctx* ctx, cos_verify_
   info->max_clusters = ctx->max_clusters[log2i(info->cluster_size)];
   info->sm_count = ctx->sm_count;
   {
-    // ordinary runs (no test hook): one launch at T = 0; else stage 0 and the one-sweep drawing stage where two
-    // channel sums describe a mass, stages 0, 1 and 2 otherwise
+    // ordinary runs (no test hook): one launch at T = 0; else stage 0 and the one-sweep drawing stage where it
+    // applies (see one_sweep_stage), stages 0, 1 and 2 otherwise
     const int mode = mode_of(ctx->cfg);
-    const bool one_sweep = (mode == kLogitSample) || (mode == kEnsembleSample && ctx->cfg.n == 2) ||
-                           (ctx->fused && ctx->draw_fused);
+    const bool one_sweep = one_sweep_stage(ctx->cfg) != 0 || (ctx->fused && ctx->draw_fused);
     info->launches_per_run = (ctx->cfg.temperature > 0.0f && !(ctx->fused && ctx->use_fused)) ? (one_sweep ? 2 : 3) : 1;
   }
   info->reserved[0] = ctx->fused ? ctx->fplan.chunks : ctx->parts;
@@ -2869,6 +3107,8 @@ extern "C" cos_status cos_verify_destroy(cos_verify_ctx* ctx) {
   cudaFree(ctx->d_wtotg);
   cudaFree(ctx->d_srung);
   cudaFree(ctx->d_srungB);
+  cudaFree(ctx->d_srungC);
+  cudaFree(ctx->d_srungD);
   cudaFree(ctx->d_part_arrivals);
   for (int k = 0; k < 4; ++k)
     if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
