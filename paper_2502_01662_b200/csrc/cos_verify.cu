@@ -33,6 +33,23 @@ using namespace cosv;
 
 namespace {
 
+// Optional timeline of the one-sweep drawing stage (build with -DCOS_STAGE_PROFILE): thread 0 of every block stamps
+// the global timer at eight points into g_sprof[block][point].  Compiled out of ordinary builds.
+#ifdef COS_STAGE_PROFILE
+constexpr int kSprofBlocks = 1024;
+__device__ unsigned long long g_sprof[kSprofBlocks * 8];
+#define SPROF(k)                                                                                  \
+  do {                                                                                            \
+    if (threadIdx.x == 0 && blockIdx.x < kSprofBlocks) {                                          \
+      unsigned long long t_;                                                                      \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                       \
+      g_sprof[blockIdx.x * 8 + (k)] = t_;                                                         \
+    }                                                                                             \
+  } while (0)
+#else
+#define SPROF(k)
+#endif
+
 struct Xchg {  // one per block and barrier parity; peers read it through DSMEM
   SoftPart soft[kMaxSlots];
   ArgPart arg[kMaxSlots];
@@ -547,6 +564,288 @@ __device__ __forceinline__ void one_sweep_channels(const KParams& p, Shared& sh,
       sh.wsoft[warp][i].ref = (i < p.n) ? sh.fsoft[i].ref : 0.f;
     }
   }
+}
+
+// The one-sweep drawing stage with two channel sums per step (stage 3), the sweep itself.  (Inline: as a function
+// of its own, with or without copies of the launch parameters it uses, its loop was slower by a quarter to a half.)
+template <int DT, int MODE>
+__device__ __forceinline__ void one_sweep_pair(const KParams& p, Shared& sh, uint4* ring, const char* base, int b, int rank, int lparts,
+                                            int pis, bool masked, float thr, bool is_bonus, bool draw_q, int emit, bool vec_ok,
+                                            double (&kc)[4]) {
+  constexpr int E = Elem<DT>::E;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  auto row_of = [&](int i) -> const void* { return base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes; };
+  // what the loop needs of the launch parameters, in registers (through `p` it would be read again after every store)
+  const float cT = p.cT, w0 = p.w[0], w1 = p.w[1];
+  const int n = p.n, mask_model = p.mask_model;
+  double* const rec_a = p.srung;
+  double* const rec_b = p.srungB;
+  // ---- the drawing stages in one sweep.  A token's mass is k_A e_A / Z_A + k_B e_B / Z_B clipped at zero,
+  // where the two channels are the two models (ensemble, n = 2) or the proposer's and the combined logits
+  // (logit level), and (k_A, k_B) says what is drawn: max(0, r - q), r, or q.  The set of tokens with a
+  // positive mass is decided with the normalisers stage 0 left (they are good to 1e-7, and a token whose sign
+  // that could change carries no mass to speak of); over that set the mass is LINEAR in 1/Z_A and 1/Z_B,
+  // so this sweep only adds up e_A and e_B over that set, step by step, and over everything for the refined
+  // normalisers of stage 1.  Whoever locates the token turns the sums into masses once the normalisers are
+  // complete.
+  // Terms above 2^-8 of a normaliser go through fp64, as in stage 1.
+  double kA, kB;
+  if (MODE == kEnsembleSample) {
+    const double selA = (pis == 0) ? 1.0 : 0.0, selB = (pis == 1) ? 1.0 : 0.0;
+    kA = !is_bonus ? p.w64[0] - selA : (draw_q ? selA : p.w64[0]);
+    kB = !is_bonus ? p.w64[1] - selB : (draw_q ? selB : p.w64[1]);
+  } else {
+    kA = !is_bonus ? -1.0 : (draw_q ? 1.0 : 0.0);
+    kB = (is_bonus && draw_q) ? 0.0 : 1.0;
+  }
+  const double ctA64 = kA / sh.fsoft[0].s, ctB64 = kB / sh.fsoft[1].s;  // with the first estimates: signs only
+  const float ctA = static_cast<float>(ctA64), ctB = static_cast<float>(ctB64);
+  const float nrefA = -sh.fsoft[0].ref, nrefB = -sh.fsoft[1].ref;
+  const float btA = sh.big_thr[0], btB = sh.big_thr[1];
+  const double drefA = static_cast<double>(sh.fsoft[0].ref), drefB = static_cast<double>(sh.fsoft[1].ref);
+  const char* row0 = reinterpret_cast<const char*>(row_of(0));
+  const long long row_step = p.s_model * Elem<DT>::bytes;
+  // this block's steps [blk_lo, blk_hi); its warps take them in turn, so that the block reads 8 KB of
+  // every row at a time; every step (32 lanes x E entries, in token order) leaves its two sums on record
+  const int blk_lo = static_cast<int>(static_cast<long long>(rank) * p.nsteps / lparts);
+  const int blk_hi = static_cast<int>(static_cast<long long>(rank + 1) * p.nsteps / lparts);
+  const size_t rec_at = static_cast<size_t>(b) * p.nsteps;
+  const int nfull = vec_ok ? p.V / (32 * E) : 0;  // steps below this are whole aligned vectors
+  float zsA = 0.f, zsB = 0.f, aA = 0.f, aB = 0.f;  // small terms: normalisers (all steps), sums of the step
+  // the big terms of the same four sums sit in shared memory (the staging ring is idle during this sweep),
+  // one slot per thread and sum: [0] Z_A, [1] Z_B, [2] and [3] the step's sums
+  double* bigacc = reinterpret_cast<double*>(ring) + tid;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) bigacc[q * kThreads] = 0.0;
+  bool hasbig = false;
+  if (tid == 0) {
+    OneSweep& c = one_sweep_consts(sh);
+    c.ctA = ctA;
+    c.ctB = ctB;
+    c.nrefA = nrefA;
+    c.nrefB = nrefB;
+    c.btA = btA;
+    c.btB = btB;
+    c.ctA64 = ctA64;
+    c.ctB64 = ctB64;
+    c.drefA = drefA;
+    c.drefB = drefB;
+  }
+  __syncthreads();
+  // one vector of entries: channel arguments xa (proposer's or model 0's logits) and xb (model 1's or the
+  // combined logits)
+  // (entries outside the mask arrive with xb = -inf: their e_B is zero)
+  const float nctA = -ctA;
+  auto eat = [&](const float (&xa)[E], const float (&xb)[E]) -> bool {
+    float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+      const float eA = ex2_approx(fmaf(xa[k], cT, nrefA));
+      const float eB = ex2_approx(fmaf(xb[k], cT, nrefB));
+      // k_A e_A / Z_A + k_B e_B / Z_B > 0 with the products rounded one by one: where r and q coincide
+      // neither side exceeds the other, as in exact arithmetic
+      const float in_p = (__fmul_rn(ctB, eB) > __fmul_rn(nctA, eA)) ? 1.f : 0.f;
+      vzA += eA;
+      vzB += eB;
+      vaA = fmaf(in_p, eA, vaA);
+      vaB = fmaf(in_p, eB, vaB);
+    }
+    // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum
+    // big); the caller does the vector again, big entries in fp64
+    if (vzA > btA || vzB > btB) return true;
+    zsA += vzA;
+    zsB += vzB;
+    aA += vaA;
+    aB += vaB;
+    return false;
+  };
+  // a vector with a big entry, entry by entry from the stored logits, out of line (ragged steps)
+  auto redo_from_memory = [&](int e0) {
+    const float4 r = one_sweep_big_vector<DT, MODE>(p, one_sweep_consts(sh), base, e0, pis, masked, thr, bigacc);
+    zsA += r.x;
+    zsB += r.y;
+    aA += r.z;
+    aB += r.w;
+    hasbig = true;
+  };
+  // the same from the two vectors at hand (models beyond the second are read again, entry by entry)
+  auto redo = [&](const uint4& r0, const uint4& r1, int e0) {
+    float x0[E], x1[E];
+    Elem<DT>::unpack(r0, x0);
+    Elem<DT>::unpack(r1, x1);
+    float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f;
+#pragma unroll
+    for (int k = 0; k < E; ++k) {
+      float xa, xb;
+      bool in = true;
+      if (MODE == kEnsembleSample) {
+        xa = x0[k];
+        xb = x1[k];
+      } else {
+        xb = fmaf(p.w[0], x0[k], 0.f);
+        if (p.n >= 2) xb = fmaf(p.w[1], x1[k], xb);
+        for (int i = 2; i < p.n; ++i) xb = fmaf(p.w[i], Elem<DT>::load1(row_of(i), e0 + k), xb);
+        xa = (pis == 0) ? x0[k] : (pis == 1 ? x1[k] : Elem<DT>::load1(row_of(pis), e0 + k));
+        if (masked) {
+          const int mm = p.mask_model;
+          const float xm = (mm == 0) ? x0[k] : (mm == 1 ? x1[k] : Elem<DT>::load1(row_of(mm), e0 + k));
+          in = (xm >= thr);
+        }
+      }
+      const float eA = ex2_approx(fmaf(xa, p.cT, nrefA));
+      const float eB = in ? ex2_approx(fmaf(xb, p.cT, nrefB)) : 0.f;
+      if (eA > btA || eB > btB) {
+        double cb;
+        if (MODE == kEnsembleSample) {
+          cb = static_cast<double>(xb);
+        } else {
+          cb = fma(p.w64[0], static_cast<double>(x0[k]), 0.0);
+          if (p.n >= 2) cb = fma(p.w64[1], static_cast<double>(x1[k]), cb);
+          for (int i = 2; i < p.n; ++i) cb = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e0 + k)), cb);
+        }
+        const double2 d = big_pair(static_cast<double>(xa) * p.cT64 - drefA, cb * p.cT64 - drefB, in);
+        bigacc[0] += d.x;
+        bigacc[kThreads] += d.y;
+        if (ctA64 * d.x + ctB64 * d.y > 0.0) {
+          bigacc[2 * kThreads] += d.x;
+          bigacc[3 * kThreads] += d.y;
+        }
+      } else {
+        const bool pos = __fadd_rn(__fmul_rn(ctA, eA), __fmul_rn(ctB, eB)) > 0.f;
+        vzA += eA;
+        vzB += eB;
+        vaA += pos ? eA : 0.f;
+        vaB += pos ? eB : 0.f;
+      }
+    }
+    zsA += vzA;
+    zsB += vzB;
+    aA += vaA;
+    aB += vaB;
+    hasbig = true;
+  };
+  // the channel arguments of one step from the lane's vectors (the first two models' fetched ahead)
+  auto feed = [&](const uint4& r0, const uint4& r1, int s) {
+    const int e0 = (s * 32 + lane) * E;
+    if (MODE == kEnsembleSample) {
+      float xa[E], xb[E];
+      Elem<DT>::unpack(r0, xa);
+      Elem<DT>::unpack(r1, xb);
+      if (eat(xa, xb)) redo(r0, r1, e0);
+    } else {
+      float cmb[E], vq[E];
+      unsigned inb = 0u;
+#pragma unroll
+      for (int k = 0; k < E; ++k) cmb[k] = 0.f;
+      auto take = [&](int i, const uint4& raw) {
+        float x[E];
+        Elem<DT>::unpack(raw, x);
+        const float wi = (i == 0) ? w0 : (i == 1 ? w1 : p.w[i]);
+#pragma unroll
+        for (int k = 0; k < E; ++k) {
+          cmb[k] = fmaf(wi, x[k], cmb[k]);
+          if (i == pis) vq[k] = x[k];
+          if (masked && i == mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
+        }
+      };
+      take(0, r0);
+      if (n >= 2) take(1, r1);
+      for (int i = 2; i < n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(s * 32 + lane) * 16));
+      if (masked) {
+#pragma unroll
+        for (int k = 0; k < E; ++k) cmb[k] = ((inb >> k) & 1u) ? cmb[k] : -INFINITY;
+      }
+      if (eat(vq, cmb)) redo(r0, r1, e0);
+    }
+  };
+  const bool pair = (MODE == kEnsembleSample) || (n >= 2);
+  uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
+  if (blk_lo + warp < blk_hi && blk_lo + warp < nfull) {
+    const char* src = row0 + static_cast<long long>((blk_lo + warp) * 32 + lane) * 16;
+    nx0 = ldg_stream16(src);
+    if (pair) nx1 = ldg_stream16(src + row_step);
+  }
+  for (int s = blk_lo + warp; s < blk_hi; s += kWarps) {
+    if (s < nfull) {
+      const uint4 a0 = nx0, a1 = nx1;
+      const int sn = s + kWarps;
+      if (sn < blk_hi && sn < nfull) {
+        const char* src = row0 + static_cast<long long>(sn * 32 + lane) * 16;
+        nx0 = ldg_stream16(src);
+        if (pair) nx1 = ldg_stream16(src + row_step);
+      }
+      feed(a0, a1, s);
+    } else {
+      // ragged or unaligned step: entry by entry; entries beyond V read as -inf (no mass, outside every set)
+      const int e0 = (s * 32 + lane) * E;
+      if (MODE == kEnsembleSample) {
+        float xa[E], xb[E];
+        load_chunk<DT>(row_of(0), e0, p.V, vec_ok, xa);
+        load_chunk<DT>(row_of(1), e0, p.V, vec_ok, xb);
+        if (eat(xa, xb)) redo_from_memory(e0);
+      } else {
+        float cmb[E], vq[E];
+        unsigned inb = 0u;
+#pragma unroll
+        for (int k = 0; k < E; ++k) cmb[k] = 0.f;
+        for (int i = 0; i < p.n; ++i) {
+          float x[E];
+          load_chunk<DT>(row_of(i), e0, p.V, vec_ok, x);
+#pragma unroll
+          for (int k = 0; k < E; ++k) {
+            cmb[k] = (e0 + k < p.V) ? fmaf(p.w[i], x[k], cmb[k]) : -INFINITY;
+            if (i == pis) vq[k] = x[k];
+            if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
+          }
+        }
+        if (masked) {
+#pragma unroll
+          for (int k = 0; k < E; ++k) cmb[k] = ((inb >> k) & 1u) ? cmb[k] : -INFINITY;
+        }
+        if (eat(vq, cmb)) redo_from_memory(e0);
+      }
+    }
+    // the step's two sums over the warp
+    float ra = aA, rb = aB;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      ra += __shfl_xor_sync(0xffffffffu, ra, d);
+      rb += __shfl_xor_sync(0xffffffffu, rb, d);
+    }
+    double da = static_cast<double>(ra), db = static_cast<double>(rb);
+    if (__any_sync(0xffffffffu, hasbig)) {
+      double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
+      bigacc[2 * kThreads] = bigacc[3 * kThreads] = 0.0;
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) {
+        ta += shfl_double(ta, lane ^ d);
+        tb += shfl_double(tb, lane ^ d);
+      }
+      da += ta;
+      db += tb;
+    }
+    if (lane == 0 && emit) {
+      rec_a[rec_at + s] = da;
+      rec_b[rec_at + s] = db;
+    }
+    aA = aB = 0.f;
+  }
+  {
+    double tA = static_cast<double>(zsA) + bigacc[0], tB = static_cast<double>(zsB) + bigacc[kThreads];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      tA += shfl_double(tA, lane ^ d);
+      tB += shfl_double(tB, lane ^ d);
+    }
+    if (lane == 0) {
+      sh.wsoft[warp][0].s = tA;
+      sh.wsoft[warp][0].ref = sh.fsoft[0].ref;
+      sh.wsoft[warp][1].s = tB;
+      sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
+    }
+  }
+  kc[0] = kA;
+  kc[1] = kB;
 }
 
 // Combined logit of one token in fp64, from the stored logits: the chain of fused multiply-adds that
@@ -1118,6 +1417,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   // later stages are launched while the previous one drains (programmatic dependent launch);
   // nothing it wrote is read before this point
   if (STAGE >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (kOneSweep) SPROF(0);
   if ((STAGE == 1 || kOneSweep) && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
   const int job_stride = gridDim.x / lparts;
   int unit = cluster_id, emit = 0, job_it = 0, njobs = 0;
@@ -1476,278 +1776,15 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
       } else {
       bool do_locate = false;
       if (kOneSweep) {
+        SPROF(1);
         double kc[4] = {0.0, 0.0, 0.0, 0.0};  // coefficient of every channel in what is drawn
         if (STAGE == 4) {
           one_sweep_channels<DT>(p, sh, ring, base, b, rank, lparts, pis, is_bonus, draw_q, emit, vec_ok, kc);
         } else {
-        // ---- the drawing stages in one sweep.  A token's mass is k_A e_A / Z_A + k_B e_B / Z_B clipped at zero,
-        // where the two channels are the two models (ensemble, n = 2) or the proposer's and the combined logits
-        // (logit level), and (k_A, k_B) says what is drawn: max(0, r - q), r, or q.  The set of tokens with a
-        // positive mass is decided with the normalisers stage 0 left (they are good to 1e-7, and a token whose sign
-        // that could change carries no mass to speak of); over that set the mass is LINEAR in 1/Z_A and 1/Z_B,
-        // so this sweep only adds up e_A and e_B over that set, step by step, and over everything for the refined
-        // normalisers of stage 1.  Whoever locates the token turns the sums into masses once the normalisers are
-        // complete.
-        // Terms above 2^-8 of a normaliser go through fp64, as in stage 1.
-        double kA, kB;
-        if (MODE == kEnsembleSample) {
-          const double selA = (pis == 0) ? 1.0 : 0.0, selB = (pis == 1) ? 1.0 : 0.0;
-          kA = !is_bonus ? p.w64[0] - selA : (draw_q ? selA : p.w64[0]);
-          kB = !is_bonus ? p.w64[1] - selB : (draw_q ? selB : p.w64[1]);
-        } else {
-          kA = !is_bonus ? -1.0 : (draw_q ? 1.0 : 0.0);
-          kB = (is_bonus && draw_q) ? 0.0 : 1.0;
-        }
-        const double ctA64 = kA / sh.fsoft[0].s, ctB64 = kB / sh.fsoft[1].s;  // with the first estimates: signs only
-        const float ctA = static_cast<float>(ctA64), ctB = static_cast<float>(ctB64);
-        const float nrefA = -sh.fsoft[0].ref, nrefB = -sh.fsoft[1].ref;
-        const float btA = sh.big_thr[0], btB = sh.big_thr[1];
-        const double drefA = static_cast<double>(sh.fsoft[0].ref), drefB = static_cast<double>(sh.fsoft[1].ref);
-        const char* row0 = reinterpret_cast<const char*>(row_of(0));
-        const long long row_step = p.s_model * Elem<DT>::bytes;
-        // this block's steps [blk_lo, blk_hi); its warps take them in turn, so that the block reads 8 KB of
-        // every row at a time; every step (32 lanes x E entries, in token order) leaves its two sums on record
-        const int blk_lo = static_cast<int>(static_cast<long long>(rank) * p.nsteps / lparts);
-        const int blk_hi = static_cast<int>(static_cast<long long>(rank + 1) * p.nsteps / lparts);
-        const size_t rec_at = static_cast<size_t>(b) * p.nsteps;
-        const int nfull = vec_ok ? p.V / (32 * E) : 0;  // steps below this are whole aligned vectors
-        float zsA = 0.f, zsB = 0.f, aA = 0.f, aB = 0.f;  // small terms: normalisers (all steps), sums of the step
-        // the big terms of the same four sums sit in shared memory (the staging ring is idle during this sweep),
-        // one slot per thread and sum: [0] Z_A, [1] Z_B, [2] and [3] the step's sums
-        double* bigacc = reinterpret_cast<double*>(ring) + tid;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) bigacc[q * kThreads] = 0.0;
-        bool hasbig = false;
-        if (tid == 0) {
-          OneSweep& c = one_sweep_consts(sh);
-          c.ctA = ctA;
-          c.ctB = ctB;
-          c.nrefA = nrefA;
-          c.nrefB = nrefB;
-          c.btA = btA;
-          c.btB = btB;
-          c.ctA64 = ctA64;
-          c.ctB64 = ctB64;
-          c.drefA = drefA;
-          c.drefB = drefB;
+          one_sweep_pair<DT, MODE>(p, sh, ring, base, b, rank, lparts, pis, masked, thr, is_bonus, draw_q, emit, vec_ok, kc);
         }
         __syncthreads();
-        // one vector of entries: channel arguments xa (proposer's or model 0's logits) and xb (model 1's or the
-        // combined logits)
-        // (entries outside the mask arrive with xb = -inf: their e_B is zero)
-        const float nctA = -ctA;
-        auto eat = [&](const float (&xa)[E], const float (&xb)[E]) -> bool {
-          float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f;
-#pragma unroll
-          for (int k = 0; k < E; ++k) {
-            const float eA = ex2_approx(fmaf(xa[k], p.cT, nrefA));
-            const float eB = ex2_approx(fmaf(xb[k], p.cT, nrefB));
-            // k_A e_A / Z_A + k_B e_B / Z_B > 0 with the products rounded one by one: where r and q coincide
-            // neither side exceeds the other, as in exact arithmetic
-            const float in_p = (__fmul_rn(ctB, eB) > __fmul_rn(nctA, eA)) ? 1.f : 0.f;
-            vzA += eA;
-            vzB += eB;
-            vaA = fmaf(in_p, eA, vaA);
-            vaB = fmaf(in_p, eB, vaB);
-          }
-          // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum
-          // big); the caller does the vector again, big entries in fp64
-          if (vzA > btA || vzB > btB) return true;
-          zsA += vzA;
-          zsB += vzB;
-          aA += vaA;
-          aB += vaB;
-          return false;
-        };
-        // a vector with a big entry, entry by entry from the stored logits, out of line (ragged steps)
-        auto redo_from_memory = [&](int e0) {
-          const float4 r = one_sweep_big_vector<DT, MODE>(p, one_sweep_consts(sh), base, e0, pis, masked, thr, bigacc);
-          zsA += r.x;
-          zsB += r.y;
-          aA += r.z;
-          aB += r.w;
-          hasbig = true;
-        };
-        // the same from the two vectors at hand (models beyond the second are read again, entry by entry)
-        auto redo = [&](const uint4& r0, const uint4& r1, int e0) {
-          float x0[E], x1[E];
-          Elem<DT>::unpack(r0, x0);
-          Elem<DT>::unpack(r1, x1);
-          float vzA = 0.f, vzB = 0.f, vaA = 0.f, vaB = 0.f;
-#pragma unroll
-          for (int k = 0; k < E; ++k) {
-            float xa, xb;
-            bool in = true;
-            if (MODE == kEnsembleSample) {
-              xa = x0[k];
-              xb = x1[k];
-            } else {
-              xb = fmaf(p.w[0], x0[k], 0.f);
-              if (p.n >= 2) xb = fmaf(p.w[1], x1[k], xb);
-              for (int i = 2; i < p.n; ++i) xb = fmaf(p.w[i], Elem<DT>::load1(row_of(i), e0 + k), xb);
-              xa = (pis == 0) ? x0[k] : (pis == 1 ? x1[k] : Elem<DT>::load1(row_of(pis), e0 + k));
-              if (masked) {
-                const int mm = p.mask_model;
-                const float xm = (mm == 0) ? x0[k] : (mm == 1 ? x1[k] : Elem<DT>::load1(row_of(mm), e0 + k));
-                in = (xm >= thr);
-              }
-            }
-            const float eA = ex2_approx(fmaf(xa, p.cT, nrefA));
-            const float eB = in ? ex2_approx(fmaf(xb, p.cT, nrefB)) : 0.f;
-            if (eA > btA || eB > btB) {
-              double cb;
-              if (MODE == kEnsembleSample) {
-                cb = static_cast<double>(xb);
-              } else {
-                cb = fma(p.w64[0], static_cast<double>(x0[k]), 0.0);
-                if (p.n >= 2) cb = fma(p.w64[1], static_cast<double>(x1[k]), cb);
-                for (int i = 2; i < p.n; ++i) cb = fma(p.w64[i], static_cast<double>(Elem<DT>::load1(row_of(i), e0 + k)), cb);
-              }
-              const double2 d = big_pair(static_cast<double>(xa) * p.cT64 - drefA, cb * p.cT64 - drefB, in);
-              bigacc[0] += d.x;
-              bigacc[kThreads] += d.y;
-              if (ctA64 * d.x + ctB64 * d.y > 0.0) {
-                bigacc[2 * kThreads] += d.x;
-                bigacc[3 * kThreads] += d.y;
-              }
-            } else {
-              const bool pos = __fadd_rn(__fmul_rn(ctA, eA), __fmul_rn(ctB, eB)) > 0.f;
-              vzA += eA;
-              vzB += eB;
-              vaA += pos ? eA : 0.f;
-              vaB += pos ? eB : 0.f;
-            }
-          }
-          zsA += vzA;
-          zsB += vzB;
-          aA += vaA;
-          aB += vaB;
-          hasbig = true;
-        };
-        // the channel arguments of one step from the lane's vectors (the first two models' fetched ahead)
-        auto feed = [&](const uint4& r0, const uint4& r1, int s) {
-          const int e0 = (s * 32 + lane) * E;
-          if (MODE == kEnsembleSample) {
-            float xa[E], xb[E];
-            Elem<DT>::unpack(r0, xa);
-            Elem<DT>::unpack(r1, xb);
-            if (eat(xa, xb)) redo(r0, r1, e0);
-          } else {
-            float cmb[E], vq[E];
-            unsigned inb = 0u;
-#pragma unroll
-            for (int k = 0; k < E; ++k) cmb[k] = 0.f;
-            auto take = [&](int i, const uint4& raw) {
-              float x[E];
-              Elem<DT>::unpack(raw, x);
-              const float wi = p.w[i];
-#pragma unroll
-              for (int k = 0; k < E; ++k) {
-                cmb[k] = fmaf(wi, x[k], cmb[k]);
-                if (i == pis) vq[k] = x[k];
-                if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
-              }
-            };
-            take(0, r0);
-            if (p.n >= 2) take(1, r1);
-            for (int i = 2; i < p.n; ++i) take(i, ldg_stream16(row0 + i * row_step + static_cast<long long>(s * 32 + lane) * 16));
-            if (masked) {
-#pragma unroll
-              for (int k = 0; k < E; ++k) cmb[k] = ((inb >> k) & 1u) ? cmb[k] : -INFINITY;
-            }
-            if (eat(vq, cmb)) redo(r0, r1, e0);
-          }
-        };
-        const bool pair = (MODE == kEnsembleSample) || (p.n >= 2);
-        uint4 nx0 = make_uint4(0u, 0u, 0u, 0u), nx1 = nx0;
-        if (blk_lo + warp < blk_hi && blk_lo + warp < nfull) {
-          const char* src = row0 + static_cast<long long>((blk_lo + warp) * 32 + lane) * 16;
-          nx0 = ldg_stream16(src);
-          if (pair) nx1 = ldg_stream16(src + row_step);
-        }
-        for (int s = blk_lo + warp; s < blk_hi; s += kWarps) {
-          if (s < nfull) {
-            const uint4 a0 = nx0, a1 = nx1;
-            const int sn = s + kWarps;
-            if (sn < blk_hi && sn < nfull) {
-              const char* src = row0 + static_cast<long long>(sn * 32 + lane) * 16;
-              nx0 = ldg_stream16(src);
-              if (pair) nx1 = ldg_stream16(src + row_step);
-            }
-            feed(a0, a1, s);
-          } else {
-            // ragged or unaligned step: entry by entry; entries beyond V read as -inf (no mass, outside every set)
-            const int e0 = (s * 32 + lane) * E;
-            if (MODE == kEnsembleSample) {
-              float xa[E], xb[E];
-              load_chunk<DT>(row_of(0), e0, p.V, vec_ok, xa);
-              load_chunk<DT>(row_of(1), e0, p.V, vec_ok, xb);
-              if (eat(xa, xb)) redo_from_memory(e0);
-            } else {
-              float cmb[E], vq[E];
-              unsigned inb = 0u;
-#pragma unroll
-              for (int k = 0; k < E; ++k) cmb[k] = 0.f;
-              for (int i = 0; i < p.n; ++i) {
-                float x[E];
-                load_chunk<DT>(row_of(i), e0, p.V, vec_ok, x);
-#pragma unroll
-                for (int k = 0; k < E; ++k) {
-                  cmb[k] = (e0 + k < p.V) ? fmaf(p.w[i], x[k], cmb[k]) : -INFINITY;
-                  if (i == pis) vq[k] = x[k];
-                  if (masked && i == p.mask_model) inb |= (x[k] >= thr) ? (1u << k) : 0u;
-                }
-              }
-              if (masked) {
-#pragma unroll
-                for (int k = 0; k < E; ++k) cmb[k] = ((inb >> k) & 1u) ? cmb[k] : -INFINITY;
-              }
-              if (eat(vq, cmb)) redo_from_memory(e0);
-            }
-          }
-          // the step's two sums over the warp
-          float ra = aA, rb = aB;
-#pragma unroll
-          for (int d = 16; d > 0; d >>= 1) {
-            ra += __shfl_xor_sync(0xffffffffu, ra, d);
-            rb += __shfl_xor_sync(0xffffffffu, rb, d);
-          }
-          double da = static_cast<double>(ra), db = static_cast<double>(rb);
-          if (__any_sync(0xffffffffu, hasbig)) {
-            double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
-            bigacc[2 * kThreads] = bigacc[3 * kThreads] = 0.0;
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-              ta += shfl_double(ta, lane ^ d);
-              tb += shfl_double(tb, lane ^ d);
-            }
-            da += ta;
-            db += tb;
-          }
-          if (lane == 0 && emit) {
-            p.srung[rec_at + s] = da;
-            p.srungB[rec_at + s] = db;
-          }
-          aA = aB = 0.f;
-        }
-        {
-          double tA = static_cast<double>(zsA) + bigacc[0], tB = static_cast<double>(zsB) + bigacc[kThreads];
-#pragma unroll
-          for (int d = 16; d > 0; d >>= 1) {
-            tA += shfl_double(tA, lane ^ d);
-            tB += shfl_double(tB, lane ^ d);
-          }
-          if (lane == 0) {
-            sh.wsoft[warp][0].s = tA;
-            sh.wsoft[warp][0].ref = sh.fsoft[0].ref;
-            sh.wsoft[warp][1].s = tB;
-            sh.wsoft[warp][1].ref = sh.fsoft[1].ref;
-          }
-        }
-        kc[0] = kA;
-        kc[1] = kB;
-        }
-        __syncthreads();
+        SPROF(2);
         if (warp < NCH) {
           float ref = (lane < kWarps) ? sh.wsoft[lane][warp].ref : -INFINITY;
           double sum = (lane < kWarps) ? sh.wsoft[lane][warp].s : 0.0;
@@ -1761,13 +1798,14 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           const int prev = atomicAdd(&p.part_arrivals[uidx], 1);
           sh.win_g = (prev == p.parts - 1) ? 1 : 0;
           if (prev == p.parts - 1) {
-            p.part_arrivals[uidx] = 0;  // ready for the next run
-            __threadfence();
+            __threadfence();            // what the other blocks wrote before they arrived is visible from here on
+            p.part_arrivals[uidx] = 0;  // ready for the next run (a later launch: nothing waits for this store)
           }
         }
         __syncthreads();
         do_locate = (sh.win_g != 0) && emit;  // (every unit listed for this stage is its row's drawing unit)
         __syncthreads();
+        SPROF(3);
         if (do_locate) {
           if (tid < NCH) {
             double z = 0.0;
@@ -1780,6 +1818,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             one_sweep_coef(sh)[tid] = live ? kmine / z : 0.0;
           }
           __syncthreads();
+          SPROF(4);
         }
       }
       if (!kOneSweep || do_locate) {
@@ -1998,11 +2037,23 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         int token = -1, last_pos = -1;
         const int rs_begin = sb + grp * gszv;
         const int rs_end = (rs_begin + gszv < se) ? rs_begin + gszv : se;
+        const int wfull = vec_ok ? p.V / (32 * E) : 0;  // steps below this are whole aligned vectors
         for (int s = rs_begin; s < rs_end && token < 0; ++s) {
           float mass32[E];
           unsigned bigbits;
           const int e0 = (s * 32 + lane) * E;
-          chunk_mass(e0, use_r, mass32, bigbits, nullptr);
+          // the lane's vectors of the step go through its slots of the staging ring (idle by now), so that the big
+          // tokens, which are evaluated one by one, find their logits there instead of in global memory.  (Ensembles
+          // only: at logit level the same made the whole stage 4 % slower on the largest workload; the compiler's
+          // register allocation for the sweep changes with it.)
+          const uint4* st = nullptr;
+          if (MODE == kEnsembleSample && s < wfull && p.n <= kRingVecs) {
+            const char* src = reinterpret_cast<const char*>(row_of(0)) + static_cast<long long>(s * 32 + lane) * 16;
+            for (int i = 0; i < p.n; ++i) myring[i * 32] = ldg_stream16(src + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes);
+            st = myring;
+          }
+          chunk_mass(e0, use_r, mass32, bigbits, st);
+          if (kOneSweep) SPROF(7);
           // per-token masses of this lane in fp64 (big tokens from their fp64 evaluation)
           double m64[E];
 #pragma unroll
@@ -2010,7 +2061,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           if (bigbits) {
 #pragma unroll
             for (int k = 0; k < E; ++k)
-              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, nullptr, k);
+              if (bigbits & (1u << k)) m64[k] = big_mass(e0 + k, use_r, st, k);
           }
           // the lane's mass exactly as lane_mass() forms it (fp32 sum of the small tokens, then the big ones
           // in token order), from the values already at hand
@@ -2148,8 +2199,8 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           const int prev = atomicAdd(&p.part_arrivals[uidx], 1);
           sh.win_g = (prev == p.parts - 1) ? 1 : 0;
           if (prev == p.parts - 1) {
-            p.part_arrivals[uidx] = 0;  // ready for the next run
-            __threadfence();
+            __threadfence();            // what the other blocks wrote before they arrived is visible from here on
+            p.part_arrivals[uidx] = 0;  // ready for the next run (a later launch: nothing waits for this store)
           }
         }
         __syncthreads();
@@ -2177,8 +2228,17 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             }
             return fmax(0.0, acc);
           };
+          // (the masses of a thread's first four steps stay in registers for the second pass)
+          double mkeep[4] = {0.0, 0.0, 0.0, 0.0};
           double mine = 0.0;
-          for (int st = lo; st < hi; ++st) mine += step_mass(st);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (lo + q < hi) {
+              mkeep[q] = step_mass(lo + q);
+              mine += mkeep[q];
+            }
+          }
+          for (int st = lo + 4; st < hi; ++st) mine += step_mass(st);
           double incl = mine;
 #pragma unroll
           for (int d = 1; d < 32; d <<= 1) {
@@ -2205,8 +2265,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           double before = sh.wincl[warp] + (incl - mine);
           int first = 0x7fffffff, last = -1;
           double first_base = 0.0, first_m = 0.0, last_base = 0.0, last_m = 0.0;
-          for (int st = lo; st < hi; ++st) {
-            const double m = step_mass(st);
+          auto look = [&](int st, double m) {
             if (m > 0.0) {
               last = st;
               last_base = before;
@@ -2218,7 +2277,11 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
               }
             }
             before += m;
-          }
+          };
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (lo + q < hi) look(lo + q, mkeep[q]);
+          for (int st = lo + 4; st < hi; ++st) look(st, step_mass(st));
           if (first != 0x7fffffff) atomicMin(&sh.win_g, first);
           if (last >= 0) atomicMax(&sh.win_rank, last);  // rounding corner: the last step with mass
           __syncthreads();
@@ -2238,6 +2301,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
             one_step = wlast;
           }
           if (tid == 0) sh.win_g = (one_step >= 0) ? 0 : -1;
+          SPROF(5);
         } else {
           for (int g = tid; g < G; g += kThreads) sh.gw[g] = __ldcg(&p.wtotg[static_cast<size_t>(uidx) * G + g]);
           __syncthreads();
@@ -2261,6 +2325,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
               if (is_bonus && p.bonus_prob != nullptr && token >= 0)
                 p.bonus_prob[b] = static_cast<float>(big_mass(token, true, nullptr, 0));
             }
+            SPROF(6);
           }
         } else if (!is_bonus && emit) {
           // no residual mass although a token is needed: this block draws from r instead, over the whole
@@ -2937,6 +3002,13 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
 }
 
 }  // namespace
+
+#ifdef COS_STAGE_PROFILE
+extern "C" int cos_stage_profile_read(unsigned long long* out, int blocks) {  // 8 words per block
+  const size_t n = static_cast<size_t>(blocks < kSprofBlocks ? blocks : kSprofBlocks) * 8 * sizeof(unsigned long long);
+  return cudaMemcpyFromSymbol(out, g_sprof, n) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 extern "C" cos_status cos_verify_run(cos_verify_ctx* ctx, const cos_verify_args* a, void* cuda_stream) {
   if (ctx && a && a->lse && reinterpret_cast<uintptr_t>(a->lse) % 4) {
