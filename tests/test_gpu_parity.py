@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2502_01662_b200 import synth
-from paper_2502_01662_b200 import COS_RUN_ALL_RESIDUALS
+from paper_2502_01662_b200 import COS_RUN_ALL_RESIDUALS, COS_ROW_BAD_DRAFT, COS_ROW_NONFINITE
 
 import helpers
 
@@ -84,6 +84,74 @@ def test_one_sweep_drawing_stage_with_more_than_two_models(w):
         gpum = helpers.run_gpu(w, inputs, diag=True, bonus_model=m)
         statm = helpers.check_parity(w, gpum, refm)
         assert statm["excused_accept"] + statm["excused_sample"] <= 1, statm
+
+
+# Ensembles of every size (Eq. 4).  Three or four models draw their tokens in the one-sweep stage that keeps a sum per
+# model and step; one model, or more than four, in the two-stage form.  Unaligned rows (scalar loads throughout),
+# sharp distributions (low temperature: big terms are common), fp32 and fp16 logits, negative-free weights that
+# do not sum to one in fp32, and a three-model ensemble whose fourth channel stays empty.
+def _ens(name, n, weights, T, batch, gamma, vocab, dtype, dist="gauss", **kw):
+    return synth.Workload(name, n, synth.COMBINE_PROB_ENSEMBLE, weights, T, batch, gamma, vocab, dtype, dist,
+                          proposer_rule="cycle", **kw)
+
+
+ENSEMBLE_N = [
+    _ens("ens3_bf16", 3, (0.5, 0.3, 0.2), 0.8, 6, 3, 20008, "bf16", sigma=3.0, rho=0.7),
+    _ens("ens3_sharp_f32_unaligned", 3, (0.2, 0.5, 0.3), 0.35, 5, 2, 4099, "f32", sigma=3.0, rho=0.8),
+    _ens("ens4_zipf_f16", 4, (0.4, 0.3, 0.2, 0.1), 0.7, 5, 4, 50000, "f16", "gumbel_zipf", rho=0.85),
+    _ens("ens4_sharp_ragged", 4, (0.25, 0.25, 0.25, 0.25), 0.3, 4, 3, 9001, "bf16", sigma=2.5, rho=0.6),
+    _ens("ens4_wide_gamma0", 4, (0.1, 0.2, 0.3, 0.4), 1.0, 3, 0, 128256, "bf16", "gumbel_zipf", rho=0.85),
+    _ens("ens1", 1, (1.0,), 0.9, 4, 3, 12000, "bf16", sigma=2.5, rho=0.7),
+    _ens("ens5", 5, (0.3, 0.25, 0.2, 0.15, 0.1), 0.8, 4, 3, 16008, "bf16", sigma=2.5, rho=0.7),
+    _ens("ens8_f32", 8, (0.125,) * 8, 0.6, 3, 2, 6004, "f32", sigma=2.5, rho=0.7),
+]
+
+
+@pytest.mark.parametrize("w", ENSEMBLE_N, ids=[w.name for w in ENSEMBLE_N])
+def test_ensembles_of_every_size(w):
+    inputs = synth.make_inputs(w, "cuda")
+    ref = helpers.run_oracle(w, inputs)
+    v = helpers.make_verifier(w)
+    try:
+        assert v.info()["launches_per_run"] == (2 if 2 <= w.n <= 4 else 3)
+        plain = helpers.run_gpu(w, inputs, verifier=v, diag=True)
+        stats = helpers.check_parity(w, plain, ref)
+        assert stats["excused_accept"] + stats["excused_sample"] <= 1, stats
+        again = helpers.run_gpu(w, inputs, verifier=v)                   # the scratch was left clean
+        hooked = helpers.run_gpu(w, inputs, verifier=v, flags=COS_RUN_ALL_RESIDUALS)   # stages 0, 1 and 2
+        for k in ("accept_count", "out_tokens", "row_status"):
+            assert np.array_equal(plain[k], again[k]), k
+            assert np.array_equal(plain[k], hooked[k]), k
+        for m in sorted({0, w.n - 1}):                                   # bonus token from a named model
+            refm = helpers.run_oracle(w, inputs, bonus_model=m)
+            gpum = helpers.run_gpu(w, inputs, verifier=v, diag=True, bonus_model=m)
+            statm = helpers.check_parity(w, gpum, refm)
+            assert statm["excused_accept"] + statm["excused_sample"] <= 1, statm
+    finally:
+        v.close()
+
+
+def test_ensemble_channel_stage_with_identical_models_and_missing_tokens():
+    """Four models: tokens that some models exclude (-inf), a non-finite logit, and a row on which every model is
+    the same.  There r == q in exact arithmetic and the residual is empty; with more than two models the oracle's
+    r - q is rounding noise (about 1e-17) rather than zero, so that row is checked by what must hold: no residual
+    mass to speak of, a token out of the vocabulary all the same, and the status bits that say so."""
+    w = _ens("ens4_edges", 4, (0.5, 0.25, 0.125, 0.125), 0.7, 6, 3, 8200, "bf16", sigma=2.5, rho=0.7)
+    inputs = synth.make_inputs(w, "cuda")
+    logits, drafts = inputs["logits"].clone(), inputs["drafts"].clone()
+    logits[1:, 0] = logits[0, 0]                 # row 0: every model equals the first
+    drafts[0, 0] = w.vocab + 1                   # ... and its first draft is bad: a token is forced out of an empty residual
+    logits[2, 1, :, 100:900] = float("-inf")     # model 2 excludes a range of tokens on row 1
+    logits[0, 2, 1, 7] = float("-inf")
+    logits[3, 3, 0, 11] = float("nan")           # model 3, row 3, first position
+    mod = dict(inputs, logits=logits, drafts=drafts)
+    ref = helpers.run_oracle(w, mod)
+    gpu = helpers.run_gpu(w, mod, diag=True)
+    helpers.check_parity(w, gpu, ref, rows=range(1, w.batch))
+    assert ref["S"][0, 0] < 1e-15 and gpu["diag"][0, 0, 3] < 1e-15
+    assert gpu["accept_count"][0] == 0 and 0 <= gpu["out_tokens"][0, 0] < w.vocab
+    assert gpu["row_status"][0] & COS_ROW_BAD_DRAFT
+    assert gpu["row_status"][3] & COS_ROW_NONFINITE
 
 
 # Both forms of the streaming stage at small sizes: cluster_size 1 runs it without block barriers (one block
