@@ -245,6 +245,8 @@ def kernel_names(w, info):
     names = ["cos_verify_kernel stage 0 (every position: sweep, accept tests, row scan)"]
     if info["launches_per_run"] == 2 and info.get("draw_items"):
         names.append("cos_fused_kernel, drawing items only (token draw, one sweep)")
+    elif info["launches_per_run"] == 2 and w.combine == synth.COMBINE_PROB_ENSEMBLE and w.n > 2:
+        names.append("cos_verify_kernel stage 4 (token draw, one sweep, a channel per model)")
     elif info["launches_per_run"] == 2:
         names.append("cos_verify_kernel stage 3 (token draw, one sweep)")
     elif info["launches_per_run"] == 3:
