@@ -58,6 +58,7 @@ struct KParams {
   int greedy;       // T = 0: no drawing stages; the fourth word of a unit's result carries the bonus probability
   int bonus_model;  // >= 0: the token after gamma acceptances follows this model's own distribution; -1: the combined one
   int parts;     // blocks that share one unit in stages 1 and 2
+  int early_dependents;  // stage 0: let the next launch in the stream take places while this one runs
   int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
   double w64[COS_MAX_MODELS];

@@ -1414,9 +1414,16 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   const Slice sl = slice_of<DT>(rank, C, p.V, vec_ok);
 
   const int cluster_id = (STAGE == 0) ? blockIdx.x / C : blockIdx.x / lparts;
-  // later stages are launched while the previous one drains (programmatic dependent launch);
-  // nothing it wrote is read before this point
-  if (STAGE >= 1) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Every stage is launched while the kernel before it in the stream drains (programmatic dependent launch): its
+  // blocks take their places as that kernel's blocks leave and wait here until it is complete and its writes are
+  // visible.  Nothing is read or written before this point.  (Without the launch attribute, and behind a kernel
+  // that never signals, this is the ordinary order of a stream.)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // The streaming stage of a large run and stage 1 let the next launch take places from the start (all their
+  // blocks are resident or done by the time every one of them has said so; runs of a few blocks were slower with
+  // the drawing stage's blocks waiting beside them); the drawing stages say so after their sweep, when most of
+  // their blocks are about to leave and one per row goes on alone.
+  if (STAGE == 1 || (STAGE == 0 && p.early_dependents)) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (kOneSweep) SPROF(0);
   if ((STAGE == 1 || kOneSweep) && blockIdx.x == 0 && tid == 0) *p.work_counter = 0u;  // stage 0 is over: ready for the next run
   const int job_stride = gridDim.x / lparts;
@@ -1784,6 +1791,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           one_sweep_pair<DT, MODE>(p, sh, ring, base, b, rank, lparts, pis, masked, thr, is_bonus, draw_q, emit, vec_ok, kc);
         }
         __syncthreads();
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
         SPROF(2);
         if (warp < NCH) {
           float ref = (lane < kWarps) ? sh.wsoft[lane][warp].ref : -INFINITY;
@@ -2955,7 +2963,8 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
   if (dense) p.num_clusters = p.num_units < ctx->dense_blocks ? p.num_units : ctx->dense_blocks;
   ctx->scratch_dirty = true;  // cleared below once the launches are known to be queued
   if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
-  e = launch_stage(c.dtype, mode, 0, p, c0, stream, false, dense);
+  p.early_dependents = (c0 == 1 && p.num_units >= ctx->sm_count) ? 1 : 0;
+  e = launch_stage(c.dtype, mode, 0, p, c0, stream, p.early_dependents != 0, dense);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
   ctx->ev_used = 2;

@@ -322,3 +322,40 @@ def test_a_run_can_be_captured_in_a_graph_and_replayed(name, kw):
     finally:
         v.close()
         ref_v.close()
+
+
+@pytest.mark.parametrize("name,kw", [("cfg3", dict(batch=40, vocab=20008, gamma=8)), ("cfg4", dict(batch=30, vocab=12808, gamma=5)),
+                                     ("cfg5", dict(batch=36, vocab=16000, gamma=4)), ("cfg5_greedy", dict(batch=36, vocab=16000, gamma=4)),
+                                     ("cfg2", dict(batch=8, vocab=9001, gamma=5))])
+def test_calls_queued_back_to_back_give_what_isolated_calls_give(name, kw):
+    """Every launch of a run may take its places on the device while the kernel before it in the stream drains,
+    and waits for that kernel before it reads or writes anything.  Sixteen calls queued without a pause, on
+    logits that a kernel queued just before each call writes, into output buffers of their own, must give what
+    the same calls give one by one with a synchronisation in between."""
+    w = C[name].scaled(**kw)
+    inputs = synth.make_inputs(w, "cuda")
+    B, P = w.batch, w.gamma + 1
+    v = helpers.make_verifier(w)
+    try:
+        variants = [torch.roll(inputs["logits"], shifts=7 * k, dims=-1) for k in range(4)]
+        drafts = [((inputs["drafts"] + 7 * k) % w.vocab).to(torch.int32) for k in range(4)]   # rolled with the logits
+        live = torch.empty_like(inputs["logits"])
+        queued = []
+        for k in range(16):
+            outs = v._alloc_outs(B, P, w.vocab, torch.device("cuda"), True, False)
+            live.copy_(variants[k % 4])                      # a kernel in the same stream produces the logits
+            v.run(live, drafts[k % 4], inputs["proposer"], inputs["seed"], 100 + k, outs=outs)
+            queued.append(outs)
+        torch.cuda.synchronize()
+        for k in range(16):
+            want = v.run(variants[k % 4], drafts[k % 4], inputs["proposer"], inputs["seed"], 100 + k, diag=True)
+            torch.cuda.synchronize()
+            for key in ("accept_count", "out_tokens", "row_status"):
+                assert torch.equal(queued[k][key], want[key]), (k, key)
+            assert torch.equal(torch.nan_to_num(queued[k]["diag"], nan=-7.0), torch.nan_to_num(want["diag"], nan=-7.0)), k
+        # and one of them against the oracle
+        ref = helpers.run_oracle(w, dict(inputs, logits=variants[1], drafts=drafts[1], offset=101), native=True)
+        got = {key: t.cpu().numpy() for key, t in queued[1].items()}
+        helpers.check_parity(w, got, ref)
+    finally:
+        v.close()
