@@ -73,12 +73,26 @@ enum {
                                      /* `bonus_model`'s own distribution instead of the combined one     */
                                      /* (Sec. 3.3: the verifier's bonus token, to be treated as that     */
                                      /* model's next proposal)                                           */
-  COS_RUN_EARLY_EXIT = 8             /* a hint: positions behind a rejection that their row has already  */
+  COS_RUN_EARLY_EXIT = 8,            /* a hint: positions behind a rejection that their row has already  */
                                      /* reported may be left unread (Sec. 3.1 discards them anyway).     */
                                      /* accept_count, out_tokens, row_status and bonus_prob are those of */
                                      /* the full run; diag is NaN at a position that was left unread,    */
                                      /* and which positions those are depends on timing.  Taken by       */
                                      /* cos_verify_run when no cluster size and no mask is configured.   */
+  COS_RUN_INPUTS_SETTLED = 16        /* a promise by the caller: logits, draft_tokens and proposer were  */
+                                     /* complete in device memory before the work that precedes this     */
+                                     /* call in its stream was submitted (they are not written by the    */
+                                     /* kernel queued just before the call).  The streaming launch may   */
+                                     /* then read them while that work drains - the drawing launch of    */
+                                     /* the previous call, for one - and waits for it only before it     */
+                                     /* touches anything else; calls queued back to back overlap.        */
+                                     /* Outputs and results are those of an ordinary run.  Without the   */
+                                     /* flag a run reads nothing before the work ahead of it in the      */
+                                     /* stream is complete.  Taken by cos_verify_run at T > 0 for runs   */
+                                     /* of at least one position per multiprocessor whose drawing launch */
+                                     /* is a single wave of blocks, without cluster size, mask, test     */
+                                     /* hook or COS_RUN_EARLY_EXIT; ignored otherwise (cos_verify_get_   */
+                                     /* info does not tell).                                             */
 };
 
 typedef struct {

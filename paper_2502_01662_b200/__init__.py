@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     COS_RUN_ALL_RESIDUALS,
     COS_RUN_BONUS_FROM_MODEL,
     COS_RUN_EARLY_EXIT,
+    COS_RUN_INPUTS_SETTLED,
     COS_RUN_PROPOSER_PER_POSITION,
     CosVerifier,
     CosVerifyError,

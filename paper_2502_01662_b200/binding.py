@@ -26,6 +26,7 @@ COS_RUN_ALL_RESIDUALS = 1
 COS_RUN_PROPOSER_PER_POSITION = 2   # proposer is [B, gamma+1]: the model that proposed each draft (Algorithm 2)
 COS_RUN_BONUS_FROM_MODEL = 4        # the bonus token follows one named model's own distribution (Sec. 3.3)
 COS_RUN_EARLY_EXIT = 8              # hint: positions behind a reported rejection may be left unread
+COS_RUN_INPUTS_SETTLED = 16         # promise: the inputs were complete before the work ahead of the call in its stream was submitted
 
 _STATUS_NAMES = {1: "COS_ERR_INVALID_ARG", 2: "COS_ERR_UNSUPPORTED", 3: "COS_ERR_ALIGNMENT",
                  4: "COS_ERR_CUDA", 5: "COS_ERR_NOMEM"}

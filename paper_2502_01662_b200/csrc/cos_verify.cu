@@ -1237,12 +1237,17 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
     fr.fault = 0;
   }
   __syncthreads();
-  if (tid == kThreads - 32) {  // the block's first unit is valid: one draw settles its second
+  // The inputs may be read before the kernel ahead in the stream is complete (the caller's promise): every warp then
+  // sweeps the block's first unit, which is the block's own by its index, and only then waits for that kernel;
+  // nothing but the inputs is touched before.  (The hint to leave positions unread is not taken together with it.)
+  const bool settled = p.inputs_settled != 0;
+  auto first_draw = [&]() {  // the block's first unit is valid: one draw settles its second
     const int nx = p.num_clusters + static_cast<int>(atomicAdd(p.work_counter, 1u));
     unit_of[1] = nx;
     __threadfence_block();
     unit_tag[1] = 2;
-  }
+  };
+  if (!settled && tid == kThreads - 32) first_draw();
   for (int seq = 0;; ++seq) {
     const int par = seq & 1;
     if (!wait_reach(&unit_tag[seq & 3], seq + 1, fault, lane)) {
@@ -1278,6 +1283,10 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
     }
     if (!skipped)
       sweep_unit<DT, MODE>(p, base, sl, pis, false, -INFINITY, &fr.wsoft[par][warp][0], &fr.warg[par][warp][0]);
+    if (settled && seq == 0) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");  // from here on as in an ordinary run
+      if (tid == kThreads - 32) first_draw();
+    }
     int prev = 0;
     if (lane == 0) {
       __threadfence_block();
@@ -1418,7 +1427,9 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
   // blocks take their places as that kernel's blocks leave and wait here until it is complete and its writes are
   // visible.  Nothing is read or written before this point.  (Without the launch attribute, and behind a kernel
   // that never signals, this is the ordinary order of a stream.)
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // (With COS_RUN_INPUTS_SETTLED the barrier-free streaming stage reads its inputs first and waits after the sweep
+  // of its first position: see stage0_free_running.)
+  if (!(STAGE == 0 && p.inputs_settled)) asm volatile("griddepcontrol.wait;" ::: "memory");
   // The streaming stage of a large run and stage 1 let the next launch take places from the start (all their
   // blocks are resident or done by the time every one of them has said so; runs of a few blocks were slower with
   // the drawing stage's blocks waiting beside them); the drawing stages say so after their sweep, when most of
@@ -2569,10 +2580,13 @@ int choose_parts(const cos_verify_config& c, int rows, int sm_count) {
 // free: one wave of whole units leaves some multiprocessors with twice the work of others.  Small units
 // stay at one wave: their blocks are bound by latency, not by throughput.
 int choose_parts_one(const cos_verify_config& c, int rows, int sm_count) {
-  const long long slots = (one_sweep_stage(c) == 4 ? 1LL : 2LL) * sm_count;  // blocks the device holds at once
+  const bool channels = (one_sweep_stage(c) == 4);
+  const long long slots = (channels ? 1LL : 2LL) * sm_count;  // blocks the device holds at once
   const int E = entries_per_vec(c.dtype);
   const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
-  int parts = choose_parts(c, rows, sm_count);
+  // (the stage with a channel per model, one block per multiprocessor: blocks on half of the multiprocessors
+  // were faster than blocks on all of them: workload 4 went from 96.1 to 90.1 us per call with 64 instead of 128)
+  int parts = choose_parts(c, rows, channels ? sm_count / 2 : sm_count);
   while (parts < 8 && static_cast<long long>(rows) * parts < 3 * slots && nsteps / (2 * parts * kWarps) >= 8) parts <<= 1;
   return parts;
 }
@@ -2883,7 +2897,8 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
   if (!a->logits || !a->proposer || !a->accept_count || !a->out_tokens || !a->row_status) return bad("null device pointer");
   if (c.gamma > 0 && !a->draft_tokens) return bad("draft_tokens is null although gamma > 0");
   if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return bad("negative stride");
-  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL | COS_RUN_EARLY_EXIT)) return bad("unknown flag bits");
+  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL | COS_RUN_EARLY_EXIT |
+                   COS_RUN_INPUTS_SETTLED)) return bad("unknown flag bits");
   if ((a->flags & COS_RUN_BONUS_FROM_MODEL) && (a->bonus_model < 0 || a->bonus_model >= c.n))
     return bad("bonus_model outside [0, n)");
   if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4) {
@@ -2964,6 +2979,18 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
   ctx->scratch_dirty = true;  // cleared below once the launches are known to be queued
   if (ctx->timing) cudaEventRecord(ctx->ev[0], stream);
   p.early_dependents = (c0 == 1 && p.num_units >= ctx->sm_count) ? 1 : 0;
+  {
+    const bool masked = (c.combine != COS_COMBINE_PROB_ENSEMBLE) && c.mask_model >= 0;
+    const bool hooks = (a->dump_r != nullptr) || (a->flags & COS_RUN_ALL_RESIDUALS);
+    // what it overlaps with is the end of the previous call's drawing stage, where one block per row goes on alone;
+    // a drawing stage of several waves of blocks leaves nothing to fill (workload 5 was 12 us slower with it), and
+    // greedy runs have no drawing stage
+    const int sweep_stage = one_sweep_stage(c);
+    const long long slots = (sweep_stage == 4 ? 1LL : 2LL) * ctx->sm_count;
+    const bool one_wave = draws && sweep_stage != 0 && static_cast<long long>(a->batch) * ctx->parts_one <= slots;
+    p.inputs_settled =
+        ((a->flags & COS_RUN_INPUTS_SETTLED) && p.early_dependents && one_wave && !masked && !hooks && !p.early_exit) ? 1 : 0;
+  }
   e = launch_stage(c.dtype, mode, 0, p, c0, stream, p.early_dependents != 0, dense);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
@@ -3076,6 +3103,7 @@ extern "C" cos_status cos_verify_run_host(cos_verify_ctx* ctx, const cos_verify_
   if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_proposer, a->proposer, nprop * sizeof(int), cudaMemcpyHostToDevice, stream);
   if (e != cudaSuccess) return cuda_fail(ctx, "host to device copy", e);
   cos_verify_args d = *a;
+  d.flags &= ~COS_RUN_INPUTS_SETTLED;  // the inputs are what the copies above have just written
   d.logits = ctx->d_logits;
   d.draft_tokens = ctx->d_drafts;
   d.proposer = ctx->d_proposer;
@@ -3254,7 +3282,8 @@ extern "C" cos_status cos_verify_run_static(const cos_verify_config* config, con
     return static_fail(COS_ERR_INVALID_ARG, "null device pointer");
   if (c.gamma > 0 && !a->draft_tokens) return static_fail(COS_ERR_INVALID_ARG, "draft_tokens is null although gamma > 0");
   if (a->stride_model < 0 || a->stride_row < 0 || a->stride_pos < 0) return static_fail(COS_ERR_INVALID_ARG, "negative stride");
-  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL | COS_RUN_EARLY_EXIT)) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
+  if (a->flags & ~(COS_RUN_ALL_RESIDUALS | COS_RUN_PROPOSER_PER_POSITION | COS_RUN_BONUS_FROM_MODEL | COS_RUN_EARLY_EXIT |
+                   COS_RUN_INPUTS_SETTLED)) return static_fail(COS_ERR_INVALID_ARG, "unknown flag bits");
   if ((a->flags & COS_RUN_BONUS_FROM_MODEL) && (a->bonus_model < 0 || a->bonus_model >= c.n))
     return static_fail(COS_ERR_INVALID_ARG, "bonus_model outside [0, n)");
   if (a->bonus_prob && reinterpret_cast<uintptr_t>(a->bonus_prob) % 4)

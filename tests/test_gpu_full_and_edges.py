@@ -5,7 +5,7 @@ import torch
 
 import helpers
 from paper_2502_01662_b200 import (COS_ROW_BAD_DRAFT, COS_ROW_NONFINITE, COS_ROW_Q_ZERO, COS_ROW_RESIDUAL_EMPTY,
-                                   COS_RUN_ALL_RESIDUALS, CosVerifier, CosVerifyError, synth)
+                                   COS_RUN_ALL_RESIDUALS, COS_RUN_INPUTS_SETTLED, CosVerifier, CosVerifyError, synth)
 from oracle import cos_oracle as orc
 
 pytestmark = pytest.mark.gpu
@@ -327,11 +327,14 @@ def test_a_run_can_be_captured_in_a_graph_and_replayed(name, kw):
 @pytest.mark.parametrize("name,kw", [("cfg3", dict(batch=40, vocab=20008, gamma=8)), ("cfg4", dict(batch=30, vocab=12808, gamma=5)),
                                      ("cfg5", dict(batch=36, vocab=16000, gamma=4)), ("cfg5_greedy", dict(batch=36, vocab=16000, gamma=4)),
                                      ("cfg2", dict(batch=8, vocab=9001, gamma=5))])
-def test_calls_queued_back_to_back_give_what_isolated_calls_give(name, kw):
+@pytest.mark.parametrize("settled", [False, True])
+def test_calls_queued_back_to_back_give_what_isolated_calls_give(name, kw, settled):
     """Every launch of a run may take its places on the device while the kernel before it in the stream drains,
     and waits for that kernel before it reads or writes anything.  Sixteen calls queued without a pause, on
     logits that a kernel queued just before each call writes, into output buffers of their own, must give what
-    the same calls give one by one with a synchronisation in between."""
+    the same calls give one by one with a synchronisation in between.  With COS_RUN_INPUTS_SETTLED (inputs that
+    were complete long before: no producer kernel) the streaming launch reads them while the previous call's
+    drawing launch drains, and the results are the same again."""
     w = C[name].scaled(**kw)
     inputs = synth.make_inputs(w, "cuda")
     B, P = w.batch, w.gamma + 1
@@ -343,8 +346,12 @@ def test_calls_queued_back_to_back_give_what_isolated_calls_give(name, kw):
         queued = []
         for k in range(16):
             outs = v._alloc_outs(B, P, w.vocab, torch.device("cuda"), True, False)
-            live.copy_(variants[k % 4])                      # a kernel in the same stream produces the logits
-            v.run(live, drafts[k % 4], inputs["proposer"], inputs["seed"], 100 + k, outs=outs)
+            if settled:
+                v.run(variants[k % 4], drafts[k % 4], inputs["proposer"], inputs["seed"], 100 + k, outs=outs,
+                      flags=COS_RUN_INPUTS_SETTLED)
+            else:
+                live.copy_(variants[k % 4])                  # a kernel in the same stream produces the logits
+                v.run(live, drafts[k % 4], inputs["proposer"], inputs["seed"], 100 + k, outs=outs)
             queued.append(outs)
         torch.cuda.synchronize()
         for k in range(16):
