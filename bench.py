@@ -26,7 +26,7 @@ import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 from paper_2502_01662_b200 import synth  # noqa: E402
-from paper_2502_01662_b200.binding import COS_RUN_EARLY_EXIT  # noqa: E402,F401
+from paper_2502_01662_b200.binding import COS_RUN_EARLY_EXIT, COS_RUN_INPUTS_SETTLED  # noqa: E402,F401
 
 HEADLINE = "cfg3"
 # dram read + write bytes of one launch of the dominant kernel, as RECORDED in the ncu capture summarised under
@@ -120,13 +120,21 @@ def time_device(w, verifier, sets, steps, warmup, row_base, sampler=None, flags=
         s = sets[k % len(sets)]
         verifier.run(s["logits"], s["drafts"], s["proposer"], s["seed"], s["offset"] + k, row_base=row_base, outs=outs,
                      flags=flags)
+    if sampler:
+        # nvidia-smi takes a third of a second to start; the device is kept busy afterwards for 50 ms before the
+        # warm-up steps, so that the timed region does not begin on a device that has just sat idle
+        sampler.__enter__()
+        t_busy = time.perf_counter()
+        k = 0
+        while time.perf_counter() - t_busy < 0.05:
+            step(k)
+            k += 1
+            if k % 64 == 0:
+                torch.cuda.synchronize(dev)
     for k in range(warmup):
         step(k)
     torch.cuda.synchronize(dev)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if sampler:
-        sampler.__enter__()
-    # a long enough region for the clock sampler to see the load
     start.record()
     for k in range(steps):
         step(warmup + k)
@@ -265,6 +273,20 @@ def measure_workload(w, dev, local, steps, warmup, row_base=0, sampler=None, clu
         verifier.set_one_launch(True)
     info = verifier.info()
     elapsed, outs = time_device(w, verifier, sets, steps, warmup, row_base, sampler)
+    # the same calls with the promise that the inputs were complete before the timed region (they were): the
+    # streaming launch of a call then overlaps the end of the previous call's drawing launch
+    settled_steps = max(20, steps // 4)
+    t_settled, _ = time_device(w, verifier, sets, settled_steps, 5, row_base, flags=COS_RUN_INPUTS_SETTLED)
+    def one_call(flags):
+        o = verifier._alloc_outs(w.batch, w.gamma + 1, w.vocab, dev, False, False)
+        s0 = sets[0]
+        for _ in range(2):          # the second of two calls in a row is the one that overlaps
+            verifier.run(s0["logits"], s0["drafts"], s0["proposer"], s0["seed"], s0["offset"] + 4242, row_base=row_base,
+                         outs=o, flags=flags)
+        torch.cuda.synchronize(dev)
+        return o
+    o_plain, o_settled = one_call(0), one_call(COS_RUN_INPUTS_SETTLED)
+    same = all(torch.equal(o_plain[k], o_settled[k]) for k in ("accept_count", "out_tokens", "row_status"))
     verifier.set_stage_timing(True)
     acc = None
     touts = verifier._alloc_outs(w.batch, w.gamma + 1, w.vocab, dev, False, False)
@@ -301,7 +323,12 @@ def measure_workload(w, dev, local, steps, warmup, row_base=0, sampler=None, clu
     res = {"us_per_call": 1e6 * per_call, "positions_per_s": w.positions / per_call, "GBps": nbytes / per_call / 1e9,
            "frac": nbytes / per_call / 1e9 / peak, "frac_of_nominal_8TBps": nbytes / per_call / 1e9 / NOMINAL_HBM_GBS,
            "bytes_per_call": nbytes, "launches_per_call": info["launches_per_run"], "stages": stages,
-           "buffers": len(sets), "one_launch": info["one_launch"]}
+           "buffers": len(sets), "one_launch": info["one_launch"],
+           "inputs_settled": {"us_per_call": 1e6 * t_settled / settled_steps,
+                              "frac": nbytes / (t_settled / settled_steps) / 1e9 / peak,
+                              "what": "the same calls with COS_RUN_INPUTS_SETTLED: a call's streaming launch may read "
+                                      "its inputs while the previous call's drawing launch drains"}}
+    res["inputs_settled"]["same_rows_as_ordinary_calls"] = bool(same)
     if one_launch_us is not None:
         res["us_per_call_one_launch_form"] = one_launch_us   # the opt-in single-kernel form of the same run
         res["us_per_call_persistent_drawing_launch"] = drawing_launch_us   # staged streaming + the persistent kernel's drawing items
@@ -469,6 +496,7 @@ def main():
         "config": {"workload": w.name, "n": w.n, "combine": "prob_ensemble" if w.combine == 0 else "logit_linear",
                    "T": w.temperature, "B": w.batch, "gamma": w.gamma, "V": w.vocab, "logits": w.dtype,
                    "l2": "inputs larger than L2" if n_sets == 1 else f"rotating over {n_sets} input copies",
+                   "before_warmup": "clock sampler started, then 50 ms of untimed calls, then the W warm-up steps",
                    "cluster_size": info["cluster_size"], "resident_clusters": info["max_clusters"],
                    "one_launch": info["one_launch"], "items_per_position": info["items_per_position"],
                    "mean_accept_count": mean_accept},
@@ -476,7 +504,10 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": TRAFFIC_BYTES.get(dominant), "peak_kind": peak_kind, "bytes_per_launch": bytes_per_call,
                      "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS, "kernel": head["stages"][0]["kernel"],
-                     "launches_per_call": head["launches_per_call"], "stages": head["stages"]},
+                     "launches_per_call": head["launches_per_call"], "stages": head["stages"],
+                     # not the headline: the same calls under the caller's promise that their inputs were complete
+                     # earlier (true of this loop), which lets consecutive calls overlap
+                     "inputs_settled": head.get("inputs_settled")},
         "gpu_launches": args.steps * info["launches_per_run"],
         "clocks": sampler.summary() if sampler else None,
     }
