@@ -229,8 +229,9 @@ int choose_parts_one(const cos_verify_config& c, int rows, int sm_count) {
   const long long slots = (channels ? 1LL : 2LL) * sm_count;  // blocks the device holds at once
   const int E = entries_per_vec(c.dtype);
   const int nsteps = (c.vocab + 32 * E - 1) / (32 * E);
-  // (the stage with a channel per model, one block per multiprocessor: blocks on half of the multiprocessors
-  // were faster than blocks on all of them: workload 4 went from 96.1 to 90.1 us per call with 64 instead of 128)
+  // (choose_parts counts two blocks per multiprocessor; the stage with a channel per model holds one, so it is
+  // asked for half the device: one wave of blocks instead of two.  Workload 4: 96.1 -> 90.1 us per call with 128
+  // blocks instead of 256; 64 blocks: 104.8 us)
   int parts = choose_parts(c, rows, channels ? sm_count / 2 : sm_count);
   while (parts < 8 && static_cast<long long>(rows) * parts < 3 * slots && nsteps / (2 * parts * kWarps) >= 8) parts <<= 1;
   return parts;
