@@ -21,8 +21,18 @@ __device__ unsigned long long g_sprof[kSprofBlocks * 8];
       g_sprof[blockIdx.x * 8 + (k)] = t_;                                                         \
     }                                                                                             \
   } while (0)
+// (the same by lane 0 of whichever warp gets there: the barrier-free streaming stage)
+#define SPROFL(k)                                                                                 \
+  do {                                                                                            \
+    if ((threadIdx.x & 31) == 0 && blockIdx.x < kSprofBlocks) {                                   \
+      unsigned long long t_;                                                                      \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                                       \
+      g_sprof[blockIdx.x * 8 + (k)] = t_;                                                         \
+    }                                                                                             \
+  } while (0)
 #else
 #define SPROF(k)
+#define SPROFL(k)
 #endif
 
 struct Xchg {  // one per block and barrier parity; peers read it through DSMEM

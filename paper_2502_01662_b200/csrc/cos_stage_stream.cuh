@@ -409,6 +409,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
     unit_tag[1] = 2;
   };
   if (!settled && tid == kThreads - 32) first_draw();
+  if (warp == 0) SPROFL(0);
   for (int seq = 0;; ++seq) {
     const int par = seq & 1;
     if (!wait_reach(&unit_tag[seq & 3], seq + 1, fault, lane)) {
@@ -484,6 +485,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       __syncwarp();
     } else if (prev == kWarps - 1) {
       // last to finish: merge, decide, publish
+      SPROFL(1);
       const int uidx = b * p.P + j;
       const bool is_bonus = (j == p.gamma);
       const int draft = is_bonus ? 0 : p.drafts[b * p.gamma + j];
@@ -526,8 +528,10 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
                           sh.fsoft[lane].s;
       }
       __syncwarp();
+      SPROFL(2);
       if (lane == 0) decide_unit<DT, MODE>(p, sh, is_bonus, draft, draft_ok, pi, pi_ok, pis, false);
       __syncwarp();
+      SPROFL(3);
       if (kSample && lane < nsoft) {  // kept for the drawing stages
         p.ustats[uidx].s[lane] = sh.fsoft[lane].s;
         p.ustats[uidx].ref[lane] = sh.fsoft[lane].ref;
@@ -543,6 +547,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
         *epi_done = seq + 1;
       }
       __syncwarp();
+      SPROFL(4);
     }
   }
   // the last warp of the block to run out of units reports the block's departure
