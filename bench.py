@@ -369,6 +369,16 @@ def sustained_small_calls(w, dev, local, calls=256, contexts=8):
             "GBps_sustained": nbytes / sec / 1e9, "contexts": contexts, "calls": calls, "buffers": len(sets)}
 
 
+def three_streams(w, dev, local):
+    """Independent calls of a workload dealt out over three contexts and streams: while one call's drawing launch
+    finishes with one block per row, another call's streaming launch has the rest of the device."""
+    peak, _ = measured_peak()
+    r = sustained_small_calls(w, dev, local, calls=120 if w.positions * w.bytes_per_position < (1 << 30) else 45, contexts=3)
+    return {"us_per_call": r["us_per_call_sustained"], "positions_per_s": r["positions_per_s_sustained"],
+            "GBps": r["GBps_sustained"], "frac": r["GBps_sustained"] / peak, "contexts": 3, "calls": r["calls"],
+            "what": "independent calls on three contexts and streams, between two events on the stream they fork from"}
+
+
 def ceilings(dev):
     """Read-only and read-plus-exponential streaming ceilings of this device (library micro-kernels)."""
     from paper_2502_01662_b200.binding import measure_ceiling
@@ -468,6 +478,7 @@ def main():
             torch.cuda.empty_cache()
             if name == w.name:
                 table[name] = {k: v for k, v in head.items()}
+                table[name]["three_streams"] = three_streams(ww, dev, local)
                 continue
             k2 = 400 if ww.positions * ww.bytes_per_position < (1 << 30) else 100
             res, _, _, inf2, s2 = measure_workload(ww, dev, local, k2, 5, stage_runs=20, try_one_launch=True)
@@ -475,6 +486,7 @@ def main():
             extra_launches += (k2 + 5 + 25) * inf2["launches_per_run"]
             if name == "cfg2":
                 res.update(sustained_small_calls(ww, dev, local))
+            res["three_streams"] = three_streams(ww, dev, local)
             table[name] = res
         torch.cuda.empty_cache()
         ceil = ceilings(dev)
@@ -507,7 +519,10 @@ def main():
                      "launches_per_call": head["launches_per_call"], "stages": head["stages"],
                      # not the headline: the same calls under the caller's promise that their inputs were complete
                      # earlier (true of this loop), which lets consecutive calls overlap
-                     "inputs_settled": head.get("inputs_settled")},
+                     "inputs_settled": head.get("inputs_settled"),
+                     # not the headline either: independent calls on three contexts and streams overlap one call's
+                     # drawing launch with another's streaming launch
+                     "three_streams": (table or {}).get(w.name, {}).get("three_streams")},
         "gpu_launches": args.steps * info["launches_per_run"],
         "clocks": sampler.summary() if sampler else None,
     }
