@@ -32,6 +32,18 @@ def test_full_size_workloads(name, nrows):
     again = helpers.run_gpu(w, inputs, diag=True)
     for k in ("accept_count", "out_tokens", "row_status"):
         assert np.array_equal(gpu[k], again[k]), k
+    # four calls queued without a pause on inputs that were complete long before (COS_RUN_INPUTS_SETTLED: a call's
+    # streaming launch overlaps the end of the previous call's drawing launch): every one gives the same rows
+    v = helpers.make_verifier(w)
+    try:
+        queued = [v.run(inputs["logits"], inputs["drafts"], inputs["proposer"], inputs["seed"], inputs["offset"],
+                        flags=COS_RUN_INPUTS_SETTLED) for _ in range(4)]
+        torch.cuda.synchronize()
+        for outs in queued:
+            for k in ("accept_count", "out_tokens", "row_status"):
+                assert np.array_equal(gpu[k], outs[k].cpu().numpy()), k
+    finally:
+        v.close()
     del inputs
     torch.cuda.empty_cache()
 
