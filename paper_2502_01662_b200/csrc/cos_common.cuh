@@ -60,6 +60,7 @@ struct KParams {
   int parts;     // blocks that share one unit in stages 1 and 2
   int early_dependents;  // stage 0: let the next launch in the stream take places while this one runs
   int inputs_settled;    // stage 0, barrier-free form: the inputs may be read before the kernel ahead in the stream is complete
+  int draw_cluster;      // one-sweep drawing stages: the blocks of a unit are a thread-block cluster and meet at its barrier
   int max_jobs;  // capacity of the job list
   float w[COS_MAX_MODELS];
   double w64[COS_MAX_MODELS];

@@ -432,6 +432,12 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
           SoftPart o = warp_reduce_soft(ref, sum);
           if (lane == 0) p.zpart[(static_cast<size_t>(uidx) * p.parts + rank) * 8 + warp] = o.s;
         }
+        if (p.draw_cluster) {
+          // the blocks of a unit are one thread-block cluster: its hardware barrier (release on arrival, acquire on
+          // leaving) makes the partial sums and step records of all of them visible, and the first block goes on
+          cluster.sync();
+          do_locate = (rank == 0) && emit;
+        } else {
         // the last block of the unit to get here completes the normalisers and locates the token
         __syncthreads();
         if (tid == 0) {
@@ -446,6 +452,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
         __syncthreads();
         do_locate = (sh.win_g != 0) && emit;  // (every unit listed for this stage is its row's drawing unit)
         __syncthreads();
+        }
         SPROF(3);
         if (do_locate) {
           if (tid < NCH) {
@@ -1002,7 +1009,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     if (STAGE >= 1) __syncthreads();
     unit = next_unit;
   }
-  cluster.sync();  // no block leaves while a peer may still read its shared memory
+  if (STAGE == 0) cluster.sync();  // no block leaves while a peer may still read its shared memory
   if (((STAGE == 0 && p.greedy) || STAGE >= 2) && tid == 0) stage_exit(p, STAGE == 0 ? 0 : 1);
 }
 

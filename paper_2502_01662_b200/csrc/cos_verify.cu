@@ -665,7 +665,17 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
     if (one_sweep) {
       p.parts = ctx->parts_one;
       p.num_clusters = (most < cap ? most : cap) * p.parts;
-      e = launch_stage(c.dtype, mode, sweep_stage, p, 1, stream, true);
+      int draw_cs = 1;
+      // the blocks of a unit as one cluster (portable sizes), where the launch is a single wave of blocks: with
+      // several waves the clusters wait for four free places at once (workload 5: +17 us per call), with one the
+      // barrier is cheaper than fence and counter (workloads 1 to 4: -1.4 to -1.7 us)
+      const long long draw_slots = (sweep_stage == 4 ? 1LL : 2LL) * ctx->sm_count;
+      if (p.parts > 1 && p.parts <= 8 && static_cast<long long>(most) * p.parts <= draw_slots) {
+        draw_cs = p.parts;
+        p.draw_cluster = 1;
+        p.num_clusters = (most < cap ? most : cap);
+      }
+      e = launch_stage(c.dtype, mode, sweep_stage, p, draw_cs, stream, true);
       if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (drawing stage)", e);
       if (ctx->timing) cudaEventRecord(ctx->ev[2], stream);
       ctx->ev_used = 3;
