@@ -156,9 +156,12 @@ typedef struct {
   int32_t threads_per_block;
   int32_t max_clusters;      /* clusters that can be resident at once on the device                   */
   int32_t sm_count;
-  int32_t launches_per_run;  /* kernels an ordinary cos_verify_run enqueues: 1 at T = 0 and wherever the  */
-                             /* one-launch form covers the configuration (reserved[2] == 1); else 2   */
-                             /* for logit-level combines and two-model ensembles, 3 otherwise         */
+  int32_t launches_per_run;  /* kernels an ordinary cos_verify_run enqueues: 1 at T = 0 and where the     */
+                             /* one-launch form was chosen (reserved[2] bit 0); else 2 for logit-level */
+                             /* combines and ensembles of two to four models, 3 otherwise.  Every      */
+                             /* launch takes its places on the device while the kernel before it in    */
+                             /* the stream drains, and reads or writes nothing until that kernel is    */
+                             /* complete (unless COS_RUN_INPUTS_SETTLED says the inputs may be read)   */
   int32_t reserved[3];       /* [0], [1]: work items per position when streaming / drawing; [2]: bit  */
                              /* 0: an ordinary run is one launch; bit 1: the tokens of a staged run   */
                              /* are drawn by the persistent kernel's drawing items                    */

@@ -34,3 +34,25 @@ def test_create_validates_before_touching_the_device():
             assert e.status == 1, (kw, e)
         else:
             raise AssertionError(f"accepted {kw}")
+
+
+def test_binding_constants_are_the_headers():
+    """Every COS_* enumerator of the header has the same value in the binding (flags, status codes, row bits)."""
+    from paper_2502_01662_b200 import binding
+    with open(os.path.join(ROOT, "include", "cos_verify.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    found = {}
+    for name, value in re.findall(r"\b(COS_[A-Z0-9_]+)\s*=\s*([^,}\n]+)", text):
+        value = value.strip()
+        m = re.fullmatch(r"(\d+)u?\s*<<\s*(\d+)", value)
+        found[name] = (int(m.group(1)) << int(m.group(2))) if m else int(value.rstrip("u"), 0)
+    assert len(found) >= 20, found
+    checked = 0
+    for name, value in found.items():
+        if hasattr(binding, name):
+            assert getattr(binding, name) == value, (name, getattr(binding, name), value)
+            checked += 1
+    for name in ("COS_RUN_ALL_RESIDUALS", "COS_RUN_PROPOSER_PER_POSITION", "COS_RUN_BONUS_FROM_MODEL", "COS_RUN_EARLY_EXIT",
+                 "COS_RUN_INPUTS_SETTLED", "COS_ROW_FAULT", "COS_ROW_NONFINITE"):
+        assert name in found and hasattr(binding, name), name
+    assert checked >= 12, checked
