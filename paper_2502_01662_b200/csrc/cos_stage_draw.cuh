@@ -354,11 +354,13 @@ __device__ __forceinline__ void one_sweep_pair(const KParams& p, Shared& sh, uin
       const float eB = ex2_approx(fmaf(xb[k], cT, nrefB));
       // k_A e_A / Z_A + k_B e_B / Z_B > 0 with the products rounded one by one: where r and q coincide
       // neither side exceeds the other, as in exact arithmetic
-      const float in_p = (__fmul_rn(ctB, eB) > __fmul_rn(nctA, eA)) ? 1.f : 0.f;
+      const bool in_p = __fmul_rn(ctB, eB) > __fmul_rn(nctA, eA);
       vzA += eA;
       vzB += eB;
-      vaA = fmaf(in_p, eA, vaA);
-      vaB = fmaf(in_p, eB, vaB);
+      if (in_p) {
+        vaA += eA;
+        vaB += eB;
+      }
     }
     // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum
     // big); the caller does the vector again, big entries in fp64
