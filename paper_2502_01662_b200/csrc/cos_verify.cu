@@ -637,7 +637,7 @@ cos_status run_launches(cos_verify_ctx* ctx, const cos_verify_args* a, void* cud
     p.inputs_settled =
         ((a->flags & COS_RUN_INPUTS_SETTLED) && p.early_dependents && one_wave && !masked && !hooks && !p.early_exit) ? 1 : 0;
   }
-  e = launch_stage(c.dtype, mode, 0, p, c0, stream, p.early_dependents != 0, dense);
+  e = launch_stage(c.dtype, mode, 0, p, c0, stream, true, dense);
   if (e != cudaSuccess) return cuda_fail(ctx, "kernel launch (stage 0)", e);
   if (ctx->timing) cudaEventRecord(ctx->ev[1], stream);
   ctx->ev_used = 2;
