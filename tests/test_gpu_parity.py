@@ -101,6 +101,8 @@ ENSEMBLE_N = [
     _ens("ens4_zipf_f16", 4, (0.4, 0.3, 0.2, 0.1), 0.7, 5, 4, 50000, "f16", "gumbel_zipf", rho=0.85),
     _ens("ens4_sharp_ragged", 4, (0.25, 0.25, 0.25, 0.25), 0.3, 4, 3, 9001, "bf16", sigma=2.5, rho=0.6),
     _ens("ens4_wide_gamma0", 4, (0.1, 0.2, 0.3, 0.4), 1.0, 3, 0, 128256, "bf16", "gumbel_zipf", rho=0.85),
+    # two rows of a wide vocabulary: sixteen blocks per row, more than a portable cluster holds (arrival counter)
+    _ens("ens4_wide_two_rows", 4, (0.4, 0.3, 0.2, 0.1), 0.8, 2, 2, 151936, "bf16", "gumbel_zipf", rho=0.85),
     _ens("ens1", 1, (1.0,), 0.9, 4, 3, 12000, "bf16", sigma=2.5, rho=0.7),
     _ens("ens5", 5, (0.3, 0.25, 0.2, 0.15, 0.1), 0.8, 4, 3, 16008, "bf16", sigma=2.5, rho=0.7),
     _ens("ens8_f32", 8, (0.125,) * 8, 0.6, 3, 2, 6004, "f32", sigma=2.5, rho=0.7),
