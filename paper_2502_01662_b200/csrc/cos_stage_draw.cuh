@@ -517,29 +517,22 @@ __device__ __forceinline__ void one_sweep_pair(const KParams& p, Shared& sh, uin
         if (eat(vq, cmb)) redo_from_memory(e0);
       }
     }
-    // the step's two sums over the warp
-    float ra = aA, rb = aB;
+    // the step's two sums over the warp: the lower half of the lanes ends up with the first, the upper half with the
+    // second (one exchange, then one sum per lane instead of two)
+    const bool upper = (lane & 16) != 0;
+    float mine = (upper ? aB : aA) + __shfl_xor_sync(0xffffffffu, upper ? aA : aB, 16);
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-      ra += __shfl_xor_sync(0xffffffffu, ra, d);
-      rb += __shfl_xor_sync(0xffffffffu, rb, d);
-    }
-    double da = static_cast<double>(ra), db = static_cast<double>(rb);
+    for (int d = 8; d > 0; d >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, d);
+    double dm = static_cast<double>(mine);
     if (__any_sync(0xffffffffu, hasbig)) {
-      double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
+      const double ta = bigacc[2 * kThreads], tb = bigacc[3 * kThreads];
       bigacc[2 * kThreads] = bigacc[3 * kThreads] = 0.0;
+      double tm = (upper ? tb : ta) + shfl_double(upper ? ta : tb, lane ^ 16);
 #pragma unroll
-      for (int d = 16; d > 0; d >>= 1) {
-        ta += shfl_double(ta, lane ^ d);
-        tb += shfl_double(tb, lane ^ d);
-      }
-      da += ta;
-      db += tb;
+      for (int d = 8; d > 0; d >>= 1) tm += shfl_double(tm, lane ^ d);
+      dm += tm;
     }
-    if (lane == 0 && emit) {
-      rec_a[rec_at + s] = da;
-      rec_b[rec_at + s] = db;
-    }
+    if ((lane & 15) == 0 && emit) (upper ? rec_b : rec_a)[rec_at + s] = dm;
     aA = aB = 0.f;
   }
   {
