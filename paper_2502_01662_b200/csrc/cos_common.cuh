@@ -480,13 +480,13 @@ __device__ __forceinline__ LaneSoft soft_slice(const void* row, const Slice& sl,
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         Elem<DT>::unpack(raw[u], x);
-        acc.add_fixed(x, c);
+        acc.add_fixed2(x, c);
       }
     }
     for (; v < sl.v_hi; v += NT) {
       raw[0] = ldg_stream16(rowb + static_cast<long long>(v) * 16);
       Elem<DT>::unpack(raw[0], x);
-      acc.add_fixed(x, c);
+      acc.add_fixed2(x, c);
     }
   }
   for (int e = sl.e_lo + tid; e < sl.e_hi; e += NT) acc.add_online1(Elem<DT>::load1(row, e), c);

@@ -117,10 +117,12 @@ __device__ __forceinline__ void sweep_unit(const KParams& p, const char* base, c
         Elem<DT>::unpack(raw, x);
         const float wi = p.w[i], wa = fabsf(wi);
 #pragma unroll
-        for (int k = 0; k < E; ++k) {
-          bad |= !(x[k] < INFINITY);
-          c32[k] = fmaf(wi, x[k], c32[k]);
+        for (int k = 0; k < E; ++k) bad |= !(x[k] < INFINITY);
+#pragma unroll
+        for (int k = 0; k < E; k += 2) {  // (packed fp32 pairs: the same values, half the instructions)
+          fma2(c32[k], c32[k + 1], wi, wi, x[k], x[k + 1], c32[k], c32[k + 1]);
           bnd[k] = fmaf(wa, fabsf(x[k]), bnd[k]);
+          bnd[k + 1] = fmaf(wa, fabsf(x[k + 1]), bnd[k + 1]);
         }
         if (i == pis) {
           float xm = x[0];
