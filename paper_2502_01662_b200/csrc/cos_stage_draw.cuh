@@ -357,27 +357,16 @@ __device__ __forceinline__ void one_sweep_pair(const KParams& p, Shared& sh, uin
     for (int k = 0; k < E; ++k) {
       // k_A e_A / Z_A + k_B e_B / Z_B > 0 with the products rounded one by one: where r and q coincide
       // neither side exceeds the other, as in exact arithmetic
-      if (MODE == kEnsembleSample) {
-        // the two channels side by side in the packed fp32 instructions: the same values, half the instructions
-        // (workload 3: 89.9 -> 89.0 us per call; at logit level the same made workload 5 slower, 550 -> 588 us)
-        float tA, tB, mA, mB;
-        fma2(tA, tB, xa[k], xb[k], cT, cT, nrefA, nrefB);
-        const float eA = ex2_approx(tA);
-        const float eB = ex2_approx(tB);
-        mul2(mA, mB, nctA, ctB, eA, eB);
-        add2(vzA, vzB, vzA, vzB, eA, eB);
-        if (mB > mA) add2(vaA, vaB, vaA, vaB, eA, eB);
-      } else {
-        const float eA = ex2_approx(fmaf(xa[k], cT, nrefA));
-        const float eB = ex2_approx(fmaf(xb[k], cT, nrefB));
-        const bool in_p = __fmul_rn(ctB, eB) > __fmul_rn(nctA, eA);
-        vzA += eA;
-        vzB += eB;
-        if (in_p) {
-          vaA += eA;
-          vaB += eB;
-        }
-      }
+      // The two channels side by side in the packed fp32 instructions: the same values, half the instructions
+      // (workload 3: 89.9 -> 89.0 us per call, workload 5: 549.0 -> 547.1; the combined logits of the logit level
+      // stay scalar: in pairs they made workload 5 slower).
+      float tA, tB, mA, mB;
+      fma2(tA, tB, xa[k], xb[k], cT, cT, nrefA, nrefB);
+      const float eA = ex2_approx(tA);
+      const float eB = ex2_approx(tB);
+      mul2(mA, mB, nctA, ctB, eA, eB);
+      add2(vzA, vzB, vzA, vzB, eA, eB);
+      if (mB > mA) add2(vaA, vaB, vaA, vaB, eA, eB);
     }
     // rare: the vector may hold a big entry (no term is negative, so a big entry makes its vector's sum
     // big); the caller does the vector again, big entries in fp64
