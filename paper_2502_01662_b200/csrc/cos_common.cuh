@@ -460,10 +460,10 @@ __device__ __forceinline__ Slice slice_of(int rank, int C, int V, bool vec_ok) {
 // Softmax normaliser of one row over the slice: fixed reference exponent (seeded from the
 // thread's first vector) with four loads in flight; overflow or a non-finite input falls
 // back to the running-maximum form.
-template <int DT, int NT>
+// U: 16-byte loads a thread issues before it consumes them
+template <int DT, int NT, int U = 4>
 __device__ __forceinline__ LaneSoft soft_slice(const void* row, const Slice& sl, int tid, float c) {
   constexpr int E = Elem<DT>::E;
-  constexpr int U = 4;
   const char* rowb = reinterpret_cast<const char*>(row);
   LaneSoft acc;
   acc.init();

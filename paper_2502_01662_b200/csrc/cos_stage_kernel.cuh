@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
     // One block per unit and no step that needs the whole block twice (the plausibility mask does, and so
     // does the greedy form of the combined-distribution test hook): the warps run without block barriers.
     if (C == 1 && !masked && (kSample || p.dump_r == nullptr)) {
-      stage0_free_running<DT, MODE>(p, sh);
+      stage0_free_running<DT, MODE, (MINB >= 4) ? 4 : 6>(p, sh);
       return;
     }
   } else {
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
 
     // ================================ sweep 1: statistics ================================
     if (MODE == kEnsembleSample) {
-      sweep_unit<DT, MODE>(p, base, sl, pis, false, 0.f, &sh.wsoft[warp][0], &sh.warg[warp][0]);
+      sweep_unit<DT, MODE, (MINB >= 4) ? 4 : 6>(p, base, sl, pis, false, 0.f, &sh.wsoft[warp][0], &sh.warg[warp][0]);
       cluster_merge(sh, cluster, phase, p.n, 0, 0);
       if (tid < p.n && !is_bonus && draft_ok) {
         // probability of the draft under model tid, with the constant the sweep used
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kThreads, MINB) cos_verify_kernel(const __grid
                          sh.fsoft[tid].s;
       }
     } else if (MODE == kEnsembleGreedy) {
-      sweep_unit<DT, MODE>(p, base, sl, pis, false, 0.f, &sh.wsoft[warp][0], &sh.warg[warp][0]);
+      sweep_unit<DT, MODE, (MINB >= 4) ? 4 : 6>(p, base, sl, pis, false, 0.f, &sh.wsoft[warp][0], &sh.warg[warp][0]);
       cluster_merge(sh, cluster, phase, 0, 0, p.n);
     } else {
       // logit-level combine.  soft slot 0 = proposer, soft slot 1 = combined logits;

@@ -26,7 +26,9 @@ __device__ __noinline__ double exact_combined(const KParams& p, const char* base
 // Ensemble greedy: arg slot i = argmax of model i.  Logit-level sampling: soft slot 0 = proposer,
 // soft slot 1 = combined logits.  Logit-level greedy: arg slot 1 = proposer argmax, arg slot 2 =
 // combined argmax.  `thr` is the plausibility threshold (logit-level modes with a mask).
-template <int DT, int MODE>
+// U: loads in flight per thread in the ensemble sweep (4 in the 32-register build, 6 where 64 registers allow it:
+// workload 4 went from 88.0 to 86.0 us per call; the 32-register build spills with 6 and lost 1.9 us on workload 3)
+template <int DT, int MODE, int U = 4>
 __device__ __forceinline__ void sweep_unit(const KParams& p, const char* base, const Slice& sl, int pis, bool masked,
                                            float thr, SoftPart* wsoft, ArgPart* warg) {
   constexpr int E = Elem<DT>::E;
@@ -34,7 +36,7 @@ __device__ __forceinline__ void sweep_unit(const KParams& p, const char* base, c
   auto row_of = [&](int i) -> const void* { return base + static_cast<long long>(i) * p.s_model * Elem<DT>::bytes; };
   if (MODE == kEnsembleSample) {
     for (int i = 0; i < p.n; ++i) {
-      LaneSoft acc = soft_slice<DT, kThreads>(row_of(i), sl, tid, p.cT);
+      LaneSoft acc = soft_slice<DT, kThreads, U>(row_of(i), sl, tid, p.cT);
       warp_merge_soft(acc, &wsoft[i], lane);
     }
   } else if (MODE == kEnsembleGreedy) {
@@ -376,7 +378,7 @@ __device__ __noinline__ void raise_fault(const KParams& p, FreeRun& fr, int lane
 // The last warp to finish a unit merges the sixteen partials, takes the decision (Eq. 6) and publishes
 // it while the others are already streaming; the first warp to finish draws the unit after the next
 // from the work counter.  Partials are kept two units deep; a warp may run at most one unit ahead.
-template <int DT, int MODE>
+template <int DT, int MODE, int U = 4>
 __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh) {
   constexpr bool kSample = (MODE == kEnsembleSample || MODE == kLogitSample);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -446,7 +448,7 @@ __device__ __forceinline__ void stage0_free_running(const KParams& p, Shared& sh
       skipped = (__shfl_sync(0xffffffffu, st, 0) == 2);
     }
     if (!skipped)
-      sweep_unit<DT, MODE>(p, base, sl, pis, false, -INFINITY, &fr.wsoft[par][warp][0], &fr.warg[par][warp][0]);
+      sweep_unit<DT, MODE, U>(p, base, sl, pis, false, -INFINITY, &fr.wsoft[par][warp][0], &fr.warg[par][warp][0]);
     if (settled && seq == 0) {
       asm volatile("griddepcontrol.wait;" ::: "memory");  // from here on as in an ordinary run
       if (tid == kThreads - 32) first_draw();
